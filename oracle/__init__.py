@@ -1,0 +1,306 @@
+"""PruneTrain hot-path ORACLE -- test infrastructure, not product code.
+
+A plain fp64 CPU statement of what the CUDA library computes, written from the
+paper. Only ``tests/``, ``__graft_entry__.smoke()`` and ``bench.py``'s
+``cpu_baseline`` / ``--impl reference`` legs may import this package; the
+product package never does, and this package never imports the product's CUDA
+path. The heavy loops live in ``pt_oracle.c`` (plain C, OpenMP over one outer
+loop); the graph-level rules (keep sets, compaction, the toy network used for
+the "compacted == masked" invariant, FLOP counts) are small numpy/Python loops
+here.
+
+Layouts: activations [N][H][W][C], weights [K][R][S][C], dense, numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pt_oracle.c")
+_LIB = os.path.join(_HERE, "libpt_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile pt_oracle.c into libpt_oracle.so next to it (gcc -O2 -fopenmp, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _L():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.pto_num_threads.restype = ctypes.c_int
+        _lib.pto_out_dim.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_L().pto_num_threads())
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def out_dim(H: int, R: int, stride: int, pad: int) -> int:
+    t = H + 2 * pad - R
+    return 0 if t < 0 else t // stride + 1
+
+
+def round_bf16(a) -> np.ndarray:
+    """bf16 round-to-nearest-even of fp32 values, widened to fp64."""
+    a = _f32(a)
+    out = np.empty(a.shape, dtype=np.float64)
+    _L().pto_round_bf16(_p(a), _p(out), ctypes.c_size_t(a.size))
+    return out
+
+
+def _conv_args(N, H, W, C, K, R, S, stride, pad):
+    return [ctypes.c_int(int(v)) for v in (N, H, W, C, K, R, S, stride, pad)]
+
+
+def conv_fwd(x, w, stride: int = 1, pad: int = 0) -> np.ndarray:
+    """y[n,p,q,k] = sum_{r,s,c} x[n,p*stride-pad+r,q*stride-pad+s,c] w[k,r,s,c]  (Sec. 2.1)."""
+    x, w = _f32(x), _f32(w)
+    N, H, W, C = x.shape
+    K, R, S, C2 = w.shape
+    assert C == C2
+    P, Q = out_dim(H, R, stride, pad), out_dim(W, S, stride, pad)
+    y = np.empty((N, P, Q, K), dtype=np.float64)
+    rc = _L().pto_conv_fwd(_p(x), _p(w), _p(y), *_conv_args(N, H, W, C, K, R, S, stride, pad))
+    assert rc == 0, rc
+    return y
+
+
+def conv_dgrad(dy, w, H: int, W: int, stride: int = 1, pad: int = 0) -> np.ndarray:
+    """dx = adjoint of conv_fwd in x applied to dy (back-propagation through the layer)."""
+    dy, w = _f32(dy), _f32(w)
+    K, R, S, C = w.shape
+    N, P, Q, K2 = dy.shape
+    assert K == K2 and P == out_dim(H, R, stride, pad) and Q == out_dim(W, S, stride, pad)
+    dx = np.empty((N, H, W, C), dtype=np.float64)
+    rc = _L().pto_conv_dgrad(_p(dy), _p(w), _p(dx), *_conv_args(N, H, W, C, K, R, S, stride, pad))
+    assert rc == 0, rc
+    return dx
+
+
+def conv_wgrad(x, dy, R: int, S: int, stride: int = 1, pad: int = 0) -> np.ndarray:
+    """dw[k,r,s,c] = sum_{n,p,q} dy[n,p,q,k] x[n,p*stride-pad+r,q*stride-pad+s,c]  (Eq. 4)."""
+    x, dy = _f32(x), _f32(dy)
+    N, H, W, C = x.shape
+    N2, P, Q, K = dy.shape
+    assert N == N2 and P == out_dim(H, R, stride, pad) and Q == out_dim(W, S, stride, pad)
+    dw = np.empty((K, R, S, C), dtype=np.float64)
+    rc = _L().pto_conv_wgrad(_p(x), _p(dy), _p(dw), *_conv_args(N, H, W, C, K, R, S, stride, pad))
+    assert rc == 0, rc
+    return dw
+
+
+def _samples(fn, a, b, idx, dims):
+    a, b = _f32(a), _f32(b)
+    idx = np.ascontiguousarray(np.asarray(idx, dtype=np.int64))
+    out = np.empty(idx.shape, dtype=np.float64)
+    rc = fn(_p(a), _p(b), _p(idx), ctypes.c_int64(idx.size), _p(out), *_conv_args(*dims))
+    assert rc == 0, rc
+    return out
+
+
+def conv_fwd_samples(x, w, idx, stride=1, pad=0) -> np.ndarray:
+    """Selected elements (flat indices into y[N][P][Q][K]) of conv_fwd, each summed alone."""
+    N, H, W, C = np.shape(x)
+    K, R, S, _ = np.shape(w)
+    return _samples(_L().pto_conv_fwd_samples, x, w, idx, (N, H, W, C, K, R, S, stride, pad))
+
+
+def conv_dgrad_samples(dy, w, idx, H, W, stride=1, pad=0) -> np.ndarray:
+    """Selected elements (flat indices into dx[N][H][W][C]) of conv_dgrad."""
+    N = np.shape(dy)[0]
+    K, R, S, C = np.shape(w)
+    return _samples(_L().pto_conv_dgrad_samples, dy, w, idx, (N, H, W, C, K, R, S, stride, pad))
+
+
+def conv_wgrad_samples(x, dy, idx, R, S, stride=1, pad=0) -> np.ndarray:
+    """Selected elements (flat indices into dw[K][R][S][C]) of conv_wgrad."""
+    N, H, W, C = np.shape(x)
+    K = np.shape(dy)[3]
+    return _samples(_L().pto_conv_wgrad_samples, x, dy, idx, (N, H, W, C, K, R, S, stride, pad))
+
+
+# --------------------------------------------------------------------------- lasso + SGD
+def lasso_sgd(w, g, v, lam: float, lr: float, mu: float, wd: float = 0.0,
+              reg_in: bool = True, reg_out: bool = True):
+    """One group-lasso + momentum-SGD update of a conv weight w[K][R][S][C]  (Eq. 1-2, Algorithm 1).
+
+    Returns (w_new, v_new, sumsq_out[K], sumsq_in[C], reg_sum) in fp64; reg_sum is Eq. 2
+    without lambda, from the pre-update weights.
+    """
+    w, g, v = _f32(w), _f32(g), _f32(v)
+    K, R, S, C = w.shape
+    w_new = np.empty(w.shape, np.float64)
+    v_new = np.empty(w.shape, np.float64)
+    s_out = np.empty(K, np.float64)
+    s_in = np.empty(C, np.float64)
+    reg = ctypes.c_double(0.0)
+    _L().pto_lasso_sgd(_p(w), _p(g), _p(v), ctypes.c_int(K), ctypes.c_int(C), ctypes.c_int(R * S),
+                       ctypes.c_int(int(reg_in)), ctypes.c_int(int(reg_out)),
+                       ctypes.c_double(lam), ctypes.c_double(lr), ctypes.c_double(mu), ctypes.c_double(wd),
+                       _p(w_new), _p(v_new), _p(s_out), _p(s_in), ctypes.byref(reg))
+    return w_new, v_new, s_out, s_in, reg.value
+
+
+def lasso_penalty(ws: Sequence[np.ndarray], reg_in: Sequence[bool], reg_out: Sequence[bool]) -> float:
+    """Eq. 2 without lambda: sum over layers of the input- and output-channel group L2 norms."""
+    tot = 0.0
+    for w, ri, ro in zip(ws, reg_in, reg_out):
+        w = np.asarray(w, np.float64)
+        if ro:
+            tot += float(np.sqrt((w * w).sum(axis=(1, 2, 3))).sum())
+        if ri:
+            tot += float(np.sqrt((w * w).sum(axis=(0, 1, 2))).sum())
+    return tot
+
+
+def set_coeff(loss1: float, reg_sum: float, ratio: float) -> float:
+    """Eq. 3 solved for lambda: ratio = lam*R / (loss1 + lam*R)."""
+    return ratio * loss1 / ((1.0 - ratio) * reg_sum)
+
+
+# --------------------------------------------------------------------------- detection
+def find_zero_groups(w, thr: float = 1e-4) -> Tuple[np.ndarray, np.ndarray]:
+    """(zero_out[K], zero_in[C]) uint8: group is zero iff every |w| < thr in fp32 (Sec. 4.1, Fig. 4)."""
+    w = _f32(w)
+    K, R, S, C = w.shape
+    zo = np.empty(K, np.uint8)
+    zi = np.empty(C, np.uint8)
+    _L().pto_find_zero_groups(_p(w), ctypes.c_int(K), ctypes.c_int(C), ctypes.c_int(R * S),
+                              ctypes.c_float(thr), _p(zo), _p(zi))
+    return zo, zi
+
+
+# --------------------------------------------------------------------------- keep sets + gather
+@dataclass
+class Graph:
+    """Channel spaces and the conv layers that write / read them.
+
+    A *channel space* is one set of channel indices shared by every conv that produces
+    it (its output channels) or consumes it (its input channels): the paper's "node" for
+    a residual stage, or the private tensor between two adjacent layers (Sec. 4.2).
+    ``layers[i] = (in_space, out_space)``; ``fixed[s]`` marks spaces never pruned (image).
+    """
+    sizes: List[int]
+    fixed: List[bool]
+    layers: List[Tuple[int, int]]
+
+
+def keep_sets(graph: Graph, zero_out: Sequence[np.ndarray], zero_in: Sequence[np.ndarray]) -> List[np.ndarray]:
+    """Surviving channel indices of every space, ascending (Sec. 4.2, intersection rule / channel union).
+
+    Channel j of a space is removed iff it is sparsified in ALL neighbouring convs: zero as an
+    output channel of every writer and zero as an input channel of every reader. Otherwise
+    (dense in at least one member: the union of dense channels) it is kept.
+    """
+    out = []
+    for s, size in enumerate(graph.sizes):
+        kept = []
+        for j in range(size):
+            keep = bool(graph.fixed[s])
+            for li, (isp, osp) in enumerate(graph.layers):
+                if osp == s and not zero_out[li][j]:
+                    keep = True
+                if isp == s and not zero_in[li][j]:
+                    keep = True
+            if keep:
+                kept.append(j)
+        out.append(np.asarray(kept, dtype=np.int32))
+    return out
+
+
+def gather_weight(w_old, mapK, mapC) -> np.ndarray:
+    """new[k',r,s,c'] = old[mapK[k'],r,s,mapC[c']], bit for bit (fp32)."""
+    w_old = _f32(w_old)
+    K, R, S, C = w_old.shape
+    mapK = np.ascontiguousarray(mapK, np.int32)
+    mapC = np.ascontiguousarray(mapC, np.int32)
+    out = np.empty((len(mapK), R, S, len(mapC)), np.float32)
+    _L().pto_gather_f32(_p(w_old), ctypes.c_int(C), ctypes.c_int(R * S), _p(mapK), ctypes.c_int(len(mapK)),
+                        _p(mapC), ctypes.c_int(len(mapC)), _p(out))
+    return out
+
+
+def gather_vector(vec, mapK) -> np.ndarray:
+    vec = np.asarray(vec)
+    out = np.empty(len(mapK), vec.dtype)
+    for i, j in enumerate(mapK):
+        out[i] = vec[j]
+    return out
+
+
+# --------------------------------------------------------------------------- FLOPs
+def conv_flops(N, H, W, C, K, R, S, stride, pad) -> int:
+    """Useful FLOPs of one conv pass (1 MAC = 2 FLOP) at the given (kept) channel counts."""
+    P, Q = out_dim(H, R, stride, pad), out_dim(W, S, stride, pad)
+    return 2 * N * P * Q * K * C * R * S
+
+
+# --------------------------------------------------------------------------- toy network (invariant only)
+def bn_affine(y, gamma, beta, mean, var, eps=1e-5):
+    """Inference-form batch norm with given running statistics, per output channel."""
+    return (y - mean) / np.sqrt(var + eps) * gamma + beta
+
+
+def toy_stage_forward(x, blocks, shortcut=None):
+    """fp64 forward of a small residual stage used to check "compacted == masked".
+
+    x: [N][H][W][C0].  shortcut: optional dict(w, bn) 1x1 projection from the input node.
+    blocks: list of dict(w1, bn1, w2, bn2): node -> conv3x3 -> BN -> ReLU -> conv3x3 -> BN -> (+node) -> ReLU.
+    Activations are NOT rounded to bf16 between layers beyond what conv_fwd does to its inputs;
+    callers pass bf16-representable data when bit-identity matters.
+    """
+    node = np.asarray(x, np.float64)
+    if shortcut is not None:
+        node = bn_affine(conv_fwd_f64(node, shortcut["w"], 1, 0), *shortcut["bn"])
+    for b in blocks:
+        t = np.maximum(bn_affine(conv_fwd_f64(node, b["w1"], 1, 1), *b["bn1"]), 0.0)
+        t = bn_affine(conv_fwd_f64(t, b["w2"], 1, 1), *b["bn2"])
+        node = np.maximum(t + node, 0.0)
+    return node
+
+
+def conv_fwd_f64(x, w, stride=1, pad=0) -> np.ndarray:
+    """The same 7-loop definition in pure fp64 numpy (no bf16 rounding), for the toy network.
+    Loops over taps and accumulates channel by channel in ascending order."""
+    x = np.asarray(x, np.float64)
+    w = np.asarray(w, np.float64)
+    N, H, W, C = x.shape
+    K, R, S, _ = w.shape
+    P, Q = out_dim(H, R, stride, pad), out_dim(W, S, stride, pad)
+    y = np.zeros((N, P, Q, K), np.float64)
+    for r in range(R):
+        for s in range(S):
+            for p in range(P):
+                h = p * stride - pad + r
+                if h < 0 or h >= H:
+                    continue
+                for q in range(Q):
+                    ww = q * stride - pad + s
+                    if ww < 0 or ww >= W:
+                        continue
+                    for c in range(C):
+                        y[:, p, q, :] += x[:, h, ww, c][:, None] * w[None, :, r, s, c]
+    return y
