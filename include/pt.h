@@ -1,0 +1,170 @@
+/*
+ * pt.h -- C ABI of the B200 (sm_100a) hot path of PruneTrain (arxiv 1901.09290).
+ *
+ * The library covers the convolution training step of a group-lasso-regularised CNN
+ * whose channel counts keep shrinking: conv forward / data gradient / weight gradient
+ * on ragged channel counts, the fused group-lasso + momentum-SGD update, zero-group
+ * detection and channel-union compaction ("reconfiguration").
+ *
+ * General conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".
+ *   - The caller allocates and frees every buffer, workspaces included. The library
+ *     allocates device memory only inside pt_create (a status word and a small table
+ *     arena) and frees it in pt_destroy.
+ *   - Every call validates its arguments on the host before any launch, enqueues its
+ *     kernels on `stream` (a cudaStream_t passed as void*) and returns without
+ *     synchronising, except pt_reconfigure_plan (documented below).
+ *   - Every call returns a pt_status. Device-side bounded waits that expire record
+ *     PT_ERR_TIMEOUT in the context's status word, read by pt_poll_device_status.
+ *   - There is no CPU fallback anywhere.
+ *
+ * Physical layouts
+ *   activations x, y, dy, dx : [N][H][W][ld]   bf16 (or fp32 outputs when out_f32 = 1), channels
+ *                              innermost, channel pitch ld >= channels, ld a multiple of 8 elements.
+ *                              Pad lanes (channel index >= channels) are never read; they are
+ *                              not written either.
+ *   master weights w, momentum v, gradient g/dw : [K][R][S][C] fp32, dense (no pitch).
+ *   bf16 weight shadow       : [K][R][S][ldw]  bf16, ldw >= C, ldw a multiple of 8.
+ *   Output size: P = floor((H + 2*pad - R)/stride) + 1, Q likewise from W and S.
+ */
+#ifndef PT_H_
+#define PT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PT_OK = 0,
+    PT_ERR_INVALID_ARG = 1,   /* null pointer, bad pitch/alignment/shape                */
+    PT_ERR_UNSUPPORTED = 2,   /* legal but not implemented (e.g. a forced algo that cannot run the shape) */
+    PT_ERR_WORKSPACE = 3,     /* workspace missing or smaller than pt_*_workspace_bytes */
+    PT_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                      */
+    PT_ERR_TIMEOUT = 5,       /* a bounded device-side wait expired                     */
+    PT_ERR_ARCH = 6           /* the device is not sm_100                               */
+} pt_status;
+
+typedef struct pt_ctx pt_ctx;  /* opaque: device id, SM count, status word, table arena, tensor-map cache */
+
+/* Create / destroy the per-device context. pt_create makes `device` current, checks that it is
+ * an sm_100 part (else PT_ERR_ARCH) and allocates the status word and table arena. */
+pt_status pt_create(pt_ctx **ctx, int device);
+pt_status pt_destroy(pt_ctx *ctx);
+const char *pt_status_string(pt_status s);
+/* Synchronises `stream`, reads and clears the device status word. PT_OK if no kernel recorded an error. */
+pt_status pt_poll_device_status(pt_ctx *ctx, void *stream);
+/* Number of kernels this context has launched since creation (for launch accounting). */
+uint64_t pt_launch_count(const pt_ctx *ctx);
+
+/* ------------------------------------------------------------------------------------------
+ * Convolutions (paper Sec. 2.1: convolution layers dominate training time; Eq. 4: weight gradient).
+ * Cross-correlation, square stride and padding, dilation 1, groups 1, no bias.
+ * C and K are the CURRENT (pruned, possibly ragged: 11, 27, 93 ...) channel counts.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    int32_t N, H, W, C, K, R, S, stride, pad;
+    int32_t ldx;      /* channel pitch of x / dx  (elements, multiple of 8, >= C)           */
+    int32_t ldy;      /* channel pitch of y / dy  (elements, multiple of 8, >= K)           */
+    int32_t ldw;      /* channel pitch of the bf16 weight shadow (multiple of 8, >= C)      */
+    int32_t out_f32;  /* fwd/dgrad: 0 = bf16 output, 1 = fp32 output (same pitch in elements) */
+    int32_t algo;     /* 0 = automatic; 1 = force the SIMT kernels; 2 = force the tcgen05 kernels */
+} pt_conv_desc;
+
+enum { PT_CONV_FWD = 0, PT_CONV_DGRAD = 1, PT_CONV_WGRAD = 2 };
+
+/* Bytes of caller-provided workspace the given pass needs for this descriptor (0 = none). */
+size_t pt_conv_workspace_bytes(const pt_ctx *ctx, const pt_conv_desc *d, int which);
+
+/* y[n,p,q,k] = sum_{r,s,c} x[n, p*stride-pad+r, q*stride-pad+s, c] * w[k,r,s,c], zero outside the image.
+ * x: bf16 [N][H][W][ldx]; w: bf16 shadow [K][R][S][ldw]; y: [N][P][Q][ldy] bf16 or fp32. fp32 accumulation. */
+pt_status pt_conv_fwd(pt_ctx *ctx, const pt_conv_desc *d, const void *x, const void *w, void *y,
+                      void *ws, size_t ws_bytes, void *stream);
+
+/* dx[n,h,w,c] = sum over (k,r,s,p,q) with p*stride-pad+r = h and q*stride-pad+s = w of dy[n,p,q,k] * w[k,r,s,c].
+ * Back-propagation through the layer (Sec. 2.1). Pixels no tap reaches are written as 0.
+ * dy: bf16 [N][P][Q][ldy]; dx: [N][H][W][ldx] bf16 or fp32. */
+pt_status pt_conv_dgrad(pt_ctx *ctx, const pt_conv_desc *d, const void *dy, const void *w, void *dx,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/* dw[k,r,s,c] = sum_{n,p,q} dy[n,p,q,k] * x[n, p*stride-pad+r, q*stride-pad+s, c]   (Eq. 4).
+ * dw: fp32 [K][R][S][C] dense. Deterministic: partial sums are combined in a fixed order. */
+pt_status pt_conv_wgrad(pt_ctx *ctx, const pt_conv_desc *d, const void *x, const void *dy, float *dw,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Group-lasso regularised momentum SGD (Eq. 1-2; Algorithm 1: GroupLassoReg(W_i) then Optimizer).
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    float *w;            /* fp32 master weights [K][RS][C], updated in place                        */
+    const float *g;      /* fp32 gradient of the data loss (wgrad output), same layout               */
+    float *v;            /* fp32 momentum, updated in place                                          */
+    void *w_bf16;        /* bf16 shadow [K][RS][ldw], rewritten from the new w; may be NULL          */
+    int32_t K, C, RS, ldw;
+    uint8_t reg_in;      /* regularise the input-channel groups (0 for the first conv: its inputs are the image) */
+    uint8_t reg_out;     /* regularise the output-channel groups                                      */
+    float *sumsq_out;    /* K floats: sum of squares of each output-channel group of the PRE-update w */
+    float *sumsq_in;     /* C floats: same for input-channel groups                                   */
+    uint8_t *zero_out;   /* K bytes, written by pt_find_zero_groups (1 = group is zero)               */
+    uint8_t *zero_in;    /* C bytes                                                                    */
+} pt_layer;
+
+typedef struct { float lambda, lr, momentum, weight_decay; } pt_sgd_hparams;
+
+/* Workspace for pt_group_lasso_sgd_step and pt_find_zero_groups over this set of layers. */
+size_t pt_group_lasso_workspace_bytes(const pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers);
+
+/* For every layer:  s_out[k] = sum_{rs,c} w^2,  s_in[c] = sum_{k,rs} w^2  (pre-update weights),
+ *   g~ = g + weight_decay*w + lambda*w*( [reg_out, s_out>1e-24]/sqrt(s_out[k]) + [reg_in, s_in>1e-24]/sqrt(s_in[c]) )
+ *   v <- momentum*v + g~ ;  w <- w - lr*v ;  shadow <- round-to-nearest-even bf16 of the new w.
+ * That is the gradient of Eq. 1 with the regulariser of Eq. 2 (one global lambda; input- and output-channel
+ * groups overlap) followed by the optimiser step of Algorithm 1. An all-zero group has subgradient 0.
+ * reg_sum_out (device, optional): receives sum over regularised groups of sqrt(sumsq) -- Eq. 2 without lambda.
+ * layers is a HOST array; the library keeps a device copy and re-uploads it only when it changes. */
+pt_status pt_group_lasso_sgd_step(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers,
+                                  const pt_sgd_hparams *hp /*host*/, double *reg_sum_out,
+                                  void *ws, size_t ws_bytes, void *stream);
+
+/* zero_out[k] = (max_{rs,c} |w| < threshold), zero_in[c] = (max_{k,rs} |w| < threshold), strict <, in fp32
+ * (Sec. 4.1: threshold 1e-4; Sec. 4.2 / Fig. 4: the absolute maximum of a channel's parameters). A NaN keeps
+ * its groups. If zero_in_place != 0 the weights, momentum and shadow of every detected group are set to 0.
+ * Uses sumsq_out / sumsq_in of each layer as scratch (their contents are destroyed). */
+pt_status pt_find_zero_groups(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers, float threshold,
+                              int32_t zero_in_place, void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Reconfiguration (Sec. 4.2: prune only the intersection of the sparsified channels of adjacent layers;
+ * channel union across all convs that share a residual node; surviving training variables kept as is).
+ * A channel space is one set of channel indices shared by the convs that write it (as output channels)
+ * and read it (as input channels).
+ * ------------------------------------------------------------------------------------------ */
+typedef struct { int32_t size; uint8_t fixed; } pt_space;      /* fixed: never pruned (the image, the classifier input) */
+typedef struct {
+    int32_t in_space, out_space;
+    float *bn[4];                                              /* gamma, beta, running mean, running var (K floats each) or NULL */
+} pt_layer_link;
+typedef struct {
+    const pt_space *spaces; int32_t n_spaces;                  /* host arrays */
+    const pt_layer *layers; const pt_layer_link *links; int32_t n_layers;
+} pt_graph;
+
+/* Phase 0. From the zero masks of g's layers, for every space:
+ *   keep[j] = fixed  OR  some writer has zero_out[j] = 0  OR  some reader has zero_in[j] = 0
+ * new2old (device, sum of space sizes int32; space s starts at the sum of the sizes before it) receives
+ * the kept indices in ascending order (entries past the count are -1); new_sizes (HOST, n_spaces) receives the
+ * counts. This call synchronises `stream` once to return the counts. A count of 0 is reported, not clamped. */
+pt_status pt_reconfigure_plan(pt_ctx *ctx, const pt_graph *g, int32_t *new2old, int32_t *new_sizes /*host*/, void *stream);
+
+/* Phase 1. Gather every layer of old_g into the caller-allocated tensors of new_g:
+ *   new.w[k',rs,c'] = old.w[new2old_out[k'], rs, new2old_in[c']]   (same for v and the bf16 shadow, bit for bit)
+ *   new.bn[i][k']   = old.bn[i][new2old_out[k']]
+ * new_g must have the same topology, and each space size equal to the count pt_reconfigure_plan returned.
+ * Layers whose new K or C is 0 are skipped. */
+pt_status pt_reconfigure(pt_ctx *ctx, const pt_graph *old_g, const int32_t *new2old, const pt_graph *new_g, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PT_H_ */

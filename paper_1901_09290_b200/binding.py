@@ -1,0 +1,229 @@
+"""Thin ctypes binding of the C ABI in ``include/pt.h``: same names, argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device memory; their ``data_ptr()`` is what the
+library sees. Every computation happens inside the library's CUDA kernels; if the shared
+library is missing or a call fails, this module raises -- there is no CPU path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import (POINTER, Structure, byref, c_char_p, c_double, c_float, c_int32, c_size_t, c_uint8, c_uint64,
+                    c_void_p)
+from typing import List, Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpt_b200.so")
+
+PT_OK = 0
+PT_CONV_FWD, PT_CONV_DGRAD, PT_CONV_WGRAD = 0, 1, 2
+STATUS_NAMES = ["PT_OK", "PT_ERR_INVALID_ARG", "PT_ERR_UNSUPPORTED", "PT_ERR_WORKSPACE", "PT_ERR_CUDA",
+                "PT_ERR_TIMEOUT", "PT_ERR_ARCH"]
+
+
+class PtError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{what} failed: {name}")
+
+
+class pt_conv_desc(Structure):
+    _fields_ = [(n, c_int32) for n in ("N", "H", "W", "C", "K", "R", "S", "stride", "pad",
+                                       "ldx", "ldy", "ldw", "out_f32", "algo")]
+
+
+class pt_layer(Structure):
+    _fields_ = [("w", c_void_p), ("g", c_void_p), ("v", c_void_p), ("w_bf16", c_void_p),
+                ("K", c_int32), ("C", c_int32), ("RS", c_int32), ("ldw", c_int32),
+                ("reg_in", c_uint8), ("reg_out", c_uint8),
+                ("sumsq_out", c_void_p), ("sumsq_in", c_void_p), ("zero_out", c_void_p), ("zero_in", c_void_p)]
+
+
+class pt_sgd_hparams(Structure):
+    _fields_ = [("lambda_", c_float), ("lr", c_float), ("momentum", c_float), ("weight_decay", c_float)]
+
+
+class pt_space(Structure):
+    _fields_ = [("size", c_int32), ("fixed", c_uint8)]
+
+
+class pt_layer_link(Structure):
+    _fields_ = [("in_space", c_int32), ("out_space", c_int32), ("bn", c_void_p * 4)]
+
+
+class pt_graph(Structure):
+    _fields_ = [("spaces", POINTER(pt_space)), ("n_spaces", c_int32),
+                ("layers", POINTER(pt_layer)), ("links", POINTER(pt_layer_link)), ("n_layers", c_int32)]
+
+
+EXPORTS = {
+    "pt_create": (c_int32, [POINTER(c_void_p), c_int32]),
+    "pt_destroy": (c_int32, [c_void_p]),
+    "pt_status_string": (c_char_p, [c_int32]),
+    "pt_poll_device_status": (c_int32, [c_void_p, c_void_p]),
+    "pt_launch_count": (c_uint64, [c_void_p]),
+    "pt_conv_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_conv_desc), c_int32]),
+    "pt_conv_fwd": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "pt_conv_dgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "pt_conv_wgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "pt_group_lasso_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_layer), c_int32]),
+    "pt_group_lasso_sgd_step": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, POINTER(pt_sgd_hparams), c_void_p,
+                                          c_void_p, c_size_t, c_void_p]),
+    "pt_find_zero_groups": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_float, c_int32, c_void_p, c_size_t, c_void_p]),
+    "pt_reconfigure_plan": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(c_int32), c_void_p]),
+    "pt_reconfigure": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(pt_graph), c_void_p]),
+}
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library. Raises if it has not been built (run ``python -m paper_1901_09290_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"CUDA library not built: {LIB_PATH} is missing (python -m paper_1901_09290_b200.build)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(L, name)          # AttributeError if a declared symbol is not exported
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(status: int, what: str):
+    if status != PT_OK:
+        raise PtError(status, what)
+
+
+class Context:
+    """Owns a pt_ctx for one device."""
+
+    def __init__(self, device: int = 0):
+        self.handle = c_void_p()
+        _check(lib().pt_create(byref(self.handle), device), "pt_create")
+        self.device = device
+
+    def close(self):
+        if self.handle:
+            lib().pt_destroy(self.handle)
+            self.handle = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def launch_count(self) -> int:
+        return int(lib().pt_launch_count(self.handle))
+
+    def poll(self, stream=None):
+        _check(lib().pt_poll_device_status(self.handle, _stream(stream)), "pt_poll_device_status")
+
+
+def make_conv_desc(N, H, W, C, K, R, S, stride, pad, ldx=None, ldy=None, ldw=None, out_f32=0, algo=0) -> pt_conv_desc:
+    p8 = lambda c: (c + 7) // 8 * 8
+    return pt_conv_desc(N, H, W, C, K, R, S, stride, pad, ldx or p8(C), ldy or p8(K), ldw or p8(C), out_f32, algo)
+
+
+def pt_conv_workspace_bytes(ctx: Context, d: pt_conv_desc, which: int) -> int:
+    return int(lib().pt_conv_workspace_bytes(ctx.handle, byref(d), which))
+
+
+def _ws(ws):
+    return (None, 0) if ws is None else (ws.data_ptr(), ws.numel() * ws.element_size())
+
+
+def pt_conv_fwd(ctx, d, x, w, y, ws=None, stream=None):
+    p, n = _ws(ws)
+    _check(lib().pt_conv_fwd(ctx.handle, byref(d), _ptr(x), _ptr(w), _ptr(y), p, n, _stream(stream)), "pt_conv_fwd")
+
+
+def pt_conv_dgrad(ctx, d, dy, w, dx, ws=None, stream=None):
+    p, n = _ws(ws)
+    _check(lib().pt_conv_dgrad(ctx.handle, byref(d), _ptr(dy), _ptr(w), _ptr(dx), p, n, _stream(stream)), "pt_conv_dgrad")
+
+
+def pt_conv_wgrad(ctx, d, x, dy, dw, ws=None, stream=None):
+    p, n = _ws(ws)
+    _check(lib().pt_conv_wgrad(ctx.handle, byref(d), _ptr(x), _ptr(dy), _ptr(dw), p, n, _stream(stream)), "pt_conv_wgrad")
+
+
+def make_layer(w, g, v, w_bf16, K, C, RS, ldw, reg_in, reg_out, sumsq_out, sumsq_in, zero_out, zero_in) -> pt_layer:
+    return pt_layer(_ptr(w), _ptr(g), _ptr(v), _ptr(w_bf16), K, C, RS, ldw, int(bool(reg_in)), int(bool(reg_out)),
+                    _ptr(sumsq_out), _ptr(sumsq_in), _ptr(zero_out), _ptr(zero_in))
+
+
+def layer_array(layers: Sequence[pt_layer]):
+    return (pt_layer * len(layers))(*layers)
+
+
+def pt_group_lasso_workspace_bytes(ctx, layers) -> int:
+    arr = layers if not isinstance(layers, (list, tuple)) else layer_array(layers)
+    return int(lib().pt_group_lasso_workspace_bytes(ctx.handle, arr, len(arr)))
+
+
+def pt_group_lasso_sgd_step(ctx, layers, lam, lr, momentum, weight_decay=0.0, reg_sum_out=None, ws=None, stream=None):
+    arr = layers if not isinstance(layers, (list, tuple)) else layer_array(layers)
+    hp = pt_sgd_hparams(lam, lr, momentum, weight_decay)
+    p, n = _ws(ws)
+    _check(lib().pt_group_lasso_sgd_step(ctx.handle, arr, len(arr), byref(hp), _ptr(reg_sum_out), p, n, _stream(stream)),
+           "pt_group_lasso_sgd_step")
+
+
+def pt_find_zero_groups(ctx, layers, threshold=1e-4, zero_in_place=False, ws=None, stream=None):
+    arr = layers if not isinstance(layers, (list, tuple)) else layer_array(layers)
+    p, n = _ws(ws)
+    _check(lib().pt_find_zero_groups(ctx.handle, arr, len(arr), threshold, int(bool(zero_in_place)), p, n, _stream(stream)),
+           "pt_find_zero_groups")
+
+
+class GraphHandle:
+    """Keeps the ctypes arrays of a pt_graph alive."""
+
+    def __init__(self, sizes: Sequence[int], fixed: Sequence[bool], layers: Sequence[pt_layer],
+                 links: Sequence[tuple], bn: Optional[Sequence[Optional[Sequence]]] = None):
+        self.spaces = (pt_space * len(sizes))(*[pt_space(int(s), int(bool(f))) for s, f in zip(sizes, fixed)])
+        self.layers = layer_array(layers)
+        lk = []
+        for i, (isp, osp) in enumerate(links):
+            ptrs = (c_void_p * 4)()
+            if bn is not None and bn[i] is not None:
+                for b in range(4):
+                    ptrs[b] = _ptr(bn[i][b])
+            lk.append(pt_layer_link(isp, osp, ptrs))
+        self.links = (pt_layer_link * len(lk))(*lk)
+        self.graph = pt_graph(self.spaces, len(sizes), self.layers, self.links, len(lk))
+
+
+def pt_reconfigure_plan(ctx, graph: GraphHandle, new2old, stream=None) -> List[int]:
+    n = graph.graph.n_spaces
+    sizes = (c_int32 * n)()
+    _check(lib().pt_reconfigure_plan(ctx.handle, byref(graph.graph), _ptr(new2old), sizes, _stream(stream)),
+           "pt_reconfigure_plan")
+    return list(sizes)
+
+
+def pt_reconfigure(ctx, old: GraphHandle, new2old, new: GraphHandle, stream=None):
+    _check(lib().pt_reconfigure(ctx.handle, byref(old.graph), _ptr(new2old), byref(new.graph), _stream(stream)),
+           "pt_reconfigure")

@@ -1,0 +1,174 @@
+// Context management, status handling, table upload and the conv entry points' dispatch.
+#include "pt_internal.h"
+
+static const size_t kArenaBytes = 4u << 20;     // 4 MiB of tables: three regions
+static const size_t kRegionBytes = kArenaBytes / 4;
+
+extern "C" const char *pt_status_string(pt_status s)
+{
+    switch (s) {
+    case PT_OK: return "PT_OK";
+    case PT_ERR_INVALID_ARG: return "PT_ERR_INVALID_ARG";
+    case PT_ERR_UNSUPPORTED: return "PT_ERR_UNSUPPORTED";
+    case PT_ERR_WORKSPACE: return "PT_ERR_WORKSPACE";
+    case PT_ERR_CUDA: return "PT_ERR_CUDA";
+    case PT_ERR_TIMEOUT: return "PT_ERR_TIMEOUT";
+    case PT_ERR_ARCH: return "PT_ERR_ARCH";
+    }
+    return "PT_ERR_UNKNOWN";
+}
+
+extern "C" pt_status pt_create(pt_ctx **out, int device)
+{
+    if (!out) return PT_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) { (void)cudaGetLastError(); return PT_ERR_CUDA; }
+    PT_CUDA_OK(cudaSetDevice(device));
+    cudaDeviceProp prop;
+    PT_CUDA_OK(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return PT_ERR_ARCH;
+    pt_ctx *c = new pt_ctx();
+    c->device = device;
+    c->sm_count = prop.multiProcessorCount;
+    c->cc_major = prop.major;
+    c->cc_minor = prop.minor;
+    c->arena_bytes = kArenaBytes;
+    bool ok = cudaMalloc(&c->d_status, 16) == cudaSuccess && cudaMemset(c->d_status, 0, 16) == cudaSuccess &&
+              cudaMallocHost(&c->h_status, 16) == cudaSuccess && cudaMalloc(&c->d_arena, kArenaBytes) == cudaSuccess &&
+              cudaMallocHost(&c->h_stage, kArenaBytes) == cudaSuccess &&
+              cudaMallocHost(&c->h_counts, 65536 * sizeof(int32_t)) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->upload_done, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); pt_destroy(c); return PT_ERR_CUDA; }
+    c->lasso_tab.off = 0;                 c->lasso_tab.cap = 2 * kRegionBytes;
+    c->graph_tab.off = 2 * kRegionBytes;  c->graph_tab.cap = kRegionBytes;
+    c->gather_tab.off = 3 * kRegionBytes; c->gather_tab.cap = kRegionBytes;
+    // Driver entry points for tensor-map encoding, looked up at run time so the library loads without libcuda.
+    cudaDriverEntryPointQueryResult qr;
+    void *fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess) c->encode_tiled = fn;
+    fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess) c->encode_im2col = fn;
+    (void)cudaGetLastError();
+    *out = c;
+    return PT_OK;
+}
+
+extern "C" pt_status pt_destroy(pt_ctx *c)
+{
+    if (!c) return PT_OK;
+    (void)cudaSetDevice(c->device);
+    if (c->upload_done) cudaEventDestroy(c->upload_done);
+    if (c->d_status) cudaFree(c->d_status);
+    if (c->h_status) cudaFreeHost(c->h_status);
+    if (c->d_arena) cudaFree(c->d_arena);
+    if (c->h_stage) cudaFreeHost(c->h_stage);
+    if (c->h_counts) cudaFreeHost(c->h_counts);
+    (void)cudaGetLastError();
+    delete c;
+    return PT_OK;
+}
+
+extern "C" uint64_t pt_launch_count(const pt_ctx *c) { return c ? c->launches : 0; }
+
+extern "C" pt_status pt_poll_device_status(pt_ctx *c, void *stream)
+{
+    if (!c) return PT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    PT_CUDA_OK(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, st));
+    PT_CUDA_OK(cudaStreamSynchronize(st));
+    unsigned int code = c->h_status[0];
+    if (code != PT_DEV_OK) {
+        PT_CUDA_OK(cudaMemsetAsync(c->d_status, 0, 16, st));
+        PT_CUDA_OK(cudaStreamSynchronize(st));
+        return code == PT_DEV_TIMEOUT ? PT_ERR_TIMEOUT : PT_ERR_CUDA;
+    }
+    return PT_OK;
+}
+
+pt_status pt_upload_table(pt_ctx *c, pt_region *reg, const void *host, size_t bytes, cudaStream_t st, char **dev)
+{
+    if (bytes > reg->cap) return PT_ERR_UNSUPPORTED;
+    *dev = c->d_arena + reg->off;
+    if (reg->valid && reg->key.size() == bytes && memcmp(reg->key.data(), host, bytes) == 0) return PT_OK;
+    if (c->upload_pending) {                       // the staging buffer may still be the source of a copy
+        PT_CUDA_OK(cudaEventSynchronize(c->upload_done));
+        c->upload_pending = false;
+    }
+    memcpy(c->h_stage + reg->off, host, bytes);
+    PT_CUDA_OK(cudaMemcpyAsync(c->d_arena + reg->off, c->h_stage + reg->off, bytes, cudaMemcpyHostToDevice, st));
+    PT_CUDA_OK(cudaEventRecord(c->upload_done, st));
+    c->upload_pending = true;
+    reg->key.assign((const char *)host, (const char *)host + bytes);
+    reg->valid = true;
+    return PT_OK;
+}
+
+// ------------------------------------------------------------------------------------------ conv dispatch
+pt_status pt_conv_validate(const pt_ctx *c, const pt_conv_desc *d, int *P, int *Q)
+{
+    if (!c || !d) return PT_ERR_INVALID_ARG;
+    if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C <= 0 || d->K <= 0 || d->R <= 0 || d->S <= 0) return PT_ERR_INVALID_ARG;
+    if (d->stride <= 0 || d->pad < 0 || d->pad >= d->R + d->S) return PT_ERR_INVALID_ARG;
+    if (d->ldx < d->C || d->ldx % 8 || d->ldy < d->K || d->ldy % 8 || d->ldw < d->C || d->ldw % 8) return PT_ERR_INVALID_ARG;
+    if (d->algo < 0 || d->algo > 2) return PT_ERR_INVALID_ARG;
+    *P = pt_out_dim(d->H, d->R, d->stride, d->pad);
+    *Q = pt_out_dim(d->W, d->S, d->stride, d->pad);
+    if (*P <= 0 || *Q <= 0) return PT_ERR_INVALID_ARG;
+    // index arithmetic inside the kernels is 64-bit for addresses and 32-bit for pixel counts
+    if ((int64_t)d->N * d->H * d->W >= (1ll << 31) || (int64_t)d->N * *P * *Q >= (1ll << 31)) return PT_ERR_UNSUPPORTED;
+    if ((int64_t)d->K * d->R * d->S * d->ldw >= (1ll << 31)) return PT_ERR_UNSUPPORTED;
+    return PT_OK;
+}
+
+static bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
+
+extern "C" size_t pt_conv_workspace_bytes(const pt_ctx *c, const pt_conv_desc *d, int which)
+{
+    int P, Q;
+    if (which < 0 || which > 2 || pt_conv_validate(c, d, &P, &Q) != PT_OK) return 0;
+    size_t a = pt_simt_conv_workspace(c, d, which);
+    size_t b = pt_sm100_conv_supported(c, d, which) ? pt_sm100_conv_workspace(c, d, which) : 0;
+    if (d->algo == 1) return a;
+    if (d->algo == 2) return b;
+    return a > b ? a : b;
+}
+
+static pt_status conv_dispatch(pt_ctx *c, const pt_conv_desc *d, int which, const void *a, const void *b, void *out,
+                               void *ws, size_t ws_bytes, void *stream)
+{
+    int P, Q;
+    pt_status s = pt_conv_validate(c, d, &P, &Q);
+    if (s != PT_OK) return s;
+    if (!a || !b || !out) return PT_ERR_INVALID_ARG;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(out) || (ws && !aligned16(ws))) return PT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    bool fast = d->algo != 1 && pt_sm100_conv_supported(c, d, which);
+    if (d->algo == 2 && !fast) return PT_ERR_UNSUPPORTED;
+    if (fast) {
+        if (pt_sm100_conv_workspace(c, d, which) > ws_bytes || (pt_sm100_conv_workspace(c, d, which) && !ws)) return PT_ERR_WORKSPACE;
+        return pt_sm100_conv(c, d, which, a, b, out, ws, ws_bytes, st);
+    }
+    if (pt_simt_conv_workspace(c, d, which) > ws_bytes || (pt_simt_conv_workspace(c, d, which) && !ws)) return PT_ERR_WORKSPACE;
+    return pt_simt_conv(c, d, which, a, b, out, ws, ws_bytes, st);
+}
+
+extern "C" pt_status pt_conv_fwd(pt_ctx *c, const pt_conv_desc *d, const void *x, const void *w, void *y,
+                                 void *ws, size_t ws_bytes, void *stream)
+{
+    return conv_dispatch(c, d, PT_CONV_FWD, x, w, y, ws, ws_bytes, stream);
+}
+
+extern "C" pt_status pt_conv_dgrad(pt_ctx *c, const pt_conv_desc *d, const void *dy, const void *w, void *dx,
+                                   void *ws, size_t ws_bytes, void *stream)
+{
+    return conv_dispatch(c, d, PT_CONV_DGRAD, dy, w, dx, ws, ws_bytes, stream);
+}
+
+extern "C" pt_status pt_conv_wgrad(pt_ctx *c, const pt_conv_desc *d, const void *x, const void *dy, float *dw,
+                                   void *ws, size_t ws_bytes, void *stream)
+{
+    return conv_dispatch(c, d, PT_CONV_WGRAD, x, dy, dw, ws, ws_bytes, stream);
+}

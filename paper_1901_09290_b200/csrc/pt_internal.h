@@ -1,0 +1,71 @@
+// Internal declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string.h>
+#include <vector>
+#include <map>
+#include <string>
+
+#include "../../include/pt.h"
+
+#define PT_CUDA_OK(call)                                   \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) { (void)cudaGetLastError(); return PT_ERR_CUDA; } \
+    } while (0)
+
+// Device status word layout: [0] = first error code recorded (0 = none), [1] = detail (where), [2..3] spare.
+enum { PT_DEV_OK = 0, PT_DEV_TIMEOUT = 1 };
+
+struct pt_region {              // one cached table in the arena
+    size_t off = 0, cap = 0;    // byte range inside the arena
+    std::vector<char> key;      // host bytes the current device copy was built from
+    bool valid = false;
+};
+
+struct pt_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int cc_major = 0, cc_minor = 0;
+    unsigned int *d_status = nullptr;   // 4 words, device
+    unsigned int *h_status = nullptr;   // 4 words, pinned host
+    char *d_arena = nullptr;            // table arena, device
+    char *h_stage = nullptr;            // pinned staging copy of the arena
+    size_t arena_bytes = 0;
+    cudaEvent_t upload_done = nullptr;  // last staging->arena copy
+    bool upload_pending = false;
+    pt_region lasso_tab, graph_tab, gather_tab;
+    int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan
+    uint64_t launches = 0;
+    // tcgen05 conv path
+    void *encode_tiled = nullptr;       // cuTensorMapEncodeTiled
+    void *encode_im2col = nullptr;      // cuTensorMapEncodeIm2col
+    std::map<std::string, std::vector<char>> tmap_cache;
+};
+
+static inline int pt_ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline size_t pt_align_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
+static inline int pt_out_dim(int H, int R, int stride, int pad) {
+    int t = H + 2 * pad - R;
+    return t < 0 ? 0 : t / stride + 1;
+}
+
+// Copies `bytes` of host data into the region's slot of the arena if it differs from what is there.
+// Returns the device address of the slot.
+pt_status pt_upload_table(pt_ctx *ctx, pt_region *reg, const void *host, size_t bytes, cudaStream_t st, char **dev);
+
+// Validation shared by the conv entry points. Fills P, Q.
+pt_status pt_conv_validate(const pt_ctx *ctx, const pt_conv_desc *d, int *P, int *Q);
+
+// SIMT (CUDA-core) convolution kernels: every legal shape.
+pt_status pt_simt_conv(pt_ctx *ctx, const pt_conv_desc *d, int which, const void *a, const void *b, void *out,
+                       void *ws, size_t ws_bytes, cudaStream_t st);
+size_t pt_simt_conv_workspace(const pt_ctx *ctx, const pt_conv_desc *d, int which);
+
+// tcgen05 / TMEM / TMA convolution kernels: returns PT_ERR_UNSUPPORTED for shapes they do not cover.
+bool pt_sm100_conv_supported(const pt_ctx *ctx, const pt_conv_desc *d, int which);
+pt_status pt_sm100_conv(pt_ctx *ctx, const pt_conv_desc *d, int which, const void *a, const void *b, void *out,
+                        void *ws, size_t ws_bytes, cudaStream_t st);
+size_t pt_sm100_conv_workspace(const pt_ctx *ctx, const pt_conv_desc *d, int which);

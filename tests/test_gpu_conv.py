@@ -1,0 +1,111 @@
+"""Parity of the CUDA convolutions (through the C ABI) with the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_09290_b200 import binding as B
+from paper_1901_09290_b200 import workloads as W
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+ALGOS = [0, 1]
+
+# (N, H, W, C, K, R, stride)  -- odd and tiny channel counts, ragged pixel tails, stride 2, 7x7
+SMALL = [
+    (2, 5, 7, 1, 1, 1, 1), (2, 5, 7, 3, 7, 3, 1), (1, 1, 1, 8, 11, 1, 1), (3, 16, 16, 11, 27, 3, 1),
+    (2, 16, 16, 16, 16, 1, 1), (2, 9, 9, 27, 8, 3, 2), (2, 8, 8, 7, 93, 1, 2), (1, 23, 23, 3, 16, 7, 2),
+    (2, 14, 14, 93, 77, 3, 1), (1, 12, 10, 130, 70, 1, 1), (1, 7, 7, 260, 300, 3, 1),
+]
+
+
+def _case(N, H, Wd, C, K, R, stride, seed):
+    pad = R // 2
+    x = W.gen_act(N, H, Wd, C, seed)
+    w = W.bf16_round(W.gen_weight(K, R, R, C, seed + 1))
+    P, Q = (H + 2 * pad - R) // stride + 1, (Wd + 2 * pad - R) // stride + 1
+    dy = W.gen_dy(N, P, Q, K, seed + 2)
+    return x, w, dy, pad
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("shape", SMALL)
+def test_small_and_odd_shapes(shape, algo):
+    N, H, Wd, C, K, R, stride = shape
+    x, w, dy, pad = _case(*shape, seed=W.BASE_SEED + 11)
+    y32, dx32, dw, _ = Hh.run_conv_all(N, H, Wd, C, K, R, stride, pad, x, w, dy, algo=algo, out_f32=1)
+    y16, dx16, dw2, _ = Hh.run_conv_all(N, H, Wd, C, K, R, stride, pad, x, w, dy, algo=algo, out_f32=0)
+    yr = oracle.conv_fwd(x.numpy(), w.numpy(), stride, pad)
+    dxr = oracle.conv_dgrad(dy.numpy(), w.numpy(), H, Wd, stride, pad)
+    Hh.check_conv(y32, K, yr, what="fwd f32")
+    Hh.check_conv(dx32, C, dxr, what="dgrad f32")
+    Hh.check_conv(dw, C, oracle.conv_wgrad(x.numpy(), dy.numpy(), R, R, stride, pad), what="wgrad")
+    Hh.check_conv(y16, K, yr, what="fwd bf16")
+    Hh.check_conv(dx16, C, dxr, what="dgrad bf16")
+    # the bf16 output is the fp32 result rounded to nearest even, nothing else
+    assert torch.equal(y16[..., :K], y32[..., :K].to(torch.bfloat16))
+    assert torch.equal(dx16[..., :C], dx32[..., :C].to(torch.bfloat16))
+    assert torch.equal(dw, dw2)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_config1_single_layer_with_zero_groups(algo):
+    """Batch 8, 16->32 channels, 16x16, 3x3: zero input channels / zero upstream-gradient channels give
+    exactly-zero weight-gradient columns / rows (Eq. 4)."""
+    N, H, C, K, R = 8, 16, 16, 32, 3
+    seed = W.BASE_SEED + 1
+    g = np.random.default_rng(seed)
+    kz, cz = np.sort(g.permutation(K)[:5]), np.sort(g.permutation(C)[:3])
+    x, w, dy, pad = _case(N, H, H, C, K, R, 1, seed)
+    x[..., cz] = 0
+    dy[..., kz] = 0
+    w[kz] = 0
+    w[:, :, :, cz] = 0
+    y, dx, dw, _ = Hh.run_conv_all(N, H, H, C, K, R, 1, pad, x, w, dy, algo=algo)
+    Hh.check_conv(y, K, oracle.conv_fwd(x.numpy(), w.numpy(), 1, pad), what="fwd")
+    Hh.check_conv(dx, C, oracle.conv_dgrad(dy.numpy(), w.numpy(), H, H, 1, pad), what="dgrad")
+    Hh.check_conv(dw, C, oracle.conv_wgrad(x.numpy(), dy.numpy(), R, R, 1, pad), what="wgrad")
+    dwc = dw.cpu()
+    assert torch.all(dwc[kz] == 0) and torch.all(dwc[:, :, :, cz] == 0)
+    assert torch.all(y.float().cpu()[..., kz] == 0) and torch.all(dx.float().cpu()[..., cz] == 0)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_config3_pruned_bottleneck(algo):
+    """ResNet-50 stage-3 bottleneck at batch 64, 28x28, pruned to 371 -> 93 -> 77 -> 371: full-tensor parity."""
+    net = W.with_sizes(W.bottleneck_stage3(), [371, 93, 77])
+    for li, l in enumerate(net.layers):
+        seed = W.layer_seed(3, li)
+        x, w, dy, pad = _case(64, l.H, l.H, l.C, l.K, l.R, l.stride, seed)
+        y, dx, dw, _ = Hh.run_conv_all(64, l.H, l.H, l.C, l.K, l.R, l.stride, pad, x, w, dy, algo=algo)
+        Hh.check_conv(y, l.K, oracle.conv_fwd(x.numpy(), w.numpy(), l.stride, pad), what=l.name + " fwd")
+        Hh.check_conv(dx, l.C, oracle.conv_dgrad(dy.numpy(), w.numpy(), l.H, l.H, l.stride, pad), what=l.name + " dgrad")
+        Hh.check_conv(dw, l.C, oracle.conv_wgrad(x.numpy(), dy.numpy(), l.R, l.R, l.stride, pad), what=l.name + " wgrad")
+
+
+def test_wgrad_is_run_to_run_identical():
+    N, H, C, K, R = 4, 14, 27, 19, 3
+    x, w, dy, pad = _case(N, H, H, C, K, R, 1, W.BASE_SEED + 5)
+    a = Hh.run_conv_all(N, H, H, C, K, R, 1, pad, x, w, dy)[2].cpu()
+    b = Hh.run_conv_all(N, H, H, C, K, R, 1, pad, x, w, dy)[2].cpu()
+    assert torch.equal(a, b)
+
+
+def test_invalid_arguments_are_rejected_before_launch():
+    c = Hh.ctx()
+    buf = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
+    good = B.make_conv_desc(1, 4, 4, 8, 8, 3, 3, 1, 1)
+    for field, val in (("ldx", 9), ("ldy", 4), ("ldw", 12), ("C", 0), ("stride", 0), ("algo", 7)):
+        d = B.make_conv_desc(1, 4, 4, 8, 8, 3, 3, 1, 1)
+        setattr(d, field, val)
+        with pytest.raises(B.PtError) as e:
+            B.pt_conv_fwd(c, d, buf, buf, buf)
+        assert e.value.status == 1
+    with pytest.raises(B.PtError):
+        B.pt_conv_fwd(c, good, None, buf, buf)
+    d = B.make_conv_desc(2, 8, 8, 8, 8, 3, 3, 1, 1)
+    with pytest.raises(B.PtError) as e:       # wgrad needs a workspace
+        B.pt_conv_wgrad(c, d, buf, buf, torch.zeros(8 * 9 * 8, device="cuda"), None)
+    assert e.value.status == 3
+    c.poll()

@@ -1,0 +1,163 @@
+"""Parity of the group-lasso SGD step and zero-group detection with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_09290_b200 import binding as B
+from paper_1901_09290_b200 import workloads as W
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+
+class DevModel:
+    """Device copies of a workloads.Model plus the per-layer scratch the ABI wants."""
+
+    def __init__(self, model: W.Model, reg_in_first=False):
+        self.net = model.net
+        self.w = [t.clone().cuda() for t in model.w]
+        self.v = [t.clone().cuda() for t in model.v]
+        self.g = [t.clone().cuda() for t in model.g]
+        self.bn = [[b.clone().cuda() for b in bb] for bb in model.bn]
+        self.wb, self.sq_out, self.sq_in, self.z_out, self.z_in, self.layers = [], [], [], [], [], []
+        for li, l in enumerate(self.net.layers):
+            ldw = W.pad8(l.C)
+            wb = torch.full((l.K, l.R, l.R, ldw), float("nan"), dtype=torch.bfloat16, device="cuda")
+            wb[..., :l.C] = self.w[li].to(torch.bfloat16)
+            self.wb.append(wb)
+            self.sq_out.append(torch.full((l.K,), -1.0, device="cuda"))
+            self.sq_in.append(torch.full((l.C,), -1.0, device="cuda"))
+            self.z_out.append(torch.full((l.K,), 9, dtype=torch.uint8, device="cuda"))
+            self.z_in.append(torch.full((l.C,), 9, dtype=torch.uint8, device="cuda"))
+            reg_in = not self.net.space_fixed[l.in_space] or reg_in_first
+            self.layers.append(B.make_layer(self.w[li], self.g[li], self.v[li], wb, l.K, l.C, l.R * l.R, ldw,
+                                            reg_in, True, self.sq_out[li], self.sq_in[li], self.z_out[li], self.z_in[li]))
+        self.arr = B.layer_array(self.layers)
+        n = B.pt_group_lasso_workspace_bytes(Hh.ctx(), self.arr)
+        self.ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
+        self.reg = torch.zeros(1, dtype=torch.float64, device="cuda")
+
+    def graph(self):
+        links = [(l.in_space, l.out_space) for l in self.net.layers]
+        return B.GraphHandle(self.net.space_sizes, self.net.space_fixed, self.layers, links, self.bn)
+
+
+def _check_step(model: W.Model, lam, lr, mu, wd):
+    dm = DevModel(model)
+    B.pt_group_lasso_sgd_step(Hh.ctx(), dm.arr, lam, lr, mu, wd, dm.reg, dm.ws)
+    torch.cuda.synchronize()
+    Hh.ctx().poll()
+    reg_ref = 0.0
+    for li, l in enumerate(model.net.layers):
+        reg_in = not model.net.space_fixed[l.in_space]
+        w_new, v_new, s_out, s_in, reg = oracle.lasso_sgd(model.w[li].numpy(), model.g[li].numpy(), model.v[li].numpy(),
+                                                          lam, lr, mu, wd, reg_in=reg_in, reg_out=True)
+        reg_ref += reg
+        Hh.check_update(dm.w[li], w_new, f"{l.name} w")
+        Hh.check_update(dm.v[li], v_new, f"{l.name} v")
+        np.testing.assert_allclose(dm.sq_out[li].cpu().numpy(), s_out, rtol=2e-5, atol=1e-30)
+        np.testing.assert_allclose(dm.sq_in[li].cpu().numpy(), s_in, rtol=2e-5, atol=1e-30)
+        # the shadow is the round-to-nearest-even bf16 of the GPU's own new fp32 weights, bit for bit
+        assert torch.equal(dm.wb[li][..., :l.C], dm.w[li].to(torch.bfloat16)), l.name
+        assert torch.all(torch.isnan(dm.wb[li][..., l.C:].float())), "shadow pad lanes were written"
+        # zero groups stay exactly zero
+        zo = (model.w[li].abs().amax(dim=(1, 2, 3)) == 0) & (model.g[li].abs().amax(dim=(1, 2, 3)) == 0) & \
+             (model.v[li].abs().amax(dim=(1, 2, 3)) == 0)
+        if zo.any():
+            assert torch.all(dm.w[li][zo.cuda()] == 0) and torch.all(dm.v[li][zo.cuda()] == 0)
+    assert abs(dm.reg.item() - reg_ref) <= 1e-5 * reg_ref
+    return dm
+
+
+def test_step_single_layer_config1():
+    net = W.single_layer(16, 32, 3, 16)
+    kept = W.choose_kept(net, [13, 27], W.BASE_SEED + 1)
+    model = W.gen_model(net, W.BASE_SEED + 1, kept=kept)
+    _check_step(model, 1e-4, 0.1, 0.9, 0.0)
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (5, 3, 3), (33, 1, 70), (7, 3, 300), (64, 7, 3), (300, 1, 2500), (9, 3, 93)])
+def test_step_odd_shapes(shape):
+    K, R, C = shape
+    net = W.single_layer(C, K, R, 8)
+    model = W.gen_model(net, W.BASE_SEED + 50 + K)
+    _check_step(model, 3e-3, 0.05, 0.9, 1e-4)
+
+
+def test_step_resnet32_with_zero_groups_and_decoys():
+    net = W.resnet32()
+    kept = W.choose_kept(net, W.random_keep(net, W.BASE_SEED + 2), W.BASE_SEED + 2)
+    model = W.gen_model(net, W.BASE_SEED + 2, kept=kept, decoys=2)
+    _check_step(model, 1e-4, 0.1, 0.9, 0.0)
+
+
+def test_step_is_run_to_run_identical_and_table_cache_reuploads():
+    net = W.resnet32()
+    model = W.gen_model(net, W.BASE_SEED + 3)
+    a = _check_step(model, 1e-4, 0.1, 0.9, 0.0)
+    b = _check_step(model, 1e-4, 0.1, 0.9, 0.0)          # new buffers: the cached table must be refreshed
+    for x, y in zip(a.w, b.w):
+        assert torch.equal(x, y)
+
+
+def test_step_resnet50_all_layers():
+    net = W.resnet50()
+    model = W.gen_model(net, W.BASE_SEED + 4)
+    _check_step(model, 1e-4, 0.1, 0.9, 0.0)
+
+
+def _check_detection(model: W.Model, thr=1e-4, zero_in_place=False):
+    dm = DevModel(model)
+    B.pt_find_zero_groups(Hh.ctx(), dm.arr, thr, zero_in_place, dm.ws)
+    torch.cuda.synchronize()
+    Hh.ctx().poll()
+    for li, l in enumerate(model.net.layers):
+        zo, zi = oracle.find_zero_groups(model.w[li].numpy(), thr)
+        assert dm.z_out[li].cpu().numpy().tolist() == zo.tolist(), l.name
+        assert dm.z_in[li].cpu().numpy().tolist() == zi.tolist(), l.name
+        if zero_in_place:
+            w = model.w[li].clone()
+            w[torch.from_numpy(zo).bool()] = 0
+            w[:, :, :, torch.from_numpy(zi).bool()] = 0
+            assert torch.equal(dm.w[li].cpu().view(torch.int32), w.view(torch.int32))
+            assert torch.all(dm.v[li].cpu()[torch.from_numpy(zo).bool()] == 0)
+            assert torch.all(dm.wb[li][..., :l.C].float().cpu()[:, :, :, torch.from_numpy(zi).bool()] == 0)
+    return dm
+
+
+def test_detection_boundaries():
+    thr = np.float32(1e-4)
+    net = W.single_layer(5, 6, 2, 8)
+    model = W.gen_model(net, 1)
+    w = model.w[0]
+    w[:] = 1.0
+    w[0] = float(thr)
+    w[1] = float(np.nextafter(thr, np.float32(0)))
+    w[2] = 0.0
+    w[2, 0, 1, 3] = float("nan")
+    w[3] = 0.0
+    w[4] = -0.99e-4
+    w[5, 0, 0, :] = 0.0
+    w[5, 0, 1, 2] = -1e-3
+    w[:, :, :, 4] = 0.5e-4
+    dm = _check_detection(model, float(thr))
+    assert dm.z_out[0].cpu().tolist() == [0, 1, 0, 1, 1, 0] and dm.z_in[0].cpu().tolist() == [0, 0, 0, 0, 1]
+
+
+@pytest.mark.parametrize("zero_in_place", [False, True])
+def test_detection_resnet32(zero_in_place):
+    net = W.resnet32()
+    kept = W.choose_kept(net, W.random_keep(net, W.BASE_SEED + 2), W.BASE_SEED + 2)
+    model = W.gen_model(net, W.BASE_SEED + 2, kept=kept, decoys=2)
+    # near-threshold groups: scale some rows to just below / above 1e-4
+    model.w[3][1] *= 1e-6
+    model.w[5][:, :, :, 2] *= 1e-7
+    _check_detection(model, 1e-4, zero_in_place)
+
+
+def test_detection_config1_counts():
+    net = W.single_layer(16, 32, 3, 16)
+    kept = W.choose_kept(net, [13, 27], W.BASE_SEED + 1)
+    dm = _check_detection(W.gen_model(net, W.BASE_SEED + 1, kept=kept))
+    assert int(dm.z_out[0].sum()) == 5 and int(dm.z_in[0].sum()) == 3
