@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the PruneTrain hot path on B200.
+
+One step = one pass of the whole hot path on the pruned ResNet-50 workload (batch 64, 224x224, 53 conv layers,
+per-layer keep ratios drawn from a seed to give ~60 % of dense FLOPs):
+  zero-group detection + keep-set scan + channel-union compaction of the dense-shaped model  ->
+  conv fwd of every layer, conv dgrad + wgrad in reverse order                                ->
+  fused group-lasso momentum-SGD step over all conv weights.
+BN, ReLU, pooling, residual adds and the classifier are not on the path and not in the step.
+
+Prints ONE JSON line (rank 0). `--impl reference` times the CPU oracle instead (a deliberately plain program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "pruned ResNet-50 train-step conv TFLOP/s (useful FLOPs / whole step)"
+UNIT = "TFLOP/s"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons, pw = [], [], set(), []
+        for line in self.f.read().splitlines():
+            c = [t.strip() for t in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2])); pw.append(float(c[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                   "samples": len(sm), "power_w_max": max(pw)}
+        return out
+
+
+def workload(args):
+    from paper_1901_09290_b200 import workloads as W
+    net = W.resnet50()
+    seed = W.BASE_SEED + 4
+    if args.keep is not None:
+        counts = W.uniform_keep(net, args.keep)
+        name = f"resnet50-uniform-keep-{args.keep:g}"
+    else:
+        counts = W.staged_keep_to_flops(net, seed, 0.60)
+        name = "resnet50-224-53conv-keep-drawn-to-0.60-flops"
+    kept = W.choose_kept(net, counts, seed)
+    return net, counts, kept, seed, name
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+def oracle_step_sample(net_p, N_s, layer_ids, seed):
+    """One bounded sample of the step on the host cores with the oracle as it stands: fwd + dgrad + wgrad of the
+    given layers at batch N_s, and the lasso step, detection of those layers. Returns (seconds, useful conv FLOPs)."""
+    import numpy as np
+    import oracle
+    from paper_1901_09290_b200 import workloads as W
+    flops = 0
+    data = []
+    for li in layer_ids:
+        l = net_p.layers[li]
+        x = (W.gen_image if li == 0 else W.gen_act)(N_s, l.H, l.H, l.C, seed + li).numpy()
+        w = W.bf16_round(W.gen_weight(l.K, l.R, l.R, l.C, seed + 1000 + li)).numpy()
+        dy = W.gen_dy(N_s, l.P, l.P, l.K, seed + 2000 + li).numpy()
+        v = W.gen_small(w.shape, seed + 3000 + li).numpy()
+        data.append((l, li, x, w, dy, v))
+    t0 = time.perf_counter()
+    for l, li, x, w, dy, v in data:
+        oracle.conv_fwd(x, w, l.stride, l.pad)
+        fl = 2 * N_s * l.P * l.P * l.K * l.C * l.R * l.R
+        flops += 2 * fl
+        if li > 0:
+            oracle.conv_dgrad(dy, w, l.H, l.H, l.stride, l.pad)
+            flops += fl
+        dw = oracle.conv_wgrad(x, dy, l.R, l.R, l.stride, l.pad)
+        oracle.lasso_sgd(w, dw.astype(np.float32), v, 1e-4, 0.1, 0.9, reg_in=(li > 0))
+        oracle.find_zero_groups(w)
+    return time.perf_counter() - t0, flops
+
+
+def pick_sample(net_p, budget_s, seed):
+    """Chooses every s-th layer at batch 1 so that one sample costs about budget_s seconds on this host."""
+    ids = list(range(len(net_p.layers)))
+    t, f = oracle_step_sample(net_p, 1, [5], seed)          # calibration on one mid-size layer
+    rate = f / max(t, 1e-6)
+    full = sum(2 * l.P * l.P * l.K * l.C * l.R * l.R * (3 if i > 0 else 2) for i, l in enumerate(net_p.layers))
+    stride = 1
+    while full / stride / rate > budget_s and stride < len(ids):
+        stride += 1
+    return ids[::stride], stride
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, same metric and config, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_1901_09290_b200 import workloads as W
+    net, counts, kept, seed, name = workload(args)
+    net_p = W.with_sizes(net, counts)
+    per_step_budget = max(0.5, min(8.0, 150.0 / (args.steps + args.warmup)))
+    ids, stride = pick_sample(net_p, per_step_budget, seed)
+    for _ in range(args.warmup):
+        oracle_step_sample(net_p, 1, ids, seed)
+    T, F = 0.0, 0
+    for _ in range(args.steps):
+        t, f = oracle_step_sample(net_p, 1, ids, seed)
+        T += t
+        F += f
+    val = F / T / 1e12
+    sample = f"batch 1 of {args.batch}, every {stride}-th of the 53 layers ({len(ids)} layers): fwd+dgrad+wgrad+lasso+detection"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": T / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": name, "batch": args.batch, "image": 224, "kept_params": sum(l.K * l.C * l.R * l.R for l in net_p.layers)},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------ GPU leg
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1901_09290_b200 import binding as B
+    from paper_1901_09290_b200 import harness
+    from paper_1901_09290_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    pk = peaks()
+    ctx = B.Context(local)
+    net, counts, kept, seed, name = workload(args)
+    ts = harness.TrainStep(ctx, net, counts, kept, args.batch, seed + 17 * rank, algo=args.algo, host_inputs=True)
+    flops = ts.conv_flops()
+    tot_flops = sum(flops.values())
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(max(args.warmup, 3)):
+        ts.step()
+    barrier()
+    ctx.poll()
+    l0 = ctx.launch_count()
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms = timed(ts.step, args.steps)
+    launches = (ctx.launch_count() - l0)
+    # end-to-end: image batch from pinned host memory, regulariser value and new sizes read back, every step
+    for _ in range(2):
+        ts.step_e2e()
+    ms_e2e = timed(ts.step_e2e, args.steps)
+    clocks = sampler.stop() if sampler else None
+    ctx.poll()
+
+    # per-phase and per-layer device times (CUDA events around each ABI call, same stream), for the roofline
+    nL = len(ts.net.layers)
+    reps = max(2, min(5, args.steps))
+    acc = {"fwd": [0.0] * nL, "dgrad": [0.0] * nL, "wgrad": [0.0] * nL}
+    phase = {"reconfigure": 0.0, "lasso": 0.0, "lasso_dense_model": 0.0}
+
+    def ev_time(fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn()
+        b.record(stream)
+        return a, b
+
+    for _ in range(reps):
+        pend = []
+        pend.append(("reconfigure", None, ev_time(ts.reconfigure)))
+        for li in range(nL):
+            pend.append(("fwd", li, ev_time(lambda: ts.conv_fwd(li))))
+        for li in range(nL - 1, -1, -1):
+            if li > 0:
+                pend.append(("dgrad", li, ev_time(lambda: ts.conv_dgrad(li))))
+            pend.append(("wgrad", li, ev_time(lambda: ts.conv_wgrad(li))))
+        pend.append(("lasso", None, ev_time(ts.lasso)))
+        torch.cuda.synchronize()
+        for kind, li, (a, b) in pend:
+            t = a.elapsed_time(b) / reps
+            if li is None:
+                phase[kind] += t
+            else:
+                acc[kind][li] += t
+    # the lasso step on the dense-shaped model (23.45 M parameters), timed alone
+    md = ts.md
+    g_saved = [w.clone() for w in md.w]
+    v_saved = [v.clone() for v in md.v]
+    for _ in range(reps):
+        a, b = ev_time(lambda: B.pt_group_lasso_sgd_step(ctx, md.arr, 1e-4, 0.0, 0.9, 0.0, md.reg, md.ws))
+        torch.cuda.synchronize()
+        phase["lasso_dense_model"] += a.elapsed_time(b) / reps
+    for w, s in zip(md.v, v_saved):
+        w.copy_(s)
+    ctx.poll()
+
+    which_id = {"fwd": 0, "dgrad": 1, "wgrad": 2}
+    per_layer = []
+    t_roof_sum, t_meas_sum = 0.0, 0.0
+    tc_peak = pk["bf16_tflops_sustained"] * 1e12
+    bw_peak = pk["hbm_gbs"] * 1e9
+    for kind in ("fwd", "dgrad", "wgrad"):
+        for li, l in enumerate(ts.net.layers):
+            if kind == "dgrad" and li == 0:
+                continue
+            fl = 2 * args.batch * l.P * l.P * l.K * l.C * l.R * l.R
+            by = ts.layer_bytes(li, which_id[kind])
+            t = acc[kind][li] * 1e-3
+            roof = max(fl / tc_peak, by / bw_peak)
+            t_roof_sum += roof
+            t_meas_sum += t
+            per_layer.append({"layer": l.name, "pass": kind, "C": l.C, "K": l.K, "R": l.R, "stride": l.stride, "H": l.H,
+                              "us": t * 1e6, "tflops": fl / t / 1e12, "gbs": by / t / 1e9,
+                              "bound": "tensor" if fl / tc_peak > by / bw_peak else "hbm", "roofline_frac": roof / t})
+    conv_ms = {k: sum(v) for k, v in acc.items()}
+    conv_total_ms = sum(conv_ms.values())
+    dom = max(conv_ms, key=conv_ms.get)
+    dom_flops = flops[dom]
+    dom_t = conv_ms[dom] * 1e-3
+    n_dom = nL - (1 if dom == "dgrad" else 0)
+    value = world * tot_flops / (ms / args.steps * 1e-3) / 1e12
+    e2e_val = world * tot_flops / (ms_e2e / args.steps * 1e-3) / 1e12
+    h2d, d2h = ts.e2e_bytes()
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 operands, f32 accumulate (convs); f32 (lasso/SGD); u8/i32 (detection, compaction)",
+        "data": "synthetic",
+        "config": {"workload": name, "batch_per_gpu": args.batch, "image": 224, "conv_layers": nL,
+                   "kept_params": ts.mp.n_params(), "dense_params": ts.md.n_params(),
+                   "useful_conv_flops_per_step": tot_flops, "l2": "inputs larger than L2 (per-layer activations 20-400 MB, ~6 GB per step)",
+                   "parallelism": "independent data-parallel replicas, no collective" if world > 1 else "1 GPU",
+                   "algo": args.algo},
+        "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "phases_ms": {"conv_fwd": conv_ms["fwd"], "conv_dgrad": conv_ms["dgrad"], "conv_wgrad": conv_ms["wgrad"],
+                      "lasso_sgd_pruned": phase["lasso"], "detect_plan_compact": phase["reconfigure"],
+                      "lasso_sgd_dense_model": phase["lasso_dense_model"]},
+        "conv_tflops": tot_flops / (conv_total_ms * 1e-3) / 1e12,
+        "conv_pct_of_bf16_peak": {"measured_sustained": 100 * tot_flops / (conv_total_ms * 1e-3) / tc_peak,
+                                  "nominal_2250": 100 * tot_flops / (conv_total_ms * 1e-3) / 2.25e15},
+        "conv_mixed_roofline_frac": t_roof_sum / t_meas_sum,
+        "lasso_gbs": {"pruned_model": ts.lasso_bytes(ts.mp) / (phase["lasso"] * 1e-3) / 1e9,
+                      "dense_model": ts.lasso_bytes(ts.md) / (phase["lasso_dense_model"] * 1e-3) / 1e9,
+                      "bytes_per_param": 26, "peak": pk["hbm_gbs"], "peak_source": pk["source"]},
+        "reconf_gbs": ts.reconf_bytes() / (phase["reconfigure"] * 1e-3) / 1e9,
+        "roofline": {"kernel": f"conv_{dom} (all {n_dom} launches of a step)", "bound": "tensor",
+                     "achieved": dom_flops / dom_t / 1e12, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": dom_flops / dom_t / tc_peak, "traffic": None, "peak_source": pk["source"] + " sustained bf16"},
+    }
+    if rank == 0:
+        if args.per_layer:
+            os.makedirs(os.path.dirname(os.path.abspath(args.per_layer)), exist_ok=True)
+            json.dump(per_layer, open(args.per_layer, "w"), indent=0)
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            net_p = ts.net
+            ids, stride = pick_sample(net_p, 15.0, seed)
+            t, f = oracle_step_sample(net_p, 1, ids, seed)
+            out["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                   "sample": f"batch 1 of {args.batch}, every {stride}-th of the 53 layers ({len(ids)} layers): "
+                                             f"fwd+dgrad+wgrad+lasso+detection, {t:.1f} s"}
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--keep", type=float, default=None, help="uniform keep ratio instead of the seeded per-space draw")
+    ap.add_argument("--algo", type=int, default=0)
+    ap.add_argument("--per-layer", default=None, help="write the per-layer table (JSON) here")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,192 @@
+"""Device-side staging around the C ABI: argument marshalling for whole models and whole steps.
+
+Nothing here computes anything of the method: it allocates torch CUDA tensors as device memory,
+fills the ABI structs and issues the ``pt_*`` calls in the order of Algorithm 1.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+
+class DeviceModel:
+    """Device copies of a workloads.Model (fp32 w, v, g, BN vectors), the bf16 shadow and the per-layer
+    scratch the ABI wants (group sums of squares, zero masks), plus the pt_layer array."""
+
+    def __init__(self, ctx: B.Context, model: W.Model, shadow_fill: float = float("nan")):
+        self.ctx = ctx
+        self.net = model.net
+        self.w = [t.clone().cuda() for t in model.w]
+        self.v = [t.clone().cuda() for t in model.v]
+        self.g = [t.clone().cuda() for t in model.g]
+        self.bn = [[b.clone().cuda() for b in bb] for bb in model.bn]
+        self.wb, self.sq_out, self.sq_in, self.z_out, self.z_in, self.layers = [], [], [], [], [], []
+        for li, l in enumerate(self.net.layers):
+            ldw = W.pad8(l.C)
+            wb = torch.full((l.K, l.R, l.R, ldw), shadow_fill, dtype=torch.bfloat16, device="cuda")
+            wb[..., :l.C] = self.w[li].to(torch.bfloat16)       # data conversion of the initial weights
+            self.wb.append(wb)
+            self.sq_out.append(torch.full((l.K,), -1.0, device="cuda"))
+            self.sq_in.append(torch.full((l.C,), -1.0, device="cuda"))
+            self.z_out.append(torch.full((l.K,), 9, dtype=torch.uint8, device="cuda"))
+            self.z_in.append(torch.full((l.C,), 9, dtype=torch.uint8, device="cuda"))
+            reg_in = self.net.space_stage[l.in_space] != 0     # only the image's channels are exempt (stage 0)
+            self.layers.append(B.make_layer(self.w[li], self.g[li], self.v[li], wb, l.K, l.C, l.R * l.R, ldw,
+                                            reg_in, True, self.sq_out[li], self.sq_in[li], self.z_out[li], self.z_in[li]))
+        self.arr = B.layer_array(self.layers)
+        n = B.pt_group_lasso_workspace_bytes(ctx, self.arr)
+        self.ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
+        self.reg = torch.zeros(1, dtype=torch.float64, device="cuda")
+        self._graph = None
+
+    def reg_in(self, li: int) -> bool:
+        return bool(self.layers[li].reg_in)
+
+    def graph(self) -> B.GraphHandle:
+        if self._graph is None:
+            links = [(l.in_space, l.out_space) for l in self.net.layers]
+            self._graph = B.GraphHandle(self.net.space_sizes, self.net.space_fixed, self.layers, links, self.bn)
+        return self._graph
+
+    def n_params(self) -> int:
+        return sum(l.K * l.C * l.R * l.R for l in self.net.layers)
+
+
+def empty_model(net: W.Net, fill: float = 0.0) -> W.Model:
+    mk = lambda l: torch.full((l.K, l.R, l.R, l.C), fill)
+    return W.Model(net, [mk(l) for l in net.layers], [mk(l) for l in net.layers],
+                   [torch.zeros((l.K, l.R, l.R, l.C)) for l in net.layers],
+                   [[torch.full((l.K,), fill) for _ in range(4)] for l in net.layers])
+
+
+class TrainStep:
+    """The hot path on one GPU for one network: reconfiguration of a dense-shaped model with embedded zero
+    groups into the pruned model, then the pruned model's conv training step (every layer's forward, then data and
+    weight gradients in reverse order, each on its own activation buffers) and the group-lasso SGD step.
+
+    The layers are not chained through BN/ReLU/pooling (those are not on the path): every layer has its own
+    seeded input x_l and upstream gradient dy_l, as in a training step's memory footprint.
+    """
+
+    def __init__(self, ctx: B.Context, dense_net: W.Net, counts: Sequence[int], kept, N: int, seed: int,
+                 algo: int = 0, host_inputs: bool = False, decoys: int = 2, device_rng: bool = True):
+        self.ctx, self.N, self.algo = ctx, N, algo
+        self.dense_net = dense_net
+        self.net = W.with_sizes(dense_net, counts)
+        self.counts = list(counts)
+        model_d = W.gen_model(dense_net, seed, kept=kept, decoys=decoys)
+        self.md = DeviceModel(ctx, model_d)
+        self.mp = DeviceModel(ctx, empty_model(self.net))
+        self.new2old = torch.full((sum(dense_net.space_sizes),), -1, dtype=torch.int32, device="cuda")
+        self.x, self.dy, self.y, self.dx, self.desc = [], [], [], [], []
+        gen = torch.Generator(device="cuda").manual_seed(seed + 99) if device_rng else None
+        ws_bytes = 16
+        for li, l in enumerate(self.net.layers):
+            ldx, ldy = W.pad8(l.C), W.pad8(l.K)
+            P = l.P
+            d = B.make_conv_desc(N, l.H, l.H, l.C, l.K, l.R, l.R, l.stride, l.pad, ldx, ldy, W.pad8(l.C), 0, algo)
+            self.desc.append(d)
+            if device_rng:
+                if li == 0:
+                    x = torch.randn((N, l.H, l.H, ldx), generator=gen, device="cuda", dtype=torch.float32)
+                else:
+                    x = torch.randn((N, l.H, l.H, ldx), generator=gen, device="cuda", dtype=torch.float32).clamp_(min=0)
+                dy = torch.randn((N, P, P, ldy), generator=gen, device="cuda", dtype=torch.float32) * (2.0 ** -6)
+                self.x.append(x.to(torch.bfloat16))
+                self.dy.append(dy.to(torch.bfloat16))
+                del x, dy
+            else:
+                sx, sd = W.layer_seed(4, li, 1), W.layer_seed(4, li, 2)
+                xh = W.gen_image(N, l.H, l.H, l.C, sx) if li == 0 else W.gen_act(N, l.H, l.H, l.C, sx)
+                dh = W.gen_dy(N, P, P, l.K, sd)
+                xd = torch.zeros((N, l.H, l.H, ldx), dtype=torch.bfloat16, device="cuda")
+                xd[..., :l.C] = xh.to(torch.bfloat16)
+                dd = torch.zeros((N, P, P, ldy), dtype=torch.bfloat16, device="cuda")
+                dd[..., :l.K] = dh.to(torch.bfloat16)
+                self.x.append(xd)
+                self.dy.append(dd)
+            self.y.append(torch.empty((N, P, P, ldy), dtype=torch.bfloat16, device="cuda"))
+            self.dx.append(torch.empty((N, l.H, l.H, ldx), dtype=torch.bfloat16, device="cuda") if li > 0 else None)
+            for which in range(3):
+                ws_bytes = max(ws_bytes, B.pt_conv_workspace_bytes(ctx, d, which))
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        # e2e: the image batch arrives from pinned host memory every step
+        l0 = self.net.layers[0]
+        self.h_image = None
+        if host_inputs:
+            self.h_image = self.x[0].cpu().pin_memory()
+        self.h_reg = torch.zeros(1, dtype=torch.float64).pin_memory()
+
+    # ---- sizes used for reporting
+    def conv_flops(self) -> Dict[str, int]:
+        f = {"fwd": 0, "dgrad": 0, "wgrad": 0}
+        for li, l in enumerate(self.net.layers):
+            fl = 2 * self.N * l.P * l.P * l.K * l.C * l.R * l.R
+            f["fwd"] += fl
+            f["wgrad"] += fl
+            if li > 0:
+                f["dgrad"] += fl
+        return f
+
+    def layer_bytes(self, li: int, which: int) -> int:
+        """Algorithmic bytes of one conv pass: each tensor touched once (bf16 activations and weights, fp32 dw)."""
+        l = self.net.layers[li]
+        a = self.N * l.H * l.H * l.C * 2 + self.N * l.P * l.P * l.K * 2
+        return a + l.K * l.C * l.R * l.R * (4 if which == 2 else 2)
+
+    def lasso_bytes(self, model: DeviceModel) -> int:
+        return 26 * model.n_params()
+
+    def reconf_bytes(self) -> int:
+        """Detection reads the old weights once (4 B/param); the gather reads w, v (8 B) and writes w, v, shadow
+        (10 B) per kept parameter."""
+        return 4 * self.md.n_params() + 18 * self.mp.n_params()
+
+    # ---- the path
+    def reconfigure(self, stream=None):
+        c = self.ctx
+        B.pt_find_zero_groups(c, self.md.arr, 1e-4, False, self.md.ws, stream)
+        sizes = B.pt_reconfigure_plan(c, self.md.graph(), self.new2old, stream)
+        if sizes != self.counts:
+            raise RuntimeError(f"reconfiguration plan returned {sizes}, expected {self.counts}")
+        B.pt_reconfigure(c, self.md.graph(), self.new2old, self.mp.graph(), stream)
+
+    def conv_fwd(self, li, stream=None):
+        B.pt_conv_fwd(self.ctx, self.desc[li], self.x[li], self.mp.wb[li], self.y[li], self.ws, stream)
+
+    def conv_dgrad(self, li, stream=None):
+        B.pt_conv_dgrad(self.ctx, self.desc[li], self.dy[li], self.mp.wb[li], self.dx[li], self.ws, stream)
+
+    def conv_wgrad(self, li, stream=None):
+        B.pt_conv_wgrad(self.ctx, self.desc[li], self.x[li], self.dy[li], self.mp.g[li], self.ws, stream)
+
+    def lasso(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
+        B.pt_group_lasso_sgd_step(self.ctx, self.mp.arr, lam, lr, mu, 0.0, self.mp.reg, self.mp.ws, stream)
+
+    def train(self, stream=None):
+        n = len(self.net.layers)
+        for li in range(n):
+            self.conv_fwd(li, stream)
+        for li in range(n - 1, -1, -1):
+            if li > 0:
+                self.conv_dgrad(li, stream)
+            self.conv_wgrad(li, stream)
+        self.lasso(stream)
+
+    def step(self, stream=None):
+        self.reconfigure(stream)
+        self.train(stream)
+
+    def step_e2e(self, stream=None):
+        """The same step with the image batch copied from pinned host memory and the regulariser value read back."""
+        self.x[0].copy_(self.h_image, non_blocking=True)
+        self.step(stream)
+        self.h_reg.copy_(self.mp.reg, non_blocking=True)
+
+    def e2e_bytes(self):
+        return self.h_image.numel() * self.h_image.element_size(), 8 + 4 * len(self.counts)

@@ -11,36 +11,11 @@ from tests import helpers as Hh
 pytestmark = pytest.mark.gpu
 
 
-class DevModel:
-    """Device copies of a workloads.Model plus the per-layer scratch the ABI wants."""
+from paper_1901_09290_b200.harness import DeviceModel
 
-    def __init__(self, model: W.Model, reg_in_first=False):
-        self.net = model.net
-        self.w = [t.clone().cuda() for t in model.w]
-        self.v = [t.clone().cuda() for t in model.v]
-        self.g = [t.clone().cuda() for t in model.g]
-        self.bn = [[b.clone().cuda() for b in bb] for bb in model.bn]
-        self.wb, self.sq_out, self.sq_in, self.z_out, self.z_in, self.layers = [], [], [], [], [], []
-        for li, l in enumerate(self.net.layers):
-            ldw = W.pad8(l.C)
-            wb = torch.full((l.K, l.R, l.R, ldw), float("nan"), dtype=torch.bfloat16, device="cuda")
-            wb[..., :l.C] = self.w[li].to(torch.bfloat16)
-            self.wb.append(wb)
-            self.sq_out.append(torch.full((l.K,), -1.0, device="cuda"))
-            self.sq_in.append(torch.full((l.C,), -1.0, device="cuda"))
-            self.z_out.append(torch.full((l.K,), 9, dtype=torch.uint8, device="cuda"))
-            self.z_in.append(torch.full((l.C,), 9, dtype=torch.uint8, device="cuda"))
-            reg_in = not self.net.space_fixed[l.in_space] or reg_in_first
-            self.layers.append(B.make_layer(self.w[li], self.g[li], self.v[li], wb, l.K, l.C, l.R * l.R, ldw,
-                                            reg_in, True, self.sq_out[li], self.sq_in[li], self.z_out[li], self.z_in[li]))
-        self.arr = B.layer_array(self.layers)
-        n = B.pt_group_lasso_workspace_bytes(Hh.ctx(), self.arr)
-        self.ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
-        self.reg = torch.zeros(1, dtype=torch.float64, device="cuda")
 
-    def graph(self):
-        links = [(l.in_space, l.out_space) for l in self.net.layers]
-        return B.GraphHandle(self.net.space_sizes, self.net.space_fixed, self.layers, links, self.bn)
+def DevModel(model):
+    return DeviceModel(Hh.ctx(), model)
 
 
 def _check_step(model: W.Model, lam, lr, mu, wd):
@@ -50,7 +25,7 @@ def _check_step(model: W.Model, lam, lr, mu, wd):
     Hh.ctx().poll()
     reg_ref = 0.0
     for li, l in enumerate(model.net.layers):
-        reg_in = not model.net.space_fixed[l.in_space]
+        reg_in = model.net.space_stage[l.in_space] != 0
         w_new, v_new, s_out, s_in, reg = oracle.lasso_sgd(model.w[li].numpy(), model.g[li].numpy(), model.v[li].numpy(),
                                                           lam, lr, mu, wd, reg_in=reg_in, reg_out=True)
         reg_ref += reg
