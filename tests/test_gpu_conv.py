@@ -109,3 +109,21 @@ def test_invalid_arguments_are_rejected_before_launch():
         B.pt_conv_wgrad(c, d, buf, buf, torch.zeros(8 * 9 * 8, device="cuda"), None)
     assert e.value.status == 3
     c.poll()
+
+
+def test_tcgen05_path_takes_fwd_and_dgrad_when_forced():
+    """algo = 2 forces the tcgen05 kernels: the call must not fall back silently."""
+    N, H, C, K, R = 2, 12, 40, 24, 3
+    x, w, dy, pad = _case(N, H, H, C, K, R, 1, W.BASE_SEED + 9)
+    d = B.make_conv_desc(N, H, H, C, K, R, R, 1, pad, algo=2, out_f32=1)
+    xd, wd, dyd = Hh.to_dev_padded(x, d.ldx), Hh.to_dev_padded(w, d.ldw), Hh.to_dev_padded(dy, d.ldy)
+    y = Hh.out_buffer((N, H, H), K, d.ldy, True)
+    dx = Hh.out_buffer((N, H, H), C, d.ldx, True)
+    n0 = Hh.ctx().launch_count()
+    B.pt_conv_fwd(Hh.ctx(), d, xd, wd, y, Hh.conv_ws(d, 0))
+    B.pt_conv_dgrad(Hh.ctx(), d, dyd, wd, dx, Hh.conv_ws(d, 1))
+    torch.cuda.synchronize()
+    Hh.ctx().poll()
+    assert Hh.ctx().launch_count() - n0 == 2
+    Hh.check_conv(y, K, oracle.conv_fwd(x.numpy(), w.numpy(), 1, pad), what="fwd tcgen05")
+    Hh.check_conv(dx, C, oracle.conv_dgrad(dy.numpy(), w.numpy(), H, H, 1, pad), what="dgrad tcgen05")
