@@ -149,7 +149,8 @@ static pt_status conv_dispatch(pt_ctx *c, const pt_conv_desc *d, int which, cons
     if (d->algo == 2 && !fast) return PT_ERR_UNSUPPORTED;
     if (fast) {
         if (pt_sm100_conv_workspace(c, d, which) > ws_bytes || (pt_sm100_conv_workspace(c, d, which) && !ws)) return PT_ERR_WORKSPACE;
-        return pt_sm100_conv(c, d, which, a, b, out, ws, ws_bytes, st);
+        pt_status r = pt_sm100_conv(c, d, which, a, b, out, ws, ws_bytes, st);
+        if (r != PT_ERR_UNSUPPORTED || d->algo == 2) return r;     // a shape the tcgen05 path declines goes to the SIMT kernels
     }
     if (pt_simt_conv_workspace(c, d, which) > ws_bytes || (pt_simt_conv_workspace(c, d, which) && !ws)) return PT_ERR_WORKSPACE;
     return pt_simt_conv(c, d, which, a, b, out, ws, ws_bytes, st);

@@ -24,6 +24,7 @@ constexpr int kBM = 128;            // output pixels per CTA tile
 constexpr int kKC = 64;             // reduction channels per stage (one 128-byte swizzle row)
 constexpr int kMaxStages = 8;
 constexpr int kThreads = 192;
+constexpr int kMaxTaps = 64;
 
 struct GemmP {
     int M_total;        // output pixels of this launch's raster
@@ -32,11 +33,10 @@ struct GemmP {
     int n_tiles;        // tiles along the channel dimension
     int c_red;          // true number of reduction channels
     int k_chunks;       // ceil(c_red / 64)
-    int taps, S;        // R*S and S
+    int taps;           // filter taps visited by this launch (<= kMaxTaps)
     int Pd, Qd;         // raster of output pixels (rows, columns) per image
     int stride;         // traversal stride of the raster in the source tensor
     int lo_h, lo_w;     // source coordinate of raster position (0,0) for tap (0,0)
-    int flip;           // dgrad: weight tap = taps-1-tap
     int stages;
     int tmem_cols;
     // output pixel mapping: pixel (n, i, j) of the raster -> out[((n*oH + i*o_step + o_h0)*oW + j*o_step + o_w0)*ld_out]
@@ -45,6 +45,8 @@ struct GemmP {
     int zero_mask;      // stride-2 dgrad: bit (a*2+b) set => also write zeros to the pixel at parity (a,b) of each 2x2 cell
     void *out;
     unsigned int *status;
+    unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
+    unsigned short tap_wt[kMaxTaps];                    // index r*S+s of the weights the tap multiplies
 };
 
 struct __align__(8) Ctl {
@@ -104,12 +106,11 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
                 const int s = it % p.stages, ph = (it / p.stages) & 1;
                 if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 1)) break;
                 const int tap = it / p.k_chunks, kc = it - tap * p.k_chunks;
-                const int r = tap / p.S, sft = tap - r * p.S;
                 const uint32_t bar = smem_u32(&ctl->full[s]);
                 const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
                 mbar_arrive_expect_tx(bar, a_bytes + b_bytes);
-                tma_load_im2col_4d(a_dst, &tmA, bar, kc * kKC, w0, h0, n, (uint16_t)sft, (uint16_t)r);
-                const int wtap = p.flip ? p.taps - 1 - tap : tap;
+                tma_load_im2col_4d(a_dst, &tmA, bar, kc * kKC, w0, h0, n, (uint16_t)p.tap_ow[tap], (uint16_t)p.tap_oh[tap]);
+                const int wtap = p.tap_wt[tap];
                 if (!B_MN) {
                     tma_load_3d(b_dst, &tmB, bar, kc * kKC, wtap, n0);
                 } else {
@@ -236,6 +237,163 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
     }
 }
 
+// ------------------------------------------------------------------------------------------ wgrad
+// dw[k][tap][c] = sum over output pixels of dy[pixel][k] * x[pixel shifted by the tap][c]   (Eq. 4)
+//   GEMM per tap: M = 128 output channels k, N = BN input channels c, reduction = output pixels, 64 per stage.
+//   A operand: dy[pixel][k], k contiguous -> MN-major tiles (two 64-channel boxes of a 2-D tiled map).
+//   B operand: x through the im2col map (same pixel raster as the forward pass, tap offset added by the TMA unit),
+//              c contiguous -> MN-major tiles (one 64-channel box per 64 columns).
+//   The pixel range is split across CTAs (blockIdx.z); with more than one split every CTA writes its fp32 partial
+//   tile to the workspace and wgrad_reduce_kernel sums the splits in ascending order (deterministic).
+struct WgradP {
+    int K, C, taps;         // true channel counts, number of taps (R*S)
+    int BN, n_tiles;        // input-channel tile
+    int m_tiles;            // ceil(K / 128)
+    int npix;               // N*P*Q
+    int pix_per_split;      // multiple of 64
+    int splits;
+    int Pd, Qd, stride, lo_h, lo_w, S;
+    int stages, tmem_cols;
+    float *out;             // dw (splits == 1) or the partial workspace [split][K*taps*C]
+    unsigned int *status;
+};
+
+__global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy,
+                                                              const __grid_constant__ CUtensorMap tmX, const WgradP p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw);
+    const uint32_t smem_base = smem_u32(smem_raw);
+    const uint32_t data_base = (smem_base + (uint32_t)sizeof(Ctl) + 1023u) & ~1023u;
+    const uint32_t a_bytes = 2u * 8192u;
+    const uint32_t nb_b = (uint32_t)((p.BN + 63) / 64);
+    const uint32_t b_bytes = nb_b * 8192u;
+    const uint32_t stage_bytes = a_bytes + b_bytes;
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int bx = blockIdx.x;
+    const int n_tile = bx % p.n_tiles; bx /= p.n_tiles;
+    const int m_tile = bx % p.m_tiles; bx /= p.m_tiles;
+    const int tap = bx;
+    const int split = blockIdx.y;
+    const int k0 = m_tile * 128, c0 = n_tile * p.BN;
+    const int pix_beg = split * p.pix_per_split;
+    const int pix_end = min(p.npix, pix_beg + p.pix_per_split);
+    const int iters = pix_end > pix_beg ? (pix_end - pix_beg + 63) / 64 : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&ctl->accum), 1);
+        ctl->abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tmDy);
+        prefetch_tmap(&tmX);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const int r = tap / p.S, sft = tap - r * p.S;
+            int issued = 0;
+            for (int it = 0; it < iters; ++it) {
+                const int s = it % p.stages, ph = (it / p.stages) & 1;
+                if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 4)) break;
+                const int pix = pix_beg + it * 64;
+                const int q = pix % p.Qd, t = pix / p.Qd, pp = t % p.Pd, n = t / p.Pd;
+                const uint32_t bar = smem_u32(&ctl->full[s]);
+                const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
+                mbar_arrive_expect_tx(bar, a_bytes + b_bytes);
+                tma_load_2d(a_dst, &tmDy, bar, k0, pix);
+                tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
+                for (uint32_t nb = 0; nb < nb_b; ++nb)
+                    tma_load_im2col_4d(b_dst + nb * 8192u, &tmX, bar, c0 + (int)nb * 64, q * p.stride + p.lo_w,
+                                       pp * p.stride + p.lo_h, n, (uint16_t)sft, (uint16_t)r);
+                issued = it + 1;
+            }
+            if (*abort_flag) {
+                for (int it = max(0, issued - p.stages); it < issued; ++it) {
+                    const int s = it % p.stages, ph = (it / p.stages) & 1;
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!mbar_try_wait(smem_u32(&ctl->full[s]), ph) && globaltimer_ns() - t0 < 20000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(128, p.BN, 1, 1);
+            bool ok = true;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % p.stages, ph = (it / p.stages) & 1;
+                ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 5);
+                if (!ok) break;
+                tc_fence_after();
+                const int rem = pix_end - (pix_beg + it * 64);
+                const int ksteps = rem >= 64 ? 4 : (rem + 15) / 16;
+                const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
+#pragma unroll 1
+                for (int k = 0; k < ksteps; ++k) {
+                    const uint64_t ad = make_desc(a_src + (uint32_t)k * 2048u, 8192u, 1024u);
+                    const uint64_t bd = make_desc(b_src + (uint32_t)k * 2048u, 8192u, 1024u);
+                    umma_bf16(tmem_base, ad, bd, idesc, (it | k) != 0 ? 1u : 0u);
+                }
+                umma_commit(smem_u32(&ctl->empty[s]));
+            }
+            if (ok) umma_commit(smem_u32(&ctl->accum));
+        }
+    } else {
+        const int quarter = warp & 3;
+        bool ok = true;
+        if (iters > 0) ok = mbar_wait(smem_u32(&ctl->accum), 0, abort_flag, p.status, 6);
+        tc_fence_after();
+        if (ok) {
+            const int k = k0 + quarter * 32 + lane;
+            const bool row_ok = k < p.K;
+            float *orow = p.out + (size_t)split * p.K * p.taps * p.C + ((size_t)k * p.taps + tap) * p.C;
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            for (int cc = 0; cc < p.BN; cc += 16) {
+                uint32_t v[16];
+                if (iters > 0) {
+                    tmem_ld16(lane_addr + (uint32_t)cc, v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = 0u;
+                }
+                const int col = c0 + cc;
+                if (!row_ok || col >= p.C) continue;
+                const int nvalid = min(16, p.C - col);
+                for (int e = 0; e < nvalid; ++e) orow[col + e] = __uint_as_float(v[e]);
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+__global__ void wgrad_reduce_kernel(const float *__restrict__ partial, float *__restrict__ dw, size_t n, int splits)
+{
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float s = 0.f;
+    for (int z = 0; z < splits; ++z) s += partial[(size_t)z * n + i];   // ascending split order: run-to-run identical
+    dw[i] = s;
+}
+
 // ------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -290,22 +448,28 @@ int pow2_cols(int bn)
     return c;
 }
 
+// Pipeline depth: two CTAs per SM when at least four stages fit in half of the shared memory, else one CTA with more.
+int pick_stages(size_t stage_bytes, int iters, size_t *smem)
+{
+    int st = (int)((110 * 1024 - 2048) / stage_bytes);
+    if (st < 4) st = (int)((220 * 1024 - 2048) / stage_bytes);
+    if (st > kMaxStages) st = kMaxStages;
+    if (st > iters) st = iters;
+    if (st < 2) st = 2;
+    *smem = 2048 + (size_t)st * stage_bytes;
+    return st;
+}
+
 template <bool B_MN>
 pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB, GemmP &p, cudaStream_t st)
 {
     const size_t a_bytes = kBM * kKC * 2;
     const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : pt_align_up((size_t)p.BN * 128, 1024);
-    const size_t stage = a_bytes + b_bytes;
-    int stages = (int)((110 * 1024 - 2048) / stage);           // two CTAs per SM
-    if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 2) stages = 2;
-    const int iters = p.taps * p.k_chunks;
-    if (stages > iters) stages = iters < 2 ? 2 : iters;
-    p.stages = stages;
-    const size_t smem = 2048 + (size_t)stages * stage;
+    size_t smem = 0;
+    p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks, &smem);
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
-        PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr_set[B_MN ? 1 : 0] = true;
     }
     const int m_tiles = pt_ceil_div(p.M_total, kBM);
@@ -315,32 +479,100 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     return PT_OK;
 }
 
+int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
+{
+    int n_tiles;
+    tile_n(d->C, &n_tiles);
+    const int tiles = pt_ceil_div(d->K, 128) * n_tiles * d->R * d->S;
+    const long long npix = (long long)d->N * P * Q;
+    long long s = pt_ceil_div(2 * c->sm_count, tiles);
+    const long long max_s = (npix + 255) / 256;          // at least four 64-pixel stages per split
+    if (s > max_s) s = max_s;
+    if (s < 1) s = 1;
+    if (s > 512) s = 512;
+    return (int)s;
+}
+
 }  // namespace
 
 bool pt_sm100_conv_supported(const pt_ctx *c, const pt_conv_desc *d, int which)
 {
     if (!c->encode_tiled || !c->encode_im2col) return false;
-    if (d->stride > 8 || d->pad > 100 || d->R > 128 || d->S > 128) return false;
+    if (d->stride > 8 || d->pad > 100 || d->R * d->S > kMaxTaps) return false;
     if (which == PT_CONV_FWD) return true;
-    if (which == PT_CONV_DGRAD) return d->stride == 1;
-    return false;
+    if (which == PT_CONV_DGRAD) return (d->stride == 1 && d->pad <= d->R - 1 && d->pad <= d->S - 1) || d->stride == 2;
+    return true;
 }
 
-size_t pt_sm100_conv_workspace(const pt_ctx *, const pt_conv_desc *, int) { return 0; }
+size_t pt_sm100_conv_workspace(const pt_ctx *c, const pt_conv_desc *d, int which)
+{
+    if (which != PT_CONV_WGRAD) return 0;
+    const int P = pt_out_dim(d->H, d->R, d->stride, d->pad), Q = pt_out_dim(d->W, d->S, d->stride, d->pad);
+    const int s = wgrad_splits(c, d, P, Q);
+    return s > 1 ? (size_t)s * d->K * d->R * d->S * d->C * sizeof(float) : 0;
+}
 
 pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void *a, const void *b, void *out, void *ws,
                         size_t ws_bytes, cudaStream_t st)
 {
-    (void)ws; (void)ws_bytes;
     const int P = pt_out_dim(d->H, d->R, d->stride, d->pad), Q = pt_out_dim(d->W, d->S, d->stride, d->pad);
+    CUtensorMap tmA, tmB;
+    if (which == PT_CONV_WGRAD) {
+        WgradP p;
+        memset(&p, 0, sizeof(p));
+        p.K = d->K; p.C = d->C; p.taps = d->R * d->S; p.S = d->S;
+        p.BN = tile_n(d->C, &p.n_tiles);
+        p.m_tiles = pt_ceil_div(d->K, 128);
+        p.npix = d->N * P * Q;
+        p.splits = wgrad_splits(c, d, P, Q);
+        p.pix_per_split = pt_ceil_div(pt_ceil_div(p.npix, p.splits), 64) * 64;
+        p.Pd = P; p.Qd = Q; p.stride = d->stride; p.lo_h = -d->pad; p.lo_w = -d->pad;
+        p.tmem_cols = pow2_cols(p.BN);
+        p.status = c->d_status;
+        const size_t n = (size_t)d->K * p.taps * d->C;
+        if (p.splits > 1) {
+            if (!ws || ws_bytes < (size_t)p.splits * n * sizeof(float)) return PT_ERR_WORKSPACE;
+            p.out = (float *)ws;
+        } else {
+            p.out = (float *)out;
+        }
+        // A: dy as a 2-D tensor (K channels, N*P*Q pixels), box 64 channels x 64 pixels
+        if (!c->encode_tiled) return PT_ERR_CUDA;
+        {
+            cuuint64_t dims[2] = {(cuuint64_t)d->K, (cuuint64_t)p.npix};
+            cuuint64_t strides[1] = {(cuuint64_t)d->ldy * 2};
+            cuuint32_t box[2] = {64, 64}, estr[2] = {1, 1};
+            CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(b), dims, strides,
+                                                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+        }
+        const int up_w = (Q - 1) * d->stride - d->pad - (d->W - 1), up_h = (P - 1) * d->stride - d->pad - (d->H - 1);
+        if (!make_im2col_map(c, &tmB, a, d->C, d->W, d->H, d->N, d->ldx, -d->pad, -d->pad, up_w, up_h, d->stride, 64)) return PT_ERR_CUDA;
+        size_t smem = 0;
+        const size_t stage = 2 * 8192 + (size_t)pt_ceil_div(p.BN, 64) * 8192;
+        p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), &smem);
+        static bool attr_set = false;
+        if (!attr_set) {
+            PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+            attr_set = true;
+        }
+        dim3 grid((unsigned)(p.n_tiles * p.m_tiles * p.taps), (unsigned)p.splits);
+        conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, p);
+        c->launches += 1;
+        if (p.splits > 1) {
+            wgrad_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const float *)ws, (float *)out, n, p.splits);
+            c->launches += 1;
+        }
+        PT_CUDA_OK(cudaGetLastError());
+        return PT_OK;
+    }
+
     GemmP p;
     memset(&p, 0, sizeof(p));
     p.status = c->d_status;
     p.out = out;
     p.out_f32 = d->out_f32;
-    p.taps = d->R * d->S;
-    p.S = d->S;
-    CUtensorMap tmA, tmB;
     if (which == PT_CONV_FWD) {
         // raster = output pixels (P x Q per image); source = x
         p.M_total = d->N * P * Q;
@@ -348,7 +580,9 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         p.BN = tile_n(d->K, &p.n_tiles);
         p.c_red = d->C;
         p.k_chunks = pt_ceil_div(d->C, kKC);
-        p.Pd = P; p.Qd = Q; p.stride = d->stride; p.lo_h = -d->pad; p.lo_w = -d->pad; p.flip = 0;
+        p.taps = d->R * d->S;
+        for (int t = 0; t < p.taps; ++t) { p.tap_oh[t] = (unsigned char)(t / d->S); p.tap_ow[t] = (unsigned char)(t % d->S); p.tap_wt[t] = (unsigned short)t; }
+        p.Pd = P; p.Qd = Q; p.stride = d->stride; p.lo_h = -d->pad; p.lo_w = -d->pad;
         p.oH = P; p.oW = Q; p.o_step = 1; p.o_h0 = 0; p.o_w0 = 0; p.ld_out = d->ldy; p.zero_mask = 0;
         p.tmem_cols = pow2_cols(p.BN);
         // the box of base positions must hold exactly P x Q positions at the traversal stride
@@ -357,22 +591,76 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         if (!make_weight_map(c, &tmB, b, d->C, d->R * d->S, d->K, d->ldw, p.BN)) return PT_ERR_CUDA;
         return launch_gemm<false>(c, tmA, tmB, p, st);
     }
-    if (which == PT_CONV_DGRAD && d->stride == 1) {
-        // raster = input pixels (H x W per image); source = dy with padding R-1-pad and flipped taps
+    if (which != PT_CONV_DGRAD) return PT_ERR_UNSUPPORTED;
+    p.n_cols = d->C;
+    p.BN = tile_n(d->C, &p.n_tiles);
+    p.c_red = d->K;
+    p.k_chunks = pt_ceil_div(d->K, kKC);
+    p.tmem_cols = pow2_cols(p.BN);
+    p.oH = d->H; p.oW = d->W; p.ld_out = d->ldx;
+    if (!make_weight_map(c, &tmB, b, d->C, d->R * d->S, d->K, d->ldw, kKC)) return PT_ERR_CUDA;
+    if (d->stride == 1) {
+        // raster = input pixels (H x W per image); source = dy with padding R-1-pad and the taps visited flipped:
+        // dx[h,w] = sum_{r',s'} dy[h - (R-1-pad) + r', w - (S-1-pad) + s'] * w[R-1-r', S-1-s']
         const int ph = d->R - 1 - d->pad, pw = d->S - 1 - d->pad;
         if (ph < 0 || pw < 0) return PT_ERR_UNSUPPORTED;
         p.M_total = d->N * d->H * d->W;
-        p.n_cols = d->C;
-        p.BN = tile_n(d->C, &p.n_tiles);
-        p.c_red = d->K;
-        p.k_chunks = pt_ceil_div(d->K, kKC);
-        p.Pd = d->H; p.Qd = d->W; p.stride = 1; p.lo_h = -ph; p.lo_w = -pw; p.flip = 1;
-        p.oH = d->H; p.oW = d->W; p.o_step = 1; p.o_h0 = 0; p.o_w0 = 0; p.ld_out = d->ldx; p.zero_mask = 0;
-        p.tmem_cols = pow2_cols(p.BN);
+        p.taps = d->R * d->S;
+        for (int t = 0; t < p.taps; ++t) {
+            p.tap_oh[t] = (unsigned char)(t / d->S); p.tap_ow[t] = (unsigned char)(t % d->S);
+            p.tap_wt[t] = (unsigned short)(p.taps - 1 - t);
+        }
+        p.Pd = d->H; p.Qd = d->W; p.stride = 1; p.lo_h = -ph; p.lo_w = -pw;
+        p.o_step = 1; p.o_h0 = 0; p.o_w0 = 0; p.zero_mask = 0;
         const int up_w = (d->W - 1) - pw - (Q - 1), up_h = (d->H - 1) - ph - (P - 1);
         if (!make_im2col_map(c, &tmA, a, d->K, Q, P, d->N, d->ldy, -pw, -ph, up_w, up_h, 1, kBM)) return PT_ERR_CUDA;
-        if (!make_weight_map(c, &tmB, b, d->C, d->R * d->S, d->K, d->ldw, kKC)) return PT_ERR_CUDA;
         return launch_gemm<true>(c, tmA, tmB, p, st);
     }
-    return PT_ERR_UNSUPPORTED;
+    if (d->stride != 2) return PT_ERR_UNSUPPORTED;
+    // Stride 2: the input pixels split by the parity (a, b) of (h, w) into four stride-1 problems over dy.
+    // Pixel h = 2i + a receives tap r iff (a + pad - r) is even, from dy row p = i + (a + pad - r)/2.
+    // Parities no tap reaches are zero-filled by the epilogue of the first launched parity.
+    struct Par { int a, b, nt; int oh[kMaxTaps], ow[kMaxTaps], wt[kMaxTaps]; };
+    Par par[4];
+    int empty_mask = 0, first = -1;
+    for (int ab = 0; ab < 4; ++ab) {
+        Par &q = par[ab];
+        q.a = ab >> 1; q.b = ab & 1; q.nt = 0;
+        for (int r = 0; r < d->R; ++r) {
+            if ((q.a + d->pad - r) & 1) continue;
+            for (int s = 0; s < d->S; ++s) {
+                if ((q.b + d->pad - s) & 1) continue;
+                q.oh[q.nt] = (q.a + d->pad - r) / 2;      // exact: the difference is even (may be negative)
+                q.ow[q.nt] = (q.b + d->pad - s) / 2;
+                q.wt[q.nt] = r * d->S + s;
+                ++q.nt;
+            }
+        }
+        const int rows = (d->H - q.a + 1) / 2, cols = (d->W - q.b + 1) / 2;
+        if (rows <= 0 || cols <= 0) { q.nt = -1; continue; }          // no pixel has this parity
+        if (q.nt == 0) empty_mask |= 1 << ab; else if (first < 0) first = ab;
+    }
+    if (first < 0) return PT_ERR_UNSUPPORTED;
+    if (empty_mask && (par[first].a != 0 || par[first].b != 0)) return PT_ERR_UNSUPPORTED;   // cells are anchored at parity (0,0)
+    for (int ab = 0; ab < 4; ++ab) {
+        Par &q = par[ab];
+        if (q.nt <= 0) continue;
+        int min_oh = q.oh[0], min_ow = q.ow[0];
+        for (int t = 0; t < q.nt; ++t) { min_oh = q.oh[t] < min_oh ? q.oh[t] : min_oh; min_ow = q.ow[t] < min_ow ? q.ow[t] : min_ow; }
+        const int rows = (d->H - q.a + 1) / 2, cols = (d->W - q.b + 1) / 2;
+        p.M_total = d->N * rows * cols;
+        p.taps = q.nt;
+        for (int t = 0; t < q.nt; ++t) {
+            p.tap_oh[t] = (unsigned char)(q.oh[t] - min_oh); p.tap_ow[t] = (unsigned char)(q.ow[t] - min_ow);
+            p.tap_wt[t] = (unsigned short)q.wt[t];
+        }
+        p.Pd = rows; p.Qd = cols; p.stride = 1; p.lo_h = min_oh; p.lo_w = min_ow;
+        p.o_step = 2; p.o_h0 = q.a; p.o_w0 = q.b;
+        p.zero_mask = (ab == first) ? empty_mask : 0;
+        const int up_w = (cols - 1) + min_ow - (Q - 1), up_h = (rows - 1) + min_oh - (P - 1);
+        if (!make_im2col_map(c, &tmA, a, d->K, Q, P, d->N, d->ldy, min_ow, min_oh, up_w, up_h, 1, kBM)) return PT_ERR_CUDA;
+        pt_status s = launch_gemm<true>(c, tmA, tmB, p, st);
+        if (s != PT_OK) return s;
+    }
+    return PT_OK;
 }

@@ -104,26 +104,25 @@ def test_invalid_arguments_are_rejected_before_launch():
         assert e.value.status == 1
     with pytest.raises(B.PtError):
         B.pt_conv_fwd(c, good, None, buf, buf)
-    d = B.make_conv_desc(2, 8, 8, 8, 8, 3, 3, 1, 1)
-    with pytest.raises(B.PtError) as e:       # wgrad needs a workspace
+    d = B.make_conv_desc(2, 8, 8, 8, 8, 3, 3, 1, 1, algo=1)
+    with pytest.raises(B.PtError) as e:       # the SIMT wgrad needs a workspace
         B.pt_conv_wgrad(c, d, buf, buf, torch.zeros(8 * 9 * 8, device="cuda"), None)
     assert e.value.status == 3
     c.poll()
 
 
-def test_tcgen05_path_takes_fwd_and_dgrad_when_forced():
-    """algo = 2 forces the tcgen05 kernels: the call must not fall back silently."""
-    N, H, C, K, R = 2, 12, 40, 24, 3
-    x, w, dy, pad = _case(N, H, H, C, K, R, 1, W.BASE_SEED + 9)
-    d = B.make_conv_desc(N, H, H, C, K, R, R, 1, pad, algo=2, out_f32=1)
-    xd, wd, dyd = Hh.to_dev_padded(x, d.ldx), Hh.to_dev_padded(w, d.ldw), Hh.to_dev_padded(dy, d.ldy)
-    y = Hh.out_buffer((N, H, H), K, d.ldy, True)
-    dx = Hh.out_buffer((N, H, H), C, d.ldx, True)
-    n0 = Hh.ctx().launch_count()
-    B.pt_conv_fwd(Hh.ctx(), d, xd, wd, y, Hh.conv_ws(d, 0))
-    B.pt_conv_dgrad(Hh.ctx(), d, dyd, wd, dx, Hh.conv_ws(d, 1))
-    torch.cuda.synchronize()
-    Hh.ctx().poll()
-    assert Hh.ctx().launch_count() - n0 == 2
-    Hh.check_conv(y, K, oracle.conv_fwd(x.numpy(), w.numpy(), 1, pad), what="fwd tcgen05")
-    Hh.check_conv(dx, C, oracle.conv_dgrad(dy.numpy(), w.numpy(), H, H, 1, pad), what="dgrad tcgen05")
+@pytest.mark.parametrize("stride", [1, 2])
+def test_tcgen05_path_takes_all_three_passes_when_forced(stride):
+    """algo = 2 forces the tcgen05 kernels: the calls must not fall back silently."""
+    N, H, C, K, R = 3, 12, 40, 24, 3
+    x, w, dy, pad = _case(N, H, H, C, K, R, stride, W.BASE_SEED + 9)
+    y, dx, dw, d = Hh.run_conv_all(N, H, H, C, K, R, stride, pad, x, w, dy, algo=2, out_f32=1)
+    Hh.check_conv(y, K, oracle.conv_fwd(x.numpy(), w.numpy(), stride, pad), what="fwd tcgen05")
+    Hh.check_conv(dx, C, oracle.conv_dgrad(dy.numpy(), w.numpy(), H, H, stride, pad), what="dgrad tcgen05")
+    Hh.check_conv(dw, C, oracle.conv_wgrad(x.numpy(), dy.numpy(), R, R, stride, pad), what="wgrad tcgen05")
+    # a 9x9 filter has more taps than the tcgen05 path's tap table: forcing it must fail loudly, auto must fall back
+    d9 = B.make_conv_desc(1, 12, 12, 8, 8, 9, 9, 1, 4, algo=2)
+    buf = torch.zeros(1 << 16, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.PtError) as e:
+        B.pt_conv_fwd(Hh.ctx(), d9, buf, buf, buf)
+    assert e.value.status == 2
