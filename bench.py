@@ -210,6 +210,17 @@ def run_ours(args):
             ms = float(t.item())
         return ms
 
+    if args.profile_steps:
+        # a short run for profilers: one warm-up step, then the requested steps, nothing else
+        ts.step()
+        torch.cuda.synchronize()
+        for _ in range(args.profile_steps):
+            ts.step()
+        torch.cuda.synchronize()
+        ctx.poll()
+        if rank == 0:
+            print(json.dumps({"profile_steps": args.profile_steps, "launches_per_step": None, "workload": name}))
+        return
     for _ in range(max(args.warmup, 3)):
         ts.step()
     barrier()
@@ -350,6 +361,7 @@ def main():
     ap.add_argument("--algo", type=int, default=0)
     ap.add_argument("--per-layer", default=None, help="write the per-layer table (JSON) here")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-steps", type=int, default=0, help="run only this many steps after one warm-up (for ncu)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -21,8 +21,9 @@
  * Physical layouts
  *   activations x, y, dy, dx : [N][H][W][ld]   bf16 (or fp32 outputs when out_f32 = 1), channels
  *                              innermost, channel pitch ld >= channels, ld a multiple of 8 elements.
- *                              Pad lanes (channel index >= channels) are never read; they are
- *                              not written either.
+ *                              Pad lanes (channel index >= channels) are never read. Outputs may get zeros
+ *                              written into the pad lanes that share the last 16-byte granule with valid
+ *                              channels (an effect of the TMA store); other pad lanes are left untouched.
  *   master weights w, momentum v, gradient g/dw : [K][R][S][C] fp32, dense (no pitch).
  *   bf16 weight shadow       : [K][R][S][ldw]  bf16, ldw >= C, ldw a multiple of 8.
  *   Output size: P = floor((H + 2*pad - R)/stride) + 1, Q likewise from W and S.
@@ -129,8 +130,8 @@ pt_status pt_group_lasso_sgd_step(pt_ctx *ctx, const pt_layer *layers /*host*/, 
 
 /* zero_out[k] = (max_{rs,c} |w| < threshold), zero_in[c] = (max_{k,rs} |w| < threshold), strict <, in fp32
  * (Sec. 4.1: threshold 1e-4; Sec. 4.2 / Fig. 4: the absolute maximum of a channel's parameters). A NaN keeps
- * its groups. If zero_in_place != 0 the weights, momentum and shadow of every detected group are set to 0.
- * Uses sumsq_out / sumsq_in of each layer as scratch (their contents are destroyed). */
+ * its groups. If zero_in_place != 0 the weights, momentum and shadow of every detected group are set to 0
+ * (the group sums of squares are then stale until the next pt_group_lasso_sgd_step recomputes them). */
 pt_status pt_find_zero_groups(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers, float threshold,
                               int32_t zero_in_place, void *ws, size_t ws_bytes, void *stream);
 

@@ -43,6 +43,7 @@ struct GemmP {
     int oH, oW, o_step, o_h0, o_w0;
     int ld_out, out_f32;
     int zero_mask;      // stride-2 dgrad: bit (a*2+b) set => also write zeros to the pixel at parity (a,b) of each 2x2 cell
+    int tma_store;      // 1: bf16 output rows are consecutive pixels -> staged in shared memory and written by TMA stores
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
@@ -59,7 +60,8 @@ struct __align__(8) Ctl {
 
 template <bool B_MN>
 __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                              const __grid_constant__ CUtensorMap tmB, const GemmP p)
+                                                              const __grid_constant__ CUtensorMap tmB,
+                                                              const __grid_constant__ CUtensorMap tmC, const GemmP p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw);
@@ -86,6 +88,7 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
         fence_mbar_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
+        if (p.tma_store) prefetch_tmap(&tmC);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), (uint32_t)p.tmem_cols);
@@ -171,6 +174,41 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
                 row_off = ((size_t)(img * p.oH + cell_h + p.o_h0) * p.oW + cell_w + p.o_w0) * (size_t)p.ld_out;
             }
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            if (p.tma_store) {
+                // All MMAs have completed, so the pipeline stages are free: they become the staging area.
+                // Each warp stages its 32 rows x 64 channels (4 KB, 128-byte swizzle) and stores it with one TMA
+                // store, which drops the channels past the true count and the rows past the last pixel.
+                const int n_chunks = (p.BN + 63) / 64;
+                for (int ch = 0; ch < n_chunks; ++ch) {
+                    const uint32_t slab = data_base + (uint32_t)(ch * 4 + quarter) * 4096u;
+                    const int groups = min(4, (p.BN - ch * 64) / 16);
+                    for (int g = 0; g < groups; ++g) {
+                        uint32_t v[16];
+                        tmem_ld16(lane_addr + (uint32_t)(ch * 64 + g * 16), v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 0]), __uint_as_float(v[8 * h + 1]));
+                            __nv_bfloat162 b1 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 2]), __uint_as_float(v[8 * h + 3]));
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 4]), __uint_as_float(v[8 * h + 5]));
+                            __nv_bfloat162 b3 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 6]), __uint_as_float(v[8 * h + 7]));
+                            const uint32_t j = (uint32_t)(g * 2 + h);
+                            const uint32_t addr = slab + (uint32_t)lane * 128u + ((j ^ ((uint32_t)lane & 7u)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t *>(&b0)),
+                                         "r"(*reinterpret_cast<uint32_t *>(&b1)), "r"(*reinterpret_cast<uint32_t *>(&b2)),
+                                         "r"(*reinterpret_cast<uint32_t *>(&b3))
+                                         : "memory");
+                        }
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0 && m0 + quarter * 32 < p.M_total) tma_store_2d(&tmC, slab, n0 + ch * 64, m0 + quarter * 32);
+                }
+                if (lane == 0) {
+                    tma_store_commit();
+                    tma_store_wait_read();
+                }
+            } else
             for (int c0 = 0; c0 < p.BN; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld16(lane_addr + (uint32_t)c0, v);
@@ -359,21 +397,38 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
         if (ok) {
             const int k = k0 + quarter * 32 + lane;
             const bool row_ok = k < p.K;
-            float *orow = p.out + (size_t)split * p.K * p.taps * p.C + ((size_t)k * p.taps + tap) * p.C;
+            (void)row_ok;
+            float *obase = p.out + (size_t)split * p.K * p.taps * p.C;
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-            for (int cc = 0; cc < p.BN; cc += 16) {
-                uint32_t v[16];
+            // The stages are free once the accumulator is complete: each warp transposes its 32 x 32 blocks through
+            // a padded shared-memory square so that a warp writes 32 consecutive floats of one dw row at a time.
+            const uint32_t sq = data_base + (uint32_t)quarter * (32u * 33u * 4u);
+            for (int cc = 0; cc < p.BN; cc += 32) {
+                uint32_t v[32];
                 if (iters > 0) {
-                    tmem_ld16(lane_addr + (uint32_t)cc, v);
+                    uint32_t lo[16], hi[16];
+                    tmem_ld16(lane_addr + (uint32_t)cc, lo);
+                    if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)cc + 16u, hi);
                     tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) { v[e] = lo[e]; v[16 + e] = (cc + 16 < p.BN) ? hi[e] : 0u; }
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) v[e] = 0u;
+                    for (int e = 0; e < 32; ++e) v[e] = 0u;
                 }
-                const int col = c0 + cc;
-                if (!row_ok || col >= p.C) continue;
-                const int nvalid = min(16, p.C - col);
-                for (int e = 0; e < nvalid; ++e) orow[col + e] = __uint_as_float(v[e]);
+                __syncwarp();
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(sq + (uint32_t)(lane * 33 + e) * 4u), "r"(v[e]) : "memory");
+                __syncwarp();
+                const int col = c0 + cc + lane;
+                for (int rr = 0; rr < 32; ++rr) {
+                    const int kk = k0 + quarter * 32 + rr;
+                    if (kk >= p.K) break;
+                    uint32_t t;
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(t) : "r"(sq + (uint32_t)(rr * 33 + lane) * 4u) : "memory");
+                    if (col < p.C && cc + lane < p.BN) obase[((size_t)kk * p.taps + tap) * p.C + col] = __uint_as_float(t);
+                }
             }
         }
         tc_fence_before();
@@ -433,12 +488,18 @@ bool make_weight_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, 
     return r == CUDA_SUCCESS;
 }
 
+// Tile width along the output channels. One tile: the ragged count rounded up to 16. Several tiles: a multiple of
+// 64 (the TMA-store chunk) chosen to waste the fewest padded columns.
 int tile_n(int cols, int *n_tiles)
 {
-    int nt = pt_ceil_div(cols, 256);
-    int bn = pt_ceil_div(pt_ceil_div(cols, nt), 16) * 16;
-    *n_tiles = pt_ceil_div(cols, bn);
-    return bn;
+    if (cols <= 256) { *n_tiles = 1; return pt_ceil_div(cols, 16) * 16; }
+    int best = 256, best_pad = 1 << 30;
+    for (int bn = 256; bn >= 128; bn -= 64) {
+        int pad = pt_ceil_div(cols, bn) * bn;
+        if (pad < best_pad) { best_pad = pad; best = bn; }
+    }
+    *n_tiles = pt_ceil_div(cols, best);
+    return best;
 }
 
 int pow2_cols(int bn)
@@ -460,9 +521,25 @@ int pick_stages(size_t stage_bytes, int iters, size_t *smem)
     return st;
 }
 
+// bf16 output viewed as (channels, pixels) with row pitch ld: box 64 channels x 32 pixels, 128-byte swizzle.
+bool make_out_map(const pt_ctx *c, CUtensorMap *tm, void *base, int cols, int rows, int ld)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, 32}, estr[2] = {1, 1};
+    CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 template <bool B_MN>
 pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB, GemmP &p, cudaStream_t st)
 {
+    CUtensorMap tmC;
+    memset(&tmC, 0, sizeof(tmC));
+    p.tma_store = (!p.out_f32 && p.o_step == 1 && p.zero_mask == 0) ? 1 : 0;
+    if (p.tma_store && !make_out_map(c, &tmC, p.out, p.n_cols, p.M_total, p.ld_out)) return PT_ERR_CUDA;
     const size_t a_bytes = kBM * kKC * 2;
     const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : pt_align_up((size_t)p.BN * 128, 1024);
     size_t smem = 0;
@@ -473,7 +550,7 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
         attr_set[B_MN ? 1 : 0] = true;
     }
     const int m_tiles = pt_ceil_div(p.M_total, kBM);
-    conv_gemm_kernel<B_MN><<<m_tiles * p.n_tiles, kThreads, smem, st>>>(tmA, tmB, p);
+    conv_gemm_kernel<B_MN><<<m_tiles * p.n_tiles, kThreads, smem, st>>>(tmA, tmB, tmC, p);
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;

@@ -1,0 +1,79 @@
+"""Times single conv passes of one layer of the pruned ResNet-50 workload (CUDA events, rotating buffers).
+
+    python -m paper_1901_09290_b200.layerbench --layer s1b1.c3 --passes fwd,dgrad,wgrad --iters 20
+    python -m paper_1901_09290_b200.layerbench --shape 64,56,36,143,1,1 --passes fwd      # N,H,C,K,R,stride
+
+It is also the small case ncu captures are taken on.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--layer", default=None)
+    ap.add_argument("--shape", default=None, help="N,H,C,K,R,stride")
+    ap.add_argument("--passes", default="fwd,dgrad,wgrad")
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--sets", type=int, default=4, help="rotating buffer sets (footprint larger than L2)")
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--algo", type=int, default=0)
+    args = ap.parse_args()
+    if args.shape:
+        N, H, C, K, R, stride = [int(t) for t in args.shape.split(",")]
+        name = args.shape
+    else:
+        net = W.resnet50()
+        counts = W.staged_keep_to_flops(net, W.BASE_SEED + 4, 0.60)
+        l = [l for l in W.with_sizes(net, counts).layers if l.name == args.layer][0]
+        N, H, C, K, R, stride = args.batch, l.H, l.C, l.K, l.R, l.stride
+        name = l.name
+    pad = R // 2
+    P = (H + 2 * pad - R) // stride + 1
+    ctx = B.Context(0)
+    d = B.make_conv_desc(N, H, H, C, K, R, R, stride, pad, algo=args.algo)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    sets = []
+    for _ in range(args.sets):
+        x = torch.randn((N, H, H, d.ldx), generator=g, device="cuda").clamp_(min=0).to(torch.bfloat16)
+        dy = (torch.randn((N, P, P, d.ldy), generator=g, device="cuda") * 2 ** -6).to(torch.bfloat16)
+        w = (torch.randn((K, R, R, d.ldw), generator=g, device="cuda") * (2.0 / (C * R * R)) ** 0.5).to(torch.bfloat16)
+        sets.append((x, dy, w, torch.empty_like(dy), torch.empty_like(x), torch.empty((K, R, R, C), device="cuda")))
+    ws = torch.empty(max(16, max(B.pt_conv_workspace_bytes(ctx, d, i) for i in range(3))), dtype=torch.uint8, device="cuda")
+    flops = 2 * N * P * P * K * C * R * R
+    act = N * H * H * C * 2 + N * P * P * K * 2
+    out = {"layer": name, "N": N, "H": H, "C": C, "K": K, "R": R, "stride": stride}
+    for ps in args.passes.split(","):
+        def run(i):
+            x, dy, w, y, dx, dw = sets[i % len(sets)]
+            if ps == "fwd":
+                B.pt_conv_fwd(ctx, d, x, w, y, ws)
+            elif ps == "dgrad":
+                B.pt_conv_dgrad(ctx, d, dy, w, dx, ws)
+            else:
+                B.pt_conv_wgrad(ctx, d, x, dy, dw, ws)
+        for i in range(3):
+            run(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.iters):
+            run(i)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / args.iters
+        by = act + K * C * R * R * (4 if ps == "wgrad" else 2)
+        out[ps] = {"us": round(us, 2), "tflops": round(flops / us / 1e6, 1), "gbs": round(by / us / 1e3, 1)}
+    ctx.poll()
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()
