@@ -449,6 +449,98 @@ __global__ void wgrad_reduce_kernel(const float *__restrict__ partial, float *__
     dw[i] = s;
 }
 
+// ------------------------------------------------------------------------------------------ few-channel stride-2 stem
+// A stride-2 convolution over very few input channels (the 7x7 / 3-channel network stem) is rewritten as a stride-1
+// convolution over a space-to-depth copy of the input: xs[n][i][j + pl][(a,b,c)] = x[n][2i+a][2j+b][c], 16 bf16 per pixel,
+// with pl zero columns on the left and V-1-pl on the right. Consecutive pixels of a row are contiguous, so the V
+// horizontal taps x 16 lanes of one output position are ONE run of 64 elements: the tensor map below gives every output
+// column its own 128-byte row (overlapping windows, 32-byte stride), and the conv becomes U vertical taps of 64
+// "channels" each -- full swizzle rows for TMA and UMMA instead of 49 taps of 3 channels.
+//   h = 2p - pad + r = 2(p - pl) + t,  t = r + off,  off = 2*pl - pad,  u = t / 2, a = t % 2   (same for columns)
+struct StemPlan {
+    int ok;
+    int pl, off, U, V, Hs, Ws, Wp, P, Q;
+    size_t xs_bytes, w2_elems;     // padded space-to-depth input; weights / weight gradient as [K][U][64]
+};
+
+StemPlan stem_plan(const pt_conv_desc *d)
+{
+    StemPlan s;
+    memset(&s, 0, sizeof(s));
+    if (d->stride != 2 || d->C > 4 || (d->H & 1) || (d->W & 1) || d->R != d->S || d->ldx != 8) return s;
+    s.pl = (d->pad + 1) / 2;
+    s.off = 2 * s.pl - d->pad;
+    s.U = (d->R - 1 + s.off) / 2 + 1;
+    s.V = s.U;
+    if (s.V > 4) return s;
+    s.Hs = d->H / 2; s.Ws = d->W / 2;
+    s.Wp = s.Ws + 3;                        // every window is 4 pixels wide whatever V is: pl zero columns left, 3 - pl right
+    s.P = pt_out_dim(d->H, d->R, 2, d->pad);
+    s.Q = pt_out_dim(d->W, d->S, 2, d->pad);
+    if (s.Q > s.Ws || s.P > s.Hs + s.pl) return s;
+    s.xs_bytes = pt_align_up((size_t)d->N * s.Hs * s.Wp * 32, 1024);
+    s.w2_elems = (size_t)d->K * s.U * 64;
+    s.ok = 1;
+    return s;
+}
+
+__global__ void stem_s2d_x_kernel(const __nv_bfloat16 *__restrict__ x, __nv_bfloat16 *__restrict__ xs, int N, int H, int W, int C,
+                                  int Hs, int Ws, int Wp, int pl)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t total = (size_t)N * Hs * Wp;
+    if (idx >= total) return;
+    const int jp = (int)(idx % Wp);
+    const size_t t = idx / Wp;
+    const int i = (int)(t % Hs), n = (int)(t / Hs);
+    __align__(16) __nv_bfloat16 o[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) o[e] = __float2bfloat16_rn(0.f);
+    const int j = jp - pl;
+    if (j >= 0 && j < Ws) {
+#pragma unroll
+        for (int ab = 0; ab < 4; ++ab) {
+            const int a = ab >> 1, b = ab & 1;
+            const uint4 px = *reinterpret_cast<const uint4 *>(x + ((size_t)(n * H + 2 * i + a) * W + 2 * j + b) * 8);
+            const __nv_bfloat16 *pe = reinterpret_cast<const __nv_bfloat16 *>(&px);
+            for (int c = 0; c < C; ++c) o[ab * C + c] = pe[c];
+        }
+    }
+    uint4 *dst = reinterpret_cast<uint4 *>(xs + idx * 16);
+    dst[0] = *reinterpret_cast<uint4 *>(&o[0]);
+    dst[1] = *reinterpret_cast<uint4 *>(&o[8]);
+}
+
+// w2[k][u][v*16 + (a*2+b)*C + c] = w[k][2u+a-off][2v+b-off][c]  (0 where the tap falls outside the filter)
+__global__ void stem_s2d_w_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bfloat16 *__restrict__ w2, int K, int R, int S, int C,
+                                  int ldw, int U, int V, int off)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= K * U * 64) return;
+    const int l = idx & 63, u = (idx >> 6) % U, k = (idx >> 6) / U;
+    const int v = l >> 4, e = l & 15;
+    float val = 0.f;
+    if (v < V && e < 4 * C) {
+        const int ab = e / C, c = e - ab * C, a = ab >> 1, b = ab & 1;
+        const int r = 2 * u + a - off, s = 2 * v + b - off;
+        if (r >= 0 && r < R && s >= 0 && s < S) val = __bfloat162float(w[((size_t)(k * R + r) * S + s) * ldw + c]);
+    }
+    w2[idx] = __float2bfloat16_rn(val);
+}
+
+// dw[k][r][s][c] = dw2[k][u][v*16 + (a*2+b)*C + c] with (u,a) from r + off and (v,b) from s + off
+__global__ void stem_dw_back_kernel(const float *__restrict__ dw2, float *__restrict__ dw, int K, int R, int S, int C, int U, int off)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= K * R * S * C) return;
+    const int c = idx % C;
+    int t = idx / C;
+    const int s = t % S; t /= S;
+    const int r = t % R, k = t / R;
+    const int tr = r + off, ts = s + off;
+    dw[idx] = dw2[((size_t)k * U + (tr >> 1)) * 64 + (ts >> 1) * 16 + ((tr & 1) * 2 + (ts & 1)) * C + c];
+}
+
 // ------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -459,12 +551,13 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_
 
 // bf16 tensor (C, W, H, N) with channel pitch ld: im2col map loading `pixels` x 64 channels.
 bool make_im2col_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, int W, int H, int N, int ld, int lo_w, int lo_h,
-                     int up_w, int up_h, int stride, int pixels)
+                     int up_w, int up_h, int stride, int pixels, int row_pixels = 0)
 {
     if (!c->encode_im2col) return false;
     if (lo_w < -128 || lo_h < -128 || up_w < -128 || up_h < -128 || lo_w > 127 || lo_h > 127 || up_w > 127 || up_h > 127) return false;
+    const int rowp = row_pixels ? row_pixels : W;        // pixels between two image rows in memory (>= W)
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
-    cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)W * ld * 2, (cuuint64_t)H * W * ld * 2};
+    cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)rowp * ld * 2, (cuuint64_t)H * rowp * ld * 2};
     int lo[2] = {lo_w, lo_h}, up[2] = {up_w, up_h};
     cuuint32_t estr[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
     CUresult r = ((EncodeIm2colFn)c->encode_im2col)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, lo,
@@ -570,6 +663,59 @@ int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     return (int)s;
 }
 
+// Launches the weight-gradient kernel for a problem whose x operand is described by `tmX` (64 pixels x 64 channels boxes).
+pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, int lo_h, int lo_w, const CUtensorMap &tmX,
+                    const void *dy, float *out, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    WgradP p;
+    memset(&p, 0, sizeof(p));
+    p.K = d->K; p.C = d->C; p.taps = d->R * d->S; p.S = d->S;
+    p.BN = tile_n(d->C, &p.n_tiles);
+    p.m_tiles = pt_ceil_div(d->K, 128);
+    p.npix = d->N * P * Q;
+    p.splits = wgrad_splits(c, d, P, Q);
+    p.pix_per_split = pt_ceil_div(pt_ceil_div(p.npix, p.splits), 64) * 64;
+    p.Pd = P; p.Qd = Q; p.stride = stride; p.lo_h = lo_h; p.lo_w = lo_w;
+    p.tmem_cols = pow2_cols(p.BN);
+    p.status = c->d_status;
+    const size_t n = (size_t)d->K * p.taps * d->C;
+    if (p.splits > 1) {
+        if (!ws || ws_bytes < (size_t)p.splits * n * sizeof(float)) return PT_ERR_WORKSPACE;
+        p.out = (float *)ws;
+    } else {
+        p.out = out;
+    }
+    // A: dy as a 2-D tensor (K channels, N*P*Q pixels), box 64 channels x 64 pixels
+    if (!c->encode_tiled) return PT_ERR_CUDA;
+    CUtensorMap tmA;
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)d->K, (cuuint64_t)p.npix};
+        cuuint64_t strides[1] = {(cuuint64_t)d->ldy * 2};
+        cuuint32_t box[2] = {64, 64}, estr[2] = {1, 1};
+        CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(dy), dims, strides, box,
+                                                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+    }
+    size_t smem = 0;
+    const size_t stage = 2 * 8192 + (size_t)pt_ceil_div(p.BN, 64) * 8192;
+    p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), &smem);
+    static bool attr_set = false;
+    if (!attr_set) {
+        PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        attr_set = true;
+    }
+    dim3 grid((unsigned)(p.n_tiles * p.m_tiles * p.taps), (unsigned)p.splits);
+    conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(tmA, tmX, p);
+    c->launches += 1;
+    if (p.splits > 1) {
+        wgrad_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const float *)ws, out, n, p.splits);
+        c->launches += 1;
+    }
+    PT_CUDA_OK(cudaGetLastError());
+    return PT_OK;
+}
+
 }  // namespace
 
 bool pt_sm100_conv_supported(const pt_ctx *c, const pt_conv_desc *d, int which)
@@ -581,8 +727,23 @@ bool pt_sm100_conv_supported(const pt_ctx *c, const pt_conv_desc *d, int which)
     return true;
 }
 
+// The stem's weight gradient as the generic kernel sees it: U taps of 64 "channels".
+static pt_conv_desc stem_virtual_desc(const pt_conv_desc *d, const StemPlan &sp)
+{
+    pt_conv_desc v = *d;
+    v.C = 64; v.R = sp.U; v.S = 1;
+    return v;
+}
+
 size_t pt_sm100_conv_workspace(const pt_ctx *c, const pt_conv_desc *d, int which)
 {
+    const StemPlan sp = stem_plan(d);
+    if (sp.ok && which == PT_CONV_FWD) return sp.xs_bytes + pt_align_up(sp.w2_elems * 2, 1024);
+    if (sp.ok && which == PT_CONV_WGRAD) {
+        const pt_conv_desc v = stem_virtual_desc(d, sp);
+        const int s = wgrad_splits(c, &v, sp.P, sp.Q);
+        return sp.xs_bytes + pt_align_up(sp.w2_elems * 4, 1024) + (s > 1 ? (size_t)s * sp.w2_elems * 4 : 0);
+    }
     if (which != PT_CONV_WGRAD) return 0;
     const int P = pt_out_dim(d->H, d->R, d->stride, d->pad), Q = pt_out_dim(d->W, d->S, d->stride, d->pad);
     const int s = wgrad_splits(c, d, P, Q);
@@ -594,55 +755,34 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
 {
     const int P = pt_out_dim(d->H, d->R, d->stride, d->pad), Q = pt_out_dim(d->W, d->S, d->stride, d->pad);
     CUtensorMap tmA, tmB;
+    const StemPlan sp = stem_plan(d);
     if (which == PT_CONV_WGRAD) {
-        WgradP p;
-        memset(&p, 0, sizeof(p));
-        p.K = d->K; p.C = d->C; p.taps = d->R * d->S; p.S = d->S;
-        p.BN = tile_n(d->C, &p.n_tiles);
-        p.m_tiles = pt_ceil_div(d->K, 128);
-        p.npix = d->N * P * Q;
-        p.splits = wgrad_splits(c, d, P, Q);
-        p.pix_per_split = pt_ceil_div(pt_ceil_div(p.npix, p.splits), 64) * 64;
-        p.Pd = P; p.Qd = Q; p.stride = d->stride; p.lo_h = -d->pad; p.lo_w = -d->pad;
-        p.tmem_cols = pow2_cols(p.BN);
-        p.status = c->d_status;
-        const size_t n = (size_t)d->K * p.taps * d->C;
-        if (p.splits > 1) {
-            if (!ws || ws_bytes < (size_t)p.splits * n * sizeof(float)) return PT_ERR_WORKSPACE;
-            p.out = (float *)ws;
-        } else {
-            p.out = (float *)out;
-        }
-        // A: dy as a 2-D tensor (K channels, N*P*Q pixels), box 64 channels x 64 pixels
-        if (!c->encode_tiled) return PT_ERR_CUDA;
-        {
-            cuuint64_t dims[2] = {(cuuint64_t)d->K, (cuuint64_t)p.npix};
-            cuuint64_t strides[1] = {(cuuint64_t)d->ldy * 2};
-            cuuint32_t box[2] = {64, 64}, estr[2] = {1, 1};
-            CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(b), dims, strides,
-                                                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
-        }
-        const int up_w = (Q - 1) * d->stride - d->pad - (d->W - 1), up_h = (P - 1) * d->stride - d->pad - (d->H - 1);
-        if (!make_im2col_map(c, &tmB, a, d->C, d->W, d->H, d->N, d->ldx, -d->pad, -d->pad, up_w, up_h, d->stride, 64)) return PT_ERR_CUDA;
-        size_t smem = 0;
-        const size_t stage = 2 * 8192 + (size_t)pt_ceil_div(p.BN, 64) * 8192;
-        p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), &smem);
-        static bool attr_set = false;
-        if (!attr_set) {
-            PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-            attr_set = true;
-        }
-        dim3 grid((unsigned)(p.n_tiles * p.m_tiles * p.taps), (unsigned)p.splits);
-        conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, p);
-        c->launches += 1;
-        if (p.splits > 1) {
-            wgrad_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const float *)ws, (float *)out, n, p.splits);
+        if (sp.ok) {
+            // stem: space-to-depth copy of x, generic wgrad over U taps x 64 lanes, then back to [K][R][S][C]
+            char *wsb = (char *)ws;
+            __nv_bfloat16 *xs = (__nv_bfloat16 *)wsb;
+            float *dw2 = (float *)(wsb + sp.xs_bytes);
+            char *part = wsb + sp.xs_bytes + pt_align_up(sp.w2_elems * 4, 1024);
+            const pt_conv_desc v = stem_virtual_desc(d, sp);
+            const size_t tot = (size_t)d->N * sp.Hs * sp.Wp;
+            stem_s2d_x_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)a, xs, d->N, d->H, d->W, d->C, sp.Hs,
+                                                                          sp.Ws, sp.Wp, sp.pl);
             c->launches += 1;
+            CUtensorMap tmX;
+            const int up_h = (sp.P - 1) - sp.pl - (sp.Hs - 1);
+            if (!make_im2col_map(c, &tmX, xs, 64, sp.Q, sp.Hs, d->N, 16, 0, -sp.pl, 0, up_h, 1, 64, sp.Wp)) return PT_ERR_CUDA;
+            pt_status r = run_wgrad(c, &v, sp.P, sp.Q, 1, -sp.pl, 0, tmX, b, dw2, part, ws_bytes - (size_t)(part - wsb), st);
+            if (r != PT_OK) return r;
+            const int n = d->K * d->R * d->S * d->C;
+            stem_dw_back_kernel<<<(n + 255) / 256, 256, 0, st>>>(dw2, (float *)out, d->K, d->R, d->S, d->C, sp.U, sp.off);
+            c->launches += 1;
+            PT_CUDA_OK(cudaGetLastError());
+            return PT_OK;
         }
-        PT_CUDA_OK(cudaGetLastError());
-        return PT_OK;
+        CUtensorMap tmX;
+        const int up_w = (Q - 1) * d->stride - d->pad - (d->W - 1), up_h = (P - 1) * d->stride - d->pad - (d->H - 1);
+        if (!make_im2col_map(c, &tmX, a, d->C, d->W, d->H, d->N, d->ldx, -d->pad, -d->pad, up_w, up_h, d->stride, 64)) return PT_ERR_CUDA;
+        return run_wgrad(c, d, P, Q, d->stride, -d->pad, -d->pad, tmX, b, (float *)out, ws, ws_bytes, st);
     }
 
     GemmP p;
@@ -650,6 +790,30 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
     p.status = c->d_status;
     p.out = out;
     p.out_f32 = d->out_f32;
+    if (which == PT_CONV_FWD && sp.ok) {
+        char *wsb = (char *)ws;
+        __nv_bfloat16 *xs = (__nv_bfloat16 *)wsb, *w2 = (__nv_bfloat16 *)(wsb + sp.xs_bytes);
+        const size_t tot = (size_t)d->N * sp.Hs * sp.Wp;
+        stem_s2d_x_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)a, xs, d->N, d->H, d->W, d->C, sp.Hs, sp.Ws,
+                                                                      sp.Wp, sp.pl);
+        stem_s2d_w_kernel<<<(unsigned)((sp.w2_elems + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)b, w2, d->K, d->R, d->S, d->C, d->ldw,
+                                                                              sp.U, sp.V, sp.off);
+        c->launches += 2;
+        p.M_total = d->N * sp.P * sp.Q;
+        p.n_cols = d->K;
+        p.BN = tile_n(d->K, &p.n_tiles);
+        p.c_red = 64;
+        p.k_chunks = 1;
+        p.taps = sp.U;
+        for (int t = 0; t < p.taps; ++t) { p.tap_oh[t] = (unsigned char)t; p.tap_ow[t] = 0; p.tap_wt[t] = (unsigned short)t; }
+        p.Pd = sp.P; p.Qd = sp.Q; p.stride = 1; p.lo_h = -sp.pl; p.lo_w = 0;
+        p.oH = sp.P; p.oW = sp.Q; p.o_step = 1; p.o_h0 = 0; p.o_w0 = 0; p.ld_out = d->ldy; p.zero_mask = 0;
+        p.tmem_cols = pow2_cols(p.BN);
+        const int up_h = (sp.P - 1) - sp.pl - (sp.Hs - 1);
+        if (!make_im2col_map(c, &tmA, xs, 64, sp.Q, sp.Hs, d->N, 16, 0, -sp.pl, 0, up_h, 1, kBM, sp.Wp)) return PT_ERR_CUDA;
+        if (!make_weight_map(c, &tmB, w2, 64, sp.U, d->K, 64, p.BN)) return PT_ERR_CUDA;
+        return launch_gemm<false>(c, tmA, tmB, p, st);
+    }
     if (which == PT_CONV_FWD) {
         // raster = output pixels (P x Q per image); source = x
         p.M_total = d->N * P * Q;

@@ -17,6 +17,8 @@ SMALL = [
     (2, 5, 7, 1, 1, 1, 1), (2, 5, 7, 3, 7, 3, 1), (1, 1, 1, 8, 11, 1, 1), (3, 16, 16, 11, 27, 3, 1),
     (2, 16, 16, 16, 16, 1, 1), (2, 9, 9, 27, 8, 3, 2), (2, 8, 8, 7, 93, 1, 2), (1, 23, 23, 3, 16, 7, 2),
     (2, 14, 14, 93, 77, 3, 1), (1, 12, 10, 130, 70, 1, 1), (1, 7, 7, 260, 300, 3, 1),
+    # few-channel stride-2 stems (space-to-depth path): 7x7, 5x5, 3x3; C = 1, 3, 4; non-square image
+    (2, 32, 32, 3, 16, 7, 2), (1, 16, 20, 3, 55, 7, 2), (2, 12, 12, 1, 9, 5, 2), (2, 16, 16, 4, 24, 3, 2),
 ]
 
 
