@@ -3,9 +3,9 @@
 //
 // All layers are processed by one launch per phase through a chunk table. A weight tensor
 // [K][RS][C] is seen as K*RS "lines" of C contiguous floats; a chunk is a run of lines of one
-// layer. Inside a block, thread (tx, ty) owns the columns c = tx + TX*j and the lines
-// ty, ty+TY, ... of its chunk, so every access is a coalesced run of a line and per-column
-// quantities stay in registers.
+// layer restricted to a block of TX <= 256 columns. Inside a block, thread (tx, ty) owns column
+// col0 + tx and the lines ty, ty+TY, ... of its chunk (four lines in flight per thread), so every
+// access is a coalesced run of a line and per-column quantities stay in registers.
 //
 // Phases of the step:
 //   1. norms_partial : per line sum of squares, per chunk column sums of squares   (reads w)
@@ -23,22 +23,25 @@ struct LayerDev {
     uint8_t *zero_out, *zero_in;
     int K, C, RS, ldw;
     int reg_in, reg_out;
-    int chunk0, n_chunks;       // this layer's chunks in the chunk table
-    int tx_log2;                // TX = 1 << tx_log2 column lanes (32..256)
+    int tx_log2;                // TX = 1 << tx_log2 threads along a line (32..256): one column per thread
+    int n_cb;                   // column blocks of TX columns
+    int n_lc;                   // line chunks
     int pad_;
-    long long line_off;         // offset of this layer's lines in the per-line scratch
-    long long col_off;          // offset of this layer's column partials (n_chunks * C floats)
+    long long line_off;         // offset of this layer's per-line partials (lines * n_cb floats)
+    long long col_off;          // offset of this layer's column partials (n_lc * C floats)
     long long k_off, c_off;     // offsets into the per-K / per-C scratch arrays
 };
 
-struct Chunk { int layer, line0, nlines, idx; };
+// A chunk is a run of lines of one layer restricted to one block of TX columns.
+struct Chunk { int layer, line0, nlines, col0, lc, cb, pad0, pad1; };
 
 struct WsLayout {
     size_t linesum, colpart, inv_out, inv_in, layer_reg, maxbits, total;
 };
 
 constexpr int kThreads = 256;
-constexpr int kMaxColsPerThread = 8;      // columns are walked in passes of TX*8
+constexpr int kUnroll = 8;                // lines in flight per thread
+constexpr int kSweeps = 4;                // unrolled sweeps per chunk: every block does the same number of iterations
 
 __device__ __forceinline__ float warp_sum(float v)
 {
@@ -52,87 +55,94 @@ __global__ void __launch_bounds__(kThreads) norms_partial_kernel(const LayerDev 
                                                                  const Chunk *__restrict__ chunks,
                                                                  float *__restrict__ linesum, float *__restrict__ colpart)
 {
-    __shared__ float s_line[8];                 // per-warp partials of one line pass
     __shared__ float s_col[kThreads];
+    __shared__ float s_line[kThreads];           // [line in chunk][warp along the line]: TY*kUnroll*kSweeps*nwx = 256
     const Chunk ch = chunks[blockIdx.x];
     const LayerDev L = layers[ch.layer];
     const int TX = 1 << L.tx_log2, TY = kThreads >> L.tx_log2;
     const int tx = threadIdx.x & (TX - 1), ty = threadIdx.x >> L.tx_log2;
     const int lane = threadIdx.x & 31;
-    const int wx = tx >> 5, nwx = TX >> 5;      // warp index along the line, warps per line
-    (void)s_line;
-    float *cp = colpart + L.col_off + (size_t)ch.idx * L.C;
-    float *ls = linesum + L.line_off;
-    const int passes = (L.C + TX * kMaxColsPerThread - 1) / (TX * kMaxColsPerThread);
-    for (int pass = 0; pass < passes; ++pass) {
-        const int cbase = pass * TX * kMaxColsPerThread + tx;
-        float cacc[kMaxColsPerThread];
+    const int wx = tx >> 5, nwx = TX >> 5;
+    const int c = ch.col0 + tx;
+    const bool cv = c < L.C;
+    const float *wbase = L.w + (size_t)ch.line0 * L.C + c;
+    float cacc = 0.f;
+    for (int l = ty; l < ch.nlines; l += kUnroll * TY) {
+        float a[kUnroll];
 #pragma unroll
-        for (int j = 0; j < kMaxColsPerThread; ++j) cacc[j] = 0.f;
-        for (int l = ty; l < ch.nlines; l += TY) {
-            const float *row = L.w + (size_t)(ch.line0 + l) * L.C;
-            float racc = 0.f;
-#pragma unroll
-            for (int j = 0; j < kMaxColsPerThread; ++j) {
-                int c = cbase + j * TX;
-                if (c < L.C) {
-                    float a = row[c];
-                    float sq = a * a;
-                    cacc[j] += sq;
-                    racc += sq;
-                }
-            }
-            racc = warp_sum(racc);
-            // one partial per (line, warp-along-line, pass): summed in fixed order by phase 2
-            if (lane == 0) ls[((size_t)(ch.line0 + l) * passes + pass) * nwx + wx] = racc;
+        for (int u = 0; u < kUnroll; ++u) {
+            const int ll = l + u * TY;
+            a[u] = (cv && ll < ch.nlines) ? wbase[(size_t)ll * L.C] : 0.f;
         }
-        // combine the TY line-groups' column partials in fixed order through shared memory
 #pragma unroll
-        for (int j = 0; j < kMaxColsPerThread; ++j) {
-            __syncthreads();
-            s_col[threadIdx.x] = cacc[j];
-            __syncthreads();
-            int c = cbase + j * TX;
-            if (ty == 0 && c < L.C) {
-                float s = 0.f;
-                for (int y = 0; y < TY; ++y) s += s_col[y * TX + tx];
-                cp[c] = s;
+        for (int u = 0; u < kUnroll; ++u) {
+            a[u] *= a[u];
+            cacc += a[u];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) a[u] += __shfl_xor_sync(0xffffffffu, a[u], o);
+        if (lane == 0) {
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int ll = l + u * TY;
+                if (ll < ch.nlines) s_line[ll * nwx + wx] = a[u];
             }
         }
+    }
+    s_col[threadIdx.x] = cacc;
+    __syncthreads();
+    // one partial per (line, column block): the warps along a line are added in ascending order
+    if ((int)threadIdx.x < ch.nlines) {
+        float s = 0.f;
+        for (int x = 0; x < nwx; ++x) s += s_line[threadIdx.x * nwx + x];
+        linesum[L.line_off + (size_t)(ch.line0 + threadIdx.x) * L.n_cb + ch.cb] = s;
+    }
+    // combine the TY line groups' column partials in fixed order
+    if (ty == 0 && cv) {
+        float s = 0.f;
+        for (int y = 0; y < TY; ++y) s += s_col[y * TX + tx];
+        colpart[L.col_off + (size_t)ch.lc * L.C + c] = s;
     }
 }
 
-// ---- phase 2: one block per layer
+// ---- phase 2: one block per 256 groups of one layer (kind 0: output-channel groups, kind 1: input-channel groups)
+struct FinishJob { int layer, kind, start, pad; };
+
 __global__ void __launch_bounds__(kThreads) norms_finish_kernel(const LayerDev *__restrict__ layers,
+                                                                const FinishJob *__restrict__ jobs,
                                                                 const float *__restrict__ linesum,
                                                                 const float *__restrict__ colpart,
                                                                 float *__restrict__ inv_out, float *__restrict__ inv_in,
-                                                                double *__restrict__ layer_reg)
+                                                                double *__restrict__ job_reg)
 {
     __shared__ double s_red[kThreads];
-    const LayerDev L = layers[blockIdx.x];
-    const int TX = 1 << L.tx_log2;
-    const int nwx = TX >> 5;
-    const int passes = (L.C + TX * kMaxColsPerThread - 1) / (TX * kMaxColsPerThread);
-    const int per_line = passes * nwx;
+    const FinishJob J = jobs[blockIdx.x];
+    const LayerDev L = layers[J.layer];
+    const int per_line = L.n_cb;
     double reg = 0.0;
-    for (int k = threadIdx.x; k < L.K; k += kThreads) {
-        const float *p = linesum + L.line_off + (size_t)k * L.RS * per_line;
-        float s = 0.f;
-        for (int i = 0; i < L.RS * per_line; ++i) s += p[i];
-        L.sumsq_out[k] = s;
-        float inv = (L.reg_out && s > 1e-24f) ? rsqrtf(s) : 0.f;
-        inv_out[L.k_off + k] = inv;
-        if (L.reg_out) reg += (double)sqrtf(s);
-    }
-    for (int c = threadIdx.x; c < L.C; c += kThreads) {
-        const float *p = colpart + L.col_off + c;
-        float s = 0.f;
-        for (int i = 0; i < L.n_chunks; ++i) s += p[(size_t)i * L.C];
-        L.sumsq_in[c] = s;
-        float inv = (L.reg_in && s > 1e-24f) ? rsqrtf(s) : 0.f;
-        inv_in[L.c_off + c] = inv;
-        if (L.reg_in) reg += (double)sqrtf(s);
+    const int i = J.start + threadIdx.x;
+    if (J.kind == 0) {
+        if (i < L.K) {
+            const float *p = linesum + L.line_off + (size_t)i * L.RS * per_line;
+            float s = 0.f;
+#pragma unroll 8
+            for (int e = 0; e < L.RS * per_line; ++e) s += p[e];           // fixed order
+            L.sumsq_out[i] = s;
+            inv_out[L.k_off + i] = (L.reg_out && s > 1e-24f) ? rsqrtf(s) : 0.f;
+            if (L.reg_out) reg = (double)sqrtf(s);
+        }
+    } else {
+        if (i < L.C) {
+            const float *p = colpart + L.col_off + i;
+            float s = 0.f;
+#pragma unroll 8
+            for (int e = 0; e < L.n_lc; ++e) s += p[(size_t)e * L.C];        // fixed order
+            L.sumsq_in[i] = s;
+            inv_in[L.c_off + i] = (L.reg_in && s > 1e-24f) ? rsqrtf(s) : 0.f;
+            if (L.reg_in) reg = (double)sqrtf(s);
+        }
     }
     s_red[threadIdx.x] = reg;
     __syncthreads();
@@ -140,17 +150,18 @@ __global__ void __launch_bounds__(kThreads) norms_finish_kernel(const LayerDev *
         if (threadIdx.x < o) s_red[threadIdx.x] += s_red[threadIdx.x + o];
         __syncthreads();
     }
-    if (threadIdx.x == 0) layer_reg[blockIdx.x] = s_red[0];
+    if (threadIdx.x == 0) job_reg[blockIdx.x] = s_red[0];
 }
 
 // ---- phase 3
-__global__ void reg_total_kernel(const double *__restrict__ layer_reg, int n, double *__restrict__ out)
+__global__ void reg_total_kernel(const double *__restrict__ job_reg, int n, double *__restrict__ out)
 {
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        double s = 0.0;
-        for (int i = 0; i < n; ++i) s += layer_reg[i];
-        *out = s;
-    }
+    // 32 lanes take strided slices, then a fixed shuffle tree: the same order on every run
+    double s = 0.0;
+    for (int i = threadIdx.x; i < n; i += 32) s += job_reg[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (threadIdx.x == 0) *out = s;
 }
 
 // ---- phase 4
@@ -163,34 +174,32 @@ __global__ void __launch_bounds__(kThreads) update_kernel(const LayerDev *__rest
     const LayerDev L = layers[ch.layer];
     const int TX = 1 << L.tx_log2, TY = kThreads >> L.tx_log2;
     const int tx = threadIdx.x & (TX - 1), ty = threadIdx.x >> L.tx_log2;
+    const int c = ch.col0 + tx;
+    if (c >= L.C) return;
+    const float ci = inv_in[L.c_off + c];
     const float *io = inv_out + L.k_off;
-    const float *ii = inv_in + L.c_off;
-    const int passes = (L.C + TX * kMaxColsPerThread - 1) / (TX * kMaxColsPerThread);
-    for (int pass = 0; pass < passes; ++pass) {
-        const int cbase = pass * TX * kMaxColsPerThread + tx;
-        float ci[kMaxColsPerThread];
+    for (int l = ty; l < ch.nlines; l += kUnroll * TY) {
+        float w[kUnroll], g[kUnroll], v[kUnroll], ko[kUnroll];
 #pragma unroll
-        for (int j = 0; j < kMaxColsPerThread; ++j) {
-            int c = cbase + j * TX;
-            ci[j] = (c < L.C) ? ii[c] : 0.f;
+        for (int u = 0; u < kUnroll; ++u) {
+            const int line = ch.line0 + l + u * TY;
+            if (l + u * TY < ch.nlines) {
+                const size_t i = (size_t)line * L.C + c;
+                w[u] = L.w[i]; g[u] = L.g[i]; v[u] = L.v[i];
+                ko[u] = io[line / L.RS];
+            }
         }
-        for (int l = ty; l < ch.nlines; l += TY) {
-            const int line = ch.line0 + l;
-            const float ko = io[line / L.RS];
-            const size_t base = (size_t)line * L.C;
-            const size_t sbase = (size_t)line * L.ldw;
 #pragma unroll
-            for (int j = 0; j < kMaxColsPerThread; ++j) {
-                int c = cbase + j * TX;
-                if (c < L.C) {
-                    float w = L.w[base + c], g = L.g[base + c], v = L.v[base + c];
-                    float gt = g + hp.weight_decay * w + hp.lambda * w * (ko + ci[j]);
-                    float vn = hp.momentum * v + gt;
-                    float wn = w - hp.lr * vn;
-                    L.v[base + c] = vn;
-                    L.w[base + c] = wn;
-                    if (L.wb) L.wb[sbase + c] = __float2bfloat16_rn(wn);
-                }
+        for (int u = 0; u < kUnroll; ++u) {
+            const int line = ch.line0 + l + u * TY;
+            if (l + u * TY < ch.nlines) {
+                const size_t i = (size_t)line * L.C + c;
+                const float gt = g[u] + hp.weight_decay * w[u] + hp.lambda * w[u] * (ko[u] + ci);
+                const float vn = hp.momentum * v[u] + gt;
+                const float wn = w[u] - hp.lr * vn;
+                L.v[i] = vn;
+                L.w[i] = wn;
+                if (L.wb) L.wb[(size_t)line * L.ldw + c] = __float2bfloat16_rn(wn);
             }
         }
     }
@@ -205,38 +214,43 @@ __global__ void __launch_bounds__(kThreads) absmax_kernel(const LayerDev *__rest
     const int TX = 1 << L.tx_log2, TY = kThreads >> L.tx_log2;
     const int tx = threadIdx.x & (TX - 1), ty = threadIdx.x >> L.tx_log2;
     const int lane = threadIdx.x & 31;
+    __shared__ unsigned int s_line[kThreads];
     unsigned int *mk = maxbits + L.k_off + L.c_off;         // this layer's K entries, then its C entries
     unsigned int *mc = mk + L.K;
-    const int passes = (L.C + TX * kMaxColsPerThread - 1) / (TX * kMaxColsPerThread);
-    for (int pass = 0; pass < passes; ++pass) {
-        const int cbase = pass * TX * kMaxColsPerThread + tx;
-        unsigned int cm[kMaxColsPerThread];
+    const int wx = tx >> 5, nwx = TX >> 5;
+    const int c = ch.col0 + tx;
+    const bool cv = c < L.C;
+    const float *wbase = L.w + (size_t)ch.line0 * L.C + c;
+    unsigned int cm = 0u;
+    for (int l = ty; l < ch.nlines; l += kUnroll * TY) {
+        unsigned int b[kUnroll];
 #pragma unroll
-        for (int j = 0; j < kMaxColsPerThread; ++j) cm[j] = 0u;
-        for (int l = ty; l < ch.nlines; l += TY) {
-            const int line = ch.line0 + l;
-            const float *row = L.w + (size_t)line * L.C;
-            unsigned int rm = 0u;
-#pragma unroll
-            for (int j = 0; j < kMaxColsPerThread; ++j) {
-                int c = cbase + j * TX;
-                if (c < L.C) {
-                    // |w| as its bit pattern: ordered like the value for finite numbers, and any NaN sorts above +inf
-                    unsigned int bits = __float_as_uint(row[c]) & 0x7fffffffu;
-                    cm[j] = max(cm[j], bits);
-                    rm = max(rm, bits);
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) rm = max(rm, __shfl_xor_sync(0xffffffffu, rm, o));
-            if (lane == 0 && rm) atomicMax(&mk[line / L.RS], rm);
+        for (int u = 0; u < kUnroll; ++u) {
+            const int ll = l + u * TY;
+            // |w| as its bit pattern: ordered like the value for finite numbers, and any NaN sorts above +inf
+            b[u] = (cv && ll < ch.nlines) ? (__float_as_uint(wbase[(size_t)ll * L.C]) & 0x7fffffffu) : 0u;
         }
 #pragma unroll
-        for (int j = 0; j < kMaxColsPerThread; ++j) {
-            int c = cbase + j * TX;
-            if (c < L.C && cm[j]) atomicMax(&mc[c], cm[j]);
+        for (int u = 0; u < kUnroll; ++u) cm = max(cm, b[u]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) b[u] = max(b[u], __shfl_xor_sync(0xffffffffu, b[u], o));
+        if (lane == 0) {
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int ll = l + u * TY;
+                if (ll < ch.nlines) s_line[ll * nwx + wx] = b[u];
+            }
         }
     }
+    __syncthreads();
+    if ((int)threadIdx.x < ch.nlines) {
+        unsigned int m = 0u;
+        for (int x = 0; x < nwx; ++x) m = max(m, s_line[threadIdx.x * nwx + x]);
+        if (m) atomicMax(&mk[(ch.line0 + threadIdx.x) / L.RS], m);
+    }
+    if (cv && cm) atomicMax(&mc[c], cm);
 }
 
 __global__ void masks_kernel(const LayerDev *__restrict__ layers, const unsigned int *__restrict__ maxbits, float thr)
@@ -255,15 +269,15 @@ __global__ void __launch_bounds__(kThreads) zero_groups_kernel(const LayerDev *_
     const LayerDev L = layers[ch.layer];
     const int TX = 1 << L.tx_log2, TY = kThreads >> L.tx_log2;
     const int tx = threadIdx.x & (TX - 1), ty = threadIdx.x >> L.tx_log2;
+    const int c = ch.col0 + tx;
+    if (c >= L.C) return;
+    const bool zc = L.zero_in[c] != 0;
     for (int l = ty; l < ch.nlines; l += TY) {
         const int line = ch.line0 + l;
-        const bool zk = L.zero_out[line / L.RS] != 0;
-        for (int c = tx; c < L.C; c += TX) {
-            if (zk || L.zero_in[c]) {
-                L.w[(size_t)line * L.C + c] = 0.f;
-                L.v[(size_t)line * L.C + c] = 0.f;
-                if (L.wb) L.wb[(size_t)line * L.ldw + c] = __float2bfloat16_rn(0.f);
-            }
+        if (zc || L.zero_out[line / L.RS]) {
+            L.w[(size_t)line * L.C + c] = 0.f;
+            L.v[(size_t)line * L.C + c] = 0.f;
+            if (L.wb) L.wb[(size_t)line * L.ldw + c] = __float2bfloat16_rn(0.f);
         }
     }
 }
@@ -272,16 +286,17 @@ __global__ void __launch_bounds__(kThreads) zero_groups_kernel(const LayerDev *_
 struct Tables {
     std::vector<LayerDev> layers;
     std::vector<Chunk> chunks;
+    std::vector<FinishJob> jobs;
     WsLayout ws;
 };
 
-constexpr int kChunkElems = 32768;
 
 pt_status build_tables(const pt_layer *layers, int n, Tables *t)
 {
     if (!layers || n <= 0) return PT_ERR_INVALID_ARG;
     t->layers.resize(n);
     t->chunks.clear();
+    t->jobs.clear();
     long long line_off = 0, col_off = 0, k_off = 0, c_off = 0;
     for (int i = 0; i < n; ++i) {
         const pt_layer &s = layers[i];
@@ -299,21 +314,22 @@ pt_status build_tables(const pt_layer *layers, int n, Tables *t)
         d.pad_ = 0;
         const int TX = 1 << lg, TY = kThreads / TX;
         const int lines = s.K * s.RS;
-        int lines_per_chunk = kChunkElems / s.C;
-        if (lines_per_chunk < TY) lines_per_chunk = TY;
-        lines_per_chunk = pt_ceil_div(lines_per_chunk, TY) * TY;
-        d.chunk0 = (int)t->chunks.size();
-        d.n_chunks = pt_ceil_div(lines, lines_per_chunk);
-        for (int c = 0; c < d.n_chunks; ++c) {
-            Chunk ch;
-            ch.layer = i; ch.line0 = c * lines_per_chunk;
-            ch.nlines = lines - ch.line0 < lines_per_chunk ? lines - ch.line0 : lines_per_chunk;
-            ch.idx = c;
-            t->chunks.push_back(ch);
-        }
-        const int passes = pt_ceil_div(s.C, TX * kMaxColsPerThread);
-        d.line_off = line_off; line_off += (long long)lines * passes * (TX / 32);
-        d.col_off = col_off;   col_off += (long long)d.n_chunks * s.C;
+        // every chunk is TY*kUnroll*kSweeps lines x TX columns (8192 thread slots): equal trip counts, no long tail
+        const int lines_per_chunk = TY * kUnroll * kSweeps;
+        d.n_cb = pt_ceil_div(s.C, TX);
+        d.n_lc = pt_ceil_div(lines, lines_per_chunk);
+        for (int lc = 0; lc < d.n_lc; ++lc)
+            for (int cb = 0; cb < d.n_cb; ++cb) {
+                Chunk ch;
+                ch.layer = i; ch.line0 = lc * lines_per_chunk;
+                ch.nlines = lines - ch.line0 < lines_per_chunk ? lines - ch.line0 : lines_per_chunk;
+                ch.col0 = cb * TX; ch.lc = lc; ch.cb = cb; ch.pad0 = ch.pad1 = 0;
+                t->chunks.push_back(ch);
+            }
+        for (int k0 = 0; k0 < s.K; k0 += kThreads) t->jobs.push_back(FinishJob{i, 0, k0, 0});
+        for (int c0 = 0; c0 < s.C; c0 += kThreads) t->jobs.push_back(FinishJob{i, 1, c0, 0});
+        d.line_off = line_off; line_off += (long long)lines * d.n_cb;
+        d.col_off = col_off;   col_off += (long long)d.n_lc * s.C;
         d.k_off = k_off;       k_off += s.K;
         d.c_off = c_off;       c_off += s.C;
     }
@@ -323,24 +339,27 @@ pt_status build_tables(const pt_layer *layers, int n, Tables *t)
     w.colpart = o;   o = pt_align_up(o + (size_t)col_off * 4, 256);
     w.inv_out = o;   o = pt_align_up(o + (size_t)k_off * 4, 256);
     w.inv_in = o;    o = pt_align_up(o + (size_t)c_off * 4, 256);
-    w.layer_reg = o; o = pt_align_up(o + (size_t)n * 8, 256);
+    w.layer_reg = o; o = pt_align_up(o + t->jobs.size() * 8, 256);
     w.maxbits = o;   o = pt_align_up(o + (size_t)(k_off + c_off) * 4, 256);
     w.total = o;
     return PT_OK;
 }
 
 // Uploads [LayerDev * n][Chunk * m] and returns device pointers.
-pt_status upload(pt_ctx *c, const Tables &t, cudaStream_t st, const LayerDev **dl, const Chunk **dc)
+pt_status upload(pt_ctx *c, const Tables &t, cudaStream_t st, const LayerDev **dl, const Chunk **dc, const FinishJob **dj)
 {
-    size_t lb = pt_align_up(t.layers.size() * sizeof(LayerDev), 256), cb = t.chunks.size() * sizeof(Chunk);
-    std::vector<char> buf(lb + cb, 0);
+    size_t lb = pt_align_up(t.layers.size() * sizeof(LayerDev), 256), cb = pt_align_up(t.chunks.size() * sizeof(Chunk), 256);
+    size_t jb = t.jobs.size() * sizeof(FinishJob);
+    std::vector<char> buf(lb + cb + jb, 0);
     memcpy(buf.data(), t.layers.data(), t.layers.size() * sizeof(LayerDev));
-    memcpy(buf.data() + lb, t.chunks.data(), cb);
+    memcpy(buf.data() + lb, t.chunks.data(), t.chunks.size() * sizeof(Chunk));
+    memcpy(buf.data() + lb + cb, t.jobs.data(), jb);
     char *dev = nullptr;
     pt_status s = pt_upload_table(c, &c->lasso_tab, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
     *dl = (const LayerDev *)dev;
     *dc = (const Chunk *)(dev + lb);
+    *dj = (const FinishJob *)(dev + lb + cb);
     return PT_OK;
 }
 
@@ -365,8 +384,8 @@ extern "C" pt_status pt_group_lasso_sgd_step(pt_ctx *c, const pt_layer *layers, 
         if (!layers[i].g || !layers[i].sumsq_out || !layers[i].sumsq_in) return PT_ERR_INVALID_ARG;
     if (!ws || ws_bytes < t.ws.total || ((uintptr_t)ws & 255)) return PT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    const LayerDev *dl; const Chunk *dc;
-    s = upload(c, t, st, &dl, &dc);
+    const LayerDev *dl; const Chunk *dc; const FinishJob *dj;
+    s = upload(c, t, st, &dl, &dc, &dj);
     if (s != PT_OK) return s;
     char *b = (char *)ws;
     float *linesum = (float *)(b + t.ws.linesum), *colpart = (float *)(b + t.ws.colpart);
@@ -374,9 +393,10 @@ extern "C" pt_status pt_group_lasso_sgd_step(pt_ctx *c, const pt_layer *layers, 
     double *layer_reg = (double *)(b + t.ws.layer_reg);
     const unsigned nch = (unsigned)t.chunks.size();
     norms_partial_kernel<<<nch, kThreads, 0, st>>>(dl, dc, linesum, colpart);
-    norms_finish_kernel<<<n, kThreads, 0, st>>>(dl, linesum, colpart, inv_out, inv_in, layer_reg);
+    const int nj = (int)t.jobs.size();
+    norms_finish_kernel<<<nj, kThreads, 0, st>>>(dl, dj, linesum, colpart, inv_out, inv_in, layer_reg);
     c->launches += 2;
-    if (reg_sum_out) { reg_total_kernel<<<1, 32, 0, st>>>(layer_reg, n, reg_sum_out); c->launches += 1; }
+    if (reg_sum_out) { reg_total_kernel<<<1, 32, 0, st>>>(layer_reg, nj, reg_sum_out); c->launches += 1; }
     update_kernel<<<nch, kThreads, 0, st>>>(dl, dc, inv_out, inv_in, *hp);
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
@@ -394,8 +414,8 @@ extern "C" pt_status pt_find_zero_groups(pt_ctx *c, const pt_layer *layers, int3
         if (!layers[i].zero_out || !layers[i].zero_in) return PT_ERR_INVALID_ARG;
     if (!ws || ws_bytes < t.ws.total || ((uintptr_t)ws & 255)) return PT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    const LayerDev *dl; const Chunk *dc;
-    s = upload(c, t, st, &dl, &dc);
+    const LayerDev *dl; const Chunk *dc; const FinishJob *dj;
+    s = upload(c, t, st, &dl, &dc, &dj);
     if (s != PT_OK) return s;
     unsigned int *maxbits = (unsigned int *)((char *)ws + t.ws.maxbits);
     PT_CUDA_OK(cudaMemsetAsync(maxbits, 0, t.ws.total - t.ws.maxbits, st));

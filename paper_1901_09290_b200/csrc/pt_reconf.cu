@@ -67,7 +67,9 @@ struct GatherJob {
     int kind;                  // 0 = weight tensors, 1 = per-channel vector
     int pad_;
 };
-struct GatherChunk { int job, line0, nlines, pad_; };
+struct GatherChunk { int job, line0, nlines, col0; };
+
+constexpr int kGatherUnroll = 8;
 
 __global__ void __launch_bounds__(256) gather_kernel(const GatherJob *__restrict__ jobs, const GatherChunk *__restrict__ chunks)
 {
@@ -77,20 +79,37 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherJob *__restrict
         for (int k = ch.line0 + threadIdx.x; k < ch.line0 + ch.nlines; k += blockDim.x) J.nw[k] = J.ow[J.mapK[k]];
         return;
     }
-    // lines of the NEW tensor: (k', rs); threads run along c' so writes are coalesced
+    // Lines of the NEW tensor are (k', rs); a block covers a run of lines x up to 256 columns. Each thread owns one new
+    // column c' (its old column looked up once) and keeps four lines in flight; writes are coalesced, reads gathered.
     int TX = 32;
     while (TX < J.Cn && TX < 256) TX <<= 1;
     const int TY = 256 / TX, tx = threadIdx.x % TX, ty = threadIdx.x / TX;
-    for (int l = ty; l < ch.nlines; l += TY) {
-        const int line = ch.line0 + l;
-        const int kn = line / J.RS, rs = line - kn * J.RS;
-        const size_t oline = (size_t)J.mapK[kn] * J.RS + rs;
-        for (int c = tx; c < J.Cn; c += TX) {
-            const int co = J.mapC[c];
-            const size_t src = oline * J.Co + co, dst = (size_t)line * J.Cn + c;
-            J.nw[dst] = J.ow[src];
-            if (J.nv) J.nv[dst] = J.ov[src];
-            if (J.nwb) J.nwb[(size_t)line * J.ldwn + c] = J.owb[oline * J.ldwo + co];
+    const int c = ch.col0 + tx;
+    if (c >= J.Cn) return;
+    const int co = J.mapC[c];
+    for (int l = ty; l < ch.nlines; l += kGatherUnroll * TY) {
+        float w[kGatherUnroll], v[kGatherUnroll];
+        __nv_bfloat16 h[kGatherUnroll];
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int line = ch.line0 + l + u * TY;
+            if (l + u * TY < ch.nlines) {
+                const int kn = line / J.RS, rs = line - kn * J.RS;
+                const size_t oline = (size_t)J.mapK[kn] * J.RS + rs;
+                w[u] = J.ow[oline * J.Co + co];
+                if (J.nv) v[u] = J.ov[oline * J.Co + co];
+                if (J.nwb) h[u] = J.owb[oline * J.ldwo + co];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int line = ch.line0 + l + u * TY;
+            if (l + u * TY < ch.nlines) {
+                const size_t dst = (size_t)line * J.Cn + c;
+                J.nw[dst] = w[u];
+                if (J.nv) J.nv[dst] = v[u];
+                if (J.nwb) J.nwb[(size_t)line * J.ldwn + c] = h[u];
+            }
         }
     }
 }
@@ -191,9 +210,11 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         const int job = (int)jobs.size();
         jobs.push_back(J);
         const int lines = n.K * n.RS;
-        int per = 32768 / n.C;
-        if (per < 8) per = 8;
-        for (int l0 = 0; l0 < lines; l0 += per) chunks.push_back(GatherChunk{job, l0, lines - l0 < per ? lines - l0 : per, 0});
+        int TX = 32;
+        while (TX < n.C && TX < 256) TX <<= 1;
+        const int per = (256 / TX) * kGatherUnroll * 4;      // equal trip counts for every block
+        for (int l0 = 0; l0 < lines; l0 += per)
+            for (int c0 = 0; c0 < n.C; c0 += TX) chunks.push_back(GatherChunk{job, l0, lines - l0 < per ? lines - l0 : per, c0});
         for (int b = 0; b < 4; ++b) {
             if (!nl.bn[b]) continue;
             if (!ol.bn[b]) return PT_ERR_INVALID_ARG;
