@@ -23,7 +23,8 @@ namespace {
 constexpr int kBM = 128;            // output pixels per CTA tile
 constexpr int kKC = 64;             // reduction channels per stage (one 128-byte swizzle row)
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;           // wgrad kernel: 2 + 4 warps
+constexpr int kGemmThreads = 448;       // fwd/dgrad kernel: 2 + up to 12 epilogue warps
 constexpr int kMaxTaps = 64;
 
 struct GemmP {
@@ -44,6 +45,9 @@ struct GemmP {
     int ld_out, out_f32;
     int zero_mask;      // stride-2 dgrad: bit (a*2+b) set => also write zeros to the pixel at parity (a,b) of each 2x2 cell
     int tma_store;      // 1: bf16 output rows are consecutive pixels -> staged in shared memory and written by TMA stores
+    int m_tiles;        // ceil(M_total / 128)
+    int epi_groups;     // 1..3 groups of four epilogue warps
+    int a_tiled;        // 1: 1x1 stride-1 problem, the A operand is a plain 2-D (channels, pixels) tiled map
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
@@ -58,32 +62,49 @@ struct __align__(8) Ctl {
     int abort_flag;
 };
 
+// Control block of the persistent fwd/dgrad kernel.
+struct __align__(8) PCtl {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t acc_full[2];       // MMA issuer -> epilogue: accumulator buffer b holds a finished tile
+    uint64_t acc_empty[2];      // epilogue -> MMA issuer: buffer b has been read out (4 arrivals, one per epilogue warp)
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+constexpr uint32_t kSlabs = 2;                          // staging slabs per epilogue warp (TMA stores in flight)
+constexpr int kMaxEpiGroups = 3;                        // epilogue warp groups (4 warps each) working on different 64-channel chunks
+
+// Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... The TMA ring runs continuously across
+// tiles, the accumulator is double-buffered in TMEM, so the loads and MMAs of tile i+1 overlap the epilogue of tile i.
 template <bool B_MN>
-__global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                              const __grid_constant__ CUtensorMap tmB,
-                                                              const __grid_constant__ CUtensorMap tmC, const GemmP p)
+__global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                 const __grid_constant__ CUtensorMap tmB,
+                                                                 const __grid_constant__ CUtensorMap tmC, const GemmP p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw);
-    // stage buffers start at the first 1024-byte boundary after the control block
+    PCtl *ctl = reinterpret_cast<PCtl *>(smem_raw);
     const uint32_t smem_base = smem_u32(smem_raw);
-    const uint32_t data_base = (smem_base + (uint32_t)sizeof(Ctl) + 1023u) & ~1023u;
+    const uint32_t staging_base = (smem_base + (uint32_t)sizeof(PCtl) + 1023u) & ~1023u;
+    const uint32_t data_base = staging_base + (uint32_t)p.epi_groups * 4u * kSlabs * 4096u;
     const uint32_t a_bytes = kBM * kKC * 2;
     const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.BN * 128u;
     const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tile = blockIdx.x % p.n_tiles, m_tile = blockIdx.x / p.n_tiles;
-    const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
     const int iters = p.taps * p.k_chunks;
+    const int total_tiles = p.m_tiles * p.n_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
-        mbar_init(smem_u32(&ctl->accum), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), 4 * p.epi_groups);
+        }
         ctl->abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmA);
@@ -102,29 +123,33 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- TMA producer
-            const int q = m0 % p.Qd, t = m0 / p.Qd, pp = t % p.Pd, n = t / p.Pd;
-            const int w0 = q * p.stride + p.lo_w, h0 = pp * p.stride + p.lo_h;
-            int issued = 0;
-            for (int it = 0; it < iters; ++it) {
-                const int s = it % p.stages, ph = (it / p.stages) & 1;
-                if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 1)) break;
-                const int tap = it / p.k_chunks, kc = it - tap * p.k_chunks;
-                const uint32_t bar = smem_u32(&ctl->full[s]);
-                const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
-                mbar_arrive_expect_tx(bar, a_bytes + b_bytes);
-                tma_load_im2col_4d(a_dst, &tmA, bar, kc * kKC, w0, h0, n, (uint16_t)p.tap_ow[tap], (uint16_t)p.tap_oh[tap]);
-                const int wtap = p.tap_wt[tap];
-                if (!B_MN) {
-                    tma_load_3d(b_dst, &tmB, bar, kc * kKC, wtap, n0);
-                } else {
-                    for (int nb = 0; nb < (p.BN + 63) / 64; ++nb)
-                        tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
+            int g = 0;          // stage-ring position, continuous across tiles
+            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+                const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
+                const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
+                const int q = m0 % p.Qd, t = m0 / p.Qd, pp = t % p.Pd, n = t / p.Pd;
+                const int w0 = q * p.stride + p.lo_w, h0 = pp * p.stride + p.lo_h;
+                for (int it = 0; it < iters; ++it, ++g) {
+                    const int s = g % p.stages, ph = (g / p.stages) & 1;
+                    if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 1)) break;
+                    const int tap = it / p.k_chunks, kc = it - tap * p.k_chunks;
+                    const uint32_t bar = smem_u32(&ctl->full[s]);
+                    const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
+                    mbar_arrive_expect_tx(bar, a_bytes + b_bytes);
+                    if (p.a_tiled) tma_load_2d(a_dst, &tmA, bar, kc * kKC, m0);
+                    else tma_load_im2col_4d(a_dst, &tmA, bar, kc * kKC, w0, h0, n, (uint16_t)p.tap_ow[tap], (uint16_t)p.tap_oh[tap]);
+                    const int wtap = p.tap_wt[tap];
+                    if (!B_MN) {
+                        tma_load_3d(b_dst, &tmB, bar, kc * kKC, wtap, n0);
+                    } else {
+                        for (int nb = 0; nb < (p.BN + 63) / 64; ++nb)
+                            tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
+                    }
                 }
-                issued = it + 1;
             }
             if (*abort_flag) {
                 // drain: give the copies already issued a bounded time to land before the CTA's smem is released
-                for (int it = max(0, issued - p.stages); it < issued; ++it) {
+                for (int it = max(0, g - p.stages); it < g; ++it) {
                     const int s = it % p.stages, ph = (it / p.stages) & 1;
                     const uint64_t t0 = globaltimer_ns();
                     while (!mbar_try_wait(smem_u32(&ctl->full[s]), ph) && globaltimer_ns() - t0 < 20000000ull) {}
@@ -135,33 +160,101 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
         if (lane == 0) {
             // ---------------- MMA issuer
             const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
+            int g = 0, tc = 0;
             bool ok = true;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % p.stages, ph = (it / p.stages) & 1;
-                ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 2);
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tc) {
+                const int b = tc & 1, aph = (tc >> 1) & 1;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 7);
                 if (!ok) break;
                 tc_fence_after();
-                const int kc = it % p.k_chunks;
-                const int rem = p.c_red - kc * kKC;
-                const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
-                const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
+                const uint32_t d_tmem = tmem_base + (uint32_t)(b * p.BN);
+                for (int it = 0; it < iters; ++it, ++g) {
+                    const int s = g % p.stages, ph = (g / p.stages) & 1;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 2);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const int kc = it % p.k_chunks;
+                    const int rem = p.c_red - kc * kKC;
+                    const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
+                    const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
 #pragma unroll 1
-                for (int k = 0; k < ksteps; ++k) {
-                    const uint64_t ad = make_desc(a_src + (uint32_t)k * 32u, 16u, 1024u);
-                    const uint64_t bd = B_MN ? make_desc(b_src + (uint32_t)k * 2048u, 8192u, 1024u)
-                                             : make_desc(b_src + (uint32_t)k * 32u, 16u, 1024u);
-                    umma_bf16(tmem_base, ad, bd, idesc, (it | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < ksteps; ++k) {
+                        const uint64_t ad = make_desc(a_src + (uint32_t)k * 32u, 16u, 1024u);
+                        const uint64_t bd = B_MN ? make_desc(b_src + (uint32_t)k * 2048u, 8192u, 1024u)
+                                                 : make_desc(b_src + (uint32_t)k * 32u, 16u, 1024u);
+                        umma_bf16(d_tmem, ad, bd, idesc, (it | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&ctl->empty[s]));       // frees the stage when these MMAs have read it
                 }
-                umma_commit(smem_u32(&ctl->empty[s]));       // frees the stage when these MMAs have read it
+                if (ok) umma_commit(smem_u32(&ctl->acc_full[b])); // this tile's accumulator is complete
             }
-            if (ok) umma_commit(smem_u32(&ctl->accum));      // accumulator complete
         }
-    } else {
-        // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
-        const int quarter = warp & 3;
-        const bool ok = mbar_wait(smem_u32(&ctl->accum), 0, abort_flag, p.status, 3);
-        tc_fence_after();
-        if (ok) {
+    } else if (warp - 2 < 4 * p.epi_groups) {
+        // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; group = which 64-channel chunks it takes
+        const int quarter = warp & 3, group = (warp - 2) >> 2, G = p.epi_groups;
+        const uint32_t slab0 = staging_base + (uint32_t)(warp - 2) * (kSlabs * 4096u);
+        int tc = 0, sl = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tc) {
+            const int b = tc & 1, aph = (tc >> 1) & 1;
+            const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
+            const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
+            ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 3);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.BN);
+            if (p.tma_store) {
+                // Each warp stages its 32 rows x 64 channels (4 KB, 128-byte swizzle) and stores it with one TMA store,
+                // which drops the channels past the true count and the rows past the last pixel. Two slabs alternate.
+                const int n_chunks = (p.BN + 63) / 64;
+                if (group >= n_chunks) {       // nothing to read from this tile: hand the buffer back at once
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                    continue;
+                }
+                for (int ch = group; ch < n_chunks; ch += G, sl ^= 1) {
+                    const uint32_t slab = slab0 + (uint32_t)sl * 4096u;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the slab's previous store has read it
+                    __syncwarp();
+                    const int groups = min(4, (p.BN - ch * 64) / 16);
+                    uint32_t v[4][16];
+                    // all of the chunk's TMEM loads are issued before the single wait
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)
+                        if (g < groups) tmem_ld16(lane_addr + (uint32_t)(ch * 64 + g * 16), v[g]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (g >= groups) break;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 0]), __uint_as_float(v[g][8 * h + 1]));
+                            __nv_bfloat162 b1 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 2]), __uint_as_float(v[g][8 * h + 3]));
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 4]), __uint_as_float(v[g][8 * h + 5]));
+                            __nv_bfloat162 b3 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 6]), __uint_as_float(v[g][8 * h + 7]));
+                            const uint32_t j = (uint32_t)(g * 2 + h);
+                            const uint32_t addr = slab + (uint32_t)lane * 128u + ((j ^ ((uint32_t)lane & 7u)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t *>(&b0)),
+                                         "r"(*reinterpret_cast<uint32_t *>(&b1)), "r"(*reinterpret_cast<uint32_t *>(&b2)),
+                                         "r"(*reinterpret_cast<uint32_t *>(&b3))
+                                         : "memory");
+                        }
+                    }
+                    if (ch + G >= n_chunks) {
+                        // every TMEM read of this tile by this warp is done: hand the buffer back to the MMA issuer
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (m0 + quarter * 32 < p.M_total) tma_store_2d(&tmC, slab, n0 + ch * 64, m0 + quarter * 32);
+                        tma_store_commit();
+                    }
+                }
+                continue;
+            }
+            // ---- direct stores (fp32 outputs, strided stride-2 data-gradient outputs)
             const int m = m0 + quarter * 32 + lane;
             const bool row_ok = m < p.M_total;
             size_t row_off = 0;
@@ -173,46 +266,16 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
                 cell_w = j * p.o_step;
                 row_off = ((size_t)(img * p.oH + cell_h + p.o_h0) * p.oW + cell_w + p.o_w0) * (size_t)p.ld_out;
             }
-            const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-            if (p.tma_store) {
-                // All MMAs have completed, so the pipeline stages are free: they become the staging area.
-                // Each warp stages its 32 rows x 64 channels (4 KB, 128-byte swizzle) and stores it with one TMA
-                // store, which drops the channels past the true count and the rows past the last pixel.
-                const int n_chunks = (p.BN + 63) / 64;
-                for (int ch = 0; ch < n_chunks; ++ch) {
-                    const uint32_t slab = data_base + (uint32_t)(ch * 4 + quarter) * 4096u;
-                    const int groups = min(4, (p.BN - ch * 64) / 16);
-                    for (int g = 0; g < groups; ++g) {
-                        uint32_t v[16];
-                        tmem_ld16(lane_addr + (uint32_t)(ch * 64 + g * 16), v);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 0]), __uint_as_float(v[8 * h + 1]));
-                            __nv_bfloat162 b1 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 2]), __uint_as_float(v[8 * h + 3]));
-                            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 4]), __uint_as_float(v[8 * h + 5]));
-                            __nv_bfloat162 b3 = __floats2bfloat162_rn(__uint_as_float(v[8 * h + 6]), __uint_as_float(v[8 * h + 7]));
-                            const uint32_t j = (uint32_t)(g * 2 + h);
-                            const uint32_t addr = slab + (uint32_t)lane * 128u + ((j ^ ((uint32_t)lane & 7u)) << 4);
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t *>(&b0)),
-                                         "r"(*reinterpret_cast<uint32_t *>(&b1)), "r"(*reinterpret_cast<uint32_t *>(&b2)),
-                                         "r"(*reinterpret_cast<uint32_t *>(&b3))
-                                         : "memory");
-                        }
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0 && m0 + quarter * 32 < p.M_total) tma_store_2d(&tmC, slab, n0 + ch * 64, m0 + quarter * 32);
-                }
-                if (lane == 0) {
-                    tma_store_commit();
-                    tma_store_wait_read();
-                }
-            } else
-            for (int c0 = 0; c0 < p.BN; c0 += 16) {
+            if (group * 16 >= p.BN && lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+            for (int c0 = group * 16; c0 < p.BN; c0 += 16 * G) {
                 uint32_t v[16];
                 tmem_ld16(lane_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
+                if (c0 + 16 * G >= p.BN) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                }
                 const int col = n0 + c0;
                 if (!row_ok || col >= p.n_cols) continue;
                 const int nvalid = min(16, p.n_cols - col);
@@ -248,7 +311,7 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
                 }
             }
             // stride-2 data gradient: pixels of this 2x2 cell that no tap reaches are written as zeros here
-            if (row_ok && p.zero_mask && n_tile == 0) {
+            if (row_ok && p.zero_mask && n_tile == 0 && group == 0) {
                 for (int ab = 0; ab < 4; ++ab) {
                     if (!((p.zero_mask >> ab) & 1)) continue;
                     const int hh = cell_h + (ab >> 1), ww = cell_w + (ab & 1);
@@ -266,6 +329,7 @@ __global__ void __launch_bounds__(kThreads) conv_gemm_kernel(const __grid_consta
                 }
             }
         }
+        if (p.tma_store && lane == 0) tma_store_wait_read();     // the staging slabs must outlive the stores' reads
         tc_fence_before();
     }
     __syncthreads();
@@ -567,6 +631,21 @@ bool make_im2col_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, 
     return r == CUDA_SUCCESS;
 }
 
+// bf16 activations as a plain 2-D tensor (channels, pixels) with row pitch ld: box 64 channels x `pixels`.
+bool make_act2d_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, long long npix, int ld, int pixels)
+{
+    if (!c->encode_tiled) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)C, (cuuint64_t)npix};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kKC, (cuuint32_t)pixels}, estr[2] = {1, 1};
+    CUresult r = ((CUresult(*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill))c->encode_tiled)(
+        tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // bf16 weight shadow as (C, R*S, K) with row pitch ldw: box (64, 1, box_k).
 bool make_weight_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, int RS, int K, int ldw, int box_k)
 {
@@ -602,15 +681,14 @@ int pow2_cols(int bn)
     return c;
 }
 
-// Pipeline depth: two CTAs per SM when at least four stages fit in half of the shared memory, else one CTA with more.
-int pick_stages(size_t stage_bytes, int iters, size_t *smem)
+// Pipeline depth for a kernel that owns the SM: as many stages as fit beside `reserved` bytes, at most kMaxStages.
+int pick_stages(size_t stage_bytes, int iters, size_t reserved, size_t *smem)
 {
-    int st = (int)((110 * 1024 - 2048) / stage_bytes);
-    if (st < 4) st = (int)((220 * 1024 - 2048) / stage_bytes);
+    int st = (int)((220 * 1024 - 2048 - reserved) / stage_bytes);
     if (st > kMaxStages) st = kMaxStages;
-    if (st > iters) st = iters;
+    if (st > iters && iters >= 2) st = iters;
     if (st < 2) st = 2;
-    *smem = 2048 + (size_t)st * stage_bytes;
+    *smem = 2048 + reserved + (size_t)st * stage_bytes;
     return st;
 }
 
@@ -636,14 +714,22 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     const size_t a_bytes = kBM * kKC * 2;
     const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : pt_align_up((size_t)p.BN * 128, 1024);
     size_t smem = 0;
-    p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks, &smem);
+    p.m_tiles = pt_ceil_div(p.M_total, kBM);
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int per_cta = pt_ceil_div(total_tiles, c->sm_count);
+    p.epi_groups = pt_ceil_div(p.BN, 64) < kMaxEpiGroups ? pt_ceil_div(p.BN, 64) : kMaxEpiGroups;
+    if (!p.tma_store) p.epi_groups = kMaxEpiGroups;
+    const size_t staging = p.tma_store ? (size_t)p.epi_groups * 4 * kSlabs * 4096 : 0;
+    p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, (size_t)p.epi_groups * 4 * kSlabs * 4096, &smem);
+    (void)staging;
+    p.tmem_cols = pow2_cols(2 * p.BN);
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr_set[B_MN ? 1 : 0] = true;
     }
-    const int m_tiles = pt_ceil_div(p.M_total, kBM);
-    conv_gemm_kernel<B_MN><<<m_tiles * p.n_tiles, kThreads, smem, st>>>(tmA, tmB, tmC, p);
+    const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
+    conv_gemm_kernel<B_MN><<<grid, kGemmThreads, smem, st>>>(tmA, tmB, tmC, p);
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
@@ -699,7 +785,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     }
     size_t smem = 0;
     const size_t stage = 2 * 8192 + (size_t)pt_ceil_div(p.BN, 64) * 8192;
-    p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), &smem);
+    p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), 0, &smem);
     static bool attr_set = false;
     if (!attr_set) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
@@ -828,7 +914,10 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         p.tmem_cols = pow2_cols(p.BN);
         // the box of base positions must hold exactly P x Q positions at the traversal stride
         const int up_w = (Q - 1) * d->stride - d->pad - (d->W - 1), up_h = (P - 1) * d->stride - d->pad - (d->H - 1);
-        if (!make_im2col_map(c, &tmA, a, d->C, d->W, d->H, d->N, d->ldx, -d->pad, -d->pad, up_w, up_h, d->stride, kBM)) return PT_ERR_CUDA;
+        if (d->R == 1 && d->S == 1 && d->stride == 1 && d->pad == 0) {
+            p.a_tiled = 1;
+            if (!make_act2d_map(c, &tmA, a, d->C, (long long)d->N * d->H * d->W, d->ldx, kBM)) return PT_ERR_CUDA;
+        } else if (!make_im2col_map(c, &tmA, a, d->C, d->W, d->H, d->N, d->ldx, -d->pad, -d->pad, up_w, up_h, d->stride, kBM)) return PT_ERR_CUDA;
         if (!make_weight_map(c, &tmB, b, d->C, d->R * d->S, d->K, d->ldw, p.BN)) return PT_ERR_CUDA;
         return launch_gemm<false>(c, tmA, tmB, p, st);
     }
@@ -854,7 +943,10 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         p.Pd = d->H; p.Qd = d->W; p.stride = 1; p.lo_h = -ph; p.lo_w = -pw;
         p.o_step = 1; p.o_h0 = 0; p.o_w0 = 0; p.zero_mask = 0;
         const int up_w = (d->W - 1) - pw - (Q - 1), up_h = (d->H - 1) - ph - (P - 1);
-        if (!make_im2col_map(c, &tmA, a, d->K, Q, P, d->N, d->ldy, -pw, -ph, up_w, up_h, 1, kBM)) return PT_ERR_CUDA;
+        if (d->R == 1 && d->S == 1 && d->pad == 0) {
+            p.a_tiled = 1;
+            if (!make_act2d_map(c, &tmA, a, d->K, (long long)d->N * P * Q, d->ldy, kBM)) return PT_ERR_CUDA;
+        } else if (!make_im2col_map(c, &tmA, a, d->K, Q, P, d->N, d->ldy, -pw, -ph, up_w, up_h, 1, kBM)) return PT_ERR_CUDA;
         return launch_gemm<true>(c, tmA, tmB, p, st);
     }
     if (d->stride != 2) return PT_ERR_UNSUPPORTED;
