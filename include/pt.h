@@ -135,6 +135,23 @@ pt_status pt_group_lasso_sgd_step(pt_ctx *ctx, const pt_layer *layers /*host*/, 
 pt_status pt_find_zero_groups(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers, float threshold,
                               int32_t zero_in_place, void *ws, size_t ws_bytes, void *stream);
 
+/* Zero-group detection of ONE weight tensor w[K][RS][C] without any allocation and without a workspace (no counterpart in
+ * the paper: it exists for callers that may not allocate). It is for code that cannot call cudaMalloc: a host framework
+ * whose caching allocator owns the whole device heap, a latency-critical loop where an allocation's implicit device
+ * synchronisation is not acceptable, or a long-running service that must not meet an out-of-memory error in the middle
+ * of a reconfiguration. Such callers have no workspace to pass either. Same masks, bit for bit, as
+ * pt_find_zero_groups with zero_in_place = 0.
+ *   - The scratch is a 256 KiB static device array inside the library, present on every GPU that loads the library until the
+ *     process exits. Limit: K + C <= PT_NOALLOC_MAX_GROUPS, otherwise PT_ERR_UNSUPPORTED (use pt_find_zero_groups).
+ *   - Calls on one device share that array and it keeps the last call's contents; each call clears what it uses first.
+ *     Calls that overlap on the GPU (e.g. on two streams) race: serialise them.
+ *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress) with the caller's current device;
+ *     make that first call before any stream capture begins. It needs no pt_ctx.
+ * w, zero_out (K bytes), zero_in (C bytes): device pointers. */
+#define PT_NOALLOC_MAX_GROUPS 65536
+pt_status pt_find_zero_groups_noalloc(const float *w, int32_t K, int32_t C, int32_t RS, float threshold,
+                                      uint8_t *zero_out, uint8_t *zero_in, void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * Reconfiguration (Sec. 4.2: prune only the intersection of the sparsified channels of adjacent layers;
  * channel union across all convs that share a residual node; surviving training variables kept as is).

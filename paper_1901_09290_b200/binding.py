@@ -71,6 +71,7 @@ EXPORTS = {
     "pt_group_lasso_sgd_step": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, POINTER(pt_sgd_hparams), c_void_p,
                                           c_void_p, c_size_t, c_void_p]),
     "pt_find_zero_groups": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_float, c_int32, c_void_p, c_size_t, c_void_p]),
+    "pt_find_zero_groups_noalloc": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p]),
     "pt_reconfigure_plan": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(c_int32), c_void_p]),
     "pt_reconfigure": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(pt_graph), c_void_p]),
 }
@@ -196,6 +197,12 @@ def pt_find_zero_groups(ctx, layers, threshold=1e-4, zero_in_place=False, ws=Non
     p, n = _ws(ws)
     _check(lib().pt_find_zero_groups(ctx.handle, arr, len(arr), threshold, int(bool(zero_in_place)), p, n, _stream(stream)),
            "pt_find_zero_groups")
+
+
+def pt_find_zero_groups_noalloc(w, K, C, RS, threshold, zero_out, zero_in, stream=None):
+    """Detection of one weight tensor with the library's static scratch: for callers that cannot allocate a workspace."""
+    _check(lib().pt_find_zero_groups_noalloc(_ptr(w), K, C, RS, threshold, _ptr(zero_out), _ptr(zero_in), _stream(stream)),
+           "pt_find_zero_groups_noalloc")
 
 
 class GraphHandle:
