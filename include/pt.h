@@ -123,7 +123,9 @@ size_t pt_group_lasso_workspace_bytes(const pt_ctx *ctx, const pt_layer *layers 
  * That is the gradient of Eq. 1 with the regulariser of Eq. 2 (one global lambda; input- and output-channel
  * groups overlap) followed by the optimiser step of Algorithm 1. An all-zero group has subgradient 0.
  * reg_sum_out (device, optional): receives sum over regularised groups of sqrt(sumsq) -- Eq. 2 without lambda.
- * layers is a HOST array; the library keeps a device copy and re-uploads it only when it changes. */
+ * layers is a HOST array; the library keeps device copies of the last three distinct layer sets given to this call (two for
+ * pt_find_zero_groups) and uploads a table only when it is not among them. A CUDA graph captured around this call embeds
+ * the table's device address: it stays valid until three other layer sets have been used with the same context. */
 pt_status pt_group_lasso_sgd_step(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers,
                                   const pt_sgd_hparams *hp /*host*/, double *reg_sum_out,
                                   void *ws, size_t ws_bytes, void *stream);

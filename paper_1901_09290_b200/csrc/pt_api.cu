@@ -1,8 +1,8 @@
 // Context management, status handling, table upload and the conv entry points' dispatch.
 #include "pt_internal.h"
 
-static const size_t kArenaBytes = 4u << 20;     // 4 MiB of tables: three regions
-static const size_t kRegionBytes = kArenaBytes / 4;
+static const size_t kArenaBytes = 4u << 20;     // 4 MiB of tables
+static const size_t kSlotBytes = 512u << 10;    // eight slots of 512 KiB
 
 extern "C" const char *pt_status_string(pt_status s)
 {
@@ -40,9 +40,11 @@ extern "C" pt_status pt_create(pt_ctx **out, int device)
               cudaMallocHost(&c->h_counts, 65536 * sizeof(int32_t)) == cudaSuccess &&
               cudaEventCreateWithFlags(&c->upload_done, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); pt_destroy(c); return PT_ERR_CUDA; }
-    c->lasso_tab.off = 0;                 c->lasso_tab.cap = 2 * kRegionBytes;
-    c->graph_tab.off = 2 * kRegionBytes;  c->graph_tab.cap = kRegionBytes;
-    c->gather_tab.off = 3 * kRegionBytes; c->gather_tab.cap = kRegionBytes;
+    size_t off = 0;
+    for (int i = 0; i < 3; ++i) { c->lasso_tab[i].off = off; c->lasso_tab[i].cap = kSlotBytes; off += kSlotBytes; }
+    for (int i = 0; i < 2; ++i) { c->detect_tab[i].off = off; c->detect_tab[i].cap = kSlotBytes; off += kSlotBytes; }
+    c->graph_tab.off = off;  c->graph_tab.cap = kSlotBytes; off += kSlotBytes;
+    c->gather_tab.off = off; c->gather_tab.cap = 2 * kSlotBytes;
     // Driver entry points for tensor-map encoding, looked up at run time so the library loads without libcuda.
     cudaDriverEntryPointQueryResult qr;
     void *fn = nullptr;
@@ -104,6 +106,17 @@ pt_status pt_upload_table(pt_ctx *c, pt_region *reg, const void *host, size_t by
     reg->key.assign((const char *)host, (const char *)host + bytes);
     reg->valid = true;
     return PT_OK;
+}
+
+pt_status pt_upload_table_slots(pt_ctx *c, pt_region *slots, int n_slots, int *next, const void *host, size_t bytes,
+                                cudaStream_t st, char **dev)
+{
+    for (int i = 0; i < n_slots; ++i)
+        if (slots[i].valid && slots[i].key.size() == bytes && memcmp(slots[i].key.data(), host, bytes) == 0)
+            return pt_upload_table(c, &slots[i], host, bytes, st, dev);
+    pt_region *victim = &slots[*next % n_slots];
+    *next = (*next + 1) % n_slots;
+    return pt_upload_table(c, victim, host, bytes, st, dev);
 }
 
 // ------------------------------------------------------------------------------------------ conv dispatch

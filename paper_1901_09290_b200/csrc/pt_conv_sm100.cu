@@ -66,8 +66,8 @@ struct __align__(8) Ctl {
 struct __align__(8) PCtl {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    uint64_t acc_full[2];       // MMA issuer -> epilogue: accumulator buffer b holds a finished tile
-    uint64_t acc_empty[2];      // epilogue -> MMA issuer: buffer b has been read out (4 arrivals, one per epilogue warp)
+    uint64_t acc_full[3];       // MMA issuer -> epilogue: accumulator buffer b holds a finished tile
+    uint64_t acc_empty[3];      // epilogue -> MMA issuer: buffer b has been read out (4 arrivals, one per warp of its group)
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -76,7 +76,8 @@ constexpr uint32_t kSlabs = 2;                          // staging slabs per epi
 constexpr int kMaxEpiGroups = 3;                        // epilogue warp groups (4 warps each) working on different 64-channel chunks
 
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... The TMA ring runs continuously across
-// tiles, the accumulator is double-buffered in TMEM, so the loads and MMAs of tile i+1 overlap the epilogue of tile i.
+// tiles. The accumulator has G = 2 or 3 buffers in TMEM and buffer b has its own group of four epilogue warps, so the
+// loads and MMAs of the next tiles overlap the epilogues of the previous ones.
 template <bool B_MN>
 __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                  const __grid_constant__ CUtensorMap tmB,
@@ -101,9 +102,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             mbar_init(smem_u32(&ctl->full[s]), 1);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < p.epi_groups; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
-            mbar_init(smem_u32(&ctl->acc_empty[b]), 4 * p.epi_groups);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
         }
         ctl->abort_flag = 0;
         fence_mbar_init();
@@ -163,7 +164,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             int g = 0, tc = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tc) {
-                const int b = tc & 1, aph = (tc >> 1) & 1;
+                const int b = tc % p.epi_groups, aph = (tc / p.epi_groups) & 1;
                 ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 7);
                 if (!ok) break;
                 tc_fence_after();
@@ -190,13 +191,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             }
         }
     } else if (warp - 2 < 4 * p.epi_groups) {
-        // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; group = which 64-channel chunks it takes
+        // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; group g drains accumulator buffer g,
+        // i.e. the tiles tc = g, g + G, g + 2G, ... of this CTA
         const int quarter = warp & 3, group = (warp - 2) >> 2, G = p.epi_groups;
         const uint32_t slab0 = staging_base + (uint32_t)(warp - 2) * (kSlabs * 4096u);
-        int tc = 0, sl = 0;
+        int tc = group, sl = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tc) {
-            const int b = tc & 1, aph = (tc >> 1) & 1;
+        for (int tile = blockIdx.x + group * gridDim.x; tile < total_tiles && ok; tile += G * gridDim.x, tc += G) {
+            const int b = group, aph = (tc / G) & 1;
             const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
             const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
             ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 3);
@@ -207,11 +209,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                 // Each warp stages its 32 rows x 64 channels (4 KB, 128-byte swizzle) and stores it with one TMA store,
                 // which drops the channels past the true count and the rows past the last pixel. Two slabs alternate.
                 const int n_chunks = (p.BN + 63) / 64;
-                if (group >= n_chunks) {       // nothing to read from this tile: hand the buffer back at once
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
-                    continue;
-                }
-                for (int ch = group; ch < n_chunks; ch += G, sl ^= 1) {
+                for (int ch = 0; ch < n_chunks; ++ch, sl ^= 1) {
                     const uint32_t slab = slab0 + (uint32_t)sl * 4096u;
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the slab's previous store has read it
                     __syncwarp();
@@ -239,7 +237,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                                          : "memory");
                         }
                     }
-                    if (ch + G >= n_chunks) {
+                    if (ch + 1 >= n_chunks) {
                         // every TMEM read of this tile by this warp is done: hand the buffer back to the MMA issuer
                         tc_fence_before();
                         __syncwarp();
@@ -266,12 +264,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                 cell_w = j * p.o_step;
                 row_off = ((size_t)(img * p.oH + cell_h + p.o_h0) * p.oW + cell_w + p.o_w0) * (size_t)p.ld_out;
             }
-            if (group * 16 >= p.BN && lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
-            for (int c0 = group * 16; c0 < p.BN; c0 += 16 * G) {
+            for (int c0 = 0; c0 < p.BN; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld16(lane_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
-                if (c0 + 16 * G >= p.BN) {
+                if (c0 + 16 >= p.BN) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
@@ -311,7 +308,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                 }
             }
             // stride-2 data gradient: pixels of this 2x2 cell that no tap reaches are written as zeros here
-            if (row_ok && p.zero_mask && n_tile == 0 && group == 0) {
+            if (row_ok && p.zero_mask && n_tile == 0) {
                 for (int ab = 0; ab < 4; ++ab) {
                     if (!((p.zero_mask >> ab) & 1)) continue;
                     const int hh = cell_h + (ab >> 1), ww = cell_w + (ab & 1);
@@ -415,9 +412,12 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 const int q = pix % p.Qd, t = pix / p.Qd, pp = t % p.Pd, n = t / p.Pd;
                 const uint32_t bar = smem_u32(&ctl->full[s]);
                 const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
-                mbar_arrive_expect_tx(bar, a_bytes + b_bytes);
+                // output channels k0+64.. of this tile do not exist when K - k0 <= 64: their accumulator rows are never
+                // stored, so that half of the A tile is not loaded at all (the MMA reads stale shared memory there)
+                const bool second = p.K - k0 > 64;
+                mbar_arrive_expect_tx(bar, (second ? a_bytes : 8192u) + b_bytes);
                 tma_load_2d(a_dst, &tmDy, bar, k0, pix);
-                tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
+                if (second) tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
                 for (uint32_t nb = 0; nb < nb_b; ++nb)
                     tma_load_im2col_4d(b_dst + nb * 8192u, &tmX, bar, c0 + (int)nb * 64, q * p.stride + p.lo_w,
                                        pp * p.stride + p.lo_h, n, (uint16_t)sft, (uint16_t)r);
@@ -662,8 +662,9 @@ bool make_weight_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, 
 
 // Tile width along the output channels. One tile: the ragged count rounded up to 16. Several tiles: a multiple of
 // 64 (the TMA-store chunk) chosen to waste the fewest padded columns.
-int tile_n(int cols, int *n_tiles)
+int tile_n(int cols, int *n_tiles, int m_tiles = 1 << 30, int sms = 0)
 {
+    (void)m_tiles; (void)sms;
     if (cols <= 256) { *n_tiles = 1; return pt_ceil_div(cols, 16) * 16; }
     int best = 256, best_pad = 1 << 30;
     for (int bn = 256; bn >= 128; bn -= 64) {
@@ -717,12 +718,12 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     p.m_tiles = pt_ceil_div(p.M_total, kBM);
     const int total_tiles = p.m_tiles * p.n_tiles;
     const int per_cta = pt_ceil_div(total_tiles, c->sm_count);
-    p.epi_groups = pt_ceil_div(p.BN, 64) < kMaxEpiGroups ? pt_ceil_div(p.BN, 64) : kMaxEpiGroups;
-    if (!p.tma_store) p.epi_groups = kMaxEpiGroups;
-    const size_t staging = p.tma_store ? (size_t)p.epi_groups * 4 * kSlabs * 4096 : 0;
+    // accumulator buffers = epilogue groups: three when 3 * BN fits the 512 TMEM columns, else two; narrow layers whose
+    // CTAs get a single tile need no more than that
+    p.epi_groups = 3 * p.BN <= 512 ? 3 : 2;
+    if (per_cta < p.epi_groups) p.epi_groups = per_cta < 2 ? 2 : per_cta;
     p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, (size_t)p.epi_groups * 4 * kSlabs * 4096, &smem);
-    (void)staging;
-    p.tmem_cols = pow2_cols(2 * p.BN);
+    p.tmem_cols = pow2_cols(p.epi_groups * p.BN);
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
@@ -741,7 +742,7 @@ int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     tile_n(d->C, &n_tiles);
     const int tiles = pt_ceil_div(d->K, 128) * n_tiles * d->R * d->S;
     const long long npix = (long long)d->N * P * Q;
-    long long s = pt_ceil_div(2 * c->sm_count, tiles);
+    long long s = c->sm_count / tiles;                     // one CTA per SM, one wave
     const long long max_s = (npix + 255) / 256;          // at least four 64-pixel stages per split
     if (s > max_s) s = max_s;
     if (s < 1) s = 1;
@@ -904,7 +905,7 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         // raster = output pixels (P x Q per image); source = x
         p.M_total = d->N * P * Q;
         p.n_cols = d->K;
-        p.BN = tile_n(d->K, &p.n_tiles);
+        p.BN = tile_n(d->K, &p.n_tiles, pt_ceil_div(p.M_total, kBM), c->sm_count);
         p.c_red = d->C;
         p.k_chunks = pt_ceil_div(d->C, kKC);
         p.taps = d->R * d->S;
@@ -923,7 +924,7 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
     }
     if (which != PT_CONV_DGRAD) return PT_ERR_UNSUPPORTED;
     p.n_cols = d->C;
-    p.BN = tile_n(d->C, &p.n_tiles);
+    p.BN = tile_n(d->C, &p.n_tiles, pt_ceil_div(d->N * d->H * d->W / (d->stride * d->stride), kBM), c->sm_count);
     p.c_red = d->K;
     p.k_chunks = pt_ceil_div(d->K, kKC);
     p.tmem_cols = pow2_cols(p.BN);

@@ -36,7 +36,10 @@ struct pt_ctx {
     size_t arena_bytes = 0;
     cudaEvent_t upload_done = nullptr;  // last staging->arena copy
     bool upload_pending = false;
-    pt_region lasso_tab, graph_tab, gather_tab;
+    // Cached device tables. A captured CUDA graph embeds the device address of the table its kernels read, so tables of
+    // different callers must not evict each other: the lasso step and the detection have their own slot sets.
+    pt_region lasso_tab[3], detect_tab[2], graph_tab, gather_tab;
+    int lasso_next = 0, detect_next = 0;
     int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan
     uint64_t launches = 0;
     // tcgen05 conv path
@@ -55,6 +58,9 @@ static inline int pt_out_dim(int H, int R, int stride, int pad) {
 // Copies `bytes` of host data into the region's slot of the arena if it differs from what is there.
 // Returns the device address of the slot.
 pt_status pt_upload_table(pt_ctx *ctx, pt_region *reg, const void *host, size_t bytes, cudaStream_t st, char **dev);
+// Same over a set of slots: a slot already holding these bytes is reused, otherwise the oldest one is overwritten.
+pt_status pt_upload_table_slots(pt_ctx *ctx, pt_region *slots, int n_slots, int *next, const void *host, size_t bytes,
+                                cudaStream_t st, char **dev);
 
 // Validation shared by the conv entry points. Fills P, Q.
 pt_status pt_conv_validate(const pt_ctx *ctx, const pt_conv_desc *d, int *P, int *Q);

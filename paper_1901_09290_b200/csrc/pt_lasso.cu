@@ -346,7 +346,8 @@ pt_status build_tables(const pt_layer *layers, int n, Tables *t)
 }
 
 // Uploads [LayerDev * n][Chunk * m] and returns device pointers.
-pt_status upload(pt_ctx *c, const Tables &t, cudaStream_t st, const LayerDev **dl, const Chunk **dc, const FinishJob **dj)
+pt_status upload(pt_ctx *c, const Tables &t, bool detect, cudaStream_t st, const LayerDev **dl, const Chunk **dc,
+                 const FinishJob **dj)
 {
     size_t lb = pt_align_up(t.layers.size() * sizeof(LayerDev), 256), cb = pt_align_up(t.chunks.size() * sizeof(Chunk), 256);
     size_t jb = t.jobs.size() * sizeof(FinishJob);
@@ -355,7 +356,8 @@ pt_status upload(pt_ctx *c, const Tables &t, cudaStream_t st, const LayerDev **d
     memcpy(buf.data() + lb, t.chunks.data(), t.chunks.size() * sizeof(Chunk));
     memcpy(buf.data() + lb + cb, t.jobs.data(), jb);
     char *dev = nullptr;
-    pt_status s = pt_upload_table(c, &c->lasso_tab, buf.data(), buf.size(), st, &dev);
+    pt_status s = detect ? pt_upload_table_slots(c, c->detect_tab, 2, &c->detect_next, buf.data(), buf.size(), st, &dev)
+                         : pt_upload_table_slots(c, c->lasso_tab, 3, &c->lasso_next, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
     *dl = (const LayerDev *)dev;
     *dc = (const Chunk *)(dev + lb);
@@ -385,7 +387,7 @@ extern "C" pt_status pt_group_lasso_sgd_step(pt_ctx *c, const pt_layer *layers, 
     if (!ws || ws_bytes < t.ws.total || ((uintptr_t)ws & 255)) return PT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     const LayerDev *dl; const Chunk *dc; const FinishJob *dj;
-    s = upload(c, t, st, &dl, &dc, &dj);
+    s = upload(c, t, false, st, &dl, &dc, &dj);
     if (s != PT_OK) return s;
     char *b = (char *)ws;
     float *linesum = (float *)(b + t.ws.linesum), *colpart = (float *)(b + t.ws.colpart);
@@ -415,7 +417,7 @@ extern "C" pt_status pt_find_zero_groups(pt_ctx *c, const pt_layer *layers, int3
     if (!ws || ws_bytes < t.ws.total || ((uintptr_t)ws & 255)) return PT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     const LayerDev *dl; const Chunk *dc; const FinishJob *dj;
-    s = upload(c, t, st, &dl, &dc, &dj);
+    s = upload(c, t, true, st, &dl, &dc, &dj);
     if (s != PT_OK) return s;
     unsigned int *maxbits = (unsigned int *)((char *)ws + t.ws.maxbits);
     PT_CUDA_OK(cudaMemsetAsync(maxbits, 0, t.ws.total - t.ws.maxbits, st));

@@ -87,7 +87,7 @@ class TrainStep:
         gen = torch.Generator(device="cuda").manual_seed(seed + 99) if device_rng else None
         ws_bytes = 16
         for li, l in enumerate(self.net.layers):
-            ldx, ldy = W.pad8(l.C), W.pad8(l.K)
+            ldx, ldy = (8 if l.C <= 4 else W.pad16(l.C)), W.pad16(l.K)
             P = l.P
             d = B.make_conv_desc(N, l.H, l.H, l.C, l.K, l.R, l.R, l.stride, l.pad, ldx, ldy, W.pad8(l.C), 0, algo)
             self.desc.append(d)
@@ -178,9 +178,42 @@ class TrainStep:
             self.conv_wgrad(li, stream)
         self.lasso(stream)
 
+    def train_two_streams(self):
+        """The same launches with each layer's data gradient and weight gradient on two streams: they only share their
+        input dy_l, so they may overlap (the weight gradients use the workspace, the data gradients do not)."""
+        main = torch.cuda.current_stream()
+        side = self._side
+        n = len(self.net.layers)
+        for li in range(n):
+            self.conv_fwd(li, main)
+        side.wait_stream(main)
+        for li in range(n - 1, -1, -1):
+            if li > 0:
+                self.conv_dgrad(li, main)
+            self.conv_wgrad(li, side)
+        main.wait_stream(side)
+        self.lasso(main)
+
+    def build_graph(self, two_streams: bool = True):
+        """Captures the training part of the step (every launch after the reconfiguration's host sync) into a CUDA graph.
+        Call after at least one eager step, so that every table and kernel attribute is already set up."""
+        self._side = torch.cuda.Stream()
+        l0 = self.ctx.launch_count()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            if two_streams:
+                self.train_two_streams()
+            else:
+                self.train()
+        self.graph_launches = self.ctx.launch_count() - l0
+        return self.graph
+
     def step(self, stream=None):
         self.reconfigure(stream)
-        self.train(stream)
+        if getattr(self, "graph", None) is not None:
+            self.graph.replay()
+        else:
+            self.train(stream)
 
     def step_e2e(self, stream=None):
         """The same step with the image batch copied from pinned host memory and the regulariser value read back."""

@@ -25,6 +25,7 @@ def main():
     ap.add_argument("--sets", type=int, default=4, help="rotating buffer sets (footprint larger than L2)")
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--algo", type=int, default=0)
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches (includes host launch cost)")
     args = ap.parse_args()
     if args.shape:
         N, H, C, K, R, stride = [int(t) for t in args.shape.split(",")]
@@ -38,7 +39,7 @@ def main():
     pad = R // 2
     P = (H + 2 * pad - R) // stride + 1
     ctx = B.Context(0)
-    d = B.make_conv_desc(N, H, H, C, K, R, R, stride, pad, algo=args.algo)
+    d = B.make_conv_desc(N, H, H, C, K, R, R, stride, pad, 8 if C <= 4 else W.pad16(C), W.pad16(K), algo=args.algo)
     g = torch.Generator(device="cuda").manual_seed(1)
     sets = []
     for _ in range(args.sets):
@@ -63,10 +64,22 @@ def main():
             run(i)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for i in range(args.iters):
-            run(i)
-        e1.record()
+        if args.no_graph:
+            e0.record()
+            for i in range(args.iters):
+                run(i)
+            e1.record()
+        else:
+            # the launches are captured once and replayed, so the device time is not hidden behind host launch cost
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(args.iters):
+                    run(i)
+            g.replay()
+            torch.cuda.synchronize()
+            e0.record()
+            g.replay()
+            e1.record()
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) * 1e3 / args.iters
         by = act + K * C * R * R * (4 if ps == "wgrad" else 2)
