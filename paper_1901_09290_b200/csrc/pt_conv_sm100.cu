@@ -178,13 +178,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     const int rem = p.c_red - kc * kKC;
                     const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
                     const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
-#pragma unroll 1
-                    for (int k = 0; k < ksteps; ++k) {
-                        const uint64_t ad = make_desc(a_src + (uint32_t)k * 32u, 16u, 1024u);
-                        const uint64_t bd = B_MN ? make_desc(b_src + (uint32_t)k * 2048u, 8192u, 1024u)
-                                                 : make_desc(b_src + (uint32_t)k * 32u, 16u, 1024u);
-                        umma_bf16(d_tmem, ad, bd, idesc, (it | k) != 0 ? 1u : 0u);
-                    }
+                    // one descriptor per operand and stage; a k-step only moves the 14-bit start-address field
+                    // (units of 16 bytes): +32 B inside a K-major row, +2048 B (16 rows) in an MN-major tile
+                    const uint64_t ad0 = make_desc(a_src, 16u, 1024u);
+                    const uint64_t bd0 = B_MN ? make_desc(b_src, 8192u, 1024u) : make_desc(b_src, 16u, 1024u);
+                    const uint64_t bstep = B_MN ? 128ull : 2ull;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (k < ksteps) umma_bf16(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, (it | k) != 0 ? 1u : 0u);
                     umma_commit(smem_u32(&ctl->empty[s]));       // frees the stage when these MMAs have read it
                 }
                 if (ok) umma_commit(smem_u32(&ctl->acc_full[b])); // this tile's accumulator is complete
@@ -336,6 +337,277 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     }
 }
 
+// ------------------------------------------------------------------------------------------ halo kernel (RxS, stride 1)
+// For a stride-1 RxS filter the per-tap im2col loads fetch every input pixel R*S times. Here each input pixel row is
+// fetched ONCE per 64-channel chunk: a tile is `nr` output rows of one image, laid out as a raster of pitch
+// Wp = Q + S - 1 (the S - 1 extra columns per row are garbage outputs that are never stored). One tiled 4-D TMA load
+// brings the (nr + R - 1) x Wp input positions of the tile, halo included, zero-filled outside the image. In that
+// raster the input position of output position m for tap (r, s) is m + r*Wp + s, a constant row shift, and the
+// 128-byte swizzle is a function of the absolute shared-memory address, so tap (r, s) is simply the same A tile read
+// through a descriptor whose start address is (r*Wp + s) rows further on. Weights: if all taps x chunks of the CTA's
+// channel tile fit in shared memory they are loaded once and stay resident; otherwise they stream through a ring.
+struct HaloP {
+    int N, P, Q, Wp, nr, row_tiles;      // images, output rows/cols, raster pitch, output rows per tile, tiles per image
+    int n_cols, BN, n_tiles;
+    int c_red, k_chunks, taps;
+    int lo_h, lo_w;                      // source coordinate of raster position (0, 0) for tap offset (0, 0)
+    int a_box_bytes, a_alloc;            // bytes one A load brings / bytes reserved per A stage
+    int stages_a, stages_b, resident;    // ring depths; resident: weights loaded once
+    int tmem_cols, tma_store, out_f32, ld_out;
+    void *out;
+    unsigned int *status;
+    unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];
+    unsigned short tap_wt[kMaxTaps];
+};
+
+struct __align__(8) HCtl {
+    uint64_t full_a[4], empty_a[4];
+    uint64_t full_b[kMaxStages], empty_b[kMaxStages];
+    uint64_t w_full;
+    uint64_t acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+constexpr int kHaloThreads = 320;        // producer warp, MMA warp, two groups of four epilogue warps
+constexpr uint32_t kHaloStaging = 2u * 16384u;
+
+template <bool B_MN>
+__global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                     const __grid_constant__ CUtensorMap tmB,
+                                                                     const __grid_constant__ CUtensorMap tmC, const HaloP p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    HCtl *ctl = reinterpret_cast<HCtl *>(smem_raw);
+    const uint32_t smem_base = smem_u32(smem_raw);
+    const uint32_t staging_base = (smem_base + (uint32_t)sizeof(HCtl) + 1023u) & ~1023u;
+    const uint32_t b_base = staging_base + kHaloStaging;
+    const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.BN * 128u;
+    const uint32_t b_slot = (b_bytes + 1023u) & ~1023u;
+    const uint32_t n_bslots = p.resident ? (uint32_t)(p.taps * p.k_chunks) : (uint32_t)p.stages_b;
+    const uint32_t a_base = b_base + n_bslots * b_slot;
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m_tiles = p.N * p.row_tiles;
+    const int total_tiles = m_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages_a; ++s) { mbar_init(smem_u32(&ctl->full_a[s]), 1); mbar_init(smem_u32(&ctl->empty_a[s]), 1); }
+        for (int s = 0; s < p.stages_b; ++s) { mbar_init(smem_u32(&ctl->full_b[s]), 1); mbar_init(smem_u32(&ctl->empty_b[s]), 1); }
+        mbar_init(smem_u32(&ctl->w_full), 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 4); }
+        ctl->abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+        if (p.tma_store) prefetch_tmap(&tmC);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- TMA producer
+            if (p.resident) {
+                // n_tiles == 1 here: the whole weight tensor of the layer, tap by tap and chunk by chunk, once
+                const uint32_t bar = smem_u32(&ctl->w_full);
+                mbar_arrive_expect_tx(bar, (uint32_t)(p.taps * p.k_chunks) * b_bytes);
+                for (int tap = 0; tap < p.taps; ++tap)
+                    for (int kc = 0; kc < p.k_chunks; ++kc) {
+                        const uint32_t dst = b_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot;
+                        const int wtap = p.tap_wt[tap];
+                        if (!B_MN) tma_load_3d(dst, &tmB, bar, kc * kKC, wtap, 0);
+                        else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
+                    }
+            }
+            int ga = 0, gb = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+                const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
+                const int img = m_tile / p.row_tiles, p0 = (m_tile - img * p.row_tiles) * p.nr;
+                const int n0 = n_tile * p.BN;
+                bool ok = true;
+                for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++ga) {
+                    const int sa = ga % p.stages_a, pha = (ga / p.stages_a) & 1;
+                    ok = mbar_wait(smem_u32(&ctl->empty_a[sa]), pha ^ 1, abort_flag, p.status, 11);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&ctl->full_a[sa]);
+                    mbar_arrive_expect_tx(bar, (uint32_t)p.a_box_bytes);
+                    tma_load_4d(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, &tmA, bar, kc * kKC, p.lo_w, p0 + p.lo_h, img);
+                    if (p.resident) continue;
+                    for (int tap = 0; tap < p.taps; ++tap, ++gb) {
+                        const int sb = gb % p.stages_b, phb = (gb / p.stages_b) & 1;
+                        ok = mbar_wait(smem_u32(&ctl->empty_b[sb]), phb ^ 1, abort_flag, p.status, 12);
+                        if (!ok) break;
+                        const uint32_t bbar = smem_u32(&ctl->full_b[sb]);
+                        const uint32_t dst = b_base + (uint32_t)sb * b_slot;
+                        const int wtap = p.tap_wt[tap];
+                        mbar_arrive_expect_tx(bbar, b_bytes);
+                        if (!B_MN) tma_load_3d(dst, &tmB, bbar, kc * kKC, wtap, n0);
+                        else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bbar, n0 + nb * 64, wtap, kc * kKC);
+                    }
+                }
+                if (!ok) break;
+            }
+            if (*abort_flag) {       // bounded drain of the copies in flight before the shared memory is released
+                const uint64_t t0 = globaltimer_ns();
+                for (int s = 0; s < p.stages_a; ++s)
+                    while (!mbar_try_wait(smem_u32(&ctl->full_a[s]), 0) && !mbar_try_wait(smem_u32(&ctl->full_a[s]), 1) &&
+                           globaltimer_ns() - t0 < 20000000ull) {}
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer
+            const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
+            int ga = 0, gb = 0, tc = 0;
+            bool ok = true;
+            if (p.resident) ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort_flag, p.status, 13);
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tc) {
+                const int b = tc & 1, aph = (tc >> 1) & 1;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 14);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(b * p.BN);
+                for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++ga) {
+                    const int sa = ga % p.stages_a, pha = (ga / p.stages_a) & 1;
+                    ok = mbar_wait(smem_u32(&ctl->full_a[sa]), pha, abort_flag, p.status, 15);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const int rem = p.c_red - kc * kKC;
+                    const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
+                    const uint32_t a_src = a_base + (uint32_t)sa * (uint32_t)p.a_alloc;
+                    for (int tap = 0; tap < p.taps; ++tap) {
+                        uint32_t b_src;
+                        int sb = 0;
+                        if (p.resident) {
+                            b_src = b_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot;
+                        } else {
+                            sb = gb % p.stages_b;
+                            const int phb = (gb / p.stages_b) & 1;
+                            ++gb;
+                            ok = mbar_wait(smem_u32(&ctl->full_b[sb]), phb, abort_flag, p.status, 16);
+                            if (!ok) break;
+                            tc_fence_after();
+                            b_src = b_base + (uint32_t)sb * b_slot;
+                        }
+                        // the tap is a row shift of the same A tile
+                        const uint32_t a_tap = a_src + (uint32_t)(p.tap_oh[tap] * p.Wp + p.tap_ow[tap]) * 128u;
+                        const uint64_t ad0 = make_desc(a_tap, 16u, 1024u);
+                        const uint64_t bd0 = B_MN ? make_desc(b_src, 8192u, 1024u) : make_desc(b_src, 16u, 1024u);
+                        const uint64_t bstep = B_MN ? 128ull : 2ull;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (k < ksteps) umma_bf16(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, (kc | tap | k) != 0 ? 1u : 0u);
+                        if (!p.resident) umma_commit(smem_u32(&ctl->empty_b[sb]));
+                    }
+                    if (ok) umma_commit(smem_u32(&ctl->empty_a[sa]));
+                }
+                if (ok) umma_commit(smem_u32(&ctl->acc_full[b]));
+            }
+        }
+    } else {
+        // ---------------- epilogue: group g (four warps) drains accumulator buffer g
+        const int quarter = warp & 3, group = (warp - 2) >> 2;
+        const int gtid = (warp - 2 - group * 4) * 32 + lane;         // 0..127 within the group
+        const uint32_t slab = staging_base + (uint32_t)group * 16384u;
+        int tc = group;
+        bool ok = true;
+        for (int tile = blockIdx.x + group * gridDim.x; tile < total_tiles && ok; tile += 2 * gridDim.x, tc += 2) {
+            const int b = group, aph = (tc >> 1) & 1;
+            const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
+            const int img = m_tile / p.row_tiles, p0 = (m_tile - img * p.row_tiles) * p.nr;
+            const int n0 = n_tile * p.BN;
+            ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 17);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.BN);
+            const int m = quarter * 32 + lane;                       // raster position of this thread's accumulator row
+            if (p.tma_store) {
+                const int n_chunks = (p.BN + 63) / 64;
+                for (int ch = 0; ch < n_chunks; ++ch) {
+                    if (gtid == 0) tma_store_wait_read();            // the slab's previous store has read it
+                    named_barrier(1 + group, 128);
+                    const int groups = min(4, (p.BN - ch * 64) / 16);
+                    uint32_t v[4][16];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)
+                        if (g < groups) tmem_ld16(lane_addr + (uint32_t)(ch * 64 + g * 16), v[g]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (g >= groups) break;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 0]), __uint_as_float(v[g][8 * h + 1]));
+                            __nv_bfloat162 b1 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 2]), __uint_as_float(v[g][8 * h + 3]));
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 4]), __uint_as_float(v[g][8 * h + 5]));
+                            __nv_bfloat162 b3 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 6]), __uint_as_float(v[g][8 * h + 7]));
+                            const uint32_t j = (uint32_t)(g * 2 + h);
+                            const uint32_t addr = slab + (uint32_t)m * 128u + ((j ^ ((uint32_t)m & 7u)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t *>(&b0)),
+                                         "r"(*reinterpret_cast<uint32_t *>(&b1)), "r"(*reinterpret_cast<uint32_t *>(&b2)),
+                                         "r"(*reinterpret_cast<uint32_t *>(&b3))
+                                         : "memory");
+                        }
+                    }
+                    if (ch + 1 >= n_chunks) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                    }
+                    fence_proxy_async();
+                    named_barrier(1 + group, 128);
+                    // one store per tile and chunk: box = nr rows x Wp columns x 64 channels; the columns past Q, the rows
+                    // past P and the channels past the true count fall outside the tensor and are dropped
+                    if (gtid == 0) {
+                        tma_store_4d(&tmC, slab, n0 + ch * 64, 0, p0, img);
+                        tma_store_commit();
+                    }
+                }
+                continue;
+            }
+            // ---- direct stores (fp32 outputs)
+            const int i = m / p.Wp, j = m - i * p.Wp;
+            const bool row_ok = m < p.nr * p.Wp && j < p.Q && p0 + i < p.P;
+            const size_t row_off = ((size_t)(img * p.P + p0 + i) * p.Q + j) * (size_t)p.ld_out;
+            for (int c0 = 0; c0 < p.BN; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(lane_addr + (uint32_t)c0, v);
+                tmem_ld_wait();
+                if (c0 + 16 >= p.BN) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                }
+                const int col = n0 + c0;
+                if (!row_ok || col >= p.n_cols) continue;
+                const int nvalid = min(16, p.n_cols - col);
+                if (p.out_f32) {
+                    float *o = (float *)p.out + row_off + col;
+                    for (int e = 0; e < nvalid; ++e) o[e] = __uint_as_float(v[e]);
+                } else {
+                    __nv_bfloat16 *o = (__nv_bfloat16 *)p.out + row_off + col;
+                    for (int e = 0; e < nvalid; ++e) o[e] = __float2bfloat16_rn(__uint_as_float(v[e]));
+                }
+            }
+        }
+        if (p.tma_store && gtid == 0) tma_store_wait_read();
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
 // ------------------------------------------------------------------------------------------ wgrad
 // dw[k][tap][c] = sum over output pixels of dy[pixel][k] * x[pixel shifted by the tap][c]   (Eq. 4)
 //   GEMM per tap: M = 128 output channels k, N = BN input channels c, reduction = output pixels, 64 per stage.
@@ -443,12 +715,10 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 const int rem = pix_end - (pix_beg + it * 64);
                 const int ksteps = rem >= 64 ? 4 : (rem + 15) / 16;
                 const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
-#pragma unroll 1
-                for (int k = 0; k < ksteps; ++k) {
-                    const uint64_t ad = make_desc(a_src + (uint32_t)k * 2048u, 8192u, 1024u);
-                    const uint64_t bd = make_desc(b_src + (uint32_t)k * 2048u, 8192u, 1024u);
-                    umma_bf16(tmem_base, ad, bd, idesc, (it | k) != 0 ? 1u : 0u);
-                }
+                const uint64_t ad0 = make_desc(a_src, 8192u, 1024u), bd0 = make_desc(b_src, 8192u, 1024u);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (k < ksteps) umma_bf16(tmem_base, ad0 + 128ull * k, bd0 + 128ull * k, idesc, (it | k) != 0 ? 1u : 0u);
                 umma_commit(smem_u32(&ctl->empty[s]));
             }
             if (ok) umma_commit(smem_u32(&ctl->accum));
@@ -736,6 +1006,98 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     return PT_OK;
 }
 
+// Source activations as a tiled 4-D tensor (C, W, H, N): box 64 channels x box_w x box_h x 1 (the halo tile).
+bool make_halo_in_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, int W, int H, int N, int ld, int box_w, int box_h)
+{
+    if (!c->encode_tiled || box_w > 256 || box_h > 256) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+    cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)W * ld * 2, (cuuint64_t)H * W * ld * 2};
+    cuuint32_t box[4] = {(cuuint32_t)kKC, (cuuint32_t)box_w, (cuuint32_t)box_h, 1}, estr[4] = {1, 1, 1, 1};
+    CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box,
+                                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// Stride-1 RxS convolution (fwd) or its data gradient through the halo kernel. Returns PT_ERR_UNSUPPORTED when the shape
+// does not suit it (the caller then uses the per-tap im2col kernel).
+//   src: activations read (x or dy), (Cs channels, Ws x Hs pixels, pitch lds); out: (n_cols channels, Q x P pixels, pitch ld_out)
+template <bool B_MN>
+pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const void *src, int Cs, int Ws, int Hs, int lds, const void *w, void *out,
+                      int n_cols, int P, int Q, int ld_out, int pad_h, int pad_w, bool flip, cudaStream_t st)
+{
+    const int R = d->R, S = d->S, taps = R * S;
+    const int Wp = Q + S - 1;
+    if (taps < 2 || taps > kMaxTaps || Wp > 128 || Ws > 250) return PT_ERR_UNSUPPORTED;
+    HaloP p;
+    memset(&p, 0, sizeof(p));
+    p.N = d->N; p.P = P; p.Q = Q; p.Wp = Wp;
+    p.nr = 128 / Wp < P ? 128 / Wp : P;
+    p.row_tiles = pt_ceil_div(P, p.nr);
+    p.n_cols = n_cols;
+    p.BN = tile_n(n_cols, &p.n_tiles);
+    p.c_red = Cs; p.k_chunks = pt_ceil_div(Cs, kKC); p.taps = taps;
+    p.lo_h = -pad_h; p.lo_w = -pad_w;
+    for (int t = 0; t < taps; ++t) {
+        p.tap_oh[t] = (unsigned char)(t / S); p.tap_ow[t] = (unsigned char)(t % S);
+        p.tap_wt[t] = (unsigned short)(flip ? taps - 1 - t : t);
+    }
+    const int box_h = p.nr + R - 1;
+    if (box_h > 256) return PT_ERR_UNSUPPORTED;
+    p.a_box_bytes = box_h * Wp * 128;
+    const int need_rows = 128 + (R - 1) * Wp + S - 1;          // rows the M = 128 MMAs of the last tap touch
+    p.a_alloc = (int)pt_align_up((size_t)(need_rows > box_h * Wp ? need_rows : box_h * Wp) * 128, 1024);
+    const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : pt_align_up((size_t)p.BN * 128, 1024);
+    const size_t budget = 222 * 1024 - 2048 - kHaloStaging;
+    const size_t w_all = (size_t)taps * p.k_chunks * b_bytes;
+    p.resident = (p.n_tiles == 1 && w_all + 2 * (size_t)p.a_alloc <= budget) ? 1 : 0;
+    size_t left = budget - (p.resident ? w_all : 0);
+    if (!p.resident) {
+        // ring: at least two A stages, the rest for weight stages (at least 3)
+        p.stages_a = 2;
+        if (left < 2 * (size_t)p.a_alloc + 3 * b_bytes) return PT_ERR_UNSUPPORTED;
+        size_t sb = (left - 2 * (size_t)p.a_alloc) / b_bytes;
+        p.stages_b = sb > kMaxStages ? kMaxStages : (int)sb;
+        left -= (size_t)p.stages_b * b_bytes;
+        int sa = (int)(left / p.a_alloc);
+        p.stages_a = sa > 4 ? 4 : sa;
+    } else {
+        int sa = (int)(left / p.a_alloc);
+        p.stages_a = sa > 4 ? 4 : sa;
+        p.stages_b = 1;
+    }
+    if (p.stages_a < 2) return PT_ERR_UNSUPPORTED;
+    p.tmem_cols = pow2_cols(2 * p.BN);
+    p.out = out; p.ld_out = ld_out; p.out_f32 = d->out_f32;
+    p.tma_store = d->out_f32 ? 0 : 1;
+    p.status = c->d_status;
+    CUtensorMap tmA, tmB, tmC;
+    memset(&tmC, 0, sizeof(tmC));
+    if (!make_halo_in_map(c, &tmA, src, Cs, Ws, Hs, d->N, lds, Wp, box_h)) return PT_ERR_CUDA;
+    if (!make_weight_map(c, &tmB, w, d->C, taps, d->K, d->ldw, B_MN ? kKC : p.BN)) return PT_ERR_CUDA;
+    if (p.tma_store) {
+        cuuint64_t dims[4] = {(cuuint64_t)n_cols, (cuuint64_t)Q, (cuuint64_t)P, (cuuint64_t)d->N};
+        cuuint64_t strides[3] = {(cuuint64_t)ld_out * 2, (cuuint64_t)Q * ld_out * 2, (cuuint64_t)P * Q * ld_out * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)Wp, (cuuint32_t)p.nr, 1}, estr[4] = {1, 1, 1, 1};
+        CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmC, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, out, dims, strides, box, estr,
+                                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                      CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+    }
+    const size_t smem = 2048 + kHaloStaging + (p.resident ? w_all : (size_t)p.stages_b * b_bytes) + (size_t)p.stages_a * p.a_alloc;
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[B_MN ? 1 : 0]) {
+        PT_CUDA_OK(cudaFuncSetAttribute(conv_halo_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        attr_set[B_MN ? 1 : 0] = true;
+    }
+    const int total_tiles = p.N * p.row_tiles * p.n_tiles;
+    const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
+    conv_halo_kernel<B_MN><<<grid, kHaloThreads, smem, st>>>(tmA, tmB, tmC, p);
+    c->launches += 1;
+    PT_CUDA_OK(cudaGetLastError());
+    return PT_OK;
+}
+
 int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
 {
     int n_tiles;
@@ -900,6 +1262,16 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         if (!make_im2col_map(c, &tmA, xs, 64, sp.Q, sp.Hs, d->N, 16, 0, -sp.pl, 0, up_h, 1, kBM, sp.Wp)) return PT_ERR_CUDA;
         if (!make_weight_map(c, &tmB, w2, 64, sp.U, d->K, 64, p.BN)) return PT_ERR_CUDA;
         return launch_gemm<false>(c, tmA, tmB, p, st);
+    }
+    if (which == PT_CONV_FWD && d->stride == 1 && d->R * d->S > 1) {
+        pt_status r = launch_halo<false>(c, d, a, d->C, d->W, d->H, d->ldx, b, out, d->K, P, Q, d->ldy, d->pad, d->pad, false, st);
+        if (r != PT_ERR_UNSUPPORTED) return r;
+    }
+    if (which == PT_CONV_DGRAD && d->stride == 1 && d->R * d->S > 1 && d->pad <= d->R - 1 && d->pad <= d->S - 1) {
+        // dx = correlation of dy (padding R-1-pad) with the taps visited flipped
+        pt_status r = launch_halo<true>(c, d, a, d->K, Q, P, d->ldy, b, out, d->C, d->H, d->W, d->ldx, d->R - 1 - d->pad,
+                                        d->S - 1 - d->pad, true, st);
+        if (r != PT_ERR_UNSUPPORTED) return r;
     }
     if (which == PT_CONV_FWD) {
         // raster = output pixels (P x Q per image); source = x
