@@ -43,12 +43,36 @@ constexpr int kThreads = 256;
 constexpr int kUnroll = 8;                // lines in flight per thread
 constexpr int kSweeps = 4;                // unrolled sweeps per chunk: every block does the same number of iterations
 
-__device__ __forceinline__ float warp_sum(float v)
+// Eight per-lane values (one per line) are reduced over the 32 lanes with 9 shuffles instead of 40: three
+// halving exchanges leave lane l with the partial of line (l >> 2) & 7 over its 4-lane group's share, two more
+// add the four lanes of a group. The tree is fixed, so the result is run-to-run identical.
+// Returns the total of line ((lane >> 2) & 7), valid in every lane.
+template <typename T, typename Op>
+__device__ __forceinline__ T warp_reduce8(T (&v)[8], int lane, Op op)
 {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
+    for (int i = 0; i < 4; ++i) {
+        const bool hi = lane & 16;
+        const T send = hi ? v[i] : v[i + 4], keep = hi ? v[i + 4] : v[i];
+        v[i] = op(keep, __shfl_xor_sync(0xffffffffu, send, 16));
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const bool hi = lane & 8;
+        const T send = hi ? v[i] : v[i + 2], keep = hi ? v[i + 2] : v[i];
+        v[i] = op(keep, __shfl_xor_sync(0xffffffffu, send, 8));
+    }
+    {
+        const bool hi = lane & 4;
+        const T send = hi ? v[0] : v[1], keep = hi ? v[1] : v[0];
+        v[0] = op(keep, __shfl_xor_sync(0xffffffffu, send, 4));
+    }
+    v[0] = op(v[0], __shfl_xor_sync(0xffffffffu, v[0], 2));
+    v[0] = op(v[0], __shfl_xor_sync(0xffffffffu, v[0], 1));
+    return v[0];
 }
+struct OpAdd { __device__ __forceinline__ float operator()(float a, float b) const { return a + b; } };
+struct OpMax { __device__ __forceinline__ unsigned int operator()(unsigned int a, unsigned int b) const { return a > b ? a : b; } };
 
 // ---- phase 1
 __global__ void __launch_bounds__(kThreads) norms_partial_kernel(const LayerDev *__restrict__ layers,
@@ -56,7 +80,7 @@ __global__ void __launch_bounds__(kThreads) norms_partial_kernel(const LayerDev 
                                                                  float *__restrict__ linesum, float *__restrict__ colpart)
 {
     __shared__ float s_col[kThreads];
-    __shared__ float s_line[kThreads];           // [line in chunk][warp along the line]: TY*kUnroll*kSweeps*nwx = 256
+    __shared__ float s_line[2 * kThreads];       // [line in chunk][warp along the line]: at most 64 lines per TY x 8 warps
     const Chunk ch = chunks[blockIdx.x];
     const LayerDev L = layers[ch.layer];
     const int TX = 1 << L.tx_log2, TY = kThreads >> L.tx_log2;
@@ -79,25 +103,19 @@ __global__ void __launch_bounds__(kThreads) norms_partial_kernel(const LayerDev 
             a[u] *= a[u];
             cacc += a[u];
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) a[u] += __shfl_xor_sync(0xffffffffu, a[u], o);
-        if (lane == 0) {
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const int ll = l + u * TY;
-                if (ll < ch.nlines) s_line[ll * nwx + wx] = a[u];
-            }
+        const float tot = warp_reduce8(a, lane, OpAdd());
+        if ((lane & 3) == 0) {
+            const int ll = l + ((lane >> 2) & 7) * TY;      // the lane's 4-lane group holds this line's total
+            if (ll < ch.nlines) s_line[ll * nwx + wx] = tot;
         }
     }
     s_col[threadIdx.x] = cacc;
     __syncthreads();
     // one partial per (line, column block): the warps along a line are added in ascending order
-    if ((int)threadIdx.x < ch.nlines) {
+    for (int ln = threadIdx.x; ln < ch.nlines; ln += kThreads) {
         float s = 0.f;
-        for (int x = 0; x < nwx; ++x) s += s_line[threadIdx.x * nwx + x];
-        linesum[L.line_off + (size_t)(ch.line0 + threadIdx.x) * L.n_cb + ch.cb] = s;
+        for (int x = 0; x < nwx; ++x) s += s_line[ln * nwx + x];
+        linesum[L.line_off + (size_t)(ch.line0 + ln) * L.n_cb + ch.cb] = s;
     }
     // combine the TY line groups' column partials in fixed order
     if (ty == 0 && cv) {
@@ -214,7 +232,7 @@ __global__ void __launch_bounds__(kThreads) absmax_kernel(const LayerDev *__rest
     const int TX = 1 << L.tx_log2, TY = kThreads >> L.tx_log2;
     const int tx = threadIdx.x & (TX - 1), ty = threadIdx.x >> L.tx_log2;
     const int lane = threadIdx.x & 31;
-    __shared__ unsigned int s_line[kThreads];
+    __shared__ unsigned int s_line[2 * kThreads];
     unsigned int *mk = maxbits + L.k_off + L.c_off;         // this layer's K entries, then its C entries
     unsigned int *mc = mk + L.K;
     const int wx = tx >> 5, nwx = TX >> 5;
@@ -232,23 +250,17 @@ __global__ void __launch_bounds__(kThreads) absmax_kernel(const LayerDev *__rest
         }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) cm = max(cm, b[u]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) b[u] = max(b[u], __shfl_xor_sync(0xffffffffu, b[u], o));
-        if (lane == 0) {
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const int ll = l + u * TY;
-                if (ll < ch.nlines) s_line[ll * nwx + wx] = b[u];
-            }
+        const unsigned int tot = warp_reduce8(b, lane, OpMax());
+        if ((lane & 3) == 0) {
+            const int ll = l + ((lane >> 2) & 7) * TY;
+            if (ll < ch.nlines) s_line[ll * nwx + wx] = tot;
         }
     }
     __syncthreads();
-    if ((int)threadIdx.x < ch.nlines) {
+    for (int ln = threadIdx.x; ln < ch.nlines; ln += kThreads) {
         unsigned int m = 0u;
-        for (int x = 0; x < nwx; ++x) m = max(m, s_line[threadIdx.x * nwx + x]);
-        if (m) atomicMax(&mk[(ch.line0 + threadIdx.x) / L.RS], m);
+        for (int x = 0; x < nwx; ++x) m = max(m, s_line[ln * nwx + x]);
+        if (m) atomicMax(&mk[(ch.line0 + ln) / L.RS], m);
     }
     if (cv && cm) atomicMax(&mc[c], cm);
 }
@@ -314,8 +326,11 @@ pt_status build_tables(const pt_layer *layers, int n, Tables *t)
         d.pad_ = 0;
         const int TX = 1 << lg, TY = kThreads / TX;
         const int lines = s.K * s.RS;
-        // every chunk is TY*kUnroll*kSweeps lines x TX columns (8192 thread slots): equal trip counts, no long tail
-        const int lines_per_chunk = TY * kUnroll * kSweeps;
+        // a chunk is TY*kUnroll*sweeps lines x TX columns; sweeps = 4 (8192 thread slots), more for tall tensors so that no
+        // column has more than ~32 chunk partials to add up in phase 2 (the s_line staging holds at most 256 lines x warps)
+        int sweeps = kSweeps;
+        while (sweeps < 8 && lines > 32 * TY * kUnroll * sweeps) sweeps *= 2;
+        const int lines_per_chunk = TY * kUnroll * sweeps;
         d.n_cb = pt_ceil_div(s.C, TX);
         d.n_lc = pt_ceil_div(lines, lines_per_chunk);
         for (int lc = 0; lc < d.n_lc; ++lc)
