@@ -38,6 +38,8 @@ extern "C" pt_status pt_create(pt_ctx **out, int device)
               cudaMallocHost(&c->h_status, 16) == cudaSuccess && cudaMalloc(&c->d_arena, kArenaBytes) == cudaSuccess &&
               cudaMallocHost(&c->h_stage, kArenaBytes) == cudaSuccess &&
               cudaMallocHost(&c->h_counts, 65536 * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&c->d_sync, 16384 * sizeof(unsigned int)) == cudaSuccess &&
+              cudaMemset(c->d_sync, 0, 16384 * sizeof(unsigned int)) == cudaSuccess &&
               cudaEventCreateWithFlags(&c->upload_done, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); pt_destroy(c); return PT_ERR_CUDA; }
     size_t off = 0;
@@ -68,6 +70,7 @@ extern "C" pt_status pt_destroy(pt_ctx *c)
     if (c->d_arena) cudaFree(c->d_arena);
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->h_counts) cudaFreeHost(c->h_counts);
+    if (c->d_sync) cudaFree(c->d_sync);
     (void)cudaGetLastError();
     delete c;
     return PT_OK;

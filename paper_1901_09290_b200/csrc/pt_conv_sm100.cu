@@ -614,8 +614,10 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
 //   A operand: dy[pixel][k], k contiguous -> MN-major tiles (two 64-channel boxes of a 2-D tiled map).
 //   B operand: x through the im2col map (same pixel raster as the forward pass, tap offset added by the TMA unit),
 //              c contiguous -> MN-major tiles (one 64-channel box per 64 columns).
-//   The pixel range is split across CTAs (blockIdx.z); with more than one split every CTA writes its fp32 partial
-//   tile to the workspace and wgrad_reduce_kernel sums the splits in ascending order (deterministic).
+//   The pixel range is split across CTAs (blockIdx.y), at most one CTA per SM in total so that all of them are resident.
+//   With more than one split every CTA TMA-stores its fp32 partial tile to the workspace, announces it on a counter,
+//   waits (bounded) until all splits of its tile have arrived, and then sums its share of the tile's rows over the
+//   splits in ascending order: deterministic, and no second kernel.
 struct WgradP {
     int K, C, taps;         // true channel counts, number of taps (R*S)
     int BN, n_tiles;        // input-channel tile
@@ -625,12 +627,15 @@ struct WgradP {
     int splits;
     int Pd, Qd, stride, lo_h, lo_w, S;
     int stages, tmem_cols;
-    float *out;             // dw (splits == 1) or the partial workspace [split][K*taps*C]
+    float *out;             // dw
+    float *partial;         // splits > 1: workspace [blockIdx.x][split][128][BN] fp32
+    unsigned int *sync;     // splits > 1: two zeroed counters per blockIdx.x (arrived, reduced); left zero again at exit
     unsigned int *status;
 };
 
 __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy,
-                                                              const __grid_constant__ CUtensorMap tmX, const WgradP p)
+                                                              const __grid_constant__ CUtensorMap tmX,
+                                                              const __grid_constant__ CUtensorMap tmP, const WgradP p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw);
@@ -732,8 +737,57 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
             const int k = k0 + quarter * 32 + lane;
             const bool row_ok = k < p.K;
             (void)row_ok;
-            float *obase = p.out + (size_t)split * p.K * p.taps * p.C;
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            if (p.splits > 1) {
+                // ---- (1) this CTA's fp32 partial tile goes to the workspace through swizzled staging + TMA stores
+                const int gtid = (warp - 2) * 32 + lane;
+                int sl = 0;
+                for (int cc = 0; cc < p.BN; cc += 32, sl ^= 1) {
+                    const uint32_t slab = data_base + (uint32_t)(quarter * 2 + sl) * 4096u;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                    uint32_t lo[16], hi[16];
+                    if (iters > 0) {
+                        tmem_ld16(lane_addr + (uint32_t)cc, lo);
+                        if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)cc + 16u, hi);
+                        tmem_ld_wait();
+                    }
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        if (iters <= 0) lo[e] = 0u;
+                        if (iters <= 0 || cc + 16 >= p.BN) hi[e] = 0u;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t *src = j < 4 ? &lo[4 * j] : &hi[4 * (j - 4)];
+                        const uint32_t addr = slab + (uint32_t)lane * 128u + (((uint32_t)j ^ ((uint32_t)lane & 7u)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(src[0]), "r"(src[1]), "r"(src[2]), "r"(src[3])
+                                     : "memory");
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmP, slab, cc, ((int)blockIdx.x * p.splits + split) * 128 + quarter * 32);
+                        tma_store_commit();
+                    }
+                }
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // the writes have completed
+                __threadfence();
+                named_barrier(1, 128);
+                // ---- (2) every split CTA of this tile is resident (the grid is at most one CTA per SM): wait for all of them
+                unsigned int *arrived = p.sync + 2 * blockIdx.x, *reduced = arrived + 1;
+                if (gtid == 0) {
+                    atomicAdd(arrived, 1u);
+                    const uint64_t t0 = globaltimer_ns();
+                    while (atomicAdd(arrived, 0u) < (unsigned)p.splits) {
+                        if (*abort_flag) break;
+                        if (globaltimer_ns() - t0 > 2000000000ull) { record_timeout(p.status, 8); *abort_flag = 1; break; }
+                        __nanosleep(64);
+                    }
+                }
+                named_barrier(1, 128);
+            } else {
+            float *obase = p.out;
             // The stages are free once the accumulator is complete: each warp transposes its 32 x 32 blocks through
             // a padded shared-memory square so that a warp writes 32 consecutive floats of one dw row at a time.
             const uint32_t sq = data_base + (uint32_t)quarter * (32u * 33u * 4u);
@@ -764,23 +818,78 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                     if (col < p.C && cc + lane < p.BN) obase[((size_t)kk * p.taps + tap) * p.C + col] = __uint_as_float(t);
                 }
             }
+            }
         }
         tc_fence_before();
     }
     __syncthreads();
+    if (p.splits > 1 && !*abort_flag) {
+        // ---- (3) all 192 threads: this CTA sums its share of the tile's rows over the splits, in ascending split order
+        __threadfence();
+        // Work items are (row, 4-column group) of the real rows of the tile, dealt out evenly to the tile's split CTAs.
+        // T lanes share an item (T = 8 when there are many splits, else 1): lane s adds the splits [s*zc, (s+1)*zc) in
+        // ascending order, then the partial sums are combined by a fixed shuffle tree: the result does not depend on timing.
+        const int rows_real = min(128, p.K - k0);
+        const int ngrp = p.BN / 4;                                   // float4 groups per row (BN is a multiple of 16)
+        const int items = rows_real * ngrp;
+        const int per_cta = (items + p.splits - 1) / p.splits;
+        const int it_beg = split * per_cta, it_end = min(items, it_beg + per_cta);
+        const int T = p.splits > 96 ? 8 : 1;                         // lanes per item: share only very long split chains
+        const int zc = (p.splits + T - 1) / T;
+        const int sub = threadIdx.x & (T - 1);
+        const float *pt = p.partial + (size_t)blockIdx.x * p.splits * 128 * p.BN;
+        const size_t zstride = (size_t)128 * p.BN;
+        for (int base = it_beg; base < it_end; base += kThreads / T) {
+            const int item = base + threadIdx.x / T;
+            const bool live = item < it_end;
+            const int r = live ? item / ngrp : 0, col = live ? (item % ngrp) * 4 : 0;
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (live && c0 + col < p.C) {
+                const float *src = pt + (size_t)r * p.BN + col;
+                const int z_end = min(p.splits, (sub + 1) * zc);
+                int z = sub * zc;
+                for (; z + 4 <= z_end; z += 4) {
+                    float4 t[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) t[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(z + u) * zstride));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) { sum.x += t[u].x; sum.y += t[u].y; sum.z += t[u].z; sum.w += t[u].w; }
+                }
+                for (; z < z_end; ++z) {
+                    const float4 t = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)z * zstride));
+                    sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+                }
+            }
+            for (int o = 1; o < T; o <<= 1) {        // (s0+s1) + (s2+s3) ... : the same tree on every run
+                sum.x += __shfl_xor_sync(0xffffffffu, sum.x, o);
+                sum.y += __shfl_xor_sync(0xffffffffu, sum.y, o);
+                sum.z += __shfl_xor_sync(0xffffffffu, sum.z, o);
+                sum.w += __shfl_xor_sync(0xffffffffu, sum.w, o);
+            }
+            if (live && sub == 0 && c0 + col < p.C) {
+                float *dst = p.out + ((size_t)(k0 + r) * p.taps + tap) * p.C + c0 + col;
+                const int nv = min(4, p.C - (c0 + col));
+                dst[0] = sum.x;
+                if (nv > 1) dst[1] = sum.y;
+                if (nv > 2) dst[2] = sum.z;
+                if (nv > 3) dst[3] = sum.w;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned int *arrived = p.sync + 2 * blockIdx.x, *reduced = arrived + 1;
+            __threadfence();
+            if (atomicAdd(reduced, 1u) == (unsigned)p.splits - 1u) {          // last one out clears the counters
+                *arrived = 0u;
+                *reduced = 0u;
+                __threadfence();
+            }
+        }
+    }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
-}
-
-__global__ void wgrad_reduce_kernel(const float *__restrict__ partial, float *__restrict__ dw, size_t n, int splits)
-{
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    float s = 0.f;
-    for (int z = 0; z < splits; ++z) s += partial[(size_t)z * n + i];   // ascending split order: run-to-run identical
-    dw[i] = s;
 }
 
 // ------------------------------------------------------------------------------------------ few-channel stride-2 stem
@@ -1112,6 +1221,16 @@ int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     return (int)s;
 }
 
+// Workspace of the split weight gradient: one padded 128 x BN fp32 tile per (tile, split).
+size_t wgrad_partial_bytes(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
+{
+    const int s = wgrad_splits(c, d, P, Q);
+    if (s <= 1) return 0;
+    int n_tiles;
+    const int bn = tile_n(d->C, &n_tiles);
+    return (size_t)n_tiles * pt_ceil_div(d->K, 128) * d->R * d->S * s * 128 * bn * sizeof(float);
+}
+
 // Launches the weight-gradient kernel for a problem whose x operand is described by `tmX` (64 pixels x 64 channels boxes).
 pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, int lo_h, int lo_w, const CUtensorMap &tmX,
                     const void *dy, float *out, void *ws, size_t ws_bytes, cudaStream_t st)
@@ -1127,12 +1246,27 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     p.Pd = P; p.Qd = Q; p.stride = stride; p.lo_h = lo_h; p.lo_w = lo_w;
     p.tmem_cols = pow2_cols(p.BN);
     p.status = c->d_status;
-    const size_t n = (size_t)d->K * p.taps * d->C;
+    const int gx = p.n_tiles * p.m_tiles * p.taps;
+    p.out = out;
+    CUtensorMap tmP;
+    memset(&tmP, 0, sizeof(tmP));
     if (p.splits > 1) {
-        if (!ws || ws_bytes < (size_t)p.splits * n * sizeof(float)) return PT_ERR_WORKSPACE;
-        p.out = (float *)ws;
-    } else {
-        p.out = out;
+        const size_t need = (size_t)gx * p.splits * 128 * p.BN * sizeof(float);
+        if (!ws || ws_bytes < need) return PT_ERR_WORKSPACE;
+        p.partial = (float *)ws;
+        // two self-resetting counters per tile from the context's ring (kernels of one stream run in order, and the ring
+        // is far larger than the tiles of the few launches that can be in flight)
+        if (2 * gx > 8192) return PT_ERR_UNSUPPORTED;
+        if (c->sync_next + 2 * gx > 16384) c->sync_next = 0;
+        p.sync = c->d_sync + c->sync_next;
+        c->sync_next += 2 * gx;
+        cuuint64_t dims[2] = {(cuuint64_t)p.BN, (cuuint64_t)gx * p.splits * 128};
+        cuuint64_t strides[1] = {(cuuint64_t)p.BN * 4};
+        cuuint32_t box[2] = {32, 32}, estr[2] = {1, 1};
+        CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmP, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ws, dims, strides, box, estr,
+                                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                      CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
     }
     // A: dy as a 2-D tensor (K channels, N*P*Q pixels), box 64 channels x 64 pixels
     if (!c->encode_tiled) return PT_ERR_CUDA;
@@ -1154,13 +1288,9 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
         PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr_set = true;
     }
-    dim3 grid((unsigned)(p.n_tiles * p.m_tiles * p.taps), (unsigned)p.splits);
-    conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(tmA, tmX, p);
+    dim3 grid((unsigned)gx, (unsigned)p.splits);
+    conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(tmA, tmX, tmP, p);
     c->launches += 1;
-    if (p.splits > 1) {
-        wgrad_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const float *)ws, out, n, p.splits);
-        c->launches += 1;
-    }
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
 }
@@ -1190,13 +1320,11 @@ size_t pt_sm100_conv_workspace(const pt_ctx *c, const pt_conv_desc *d, int which
     if (sp.ok && which == PT_CONV_FWD) return sp.xs_bytes + pt_align_up(sp.w2_elems * 2, 1024);
     if (sp.ok && which == PT_CONV_WGRAD) {
         const pt_conv_desc v = stem_virtual_desc(d, sp);
-        const int s = wgrad_splits(c, &v, sp.P, sp.Q);
-        return sp.xs_bytes + pt_align_up(sp.w2_elems * 4, 1024) + (s > 1 ? (size_t)s * sp.w2_elems * 4 : 0);
+        return sp.xs_bytes + pt_align_up(sp.w2_elems * 4, 1024) + wgrad_partial_bytes(c, &v, sp.P, sp.Q);
     }
     if (which != PT_CONV_WGRAD) return 0;
     const int P = pt_out_dim(d->H, d->R, d->stride, d->pad), Q = pt_out_dim(d->W, d->S, d->stride, d->pad);
-    const int s = wgrad_splits(c, d, P, Q);
-    return s > 1 ? (size_t)s * d->K * d->R * d->S * d->C * sizeof(float) : 0;
+    return wgrad_partial_bytes(c, d, P, Q);
 }
 
 pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void *a, const void *b, void *out, void *ws,

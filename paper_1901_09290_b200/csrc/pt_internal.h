@@ -41,6 +41,8 @@ struct pt_ctx {
     pt_region lasso_tab[3], detect_tab[2], graph_tab, gather_tab;
     int lasso_next = 0, detect_next = 0;
     int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan
+    unsigned int *d_sync = nullptr;     // zero-initialised, self-resetting arrival counters of the split weight gradient
+    unsigned int sync_next = 0;         // ring position in d_sync
     uint64_t launches = 0;
     // tcgen05 conv path
     void *encode_tiled = nullptr;       // cuTensorMapEncodeTiled
