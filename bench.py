@@ -167,6 +167,23 @@ def run_reference(args):
     }))
 
 
+# ------------------------------------------------------------------------------------------ multi-rank aggregation
+def max_over_ranks(ms: float, world: int, device="cuda") -> float:
+    """Step time of the job = the slowest rank's device time."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_rank: float, world: int, ms_total: float, steps: int) -> float:
+    """Whole-job TFLOP/s: every rank processes its own batch (weak scaling), the job takes the slowest rank's time."""
+    return world * flops_per_rank / (ms_total / steps * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------------------------ GPU leg
 def run_ours(args):
     import torch
@@ -203,12 +220,7 @@ def run_ours(args):
             fn()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), world)
 
     if args.profile_steps:
         # a short run for profilers: one warm-up step, then the requested steps, nothing else
@@ -332,8 +344,8 @@ def run_ours(args):
     dom_flops = flops[dom]
     dom_t = conv_ms[dom] * 1e-3
     n_dom = nL - (1 if dom == "dgrad" else 0)
-    value = world * tot_flops / (ms / args.steps * 1e-3) / 1e12
-    e2e_val = world * tot_flops / (ms_e2e / args.steps * 1e-3) / 1e12
+    value = whole_job_value(tot_flops, world, ms, args.steps)
+    e2e_val = whole_job_value(tot_flops, world, ms_e2e, args.steps)
     h2d, d2h = ts.e2e_bytes()
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),

@@ -1,0 +1,105 @@
+"""Parity on whole networks and at the bench's full sizes.
+
+* config 2: every layer of the pruned ResNet-32 stack at batch 128, full tensors.
+* config 4 at batch 2: every layer of the pruned ResNet-50, full tensors (identical channel shapes to the bench).
+* config 4 / 5 at the bench's batch sizes, through the same harness buffers and launch path (CUDA-graph replay):
+  4096 seeded sampled outputs per tensor, each computed alone by the oracle, plus all of dw for the smallest layers.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_09290_b200 import binding as B
+from paper_1901_09290_b200 import harness
+from paper_1901_09290_b200 import workloads as W
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer_inputs(l, N, seed, first):
+    x = (W.gen_image if first else W.gen_act)(N, l.H, l.H, l.C, seed)
+    w = W.bf16_round(W.gen_weight(l.K, l.R, l.R, l.C, seed + 1))
+    dy = W.gen_dy(N, l.P, l.P, l.K, seed + 2)
+    return x, w, dy
+
+
+def _full_layer_check(l, N, seed, first):
+    x, w, dy = _layer_inputs(l, N, seed, first)
+    y, dx, dw, _ = Hh.run_conv_all(N, l.H, l.H, l.C, l.K, l.R, l.stride, l.pad, x, w, dy)
+    Hh.check_conv(y, l.K, oracle.conv_fwd(x.numpy(), w.numpy(), l.stride, l.pad), what=l.name + " fwd")
+    Hh.check_conv(dx, l.C, oracle.conv_dgrad(dy.numpy(), w.numpy(), l.H, l.H, l.stride, l.pad), what=l.name + " dgrad")
+    Hh.check_conv(dw, l.C, oracle.conv_wgrad(x.numpy(), dy.numpy(), l.R, l.R, l.stride, l.pad), what=l.name + " wgrad")
+
+
+def test_config2_resnet32_every_layer_batch128():
+    net = W.resnet32()
+    counts = W.random_keep(net, W.BASE_SEED + 2)
+    pruned = W.with_sizes(net, counts)
+    for li, l in enumerate(pruned.layers):
+        _full_layer_check(l, 128, W.layer_seed(2, li), li == 0)
+
+
+def test_config4_resnet50_every_layer_batch2():
+    net = W.resnet50()
+    counts = W.staged_keep_to_flops(net, W.BASE_SEED + 4)
+    pruned = W.with_sizes(net, counts)
+    for li, l in enumerate(pruned.layers):
+        _full_layer_check(l, 2, W.layer_seed(4, li), li == 0)
+
+
+def _sampled_step_check(keep, N, layer_ids, n_samples=4096, full_dw_below=40000):
+    """Runs the harness's graph-replayed training step at the bench's sizes on CPU-generated inputs and compares sampled
+    outputs of the chosen layers with the oracle."""
+    ctx = Hh.ctx()
+    net = W.resnet50()
+    seed = W.BASE_SEED + 4
+    counts = W.staged_keep_to_flops(net, seed, 0.60) if keep is None else W.uniform_keep(net, keep)
+    kept = W.choose_kept(net, counts, seed)
+    ts = harness.TrainStep(ctx, net, counts, kept, N, seed, host_inputs=False, device_rng=True)
+    ts.step()                       # eager: reconfiguration + training step (sets tables and attributes up)
+    torch.cuda.synchronize()
+    ts.build_graph(two_streams=True)
+    ts.step()                       # the launch configuration the bench times
+    torch.cuda.synchronize()
+    ctx.poll()
+    rng = np.random.default_rng(seed)
+    for li in layer_ids:
+        l = ts.net.layers[li]
+        # the buffers the step used, copied back: the oracle sees exactly the bits the kernels saw
+        x = ts.x[li][..., :l.C].float().cpu().numpy()
+        dy = ts.dy[li][..., :l.K].float().cpu().numpy()
+        # the step's lasso update has already rewritten mp.wb: the convs ran on the weights gathered from the dense model
+        wsrc = oracle.gather_weight(ts.md.wb[li][..., :ts.dense_net.layers[li].C].float().cpu().numpy(),
+                                    kept[ts.net.layers[li].out_space], kept[ts.net.layers[li].in_space])
+        y = ts.y[li][..., :l.K].float().cpu().numpy()
+        idx = rng.integers(0, y.size, n_samples)
+        ref = oracle.conv_fwd_samples(x, wsrc, idx, l.stride, l.pad)
+        rms = float(np.sqrt(np.mean(ref ** 2))) if np.any(ref) else 1.0
+        Hh.check_samples(y.ravel()[idx], ref, rms, True, f"{l.name} fwd N={N}")
+        if li > 0:
+            dx = ts.dx[li][..., :l.C].float().cpu().numpy()
+            idx = rng.integers(0, dx.size, n_samples)
+            ref = oracle.conv_dgrad_samples(dy, wsrc, idx, l.H, l.H, l.stride, l.pad)
+            rms = float(np.sqrt(np.mean(ref ** 2)))
+            Hh.check_samples(dx.ravel()[idx], ref, rms, True, f"{l.name} dgrad N={N}")
+        dw = ts.mp.g[li].cpu().numpy()
+        if dw.size <= full_dw_below:
+            idx = np.arange(dw.size)
+        else:
+            idx = rng.integers(0, dw.size, 512)
+        ref = oracle.conv_wgrad_samples(x, dy, idx, l.R, l.R, l.stride, l.pad)
+        rms = float(np.sqrt(np.mean(ref ** 2)))
+        Hh.check_samples(dw.ravel()[idx], ref, rms, False, f"{l.name} wgrad N={N}")
+    return ts
+
+
+def test_config4_full_size_sampled_batch64():
+    # stem, 1x1 / 3x3 / stride-2 / shortcut layers of every stage
+    _sampled_step_check(None, 64, [0, 1, 2, 3, 4, 10, 12, 13, 14, 24, 25, 27, 43, 44, 46, 52])
+
+
+@pytest.mark.parametrize("keep,N", [(0.3, 256), (0.6, 128), (1.0, 64)])
+def test_config5_sweep_points_sampled(keep, N):
+    _sampled_step_check(keep, N, [0, 2, 12, 26, 45], n_samples=2048)

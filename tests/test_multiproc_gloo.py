@@ -1,0 +1,42 @@
+"""The N > 1 path of bench.py shards nothing on the data path (independent replicas, no collective): what the ranks
+share is the barrier, the max-over-ranks step time and the whole-job aggregation. That host logic is exercised here with
+two gloo ranks on the CPU."""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms_local = 10.0 + 5.0 * rank                    # rank 1 is the slower replica
+    ms = bench.max_over_ranks(ms_local, world, device="cpu")
+    value = bench.whole_job_value(flops_per_rank=2.0e12, world=world, ms_total=ms, steps=4)
+    dist.barrier()
+    out[rank] = (ms, value)
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_take_the_max_time_and_sum_the_work():
+    world, port = 2, 29731
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+        for rank in range(world):
+            ms, value = out[rank]
+            assert ms == 15.0                                         # the slowest rank's time on every rank
+            assert abs(value - 2 * 2.0e12 / (15.0e-3 / 4) / 1e12) < 1e-9   # both ranks' FLOPs over that time, TFLOP/s
+
+
+def test_single_rank_is_the_identity():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(7.5, 1, device="cpu") == 7.5
+    assert abs(bench.whole_job_value(1e12, 1, 10.0, 10) - 1.0e12 / 1e-3 / 1e12) < 1e-9
