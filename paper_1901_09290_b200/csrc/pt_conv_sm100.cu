@@ -354,6 +354,7 @@ struct HaloP {
     int a_box_bytes, a_alloc;            // bytes one A load brings / bytes reserved per A stage
     int stages_a, stages_b, resident;    // ring depths; resident: weights loaded once
     int tmem_cols, tma_store, out_f32, ld_out;
+    int oH, oW, o_step, o_h0, o_w0;      // direct stores: raster (n, i, j) -> out[((n*oH + i*o_step + o_h0)*oW + j*o_step + o_w0)*ld_out]
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];
@@ -576,7 +577,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
             // ---- direct stores (fp32 outputs)
             const int i = m / p.Wp, j = m - i * p.Wp;
             const bool row_ok = m < p.nr * p.Wp && j < p.Q && p0 + i < p.P;
-            const size_t row_off = ((size_t)(img * p.P + p0 + i) * p.Q + j) * (size_t)p.ld_out;
+            const size_t row_off = ((size_t)(img * p.oH + (p0 + i) * p.o_step + p.o_h0) * p.oW + j * p.o_step + p.o_w0) * (size_t)p.ld_out;
             for (int c0 = 0; c0 < p.BN; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld16(lane_addr + (uint32_t)c0, v);
@@ -1128,37 +1129,44 @@ bool make_halo_in_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C,
     return r == CUDA_SUCCESS;
 }
 
-// Stride-1 RxS convolution (fwd) or its data gradient through the halo kernel. Returns PT_ERR_UNSUPPORTED when the shape
-// does not suit it (the caller then uses the per-tap im2col kernel).
-//   src: activations read (x or dy), (Cs channels, Ws x Hs pixels, pitch lds); out: (n_cols channels, Q x P pixels, pitch ld_out)
+// One launch of the halo kernel: a stride-1 correlation of `src` with a list of taps, written to a (possibly strided)
+// view of the output.
+struct HaloSpec {
+    const void *src; int Cs, Ws, Hs, lds;            // activations read: channels, width, height, pitch
+    int P, Q;                                        // output raster per image (rows, columns)
+    int n_taps, span_h, span_w;                      // taps and the extent of their offsets (max offset + 1)
+    int lo_h, lo_w;                                  // source coordinate of raster (0,0) at tap offset (0,0)
+    int tap_oh[kMaxTaps], tap_ow[kMaxTaps], tap_wt[kMaxTaps];
+    int n_cols, ld_out;                              // output channels and pitch
+    int oH, oW, o_step, o_h0, o_w0;                  // output view: raster (i, j) -> pixel (i*o_step + o_h0, j*o_step + o_w0) of oH x oW
+};
+
 template <bool B_MN>
-pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const void *src, int Cs, int Ws, int Hs, int lds, const void *w, void *out,
-                      int n_cols, int P, int Q, int ld_out, int pad_h, int pad_w, bool flip, cudaStream_t st)
+pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const void *w, void *out, cudaStream_t st)
 {
-    const int R = d->R, S = d->S, taps = R * S;
-    const int Wp = Q + S - 1;
-    if (taps < 2 || taps > kMaxTaps || Wp > 128 || Ws > 250) return PT_ERR_UNSUPPORTED;
+    const int Wp = h.Q + h.span_w - 1;
+    if (h.n_taps < 1 || h.n_taps > kMaxTaps || Wp > 128 || h.Ws > 250) return PT_ERR_UNSUPPORTED;
     HaloP p;
     memset(&p, 0, sizeof(p));
-    p.N = d->N; p.P = P; p.Q = Q; p.Wp = Wp;
-    p.nr = 128 / Wp < P ? 128 / Wp : P;
-    p.row_tiles = pt_ceil_div(P, p.nr);
-    p.n_cols = n_cols;
-    p.BN = tile_n(n_cols, &p.n_tiles);
-    p.c_red = Cs; p.k_chunks = pt_ceil_div(Cs, kKC); p.taps = taps;
-    p.lo_h = -pad_h; p.lo_w = -pad_w;
-    for (int t = 0; t < taps; ++t) {
-        p.tap_oh[t] = (unsigned char)(t / S); p.tap_ow[t] = (unsigned char)(t % S);
-        p.tap_wt[t] = (unsigned short)(flip ? taps - 1 - t : t);
+    p.N = d->N; p.P = h.P; p.Q = h.Q; p.Wp = Wp;
+    p.nr = 128 / Wp < h.P ? 128 / Wp : h.P;
+    p.row_tiles = pt_ceil_div(h.P, p.nr);
+    p.n_cols = h.n_cols;
+    p.BN = tile_n(h.n_cols, &p.n_tiles);
+    p.c_red = h.Cs; p.k_chunks = pt_ceil_div(h.Cs, kKC); p.taps = h.n_taps;
+    p.lo_h = h.lo_h; p.lo_w = h.lo_w;
+    for (int t = 0; t < h.n_taps; ++t) {
+        p.tap_oh[t] = (unsigned char)h.tap_oh[t]; p.tap_ow[t] = (unsigned char)h.tap_ow[t];
+        p.tap_wt[t] = (unsigned short)h.tap_wt[t];
     }
-    const int box_h = p.nr + R - 1;
+    const int box_h = p.nr + h.span_h - 1;
     if (box_h > 256) return PT_ERR_UNSUPPORTED;
     p.a_box_bytes = box_h * Wp * 128;
-    const int need_rows = 128 + (R - 1) * Wp + S - 1;          // rows the M = 128 MMAs of the last tap touch
+    const int need_rows = 128 + (h.span_h - 1) * Wp + h.span_w - 1;   // rows the M = 128 MMAs of the last tap touch
     p.a_alloc = (int)pt_align_up((size_t)(need_rows > box_h * Wp ? need_rows : box_h * Wp) * 128, 1024);
     const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : pt_align_up((size_t)p.BN * 128, 1024);
     const size_t budget = 222 * 1024 - 2048 - kHaloStaging;
-    const size_t w_all = (size_t)taps * p.k_chunks * b_bytes;
+    const size_t w_all = (size_t)h.n_taps * p.k_chunks * b_bytes;
     p.resident = (p.n_tiles == 1 && w_all + 2 * (size_t)p.a_alloc <= budget) ? 1 : 0;
     size_t left = budget - (p.resident ? w_all : 0);
     if (!p.resident) {
@@ -1177,18 +1185,23 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const void *src, int Cs,
     }
     if (p.stages_a < 2) return PT_ERR_UNSUPPORTED;
     p.tmem_cols = pow2_cols(2 * p.BN);
-    p.out = out; p.ld_out = ld_out; p.out_f32 = d->out_f32;
+    p.out = out; p.ld_out = h.ld_out; p.out_f32 = d->out_f32;
+    p.oH = h.oH; p.oW = h.oW; p.o_step = h.o_step; p.o_h0 = h.o_h0; p.o_w0 = h.o_w0;
     p.tma_store = d->out_f32 ? 0 : 1;
     p.status = c->d_status;
     CUtensorMap tmA, tmB, tmC;
     memset(&tmC, 0, sizeof(tmC));
-    if (!make_halo_in_map(c, &tmA, src, Cs, Ws, Hs, d->N, lds, Wp, box_h)) return PT_ERR_CUDA;
-    if (!make_weight_map(c, &tmB, w, d->C, taps, d->K, d->ldw, B_MN ? kKC : p.BN)) return PT_ERR_CUDA;
+    if (!make_halo_in_map(c, &tmA, h.src, h.Cs, h.Ws, h.Hs, d->N, h.lds, Wp, box_h)) return PT_ERR_CUDA;
+    if (!make_weight_map(c, &tmB, w, d->C, d->R * d->S, d->K, d->ldw, B_MN ? kKC : p.BN)) return PT_ERR_CUDA;
     if (p.tma_store) {
-        cuuint64_t dims[4] = {(cuuint64_t)n_cols, (cuuint64_t)Q, (cuuint64_t)P, (cuuint64_t)d->N};
-        cuuint64_t strides[3] = {(cuuint64_t)ld_out * 2, (cuuint64_t)Q * ld_out * 2, (cuuint64_t)P * Q * ld_out * 2};
+        // the output view as a 4-D tensor (channels, raster columns, raster rows, images); strided when o_step > 1
+        const size_t es = 2;
+        char *base = (char *)out + ((size_t)h.o_h0 * h.oW + h.o_w0) * h.ld_out * es;
+        cuuint64_t dims[4] = {(cuuint64_t)h.n_cols, (cuuint64_t)h.Q, (cuuint64_t)h.P, (cuuint64_t)d->N};
+        cuuint64_t strides[3] = {(cuuint64_t)h.o_step * h.ld_out * es, (cuuint64_t)h.o_step * h.oW * h.ld_out * es,
+                                 (cuuint64_t)h.oH * h.oW * h.ld_out * es};
         cuuint32_t box[4] = {64, (cuuint32_t)Wp, (cuuint32_t)p.nr, 1}, estr[4] = {1, 1, 1, 1};
-        CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmC, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, out, dims, strides, box, estr,
+        CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmC, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
                                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                       CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
@@ -1205,6 +1218,22 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const void *src, int Cs,
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
+}
+
+// Stride-1 RxS forward (flip = false, src = x) or data gradient (flip = true, src = dy, padding R-1-pad).
+void halo_spec_stride1(const pt_conv_desc *d, HaloSpec *h, const void *src, int Cs, int Ws, int Hs, int lds, int n_cols, int P, int Q,
+                       int ld_out, int pad_h, int pad_w, bool flip)
+{
+    memset(h, 0, sizeof(*h));
+    h->src = src; h->Cs = Cs; h->Ws = Ws; h->Hs = Hs; h->lds = lds;
+    h->P = P; h->Q = Q; h->n_taps = d->R * d->S; h->span_h = d->R; h->span_w = d->S;
+    h->lo_h = -pad_h; h->lo_w = -pad_w;
+    for (int t = 0; t < h->n_taps && t < kMaxTaps; ++t) {
+        h->tap_oh[t] = t / d->S; h->tap_ow[t] = t % d->S;
+        h->tap_wt[t] = flip ? h->n_taps - 1 - t : t;
+    }
+    h->n_cols = n_cols; h->ld_out = ld_out;
+    h->oH = P; h->oW = Q; h->o_step = 1; h->o_h0 = 0; h->o_w0 = 0;
 }
 
 int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
@@ -1292,6 +1321,59 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(tmA, tmX, tmP, p);
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
+    return PT_OK;
+}
+
+// Stride-2 data gradient of a bf16 dx with even H and W: the input pixels split by the parity (a, b) of (h, w) into four
+// stride-1 correlations over dy (pixel h = 2i + a receives tap r iff a + pad - r is even, from dy row i + (a + pad - r)/2).
+// Each parity with taps is one halo-kernel launch that TMA-stores into the strided view of dx holding that parity; if some
+// parity has no tap (1x1 stride 2), dx is cleared first. Returns PT_ERR_UNSUPPORTED for shapes the halo kernel declines
+// (nothing has been launched then).
+pt_status dgrad_stride2_halo(pt_ctx *c, const pt_conv_desc *d, int P, int Q, const void *dy, const void *w, void *dx, cudaStream_t st)
+{
+    HaloSpec hs[4];
+    int n_launch = 0;
+    bool any_empty = false;
+    for (int ab = 0; ab < 4; ++ab) {
+        const int pa = ab >> 1, pb = ab & 1;
+        HaloSpec &h = hs[n_launch];
+        memset(&h, 0, sizeof(h));
+        int oh[kMaxTaps], ow[kMaxTaps], nt = 0;
+        for (int r = 0; r < d->R; ++r) {
+            if ((pa + d->pad - r) & 1) continue;
+            for (int sft = 0; sft < d->S; ++sft) {
+                if ((pb + d->pad - sft) & 1) continue;
+                if (nt >= kMaxTaps) return PT_ERR_UNSUPPORTED;
+                oh[nt] = (pa + d->pad - r) / 2; ow[nt] = (pb + d->pad - sft) / 2;
+                h.tap_wt[nt] = r * d->S + sft;
+                ++nt;
+            }
+        }
+        if (nt == 0) { any_empty = true; continue; }
+        int min_oh = oh[0], min_ow = ow[0], max_oh = oh[0], max_ow = ow[0];
+        for (int t = 0; t < nt; ++t) {
+            min_oh = oh[t] < min_oh ? oh[t] : min_oh; max_oh = oh[t] > max_oh ? oh[t] : max_oh;
+            min_ow = ow[t] < min_ow ? ow[t] : min_ow; max_ow = ow[t] > max_ow ? ow[t] : max_ow;
+        }
+        for (int t = 0; t < nt; ++t) { h.tap_oh[t] = oh[t] - min_oh; h.tap_ow[t] = ow[t] - min_ow; }
+        h.src = dy; h.Cs = d->K; h.Ws = Q; h.Hs = P; h.lds = d->ldy;
+        h.P = d->H / 2; h.Q = d->W / 2;
+        h.n_taps = nt; h.span_h = max_oh - min_oh + 1; h.span_w = max_ow - min_ow + 1;
+        h.lo_h = min_oh; h.lo_w = min_ow;
+        h.n_cols = d->C; h.ld_out = d->ldx;
+        h.oH = d->H; h.oW = d->W; h.o_step = 2; h.o_h0 = pa; h.o_w0 = pb;
+        if (h.Q + h.span_w - 1 > 128) return PT_ERR_UNSUPPORTED;
+        ++n_launch;
+    }
+    if (n_launch == 0) return PT_ERR_UNSUPPORTED;
+    // a 1x1 filter on tiny images: one image fills less than half of a 128-row tile and the reduction is deep, so the
+    // pixel-linear tiles of the im2col kernel do better
+    if (d->R * d->S == 1 && (d->H / 2) * (d->W / 2) < 64) return PT_ERR_UNSUPPORTED;
+    if (any_empty) PT_CUDA_OK(cudaMemsetAsync(dx, 0, (size_t)d->N * d->H * d->W * d->ldx * 2, st));
+    for (int i = 0; i < n_launch; ++i) {
+        pt_status r = launch_halo<true>(c, d, hs[i], w, dx, st);
+        if (r != PT_OK) return r == PT_ERR_UNSUPPORTED && i == 0 && !any_empty ? r : (r == PT_ERR_UNSUPPORTED ? PT_ERR_CUDA : r);
+    }
     return PT_OK;
 }
 
@@ -1391,14 +1473,22 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         if (!make_weight_map(c, &tmB, w2, 64, sp.U, d->K, 64, p.BN)) return PT_ERR_CUDA;
         return launch_gemm<false>(c, tmA, tmB, p, st);
     }
-    if (which == PT_CONV_FWD && d->stride == 1 && d->R * d->S > 1) {
-        pt_status r = launch_halo<false>(c, d, a, d->C, d->W, d->H, d->ldx, b, out, d->K, P, Q, d->ldy, d->pad, d->pad, false, st);
+    if (which == PT_CONV_FWD && d->stride == 1 && d->R * d->S > 1 && d->R * d->S <= kMaxTaps) {
+        HaloSpec h;
+        halo_spec_stride1(d, &h, a, d->C, d->W, d->H, d->ldx, d->K, P, Q, d->ldy, d->pad, d->pad, false);
+        pt_status r = launch_halo<false>(c, d, h, b, out, st);
         if (r != PT_ERR_UNSUPPORTED) return r;
     }
-    if (which == PT_CONV_DGRAD && d->stride == 1 && d->R * d->S > 1 && d->pad <= d->R - 1 && d->pad <= d->S - 1) {
+    if (which == PT_CONV_DGRAD && d->stride == 1 && d->R * d->S > 1 && d->R * d->S <= kMaxTaps && d->pad <= d->R - 1 &&
+        d->pad <= d->S - 1) {
         // dx = correlation of dy (padding R-1-pad) with the taps visited flipped
-        pt_status r = launch_halo<true>(c, d, a, d->K, Q, P, d->ldy, b, out, d->C, d->H, d->W, d->ldx, d->R - 1 - d->pad,
-                                        d->S - 1 - d->pad, true, st);
+        HaloSpec h;
+        halo_spec_stride1(d, &h, a, d->K, Q, P, d->ldy, d->C, d->H, d->W, d->ldx, d->R - 1 - d->pad, d->S - 1 - d->pad, true);
+        pt_status r = launch_halo<true>(c, d, h, b, out, st);
+        if (r != PT_ERR_UNSUPPORTED) return r;
+    }
+    if (which == PT_CONV_DGRAD && d->stride == 2 && !d->out_f32 && (d->H % 2 == 0) && (d->W % 2 == 0)) {
+        pt_status r = dgrad_stride2_halo(c, d, P, Q, a, b, out, st);
         if (r != PT_ERR_UNSUPPORTED) return r;
     }
     if (which == PT_CONV_FWD) {
