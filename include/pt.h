@@ -48,7 +48,7 @@ typedef enum {
     PT_ERR_ARCH = 6           /* the device is not sm_100                               */
 } pt_status;
 
-typedef struct pt_ctx pt_ctx;  /* opaque: device id, SM count, status word, table arena, tensor-map cache */
+typedef struct pt_ctx pt_ctx;  /* opaque: device id, SM count, status word, table arena, arrival counters */
 
 /* Create / destroy the per-device context. pt_create makes `device` current, checks that it is
  * an sm_100 part (else PT_ERR_ARCH) and allocates the status word and table arena. */

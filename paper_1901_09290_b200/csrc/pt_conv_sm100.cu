@@ -1,17 +1,16 @@
 // tcgen05 / TMEM / TMA implicit-GEMM convolutions for sm_100a.
 //
-// conv_gemm_kernel  (fwd, dgrad):  D[pixel][channel] = sum over taps and reduction channels.
-//   A operand: 128 output pixels x 64 reduction channels per stage, fetched by ONE im2col-mode TMA load
-//              (the TMA unit walks the output-pixel raster with the conv stride and adds the tap offset,
-//              zero-filling the padding halo and the channels past the true, ragged channel count).
-//   B operand: the bf16 weight shadow [K][R*S][ldw].
-//              fwd   : rows = output channels, 64 input channels contiguous  -> K-major tile, one 3-D TMA box.
-//              dgrad : rows = 64 output channels (the reduction), input channels contiguous -> MN-major tiles
-//                      straight from the same shadow, taps visited flipped. No transposed copy of the weights.
-//   Accumulator: fp32 in TMEM, 128 lanes x BN columns (BN = the ragged channel count rounded up to 16, <= 256).
-//   Roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue
-//          (tcgen05.ld -> bf16/fp32 -> predicated stores at the true channel count).
-// Every mbarrier wait is bounded; on expiry the CTA records PT_DEV_TIMEOUT in the status word, drains and exits.
+//   conv_gemm_kernel   fwd and dgrad of 1x1 / strided layers: persistent CTAs, im2col-mode (or plain 2-D) TMA loads of
+//                      128 pixels x 64 channels, K-major (fwd) or MN-major (dgrad) weight tiles from the same bf16 shadow,
+//                      double/triple-buffered fp32 accumulators in TMEM, TMA-store epilogue.
+//   conv_halo_kernel   stride-1 RxS fwd/dgrad and the parities of a stride-2 dgrad: one halo tile per 64-channel chunk,
+//                      filter taps as row-shifted UMMA descriptors of that tile.
+//   conv_wgrad_kernel  weight gradient: both operands MN-major, reduction over pixels split across CTAs, partial tiles
+//                      summed in-kernel in a fixed order.
+//   stem_* kernels     space-to-depth layout kernels of the few-channel stride-2 stem.
+// Ragged channel counts are handled by the TMA unit (true extents in the tensor maps: zero-fill on load, clipping on
+// store) and by skipping the 16-wide k-steps past the last valid channel.
+// Every wait is bounded; on expiry the CTA records PT_DEV_TIMEOUT in the status word, drains its copies and exits.
 #include "pt_internal.h"
 #include "pt_sm100_ptx.cuh"
 #include <cudaTypedefs.h>

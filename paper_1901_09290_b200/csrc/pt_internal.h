@@ -5,8 +5,6 @@
 #include <stdint.h>
 #include <string.h>
 #include <vector>
-#include <map>
-#include <string>
 
 #include "../../include/pt.h"
 
@@ -47,7 +45,6 @@ struct pt_ctx {
     // tcgen05 conv path
     void *encode_tiled = nullptr;       // cuTensorMapEncodeTiled
     void *encode_im2col = nullptr;      // cuTensorMapEncodeIm2col
-    std::map<std::string, std::vector<char>> tmap_cache;
 };
 
 static inline int pt_ceil_div(int a, int b) { return (a + b - 1) / b; }
