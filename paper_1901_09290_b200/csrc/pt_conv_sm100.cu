@@ -622,13 +622,14 @@ struct WgradP {
     int K, C, taps;         // true channel counts, number of taps (R*S)
     int BN, n_tiles;        // input-channel tile
     int m_tiles;            // ceil(K / 128)
+    int tpc, tap_groups;    // taps per CTA (they share the dy tile; one accumulator of BN columns each) and groups of taps
     int npix;               // N*P*Q
     int pix_per_split;      // multiple of 64
     int splits;
     int Pd, Qd, stride, lo_h, lo_w, S;
     int stages, tmem_cols;
     float *out;             // dw
-    float *partial;         // splits > 1: workspace [blockIdx.x][split][128][BN] fp32
+    float *partial;         // splits > 1: workspace [blockIdx.x][tap in group][split][128][BN] fp32
     unsigned int *sync;     // splits > 1: two zeroed counters per blockIdx.x (arrived, reduced); left zero again at exit
     unsigned int *status;
 };
@@ -643,15 +644,16 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
     const uint32_t data_base = (smem_base + (uint32_t)sizeof(Ctl) + 1023u) & ~1023u;
     const uint32_t a_bytes = 2u * 8192u;
     const uint32_t nb_b = (uint32_t)((p.BN + 63) / 64);
-    const uint32_t b_bytes = nb_b * 8192u;
-    const uint32_t stage_bytes = a_bytes + b_bytes;
+    const uint32_t b_bytes = nb_b * 8192u;                            // one tap's x tile
+    const uint32_t stage_bytes = a_bytes + (uint32_t)p.tpc * b_bytes;
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int bx = blockIdx.x;
     const int n_tile = bx % p.n_tiles; bx /= p.n_tiles;
     const int m_tile = bx % p.m_tiles; bx /= p.m_tiles;
-    const int tap = bx;
+    const int tap0 = bx * p.tpc;                                      // this CTA's taps: tap0 .. tap0 + ntap - 1
+    const int ntap = min(p.tpc, p.taps - tap0);
     const int split = blockIdx.y;
     const int k0 = m_tile * 128, c0 = n_tile * p.BN;
     const int pix_beg = split * p.pix_per_split;
@@ -680,7 +682,6 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
 
     if (warp == 0) {
         if (lane == 0) {
-            const int r = tap / p.S, sft = tap - r * p.S;
             int issued = 0;
             for (int it = 0; it < iters; ++it) {
                 const int s = it % p.stages, ph = (it / p.stages) & 1;
@@ -692,12 +693,15 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 // output channels k0+64.. of this tile do not exist when K - k0 <= 64: their accumulator rows are never
                 // stored, so that half of the A tile is not loaded at all (the MMA reads stale shared memory there)
                 const bool second = p.K - k0 > 64;
-                mbar_arrive_expect_tx(bar, (second ? a_bytes : 8192u) + b_bytes);
+                mbar_arrive_expect_tx(bar, (second ? a_bytes : 8192u) + (uint32_t)ntap * b_bytes);
                 tma_load_2d(a_dst, &tmDy, bar, k0, pix);
                 if (second) tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
-                for (uint32_t nb = 0; nb < nb_b; ++nb)
-                    tma_load_im2col_4d(b_dst + nb * 8192u, &tmX, bar, c0 + (int)nb * 64, q * p.stride + p.lo_w,
-                                       pp * p.stride + p.lo_h, n, (uint16_t)sft, (uint16_t)r);
+                for (int tt = 0; tt < ntap; ++tt) {                  // the dy tile is fetched once for all of these taps
+                    const int r = (tap0 + tt) / p.S, sft = (tap0 + tt) - r * p.S;
+                    for (uint32_t nb = 0; nb < nb_b; ++nb)
+                        tma_load_im2col_4d(b_dst + (uint32_t)tt * b_bytes + nb * 8192u, &tmX, bar, c0 + (int)nb * 64,
+                                           q * p.stride + p.lo_w, pp * p.stride + p.lo_h, n, (uint16_t)sft, (uint16_t)r);
+                }
                 issued = it + 1;
             }
             if (*abort_flag) {
@@ -720,10 +724,14 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 const int rem = pix_end - (pix_beg + it * 64);
                 const int ksteps = rem >= 64 ? 4 : (rem + 15) / 16;
                 const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
-                const uint64_t ad0 = make_desc(a_src, 8192u, 1024u), bd0 = make_desc(b_src, 8192u, 1024u);
+                const uint64_t ad0 = make_desc(a_src, 8192u, 1024u);
+                for (int tt = 0; tt < ntap; ++tt) {
+                    const uint64_t bd0 = make_desc(b_src + (uint32_t)tt * b_bytes, 8192u, 1024u);
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(tt * p.BN);
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    if (k < ksteps) umma_bf16(tmem_base, ad0 + 128ull * k, bd0 + 128ull * k, idesc, (it | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < 4; ++k)
+                        if (k < ksteps) umma_bf16(d_tmem, ad0 + 128ull * k, bd0 + 128ull * k, idesc, (it | k) != 0 ? 1u : 0u);
+                }
                 umma_commit(smem_u32(&ctl->empty[s]));
             }
             if (ok) umma_commit(smem_u32(&ctl->accum));
@@ -742,14 +750,15 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 // ---- (1) this CTA's fp32 partial tile goes to the workspace through swizzled staging + TMA stores
                 const int gtid = (warp - 2) * 32 + lane;
                 int sl = 0;
+                for (int tt = 0; tt < ntap; ++tt)
                 for (int cc = 0; cc < p.BN; cc += 32, sl ^= 1) {
                     const uint32_t slab = data_base + (uint32_t)(quarter * 2 + sl) * 4096u;
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                     uint32_t lo[16], hi[16];
                     if (iters > 0) {
-                        tmem_ld16(lane_addr + (uint32_t)cc, lo);
-                        if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)cc + 16u, hi);
+                        tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc), lo);
+                        if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc) + 16u, hi);
                         tmem_ld_wait();
                     }
 #pragma unroll
@@ -767,7 +776,7 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                     fence_proxy_async();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_2d(&tmP, slab, cc, ((int)blockIdx.x * p.splits + split) * 128 + quarter * 32);
+                        tma_store_2d(&tmP, slab, cc, (((int)blockIdx.x * p.tpc + tt) * p.splits + split) * 128 + quarter * 32);
                         tma_store_commit();
                     }
                 }
@@ -791,12 +800,14 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
             // The stages are free once the accumulator is complete: each warp transposes its 32 x 32 blocks through
             // a padded shared-memory square so that a warp writes 32 consecutive floats of one dw row at a time.
             const uint32_t sq = data_base + (uint32_t)quarter * (32u * 33u * 4u);
+            for (int tt = 0; tt < ntap; ++tt)
             for (int cc = 0; cc < p.BN; cc += 32) {
+                const int tap = tap0 + tt;
                 uint32_t v[32];
                 if (iters > 0) {
                     uint32_t lo[16], hi[16];
-                    tmem_ld16(lane_addr + (uint32_t)cc, lo);
-                    if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)cc + 16u, hi);
+                    tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc), lo);
+                    if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc) + 16u, hi);
                     tmem_ld_wait();
 #pragma unroll
                     for (int e = 0; e < 16; ++e) { v[e] = lo[e]; v[16 + e] = (cc + 16 < p.BN) ? hi[e] : 0u; }
@@ -837,8 +848,10 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
         const int T = p.splits > 96 ? 8 : 1;                         // lanes per item: share only very long split chains
         const int zc = (p.splits + T - 1) / T;
         const int sub = threadIdx.x & (T - 1);
-        const float *pt = p.partial + (size_t)blockIdx.x * p.splits * 128 * p.BN;
         const size_t zstride = (size_t)128 * p.BN;
+        for (int tt = 0; tt < ntap; ++tt) {
+        const int tap = tap0 + tt;
+        const float *pt = p.partial + ((size_t)blockIdx.x * p.tpc + tt) * p.splits * 128 * p.BN;
         for (int base = it_beg; base < it_end; base += kThreads / T) {
             const int item = base + threadIdx.x / T;
             const bool live = item < it_end;
@@ -874,6 +887,7 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 if (nv > 2) dst[2] = sum.z;
                 if (nv > 3) dst[3] = sum.w;
             }
+        }
         }
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -1235,11 +1249,27 @@ void halo_spec_stride1(const pt_conv_desc *d, HaloSpec *h, const void *src, int 
     h->oH = P; h->oW = Q; h->o_step = 1; h->o_h0 = 0; h->o_w0 = 0;
 }
 
+// Taps handled by one weight-gradient CTA: they share the dy tile and get one TMEM accumulator of BN columns each.
+// Bounded by the 512 TMEM columns and by a stage of 16 KB (dy) + taps x BN/64 x 8 KB (x) staying at or below 48 KB, so
+// that at least four pipeline stages fit (measured: with two stages the kernel is slower than with one tap per CTA);
+// the taps are then dealt out in equal groups.
+int wgrad_taps_per_cta(int taps, int bn)
+{
+    int t = 512 / bn;
+    const int by_smem = 4 / pt_ceil_div(bn, 64);
+    if (t > by_smem) t = by_smem;
+    if (t < 1) t = 1;
+    if (t > taps) t = taps;
+    const int groups = pt_ceil_div(taps, t);
+    return pt_ceil_div(taps, groups);
+}
+
 int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
 {
     int n_tiles;
-    tile_n(d->C, &n_tiles);
-    const int tiles = pt_ceil_div(d->K, 128) * n_tiles * d->R * d->S;
+    const int bn = tile_n(d->C, &n_tiles);
+    const int tpc = wgrad_taps_per_cta(d->R * d->S, bn);
+    const int tiles = pt_ceil_div(d->K, 128) * n_tiles * pt_ceil_div(d->R * d->S, tpc);
     const long long npix = (long long)d->N * P * Q;
     long long s = c->sm_count / tiles;                     // one CTA per SM, one wave
     const long long max_s = (npix + 255) / 256;          // at least four 64-pixel stages per split
@@ -1256,7 +1286,8 @@ size_t wgrad_partial_bytes(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     if (s <= 1) return 0;
     int n_tiles;
     const int bn = tile_n(d->C, &n_tiles);
-    return (size_t)n_tiles * pt_ceil_div(d->K, 128) * d->R * d->S * s * 128 * bn * sizeof(float);
+    const int tpc = wgrad_taps_per_cta(d->R * d->S, bn);
+    return (size_t)n_tiles * pt_ceil_div(d->K, 128) * pt_ceil_div(d->R * d->S, tpc) * tpc * s * 128 * bn * sizeof(float);
 }
 
 // Launches the weight-gradient kernel for a problem whose x operand is described by `tmX` (64 pixels x 64 channels boxes).
@@ -1268,18 +1299,20 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     p.K = d->K; p.C = d->C; p.taps = d->R * d->S; p.S = d->S;
     p.BN = tile_n(d->C, &p.n_tiles);
     p.m_tiles = pt_ceil_div(d->K, 128);
+    p.tpc = wgrad_taps_per_cta(p.taps, p.BN);
+    p.tap_groups = pt_ceil_div(p.taps, p.tpc);
     p.npix = d->N * P * Q;
     p.splits = wgrad_splits(c, d, P, Q);
     p.pix_per_split = pt_ceil_div(pt_ceil_div(p.npix, p.splits), 64) * 64;
     p.Pd = P; p.Qd = Q; p.stride = stride; p.lo_h = lo_h; p.lo_w = lo_w;
-    p.tmem_cols = pow2_cols(p.BN);
+    p.tmem_cols = pow2_cols(p.tpc * p.BN);
     p.status = c->d_status;
-    const int gx = p.n_tiles * p.m_tiles * p.taps;
+    const int gx = p.n_tiles * p.m_tiles * p.tap_groups;
     p.out = out;
     CUtensorMap tmP;
     memset(&tmP, 0, sizeof(tmP));
     if (p.splits > 1) {
-        const size_t need = (size_t)gx * p.splits * 128 * p.BN * sizeof(float);
+        const size_t need = (size_t)gx * p.tpc * p.splits * 128 * p.BN * sizeof(float);
         if (!ws || ws_bytes < need) return PT_ERR_WORKSPACE;
         p.partial = (float *)ws;
         // two self-resetting counters per tile from the context's ring (kernels of one stream run in order, and the ring
@@ -1288,7 +1321,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
         if (c->sync_next + 2 * gx > 16384) c->sync_next = 0;
         p.sync = c->d_sync + c->sync_next;
         c->sync_next += 2 * gx;
-        cuuint64_t dims[2] = {(cuuint64_t)p.BN, (cuuint64_t)gx * p.splits * 128};
+        cuuint64_t dims[2] = {(cuuint64_t)p.BN, (cuuint64_t)gx * p.tpc * p.splits * 128};
         cuuint64_t strides[1] = {(cuuint64_t)p.BN * 4};
         cuuint32_t box[2] = {32, 32}, estr[2] = {1, 1};
         CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmP, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ws, dims, strides, box, estr,
@@ -1309,7 +1342,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
         if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
     }
     size_t smem = 0;
-    const size_t stage = 2 * 8192 + (size_t)pt_ceil_div(p.BN, 64) * 8192;
+    const size_t stage = 2 * 8192 + (size_t)p.tpc * pt_ceil_div(p.BN, 64) * 8192;
     p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), 0, &smem);
     static bool attr_set = false;
     if (!attr_set) {
