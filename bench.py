@@ -359,7 +359,8 @@ def run_ours(args):
                    "algo": args.algo,
                    "launch": "eager" if args.no_graph else ("CUDA graph replay after the reconfiguration's host sync; "
                                                             + ("1 stream" if args.one_stream else "dgrad and wgrad of a layer on 2 streams"))},
-        "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "pipeline": "one pinned-host image copy per step on a copy stream, overlapping the previous step's kernels"},
         "gpu_launches": launches,
         "clocks": clocks,
         "phases_ms": {"conv_fwd": conv_ms["fwd"], "conv_dgrad": conv_ms["dgrad"], "conv_wgrad": conv_ms["wgrad"],

@@ -216,8 +216,32 @@ class TrainStep:
             self.train(stream)
 
     def step_e2e(self, stream=None):
-        """The same step with the image batch copied from pinned host memory and the regulariser value read back."""
-        self.x[0].copy_(self.h_image, non_blocking=True)
+        """The same step with the image batch copied from pinned host memory and the regulariser value read back.
+
+        The host-to-device copy runs on a copy stream into a staging buffer, so the copy of the next step's batch
+        overlaps this step's kernels (one copy per step; the first call issues its own). The step itself starts with a
+        device-to-device move of the staged batch into the stem's input."""
+        main = torch.cuda.current_stream()
+        if getattr(self, "_copy_stream", None) is None:
+            self._copy_stream = torch.cuda.Stream()
+            self._x_stage = torch.empty_like(self.x[0])
+            self._ev_copied = torch.cuda.Event()
+            self._ev_free = torch.cuda.Event()
+            self._prefetched = False
+        cs = self._copy_stream
+        if not self._prefetched:
+            cs.wait_stream(main)
+            with torch.cuda.stream(cs):
+                self._x_stage.copy_(self.h_image, non_blocking=True)
+                self._ev_copied.record(cs)
+        main.wait_event(self._ev_copied)
+        self.x[0].copy_(self._x_stage, non_blocking=True)
+        self._ev_free.record(main)
+        cs.wait_event(self._ev_free)
+        with torch.cuda.stream(cs):                      # the next step's batch
+            self._x_stage.copy_(self.h_image, non_blocking=True)
+            self._ev_copied.record(cs)
+        self._prefetched = True
         self.step(stream)
         self.h_reg.copy_(self.mp.reg, non_blocking=True)
 
