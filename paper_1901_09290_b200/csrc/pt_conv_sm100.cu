@@ -352,6 +352,8 @@ struct HaloP {
     int lo_h, lo_w;                      // source coordinate of raster position (0, 0) for tap offset (0, 0)
     int a_box_bytes, a_alloc;            // bytes one A load brings / bytes reserved per A stage
     int stages_a, stages_b, resident;    // ring depths; resident: weights loaded once
+    int n_issuers, acc_per;              // MMA issuer warps (each with its own A ring of stages_a / n_issuers stages); accumulators per issuer (1 or 2)
+    int b_slot, b_rows, staging;         // bytes reserved per weight tile, rows a K-major weight box brings, bytes of an epilogue group's staging slab
     int tmem_cols, tma_store, out_f32, ld_out;
     int oH, oW, o_step, o_h0, o_w0;      // direct stores: raster (n, i, j) -> out[((n*oH + i*o_step + o_h0)*oW + j*o_step + o_w0)*ld_out]
     void *out;
@@ -360,18 +362,32 @@ struct HaloP {
     unsigned short tap_wt[kMaxTaps];
 };
 
+constexpr int kHaloMaxIssuers = 4;
+#ifdef PT_HALO_TRACE
+__device__ unsigned long long g_halo_trace[8][64];
+#define HTRACE(role, idx) do { if (blockIdx.x == 0 && (idx) < 64 && (threadIdx.x & 31) == 0) g_halo_trace[role][idx] = globaltimer_ns(); } while (0)
+#else
+#define HTRACE(role, idx) do { } while (0)
+#endif
+
 struct __align__(8) HCtl {
     uint64_t full_a[4], empty_a[4];
     uint64_t full_b[kMaxStages], empty_b[kMaxStages];
     uint64_t w_full;
-    uint64_t acc_full[2], acc_empty[2];
+    uint64_t acc_full[2 * kHaloMaxIssuers], acc_empty[2 * kHaloMaxIssuers];
+    uint32_t tap_aoff[kMaxTaps];         // row shift of each tap in descriptor units (16 bytes)
     uint32_t tmem_base;
     int abort_flag;
 };
 
-constexpr int kHaloThreads = 320;        // producer warp, MMA warp, two groups of four epilogue warps
-constexpr uint32_t kHaloStaging = 2u * 16384u;
+// warp 0: TMA producer; warp 1 and warps 10..12: MMA issuers; warps 2..9: two groups of four epilogue warps
+constexpr int kHaloThreads = 416;
 
+// Issuing one tcgen05.mma costs the issuing warp 50 to 100 cycles of instruction time, more than a narrow MMA (N <= 64)
+// takes to execute, so with a single issuer the tensor pipe of a small-channel layer idles most of the time. The
+// kernel therefore runs up to four issuer warps, each on its own scheduler: issuer i owns accumulator buffer i and
+// an A ring of its own (a waiter may lag an mbarrier by at most one phase, so issuers cannot share a ring), and takes
+// the tiles i, i + I, i + 2I, ... of the CTA. Weights that stream through a ring keep a single issuer.
 template <bool B_MN>
 __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                      const __grid_constant__ CUtensorMap tmB,
@@ -381,9 +397,10 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     HCtl *ctl = reinterpret_cast<HCtl *>(smem_raw);
     const uint32_t smem_base = smem_u32(smem_raw);
     const uint32_t staging_base = (smem_base + (uint32_t)sizeof(HCtl) + 1023u) & ~1023u;
-    const uint32_t b_base = staging_base + kHaloStaging;
-    const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.BN * 128u;
-    const uint32_t b_slot = (b_bytes + 1023u) & ~1023u;
+    const uint32_t b_base = staging_base + 2u * (uint32_t)p.staging;
+    // bytes one weight tile brings: a K-major tile only holds the rows (output channels) that exist
+    const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.b_rows * 128u;
+    const uint32_t b_slot = (uint32_t)p.b_slot;
     const uint32_t n_bslots = p.resident ? (uint32_t)(p.taps * p.k_chunks) : (uint32_t)p.stages_b;
     const uint32_t a_base = b_base + n_bslots * b_slot;
     volatile int *abort_flag = &ctl->abort_flag;
@@ -391,18 +408,20 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m_tiles = p.N * p.row_tiles;
     const int total_tiles = m_tiles * p.n_tiles;
+    const int NI = p.n_issuers, SR = p.stages_a / NI;        // issuers, A stages per issuer ring
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages_a; ++s) { mbar_init(smem_u32(&ctl->full_a[s]), 1); mbar_init(smem_u32(&ctl->empty_a[s]), 1); }
         for (int s = 0; s < p.stages_b; ++s) { mbar_init(smem_u32(&ctl->full_b[s]), 1); mbar_init(smem_u32(&ctl->empty_b[s]), 1); }
         mbar_init(smem_u32(&ctl->w_full), 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 4); }
+        for (int b = 0; b < 2 * kHaloMaxIssuers; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 4); }
         ctl->abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
         if (p.tma_store) prefetch_tmap(&tmC);
     }
+    if (threadIdx.x < p.taps) ctl->tap_aoff[threadIdx.x] = (uint32_t)(p.tap_oh[threadIdx.x] * p.Wp + p.tap_ow[threadIdx.x]) * 8u;
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), (uint32_t)p.tmem_cols);
         tmem_relinquish();
@@ -411,6 +430,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    const int issuer = warp == 1 ? 0 : warp - 9;             // warps 10, 11, 12 -> issuers 1, 2, 3
 
     if (warp == 0) {
         if (lane == 0) {
@@ -427,17 +447,20 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
                     }
             }
-            int ga = 0, gb = 0;
-            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+            int gb = 0, tc = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tc) {
                 const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
                 const int img = m_tile / p.row_tiles, p0 = (m_tile - img * p.row_tiles) * p.nr;
                 const int n0 = n_tile * p.BN;
+                const int ring = tc % NI;
+                int cnt = (tc / NI) * p.k_chunks;              // chunks this ring has carried before this tile
                 bool ok = true;
-                for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++ga) {
-                    const int sa = ga % p.stages_a, pha = (ga / p.stages_a) & 1;
+                for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++cnt) {
+                    const int sa = ring * SR + cnt % SR, pha = (cnt / SR) & 1;
                     ok = mbar_wait(smem_u32(&ctl->empty_a[sa]), pha ^ 1, abort_flag, p.status, 11);
                     if (!ok) break;
                     const uint32_t bar = smem_u32(&ctl->full_a[sa]);
+                    HTRACE(0, tc);
                     mbar_arrive_expect_tx(bar, (uint32_t)p.a_box_bytes);
                     tma_load_4d(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, &tmA, bar, kc * kKC, p.lo_w, p0 + p.lo_h, img);
                     if (p.resident) continue;
@@ -462,70 +485,93 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                            globaltimer_ns() - t0 < 20000000ull) {}
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
-            const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
-            int ga = 0, gb = 0, tc = 0;
-            bool ok = true;
-            if (p.resident) ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort_flag, p.status, 13);
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tc) {
-                const int b = tc & 1, aph = (tc >> 1) & 1;
-                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 14);
+    } else if (warp == 1 || (warp >= 10 && issuer < NI)) {
+        // ---------------- MMA issuer `issuer`: the whole warp walks the loops in lockstep, lane 0 issues
+        const uint32_t leader = lane == 0 ? 1u : 0u;
+        const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
+        const uint64_t bstep = B_MN ? 128ull : 2ull;
+        const uint32_t b_lbo = B_MN ? 8192u : 16u;
+        int gb = 0;
+        int s_loc = 0, pha = 0;                               // position in this issuer's A ring
+        bool ok = true;
+        if (p.resident) ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort_flag, p.status, 13);
+        int nt = 0;                                           // tiles this issuer has started
+        for (int tc = issuer; ok; tc += NI, ++nt) {
+            const int tile = blockIdx.x + tc * (int)gridDim.x;
+            if (tile >= total_tiles) break;
+            // accumulator buffers issuer*acc_per .. +acc_per-1, used in turn
+            const int b = p.acc_per == 2 ? issuer * 2 + (nt & 1) : issuer, aph = p.acc_per == 2 ? (nt >> 1) & 1 : nt & 1;
+            ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 14);
+            if (!ok) break;
+            HTRACE(1, tc);
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(b * p.BN);
+            uint32_t accumulate = 0u;
+            for (int kc = 0; kc < p.k_chunks && ok; ++kc) {
+                const int sa = issuer * SR + s_loc;
+                ok = mbar_wait(smem_u32(&ctl->full_a[sa]), pha, abort_flag, p.status, 15);
                 if (!ok) break;
+                HTRACE(2, tc);
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(b * p.BN);
-                for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++ga) {
-                    const int sa = ga % p.stages_a, pha = (ga / p.stages_a) & 1;
-                    ok = mbar_wait(smem_u32(&ctl->full_a[sa]), pha, abort_flag, p.status, 15);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const int rem = p.c_red - kc * kKC;
-                    const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
-                    const uint32_t a_src = a_base + (uint32_t)sa * (uint32_t)p.a_alloc;
-                    for (int tap = 0; tap < p.taps; ++tap) {
-                        uint32_t b_src;
-                        int sb = 0;
-                        if (p.resident) {
-                            b_src = b_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot;
-                        } else {
-                            sb = gb % p.stages_b;
-                            const int phb = (gb / p.stages_b) & 1;
-                            ++gb;
-                            ok = mbar_wait(smem_u32(&ctl->full_b[sb]), phb, abort_flag, p.status, 16);
-                            if (!ok) break;
-                            tc_fence_after();
-                            b_src = b_base + (uint32_t)sb * b_slot;
+                const int rem = p.c_red - kc * kKC;
+                const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
+                const uint64_t abase = make_desc(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, 16u, 1024u);
+                if (p.resident) {
+                    // every tap is the same A tile read through a descriptor that starts (r*Wp + s) rows further on
+                    uint64_t bd0 = make_desc(b_base + (uint32_t)kc * b_slot, b_lbo, 1024u);
+                    const uint64_t b_tap_step = (uint64_t)(((uint32_t)p.k_chunks * b_slot) >> 4);
+                    if (ksteps == 4) {
+                        for (int tap = 0; tap < p.taps; ++tap, bd0 += b_tap_step) {
+                            const uint64_t ad0 = abase + ctl->tap_aoff[tap];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) { umma_bf16_lead(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, accumulate, leader); accumulate = 1u; }
                         }
-                        // the tap is a row shift of the same A tile
-                        const uint32_t a_tap = a_src + (uint32_t)(p.tap_oh[tap] * p.Wp + p.tap_ow[tap]) * 128u;
-                        const uint64_t ad0 = make_desc(a_tap, 16u, 1024u);
-                        const uint64_t bd0 = B_MN ? make_desc(b_src, 8192u, 1024u) : make_desc(b_src, 16u, 1024u);
-                        const uint64_t bstep = B_MN ? 128ull : 2ull;
+                    } else {
+                        for (int tap = 0; tap < p.taps; ++tap, bd0 += b_tap_step) {
+                            const uint64_t ad0 = abase + ctl->tap_aoff[tap];
+                            for (int k = 0; k < ksteps; ++k) { umma_bf16_lead(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, accumulate, leader); accumulate = 1u; }
+                        }
+                    }
+                } else {
+                    for (int tap = 0; tap < p.taps; ++tap, ++gb) {
+                        const int sb = gb % p.stages_b, phb = (gb / p.stages_b) & 1;
+                        ok = mbar_wait(smem_u32(&ctl->full_b[sb]), phb, abort_flag, p.status, 16);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t ad0 = abase + ctl->tap_aoff[tap];
+                        const uint64_t bd0 = make_desc(b_base + (uint32_t)sb * b_slot, b_lbo, 1024u);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            if (k < ksteps) umma_bf16(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, (kc | tap | k) != 0 ? 1u : 0u);
-                        if (!p.resident) umma_commit(smem_u32(&ctl->empty_b[sb]));
+                            if (k < ksteps) { umma_bf16_lead(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, accumulate, leader); accumulate = 1u; }
+                        umma_commit_lead(smem_u32(&ctl->empty_b[sb]), leader);
                     }
-                    if (ok) umma_commit(smem_u32(&ctl->empty_a[sa]));
                 }
-                if (ok) umma_commit(smem_u32(&ctl->acc_full[b]));
+                if (ok) umma_commit_lead(smem_u32(&ctl->empty_a[sa]), leader);
+                if (++s_loc == SR) { s_loc = 0; pha ^= 1; }
             }
+            if (ok) umma_commit_lead(smem_u32(&ctl->acc_full[b]), leader);
+            HTRACE(3, tc);
         }
-    } else {
-        // ---------------- epilogue: group g (four warps) drains accumulator buffer g
+    } else if (warp >= 2 && warp < 10) {
+        // ---------------- epilogue: group g (four warps) drains the accumulator buffers of its parity
         const int quarter = warp & 3, group = (warp - 2) >> 2;
         const int gtid = (warp - 2 - group * 4) * 32 + lane;         // 0..127 within the group
-        const uint32_t slab = staging_base + (uint32_t)group * 16384u;
-        int tc = group;
+        const uint32_t slab = staging_base + (uint32_t)group * (uint32_t)p.staging;
         bool ok = true;
-        for (int tile = blockIdx.x + group * gridDim.x; tile < total_tiles && ok; tile += 2 * gridDim.x, tc += 2) {
-            const int b = group, aph = (tc >> 1) & 1;
+        const int step = NI == 1 ? 1 : 2;                     // one issuer: the groups alternate tiles like its two buffers
+        for (int tc = group; ok; tc += 2) {
+            const int tile = blockIdx.x + tc * (int)gridDim.x;
+            if (tile >= total_tiles) break;
+            // tile tc is the nt-th tile of issuer tc % NI (NI is 1 or even, so a group always serves the same issuers)
+            const int iss = NI == 1 ? 0 : tc % NI, nt = NI == 1 ? tc : tc / NI;
+            const int b = p.acc_per == 2 ? iss * 2 + (nt & 1) : iss, aph = p.acc_per == 2 ? (nt >> 1) & 1 : nt & 1;
+            (void)step;
             const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
             const int img = m_tile / p.row_tiles, p0 = (m_tile - img * p.row_tiles) * p.nr;
             const int n0 = n_tile * p.BN;
             ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 17);
             if (!ok) break;
+            if (gtid == 0) HTRACE(4, tc);
             tc_fence_after();
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.BN);
             const int m = quarter * 32 + lane;                       // raster position of this thread's accumulator row
@@ -533,6 +579,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                 const int n_chunks = (p.BN + 63) / 64;
                 for (int ch = 0; ch < n_chunks; ++ch) {
                     if (gtid == 0) tma_store_wait_read();            // the slab's previous store has read it
+                    if (gtid == 0) HTRACE(5, tc);
                     named_barrier(1 + group, 128);
                     const int groups = min(4, (p.BN - ch * 64) / 16);
                     uint32_t v[4][16];
@@ -542,7 +589,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                     tmem_ld_wait();
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
-                        if (g >= groups) break;
+                        if (g >= groups || m >= p.nr * p.Wp) break;   // the slab only holds the tile's raster rows
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 0]), __uint_as_float(v[g][8 * h + 1]));
@@ -567,8 +614,10 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                     // one store per tile and chunk: box = nr rows x Wp columns x 64 channels; the columns past Q, the rows
                     // past P and the channels past the true count fall outside the tensor and are dropped
                     if (gtid == 0) {
+                        HTRACE(6, tc);
                         tma_store_4d(&tmC, slab, n0 + ch * 64, 0, p0, img);
                         tma_store_commit();
+                        HTRACE(7, tc);
                     }
                 }
                 continue;
@@ -1119,7 +1168,7 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     p.tmem_cols = pow2_cols(p.epi_groups * p.BN);
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
-        PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set[B_MN ? 1 : 0] = true;
     }
     const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
@@ -1175,10 +1224,19 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     const int box_h = p.nr + h.span_h - 1;
     if (box_h > 256) return PT_ERR_UNSUPPORTED;
     p.a_box_bytes = box_h * Wp * 128;
-    const int need_rows = 128 + (h.span_h - 1) * Wp + h.span_w - 1;   // rows the M = 128 MMAs of the last tap touch
-    p.a_alloc = (int)pt_align_up((size_t)(need_rows > box_h * Wp ? need_rows : box_h * Wp) * 128, 1024);
-    const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : pt_align_up((size_t)p.BN * 128, 1024);
-    const size_t budget = 222 * 1024 - 2048 - kHaloStaging;
+    // The M = 128 MMAs of the last tap read up to this many rows; the rows past the box only feed raster positions that
+    // are never stored, so consecutive A stages may overlap there (and a tail pad follows the last stage).
+    const int need_rows = 128 + (h.span_h - 1) * Wp + h.span_w - 1;
+    p.a_alloc = (int)pt_align_up((size_t)p.a_box_bytes, 1024);
+    const size_t a_tail = need_rows * 128 > p.a_alloc ? pt_align_up((size_t)need_rows * 128 - p.a_alloc, 1024) : 0;
+    // a K-major weight box only brings the output channels that exist (in whole 8-row swizzle atoms); the MMA still reads
+    // BN rows, the rest from whatever follows in shared memory: columns that are never stored
+    p.b_rows = (int)pt_align_up((size_t)(p.BN < h.n_cols ? p.BN : h.n_cols), 8);
+    const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : (size_t)p.b_rows * 128;
+    p.b_slot = (int)b_bytes;
+    // epilogue staging: one slab of the tile's raster rows x 128 bytes per group (direct-store launches use none)
+    p.staging = d->out_f32 ? 0 : (int)pt_align_up((size_t)(p.nr * Wp < 128 ? p.nr * Wp : 128) * 128, 1024);
+    const size_t budget = 227 * 1024 - 2048 - 2 * (size_t)p.staging - a_tail;
     const size_t w_all = (size_t)h.n_taps * p.k_chunks * b_bytes;
     p.resident = (p.n_tiles == 1 && w_all + 2 * (size_t)p.a_alloc <= budget) ? 1 : 0;
     size_t left = budget - (p.resident ? w_all : 0);
@@ -1197,7 +1255,15 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
         p.stages_b = 1;
     }
     if (p.stages_a < 2) return PT_ERR_UNSUPPORTED;
-    p.tmem_cols = pow2_cols(2 * p.BN);
+    // issuer warps: several only with resident weights; each needs an A stage of its own and an accumulator buffer
+    p.n_issuers = 1;
+    p.acc_per = 2;
+    if (p.resident) {
+        p.n_issuers = (p.stages_a >= 4 && 4 * p.BN <= 512) ? 4 : 2;
+        p.acc_per = p.n_issuers * 2 * p.BN <= 512 ? 2 : 1;
+    }
+    p.stages_a = p.stages_a / p.n_issuers * p.n_issuers;
+    p.tmem_cols = pow2_cols(p.n_issuers * p.acc_per * p.BN);
     p.out = out; p.ld_out = h.ld_out; p.out_f32 = d->out_f32;
     p.oH = h.oH; p.oW = h.oW; p.o_step = h.o_step; p.o_h0 = h.o_h0; p.o_w0 = h.o_w0;
     p.tma_store = d->out_f32 ? 0 : 1;
@@ -1205,7 +1271,7 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     CUtensorMap tmA, tmB, tmC;
     memset(&tmC, 0, sizeof(tmC));
     if (!make_halo_in_map(c, &tmA, h.src, h.Cs, h.Ws, h.Hs, d->N, h.lds, Wp, box_h)) return PT_ERR_CUDA;
-    if (!make_weight_map(c, &tmB, w, d->C, d->R * d->S, d->K, d->ldw, B_MN ? kKC : p.BN)) return PT_ERR_CUDA;
+    if (!make_weight_map(c, &tmB, w, d->C, d->R * d->S, d->K, d->ldw, B_MN ? kKC : p.b_rows)) return PT_ERR_CUDA;
     if (p.tma_store) {
         // the output view as a 4-D tensor (channels, raster columns, raster rows, images); strided when o_step > 1
         const size_t es = 2;
@@ -1219,10 +1285,10 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
                                                       CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
     }
-    const size_t smem = 2048 + kHaloStaging + (p.resident ? w_all : (size_t)p.stages_b * b_bytes) + (size_t)p.stages_a * p.a_alloc;
+    const size_t smem = 2048 + 2 * (size_t)p.staging + (p.resident ? w_all : (size_t)p.stages_b * b_bytes) + (size_t)p.stages_a * p.a_alloc + a_tail;
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
-        PT_CUDA_OK(cudaFuncSetAttribute(conv_halo_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        PT_CUDA_OK(cudaFuncSetAttribute(conv_halo_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set[B_MN ? 1 : 0] = true;
     }
     const int total_tiles = p.N * p.row_tiles * p.n_tiles;
@@ -1620,3 +1686,10 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
     }
     return PT_OK;
 }
+
+#ifdef PT_HALO_TRACE
+extern "C" int pt_debug_halo_trace(unsigned long long *host_out)
+{
+    return (int)cudaMemcpyFromSymbol(host_out, g_halo_trace, sizeof(unsigned long long) * 8 * 64);
+}
+#endif
