@@ -22,7 +22,7 @@ namespace {
 constexpr int kBM = 128;            // output pixels per CTA tile
 constexpr int kKC = 64;             // reduction channels per stage (one 128-byte swizzle row)
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 192;           // wgrad kernel: 2 + 4 warps
+constexpr int kThreads = 288;           // wgrad kernel: dy producer, MMA issuer, 4 epilogue warps (x producers in the main loop), 3 more MMA issuers
 constexpr int kGemmThreads = 448;       // fwd/dgrad kernel: 2 + up to 12 epilogue warps
 constexpr int kMaxTaps = 64;
 
@@ -709,12 +709,19 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
     const int pix_end = min(p.npix, pix_beg + p.pix_per_split);
     const int iters = pix_end > pix_beg ? (pix_end - pix_beg + 63) / 64 : 0;
 
+    // Issuing is what a single thread does slowly (about 200 cycles per TMA instruction, 50 to 100 per MMA), so both
+    // sides of the pipeline are spread over warps: warp 0 loads the dy tile, the four epilogue warps (idle until the
+    // accumulators are complete) load the x tiles, and up to four issuer warps each own the accumulators of the taps
+    // tt = i, i + NI, ... Every participant arrives on a stage's barriers itself.
+    const int n_x = ntap * (int)nb_b;                                 // x boxes per stage
+    const int NXP = n_x < 4 ? n_x : 4;                                // x producer warps in use
+    const int NI = ntap < 4 ? ntap : 4;                               // MMA issuer warps in use
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
+            mbar_init(smem_u32(&ctl->full[s]), 1u + (uint32_t)NXP);
+            mbar_init(smem_u32(&ctl->empty[s]), (uint32_t)NI);
         }
-        mbar_init(smem_u32(&ctl->accum), 1);
+        mbar_init(smem_u32(&ctl->accum), (uint32_t)NI);
         ctl->abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmDy);
@@ -728,64 +735,84 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    const int issuer = warp == 1 ? 0 : warp - 5;                      // warps 6, 7, 8 -> issuers 1, 2, 3
 
-    if (warp == 0) {
+    if (warp == 0 || (warp >= 2 && warp < 2 + NXP)) {
         if (lane == 0) {
-            int issued = 0;
+            // ---------------- producers: warp 0 brings dy, warp 2 + j the x boxes j, j + 4, ... of every stage
+            const bool is_dy = warp == 0;
+            const int xp = warp - 2;
+            // output channels k0+64.. of this tile do not exist when K - k0 <= 64: their accumulator rows are never
+            // stored, so that half of the A tile is not loaded at all (the MMA reads stale shared memory there)
+            const bool second = p.K - k0 > 64;
+            uint32_t my_bytes;
+            if (is_dy) my_bytes = second ? a_bytes : 8192u;
+            else my_bytes = (uint32_t)((n_x - xp + 3) / 4) * 8192u;
+            int q = pix_beg % p.Qd, t = pix_beg / p.Qd, pp = t % p.Pd, n = t / p.Pd;   // first pixel of the stage
+            int s = 0, ph = 0, issued = 0;
             for (int it = 0; it < iters; ++it) {
-                const int s = it % p.stages, ph = (it / p.stages) & 1;
                 if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 4)) break;
-                const int pix = pix_beg + it * 64;
-                const int q = pix % p.Qd, t = pix / p.Qd, pp = t % p.Pd, n = t / p.Pd;
                 const uint32_t bar = smem_u32(&ctl->full[s]);
                 const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
-                // output channels k0+64.. of this tile do not exist when K - k0 <= 64: their accumulator rows are never
-                // stored, so that half of the A tile is not loaded at all (the MMA reads stale shared memory there)
-                const bool second = p.K - k0 > 64;
-                mbar_arrive_expect_tx(bar, (second ? a_bytes : 8192u) + (uint32_t)ntap * b_bytes);
-                tma_load_2d(a_dst, &tmDy, bar, k0, pix);
-                if (second) tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
-                for (int tt = 0; tt < ntap; ++tt) {                  // the dy tile is fetched once for all of these taps
-                    const int r = (tap0 + tt) / p.S, sft = (tap0 + tt) - r * p.S;
-                    for (uint32_t nb = 0; nb < nb_b; ++nb)
-                        tma_load_im2col_4d(b_dst + (uint32_t)tt * b_bytes + nb * 8192u, &tmX, bar, c0 + (int)nb * 64,
-                                           q * p.stride + p.lo_w, pp * p.stride + p.lo_h, n, (uint16_t)sft, (uint16_t)r);
+                mbar_arrive_expect_tx(bar, my_bytes);
+                if (is_dy) {
+                    const int pix = pix_beg + it * 64;
+                    tma_load_2d(a_dst, &tmDy, bar, k0, pix);
+                    if (second) tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
+                } else {
+                    for (int j = xp; j < n_x; j += 4) {
+                        const int tt = j / (int)nb_b, nb = j - tt * (int)nb_b;
+                        const int r = (tap0 + tt) / p.S, sft = (tap0 + tt) - r * p.S;
+                        tma_load_im2col_4d(b_dst + (uint32_t)j * 8192u, &tmX, bar, c0 + nb * 64, q * p.stride + p.lo_w,
+                                           pp * p.stride + p.lo_h, n, (uint16_t)sft, (uint16_t)r);
+                    }
+                    q += 64;                                          // the next stage starts 64 pixels further on
+                    while (q >= p.Qd) { q -= p.Qd; if (++pp == p.Pd) { pp = 0; ++n; } }
                 }
                 issued = it + 1;
+                if (++s == p.stages) { s = 0; ph ^= 1; }
             }
-            if (*abort_flag) {
+            if (*abort_flag && is_dy) {
                 for (int it = max(0, issued - p.stages); it < issued; ++it) {
-                    const int s = it % p.stages, ph = (it / p.stages) & 1;
+                    const int s2 = it % p.stages, ph2 = (it / p.stages) & 1;
                     const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(smem_u32(&ctl->full[s]), ph) && globaltimer_ns() - t0 < 20000000ull) {}
+                    while (!mbar_try_wait(smem_u32(&ctl->full[s2]), ph2) && globaltimer_ns() - t0 < 20000000ull) {}
                 }
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(128, p.BN, 1, 1);
-            bool ok = true;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % p.stages, ph = (it / p.stages) & 1;
-                ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 5);
-                if (!ok) break;
-                tc_fence_after();
-                const int rem = pix_end - (pix_beg + it * 64);
-                const int ksteps = rem >= 64 ? 4 : (rem + 15) / 16;
-                const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
-                const uint64_t ad0 = make_desc(a_src, 8192u, 1024u);
-                for (int tt = 0; tt < ntap; ++tt) {
-                    const uint64_t bd0 = make_desc(b_src + (uint32_t)tt * b_bytes, 8192u, 1024u);
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(tt * p.BN);
+        __syncwarp();
+    }
+    if (warp == 1 || (warp >= 6 && issuer < NI)) {
+        // ---------------- MMA issuer `issuer`: the warp walks the loop in lockstep, lane 0 issues
+        const uint32_t leader = lane == 0 ? 1u : 0u;
+        const uint32_t idesc = make_idesc_bf16(128, p.BN, 1, 1);
+        bool ok = true;
+        int s = 0, ph = 0;
+        for (int it = 0; it < iters && ok; ++it) {
+            ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 5);
+            if (!ok) break;
+            tc_fence_after();
+            const int rem = pix_end - (pix_beg + it * 64);
+            const int ksteps = rem >= 64 ? 4 : (rem + 15) / 16;
+            const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
+            const uint64_t ad0 = make_desc(a_src, 8192u, 1024u);
+            const uint32_t acc = it != 0 ? 1u : 0u;
+            for (int tt = issuer; tt < ntap; tt += NI) {
+                const uint64_t bd0 = make_desc(b_src + (uint32_t)tt * b_bytes, 8192u, 1024u);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(tt * p.BN);
+                if (ksteps == 4) {
+                    umma_bf16_lead(d_tmem, ad0, bd0, idesc, acc, leader);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (k < ksteps) umma_bf16(d_tmem, ad0 + 128ull * k, bd0 + 128ull * k, idesc, (it | k) != 0 ? 1u : 0u);
+                    for (int k = 1; k < 4; ++k) umma_bf16_lead(d_tmem, ad0 + 128ull * k, bd0 + 128ull * k, idesc, 1u, leader);
+                } else {
+                    for (int k = 0; k < ksteps; ++k) umma_bf16_lead(d_tmem, ad0 + 128ull * k, bd0 + 128ull * k, idesc, k ? 1u : acc, leader);
                 }
-                umma_commit(smem_u32(&ctl->empty[s]));
             }
-            if (ok) umma_commit(smem_u32(&ctl->accum));
+            umma_commit_lead(smem_u32(&ctl->empty[s]), leader);
+            if (++s == p.stages) { s = 0; ph ^= 1; }
         }
-    } else {
+        if (ok) umma_commit_lead(smem_u32(&ctl->accum), leader);
+    } else if (warp >= 2 && warp < 6) {
         const int quarter = warp & 3;
         bool ok = true;
         if (iters > 0) ok = mbar_wait(smem_u32(&ctl->accum), 0, abort_flag, p.status, 6);
