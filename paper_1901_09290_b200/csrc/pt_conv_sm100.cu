@@ -23,7 +23,7 @@ constexpr int kBM = 128;            // output pixels per CTA tile
 constexpr int kKC = 64;             // reduction channels per stage (one 128-byte swizzle row)
 constexpr int kMaxStages = 8;
 constexpr int kThreads = 288;           // wgrad kernel: dy producer, MMA issuer, 4 epilogue warps (x producers in the main loop), 3 more MMA issuers
-constexpr int kGemmThreads = 448;       // fwd/dgrad kernel: 2 + up to 12 epilogue warps
+constexpr int kGemmThreads = 480;       // fwd/dgrad kernel: A producer, MMA issuer, up to 12 epilogue warps, B producer
 constexpr int kMaxTaps = 64;
 
 struct GemmP {
@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->full[s]), 2);              // the A producer and the B producer
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         for (int b = 0; b < p.epi_groups; ++b) {
@@ -120,75 +120,95 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (warp == 0) {
+    if (warp == 0 || warp == 14) {
         if (lane == 0) {
-            // ---------------- TMA producer
-            int g = 0;          // stage-ring position, continuous across tiles
+            // ---------------- TMA producers: warp 0 brings the A tile of every stage, warp 14 the B tile (issuing a TMA
+            // instruction costs its thread about 200 cycles, so the two operands are issued side by side)
+            const bool is_a = warp == 0;
+            const uint32_t my_bytes = is_a ? a_bytes : b_bytes;
+            int s = 0, ph = 0, issued = 0;   // stage-ring position, continuous across tiles
             for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
                 const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
                 const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
-                const int q = m0 % p.Qd, t = m0 / p.Qd, pp = t % p.Pd, n = t / p.Pd;
-                const int w0 = q * p.stride + p.lo_w, h0 = pp * p.stride + p.lo_h;
-                for (int it = 0; it < iters; ++it, ++g) {
-                    const int s = g % p.stages, ph = (g / p.stages) & 1;
-                    if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 1)) break;
-                    const int tap = it / p.k_chunks, kc = it - tap * p.k_chunks;
-                    const uint32_t bar = smem_u32(&ctl->full[s]);
-                    const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
-                    mbar_arrive_expect_tx(bar, a_bytes + b_bytes);
-                    if (p.a_tiled) tma_load_2d(a_dst, &tmA, bar, kc * kKC, m0);
-                    else tma_load_im2col_4d(a_dst, &tmA, bar, kc * kKC, w0, h0, n, (uint16_t)p.tap_ow[tap], (uint16_t)p.tap_oh[tap]);
+                int w0 = 0, h0 = 0, n = 0;
+                if (is_a && !p.a_tiled) {
+                    const int q = m0 % p.Qd, t = m0 / p.Qd, pp = t % p.Pd;
+                    n = t / p.Pd;
+                    w0 = q * p.stride + p.lo_w; h0 = pp * p.stride + p.lo_h;
+                }
+                bool ok = true;
+                for (int tap = 0; tap < p.taps && ok; ++tap) {
                     const int wtap = p.tap_wt[tap];
-                    if (!B_MN) {
-                        tma_load_3d(b_dst, &tmB, bar, kc * kKC, wtap, n0);
-                    } else {
-                        for (int nb = 0; nb < (p.BN + 63) / 64; ++nb)
-                            tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
+                    const uint16_t ow = (uint16_t)p.tap_ow[tap], oh = (uint16_t)p.tap_oh[tap];
+                    for (int kc = 0; kc < p.k_chunks; ++kc) {
+                        ok = mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 1);
+                        if (!ok) break;
+                        const uint32_t bar = smem_u32(&ctl->full[s]);
+                        const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
+                        mbar_arrive_expect_tx(bar, my_bytes);
+                        if (is_a) {
+                            if (p.a_tiled) tma_load_2d(a_dst, &tmA, bar, kc * kKC, m0);
+                            else tma_load_im2col_4d(a_dst, &tmA, bar, kc * kKC, w0, h0, n, ow, oh);
+                        } else if (!B_MN) {
+                            tma_load_3d(b_dst, &tmB, bar, kc * kKC, wtap, n0);
+                        } else {
+                            for (int nb = 0; nb < (p.BN + 63) / 64; ++nb)
+                                tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
+                        }
+                        ++issued;
+                        if (++s == p.stages) { s = 0; ph ^= 1; }
                     }
                 }
+                if (!ok) break;
             }
-            if (*abort_flag) {
+            if (*abort_flag && is_a) {
                 // drain: give the copies already issued a bounded time to land before the CTA's smem is released
-                for (int it = max(0, g - p.stages); it < g; ++it) {
-                    const int s = it % p.stages, ph = (it / p.stages) & 1;
+                for (int it = max(0, issued - p.stages); it < issued; ++it) {
+                    const int s2 = it % p.stages, ph2 = (it / p.stages) & 1;
                     const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(smem_u32(&ctl->full[s]), ph) && globaltimer_ns() - t0 < 20000000ull) {}
+                    while (!mbar_try_wait(smem_u32(&ctl->full[s2]), ph2) && globaltimer_ns() - t0 < 20000000ull) {}
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
-            const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
-            int g = 0, tc = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tc) {
-                const int b = tc % p.epi_groups, aph = (tc / p.epi_groups) & 1;
-                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 7);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(b * p.BN);
-                for (int it = 0; it < iters; ++it, ++g) {
-                    const int s = g % p.stages, ph = (g / p.stages) & 1;
+        // ---------------- MMA issuer: the warp walks the loops in lockstep, lane 0 issues
+        const uint32_t leader = lane == 0 ? 1u : 0u;
+        const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
+        const uint64_t bstep = B_MN ? 128ull : 2ull;
+        const uint32_t b_lbo = B_MN ? 8192u : 16u;
+        const int last_steps = (p.c_red - (p.k_chunks - 1) * kKC + 15) / 16;      // k-steps of a tap's last chunk
+        int s = 0, ph = 0, b = 0, aph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 7);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(b * p.BN);
+            uint32_t acc = 0u;
+            for (int tap = 0; tap < p.taps && ok; ++tap) {
+                for (int kc = 0; kc < p.k_chunks; ++kc) {
                     ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 2);
                     if (!ok) break;
                     tc_fence_after();
-                    const int kc = it % p.k_chunks;
-                    const int rem = p.c_red - kc * kKC;
-                    const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
                     const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
                     // one descriptor per operand and stage; a k-step only moves the 14-bit start-address field
                     // (units of 16 bytes): +32 B inside a K-major row, +2048 B (16 rows) in an MN-major tile
                     const uint64_t ad0 = make_desc(a_src, 16u, 1024u);
-                    const uint64_t bd0 = B_MN ? make_desc(b_src, 8192u, 1024u) : make_desc(b_src, 16u, 1024u);
-                    const uint64_t bstep = B_MN ? 128ull : 2ull;
+                    const uint64_t bd0 = make_desc(b_src, b_lbo, 1024u);
+                    if (kc + 1 < p.k_chunks || last_steps == 4) {
+                        umma_bf16_lead(d_tmem, ad0, bd0, idesc, acc, leader);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (k < ksteps) umma_bf16(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, (it | k) != 0 ? 1u : 0u);
-                    umma_commit(smem_u32(&ctl->empty[s]));       // frees the stage when these MMAs have read it
+                        for (int k = 1; k < 4; ++k) umma_bf16_lead(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, 1u, leader);
+                    } else {
+                        for (int k = 0; k < last_steps; ++k) umma_bf16_lead(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, k ? 1u : acc, leader);
+                    }
+                    acc = 1u;
+                    umma_commit_lead(smem_u32(&ctl->empty[s]), leader);       // frees the stage when these MMAs have read it
+                    if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
-                if (ok) umma_commit(smem_u32(&ctl->acc_full[b])); // this tile's accumulator is complete
             }
+            if (ok) umma_commit_lead(smem_u32(&ctl->acc_full[b]), leader);   // this tile's accumulator is complete
+            if (++b == p.epi_groups) { b = 0; aph ^= 1; }
         }
     } else if (warp - 2 < 4 * p.epi_groups) {
         // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; group g drains accumulator buffer g,
