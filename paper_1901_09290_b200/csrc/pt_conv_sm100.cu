@@ -703,6 +703,12 @@ struct WgradP {
     unsigned int *status;
 };
 
+#ifdef PT_HALO_TRACE
+__device__ unsigned long long g_wg_trace[8][64];
+#define WTRACE(i) do { if (blockIdx.x == 0 && blockIdx.y < 64 && (threadIdx.x & 31) == 0) g_wg_trace[i][blockIdx.y] = globaltimer_ns(); } while (0)
+#else
+#define WTRACE(i) do { } while (0)
+#endif
 __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy,
                                                               const __grid_constant__ CUtensorMap tmX,
                                                               const __grid_constant__ CUtensorMap tmP, const WgradP p)
@@ -756,6 +762,7 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int issuer = warp == 1 ? 0 : warp - 5;                      // warps 6, 7, 8 -> issuers 1, 2, 3
+    if (threadIdx.x == 0) WTRACE(0);
 
     if (warp == 0 || (warp >= 2 && warp < 2 + NXP)) {
         if (lane == 0) {
@@ -811,6 +818,7 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
         for (int it = 0; it < iters && ok; ++it) {
             ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 5);
             if (!ok) break;
+            if (it == 0 && warp == 1) WTRACE(1);
             tc_fence_after();
             const int rem = pix_end - (pix_beg + it * 64);
             const int ksteps = rem >= 64 ? 4 : (rem + 15) / 16;
@@ -832,10 +840,15 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
             if (++s == p.stages) { s = 0; ph ^= 1; }
         }
         if (ok) umma_commit_lead(smem_u32(&ctl->accum), leader);
-    } else if (warp >= 2 && warp < 6) {
-        const int quarter = warp & 3;
+        if (warp == 1) WTRACE(2);
+    }
+    if (warp >= 1) {
+        // ---------------- epilogue: the four epilogue warps and, once they are done issuing, the four issuer warps; a warp
+        // may read the TMEM lanes of quarter warp % 4, so each quarter has two warps, which take alternate 32-column chunks
+        const int quarter = warp & 3, wset = (warp >= 2 && warp < 6) ? 0 : 1;
         bool ok = true;
         if (iters > 0) ok = mbar_wait(smem_u32(&ctl->accum), 0, abort_flag, p.status, 6);
+        if (warp == 2) WTRACE(3);
         tc_fence_after();
         if (ok) {
             const int k = k0 + quarter * 32 + lane;
@@ -844,11 +857,13 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
             if (p.splits > 1) {
                 // ---- (1) this CTA's fp32 partial tile goes to the workspace through swizzled staging + TMA stores
-                const int gtid = (warp - 2) * 32 + lane;
-                int sl = 0;
+                const int gtid = (warp - 1) * 32 + lane;
+                int sl = 0, ci = 0;
                 for (int tt = 0; tt < ntap; ++tt)
-                for (int cc = 0; cc < p.BN; cc += 32, sl ^= 1) {
-                    const uint32_t slab = data_base + (uint32_t)(quarter * 2 + sl) * 4096u;
+                for (int cc = 0; cc < p.BN; cc += 32, ++ci) {
+                    if ((ci & 1) != wset) continue;
+                    sl ^= 1;
+                    const uint32_t slab = data_base + (uint32_t)((wset * 4 + quarter) * 2 + sl) * 4096u;
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                     uint32_t lo[16], hi[16];
@@ -878,7 +893,8 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 }
                 if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // the writes have completed
                 __threadfence();
-                named_barrier(1, 128);
+                if (warp == 2) WTRACE(4);
+                named_barrier(1, 256);
                 // ---- (2) every split CTA of this tile is resident (the grid is at most one CTA per SM): wait for all of them
                 unsigned int *arrived = p.sync + 2 * blockIdx.x, *reduced = arrived + 1;
                 if (gtid == 0) {
@@ -890,14 +906,17 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                         __nanosleep(64);
                     }
                 }
-                named_barrier(1, 128);
+                named_barrier(1, 256);
+                if (warp == 2) WTRACE(5);
             } else {
             float *obase = p.out;
             // The stages are free once the accumulator is complete: each warp transposes its 32 x 32 blocks through
             // a padded shared-memory square so that a warp writes 32 consecutive floats of one dw row at a time.
-            const uint32_t sq = data_base + (uint32_t)quarter * (32u * 33u * 4u);
+            const uint32_t sq = data_base + (uint32_t)(wset * 4 + quarter) * (32u * 33u * 4u);
+            int ci = 0;
             for (int tt = 0; tt < ntap; ++tt)
-            for (int cc = 0; cc < p.BN; cc += 32) {
+            for (int cc = 0; cc < p.BN; cc += 32, ++ci) {
+                if ((ci & 1) != wset) continue;
                 const int tap = tap0 + tt;
                 uint32_t v[32];
                 if (iters > 0) {
@@ -931,61 +950,54 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
     }
     __syncthreads();
     if (p.splits > 1 && !*abort_flag) {
-        // ---- (3) all 192 threads: this CTA sums its share of the tile's rows over the splits, in ascending split order
+        // ---- (3) all threads: this CTA sums its share of the tile's elements over the splits
         __threadfence();
-        // Work items are (row, 4-column group) of the real rows of the tile, dealt out evenly to the tile's split CTAs.
-        // T lanes share an item (T = 8 when there are many splits, else 1): lane s adds the splits [s*zc, (s+1)*zc) in
-        // ascending order, then the partial sums are combined by a fixed shuffle tree: the result does not depend on timing.
+        // Work items are (tap, row, 4-column group) of the real rows of the CTA's tiles, dealt out evenly to the split CTAs.
+        // The partial tiles sit in L2; what costs time is a chain of dependent loads, so every thread first issues the
+        // asynchronous 16-byte copies of its items for ALL splits into the (now idle) stage memory, and only then are the
+        // copies summed from shared memory in ascending split order: deterministic, whichever CTA does the work.
         const int rows_real = min(128, p.K - k0);
         const int ngrp = p.BN / 4;                                   // float4 groups per row (BN is a multiple of 16)
         const int items = rows_real * ngrp;
-        const int per_cta = (items + p.splits - 1) / p.splits;
-        const int it_beg = split * per_cta, it_end = min(items, it_beg + per_cta);
-        const int T = p.splits > 96 ? 8 : 1;                         // lanes per item: share only very long split chains
-        const int zc = (p.splits + T - 1) / T;
-        const int sub = threadIdx.x & (T - 1);
+        const int total = ntap * items;
+        const int per_cta = (total + p.splits - 1) / p.splits;
+        const int it_beg = split * per_cta, it_end = min(total, it_beg + per_cta);
         const size_t zstride = (size_t)128 * p.BN;
-        for (int tt = 0; tt < ntap; ++tt) {
-        const int tap = tap0 + tt;
-        const float *pt = p.partial + ((size_t)blockIdx.x * p.tpc + tt) * p.splits * 128 * p.BN;
-        for (int base = it_beg; base < it_end; base += kThreads / T) {
-            const int item = base + threadIdx.x / T;
-            const bool live = item < it_end;
-            const int r = live ? item / ngrp : 0, col = live ? (item % ngrp) * 4 : 0;
-            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (live && c0 + col < p.C) {
-                const float *src = pt + (size_t)r * p.BN + col;
-                const int z_end = min(p.splits, (sub + 1) * zc);
-                int z = sub * zc;
-                for (; z + 4 <= z_end; z += 4) {
-                    float4 t[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) t[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(z + u) * zstride));
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) { sum.x += t[u].x; sum.y += t[u].y; sum.z += t[u].z; sum.w += t[u].w; }
-                }
-                for (; z < z_end; ++z) {
-                    const float4 t = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)z * zstride));
+        const float *pbase = p.partial + (size_t)blockIdx.x * p.tpc * p.splits * zstride;
+        const int cap = (int)(((size_t)p.stages * stage_bytes) / ((size_t)p.splits * 16));   // items the stage memory holds
+        for (int c_beg = it_beg; c_beg < it_end; c_beg += cap) {
+            const int n_chunk = min(cap, it_end - c_beg);
+            for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
+                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
+                const float *src = pbase + (size_t)tt * p.splits * zstride + (size_t)item * 4;
+                uint32_t dst = data_base + (uint32_t)i * 16u;
+                for (int z = 0; z < p.splits; ++z, src += zstride, dst += (uint32_t)n_chunk * 16u)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            __syncthreads();
+            for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
+                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
+                const int r = item / ngrp, col = (item - r * ngrp) * 4;
+                if (c0 + col >= p.C) continue;
+                float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                uint32_t a = data_base + (uint32_t)i * 16u;
+                for (int z = 0; z < p.splits; ++z, a += (uint32_t)n_chunk * 16u) {
+                    float4 t;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "r"(a) : "memory");
                     sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
                 }
-            }
-            for (int o = 1; o < T; o <<= 1) {        // (s0+s1) + (s2+s3) ... : the same tree on every run
-                sum.x += __shfl_xor_sync(0xffffffffu, sum.x, o);
-                sum.y += __shfl_xor_sync(0xffffffffu, sum.y, o);
-                sum.z += __shfl_xor_sync(0xffffffffu, sum.z, o);
-                sum.w += __shfl_xor_sync(0xffffffffu, sum.w, o);
-            }
-            if (live && sub == 0 && c0 + col < p.C) {
-                float *dst = p.out + ((size_t)(k0 + r) * p.taps + tap) * p.C + c0 + col;
+                float *dst = p.out + ((size_t)(k0 + r) * p.taps + tap0 + tt) * p.C + c0 + col;
                 const int nv = min(4, p.C - (c0 + col));
                 dst[0] = sum.x;
                 if (nv > 1) dst[1] = sum.y;
                 if (nv > 2) dst[2] = sum.z;
                 if (nv > 3) dst[3] = sum.w;
             }
-        }
+            __syncthreads();
         }
         __syncthreads();
+        if (threadIdx.x == 0) WTRACE(6);
         if (threadIdx.x == 0) {
             unsigned int *arrived = p.sync + 2 * blockIdx.x, *reduced = arrived + 1;
             __threadfence();
@@ -1457,6 +1469,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     size_t smem = 0;
     const size_t stage = 2 * 8192 + (size_t)p.tpc * pt_ceil_div(p.BN, 64) * 8192;
     p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), 0, &smem);
+    if (smem < 2048 + 8 * 2 * 4096) smem = 2048 + 8 * 2 * 4096;        // the epilogue's staging slabs reuse the stage memory
     static bool attr_set = false;
     if (!attr_set) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
@@ -1735,6 +1748,10 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
 }
 
 #ifdef PT_HALO_TRACE
+extern "C" int pt_debug_wgrad_trace(unsigned long long *host_out)
+{
+    return (int)cudaMemcpyFromSymbol(host_out, g_wg_trace, sizeof(unsigned long long) * 8 * 64);
+}
 extern "C" int pt_debug_halo_trace(unsigned long long *host_out)
 {
     return (int)cudaMemcpyFromSymbol(host_out, g_halo_trace, sizeof(unsigned long long) * 8 * 64);
