@@ -18,6 +18,22 @@
 using namespace sm100;
 
 namespace {
+// Launch with programmatic stream serialization: the kernel may be scheduled while the previous kernel of the stream is
+// still draining, so its prologue (barrier setup, TMEM allocation, descriptor prefetch) and the launch latency overlap that
+// kernel's tail. Every kernel launched this way executes griddepcontrol.wait before its first global-memory access.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 
 constexpr int kBM = 128;            // output pixels per CTA tile
 constexpr int kKC = 64;             // reduction channels per stage (one 128-byte swizzle row)
@@ -119,6 +135,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    grid_dependency_wait();              // nothing above touches global memory
+    grid_launch_dependents();
 
     if (warp == 0 || warp == 14) {
         if (lane == 0) {
@@ -451,6 +469,8 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int issuer = warp == 1 ? 0 : warp - 9;             // warps 10, 11, 12 -> issuers 1, 2, 3
+    grid_dependency_wait();              // nothing above touches global memory
+    grid_launch_dependents();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -762,6 +782,8 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int issuer = warp == 1 ? 0 : warp - 5;                      // warps 6, 7, 8 -> issuers 1, 2, 3
+    grid_dependency_wait();              // nothing above touches global memory
+    grid_launch_dependents();
     if (threadIdx.x == 0) WTRACE(0);
 
     if (warp == 0 || (warp >= 2 && warp < 2 + NXP)) {
@@ -1231,7 +1253,7 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
         attr_set[B_MN ? 1 : 0] = true;
     }
     const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
-    conv_gemm_kernel<B_MN><<<grid, kGemmThreads, smem, st>>>(tmA, tmB, tmC, p);
+    PT_CUDA_OK(launch_pdl(conv_gemm_kernel<B_MN>, dim3((unsigned)grid), dim3(kGemmThreads), smem, st, tmA, tmB, tmC, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
@@ -1352,7 +1374,7 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     }
     const int total_tiles = p.N * p.row_tiles * p.n_tiles;
     const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
-    conv_halo_kernel<B_MN><<<grid, kHaloThreads, smem, st>>>(tmA, tmB, tmC, p);
+    PT_CUDA_OK(launch_pdl(conv_halo_kernel<B_MN>, dim3((unsigned)grid), dim3(kHaloThreads), smem, st, tmA, tmB, tmC, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
@@ -1476,7 +1498,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
         attr_set = true;
     }
     dim3 grid((unsigned)gx, (unsigned)p.splits);
-    conv_wgrad_kernel<<<grid, kThreads, smem, st>>>(tmA, tmX, tmP, p);
+    PT_CUDA_OK(launch_pdl(conv_wgrad_kernel, grid, dim3(kThreads), smem, st, tmA, tmX, tmP, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;

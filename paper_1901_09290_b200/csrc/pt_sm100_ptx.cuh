@@ -135,6 +135,12 @@ __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *tm)
     asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Blocks until every kernel this one depends on has completed and its memory operations are visible.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be scheduled as soon as every CTA of this grid has said so (or exited).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- TMEM
 // Whole warp. Writes the TMEM base address (lane 0, column of the allocation) to *dst_smem.
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
