@@ -358,7 +358,7 @@ def run_ours(args):
                    "parallelism": "independent data-parallel replicas, no collective" if world > 1 else "1 GPU",
                    "algo": args.algo,
                    "launch": "eager" if args.no_graph else ("CUDA graph replay after the reconfiguration's host sync; "
-                                                            + ("1 stream" if args.one_stream else "dgrad and wgrad of a layer on 2 streams"))},
+                                                            + ("1 stream" if args.one_stream else "3 streams along the network's data dependencies: wgrad of a layer beside its dgrad, projection shortcuts beside their blocks"))},
         "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "pipeline": "one pinned-host image copy per step on a copy stream, overlapping the previous step's kernels"},
         "gpu_launches": launches,

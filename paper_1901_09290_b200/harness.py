@@ -178,26 +178,64 @@ class TrainStep:
             self.conv_wgrad(li, stream)
         self.lasso(stream)
 
+    def _branches(self):
+        """(first layer of the block, index of the projection shortcut) for every block that has one: the shortcut reads
+        the block's input and is only needed at the block's output, so it is independent of the block's other layers."""
+        out = []
+        names = [l.name for l in self.net.layers]
+        for d, nm in enumerate(names):
+            if nm.endswith(".ds"):
+                pre = nm[:-3]
+                first = min(i for i, x in enumerate(names) if x.startswith(pre + "."))
+                out.append((first, d))
+        return out
+
     def train_two_streams(self):
-        """The same launches with each layer's data gradient and weight gradient on two streams: they only share their
-        input dy_l, so they may overlap (the weight gradients use the workspace, the data gradients do not)."""
+        """The same launches on three streams, following the network's own data dependencies: a layer's data gradient and
+        weight gradient only share their input dy_l (the weight gradients use the workspace, the data gradients do not),
+        and a block's projection shortcut is independent of the block's other convolutions in both directions."""
         main = torch.cuda.current_stream()
-        side = self._side
+        side, aux = self._side, self._aux
         n = len(self.net.layers)
+        br = self._branches()
+        fork_at = {f: d for f, d in br}          # before layer f: start shortcut d on the aux stream
+        ds_set = {d for _, d in br}
         for li in range(n):
+            if li in fork_at:
+                aux.wait_stream(main)
+                self.conv_fwd(fork_at[li], aux)
+            if li in ds_set:
+                main.wait_stream(aux)            # the block's output needs both branches
+                continue
             self.conv_fwd(li, main)
-        side.wait_stream(main)
+        first_of = {d: f for f, d in br}
+        join_after = None
         for li in range(n - 1, -1, -1):
+            # dy_l exists once the data gradients above layer l are done: the weight gradient of layer l starts there, next
+            # to the layer's own data gradient
+            side.wait_stream(main)
+            if li in ds_set:
+                aux.wait_stream(main)            # both branches start from the gradient of the block's output
+                if li > 0:
+                    self.conv_dgrad(li, aux)
+                self.conv_wgrad(li, side)
+                join_after = first_of[li]
+                continue
             if li > 0:
                 self.conv_dgrad(li, main)
             self.conv_wgrad(li, side)
+            if join_after == li:
+                main.wait_stream(aux)            # the gradient of the block's input sums both branches
+                join_after = None
         main.wait_stream(side)
+        main.wait_stream(aux)
         self.lasso(main)
 
     def build_graph(self, two_streams: bool = True):
         """Captures the training part of the step (every launch after the reconfiguration's host sync) into a CUDA graph.
         Call after at least one eager step, so that every table and kernel attribute is already set up."""
         self._side = torch.cuda.Stream()
+        self._aux = torch.cuda.Stream()
         l0 = self.ctx.launch_count()
         self.graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.graph):
