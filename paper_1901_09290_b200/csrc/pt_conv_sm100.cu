@@ -63,6 +63,7 @@ struct GemmP {
     int m_tiles;        // ceil(M_total / 128)
     int epi_groups;     // 1..3 groups of four epilogue warps
     int a_tiled;        // 1: 1x1 stride-1 problem, the A operand is a plain 2-D (channels, pixels) tiled map
+    int resident;       // 1: every weight tile of the launch stays in shared memory (loaded once); the ring carries A only
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
@@ -83,6 +84,7 @@ struct __align__(8) PCtl {
     uint64_t empty[kMaxStages];
     uint64_t acc_full[3];       // MMA issuer -> epilogue: accumulator buffer b holds a finished tile
     uint64_t acc_empty[3];      // epilogue -> MMA issuer: buffer b has been read out (4 arrivals, one per warp of its group)
+    uint64_t w_full;            // resident weights have landed
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -102,10 +104,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     PCtl *ctl = reinterpret_cast<PCtl *>(smem_raw);
     const uint32_t smem_base = smem_u32(smem_raw);
     const uint32_t staging_base = (smem_base + (uint32_t)sizeof(PCtl) + 1023u) & ~1023u;
-    const uint32_t data_base = staging_base + (uint32_t)p.epi_groups * 4u * kSlabs * 4096u;
     const uint32_t a_bytes = kBM * kKC * 2;
     const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.BN * 128u;
-    const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
+    const uint32_t b_slot = (b_bytes + 1023u) & ~1023u;
+    // resident weights: all taps x chunks sit in front of the ring, whose stages then hold an A tile only
+    const uint32_t w_base = staging_base + (uint32_t)p.epi_groups * 4u * kSlabs * 4096u;
+    const uint32_t stage_bytes = p.resident ? a_bytes : a_bytes + b_slot;
+    const uint32_t data_base = w_base + (p.resident ? (uint32_t)(p.taps * p.k_chunks) * b_slot : 0u);
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -114,9 +119,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 2);              // the A producer and the B producer
+            mbar_init(smem_u32(&ctl->full[s]), p.resident ? 1 : 2);   // the A producer and, with streamed weights, the B producer
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
+        mbar_init(smem_u32(&ctl->w_full), 1);
         for (int b = 0; b < p.epi_groups; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
@@ -145,7 +151,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             const bool is_a = warp == 0;
             const uint32_t my_bytes = is_a ? a_bytes : b_bytes;
             int s = 0, ph = 0, issued = 0;   // stage-ring position, continuous across tiles
-            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+            if (!is_a && p.resident) {
+                // n_tiles == 1 here: every weight tile of the launch, once
+                const uint32_t bar = smem_u32(&ctl->w_full);
+                mbar_arrive_expect_tx(bar, (uint32_t)iters * b_bytes);
+                for (int tap = 0; tap < p.taps; ++tap)
+                    for (int kc = 0; kc < p.k_chunks; ++kc) {
+                        const uint32_t dst = w_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot;
+                        const int wtap = p.tap_wt[tap];
+                        if (!B_MN) tma_load_3d(dst, &tmB, bar, kc * kKC, wtap, 0);
+                        else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
+                    }
+            }
+            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag && (is_a || !p.resident); tile += gridDim.x) {
                 const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
                 const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
                 int w0 = 0, h0 = 0, n = 0;
@@ -197,6 +215,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         const int last_steps = (p.c_red - (p.k_chunks - 1) * kKC + 15) / 16;      // k-steps of a tap's last chunk
         int s = 0, ph = 0, b = 0, aph = 0;
         bool ok = true;
+        if (p.resident) ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort_flag, p.status, 8);
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 7);
             if (!ok) break;
@@ -208,7 +227,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 2);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
+                    const uint32_t a_src = data_base + (uint32_t)s * stage_bytes;
+                    const uint32_t b_src = p.resident ? w_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot : a_src + a_bytes;
                     // one descriptor per operand and stage; a k-step only moves the 14-bit start-address field
                     // (units of 16 bytes): +32 B inside a K-major row, +2048 B (16 rows) in an MN-major tile
                     const uint64_t ad0 = make_desc(a_src, 16u, 1024u);
@@ -1245,7 +1265,13 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     // CTAs get a single tile need no more than that
     p.epi_groups = 3 * p.BN <= 512 ? 3 : 2;
     if (per_cta < p.epi_groups) p.epi_groups = per_cta < 2 ? 2 : per_cta;
-    p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, (size_t)p.epi_groups * 4 * kSlabs * 4096, &smem);
+    // Small weights (one channel tile, all taps x chunks within 64 KB) stay resident: the ring then carries A tiles only and
+    // holds more of them, which is what an activation-bound layer needs to cover the memory latency.
+    const size_t staging = (size_t)p.epi_groups * 4 * kSlabs * 4096;
+    const size_t w_all = (size_t)p.taps * p.k_chunks * b_bytes;
+    p.resident = (p.n_tiles == 1 && w_all <= 64 * 1024 && per_cta >= 2) ? 1 : 0;
+    if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging + w_all, &smem);
+    else p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging, &smem);
     p.tmem_cols = pow2_cols(p.epi_groups * p.BN);
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
