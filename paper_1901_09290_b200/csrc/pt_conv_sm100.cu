@@ -39,7 +39,7 @@ constexpr int kBM = 128;            // output pixels per CTA tile
 constexpr int kKC = 64;             // reduction channels per stage (one 128-byte swizzle row)
 constexpr int kMaxStages = 8;
 constexpr int kThreads = 288;           // wgrad kernel: dy producer, MMA issuer, 4 epilogue warps (x producers in the main loop), 3 more MMA issuers
-constexpr int kGemmThreads = 480;       // fwd/dgrad kernel: A producer, MMA issuer, up to 12 epilogue warps, B producer
+constexpr int kGemmThreads = 512;       // fwd/dgrad kernel: A producer, MMA issuer, up to 12 epilogue warps, B producer, second MMA issuer
 constexpr int kMaxTaps = 64;
 
 struct GemmP {
@@ -64,6 +64,8 @@ struct GemmP {
     int epi_groups;     // 1..3 groups of four epilogue warps
     int a_tiled;        // 1: 1x1 stride-1 problem, the A operand is a plain 2-D (channels, pixels) tiled map
     int resident;       // 1: every weight tile of the launch stays in shared memory (loaded once); the ring carries A only
+    int n_issuers;      // 2 (resident weights only): two MMA issuer warps take alternate tiles, each with half of the ring's stages
+    int acc_per;        // two issuers: accumulator buffers per issuer (1 or 2)
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
@@ -82,8 +84,8 @@ struct __align__(8) Ctl {
 struct __align__(8) PCtl {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    uint64_t acc_full[3];       // MMA issuer -> epilogue: accumulator buffer b holds a finished tile
-    uint64_t acc_empty[3];      // epilogue -> MMA issuer: buffer b has been read out (4 arrivals, one per warp of its group)
+    uint64_t acc_full[4];       // MMA issuer -> epilogue: accumulator buffer b holds a finished tile
+    uint64_t acc_empty[4];      // epilogue -> MMA issuer: buffer b has been read out (4 arrivals, one per warp of its group)
     uint64_t w_full;            // resident weights have landed
     uint32_t tmem_base;
     int abort_flag;
@@ -123,7 +125,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->w_full), 1);
-        for (int b = 0; b < p.epi_groups; ++b) {
+        for (int b = 0; b < 4; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
         }
@@ -151,6 +153,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             const bool is_a = warp == 0;
             const uint32_t my_bytes = is_a ? a_bytes : b_bytes;
             int s = 0, ph = 0, issued = 0;   // stage-ring position, continuous across tiles
+            int s1 = 0, ph1 = 0;             // position in the second issuer's ring
+            const int SR = p.stages / p.n_issuers;
             if (!is_a && p.resident) {
                 // n_tiles == 1 here: every weight tile of the launch, once
                 const uint32_t bar = smem_u32(&ctl->w_full);
@@ -163,9 +167,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
                     }
             }
-            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag && (is_a || !p.resident); tile += gridDim.x) {
+            int ring = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag && (is_a || !p.resident); tile += gridDim.x,
+                     ring = p.n_issuers == 2 ? ring ^ 1 : 0) {
                 const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
                 const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
+                if (ring) { int t = s; s = s1; s1 = t; t = ph; ph = ph1; ph1 = t; }     // work on the second ring's position
+                const int sbase = ring * SR;
                 int w0 = 0, h0 = 0, n = 0;
                 if (is_a && !p.a_tiled) {
                     const int q = m0 % p.Qd, t = m0 / p.Qd, pp = t % p.Pd;
@@ -177,10 +185,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     const int wtap = p.tap_wt[tap];
                     const uint16_t ow = (uint16_t)p.tap_ow[tap], oh = (uint16_t)p.tap_oh[tap];
                     for (int kc = 0; kc < p.k_chunks; ++kc) {
-                        ok = mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 1);
+                        ok = mbar_wait(smem_u32(&ctl->empty[sbase + s]), ph ^ 1, abort_flag, p.status, 1);
                         if (!ok) break;
-                        const uint32_t bar = smem_u32(&ctl->full[s]);
-                        const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
+                        const uint32_t bar = smem_u32(&ctl->full[sbase + s]);
+                        const uint32_t a_dst = data_base + (uint32_t)(sbase + s) * stage_bytes, b_dst = a_dst + a_bytes;
                         mbar_arrive_expect_tx(bar, my_bytes);
                         if (is_a) {
                             if (p.a_tiled) tma_load_2d(a_dst, &tmA, bar, kc * kKC, m0);
@@ -192,31 +200,35 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                                 tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
                         }
                         ++issued;
-                        if (++s == p.stages) { s = 0; ph ^= 1; }
+                        if (++s == SR) { s = 0; ph ^= 1; }
                     }
                 }
+                if (ring) { int t = s; s = s1; s1 = t; t = ph; ph = ph1; ph1 = t; }
                 if (!ok) break;
             }
             if (*abort_flag && is_a) {
                 // drain: give the copies already issued a bounded time to land before the CTA's smem is released
-                for (int it = max(0, issued - p.stages); it < issued; ++it) {
-                    const int s2 = it % p.stages, ph2 = (it / p.stages) & 1;
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(smem_u32(&ctl->full[s2]), ph2) && globaltimer_ns() - t0 < 20000000ull) {}
-                }
+                const uint64_t t0 = globaltimer_ns();
+                for (int s2 = 0; s2 < p.stages && issued > 0; ++s2)
+                    while (!mbar_try_wait(smem_u32(&ctl->full[s2]), 0) && !mbar_try_wait(smem_u32(&ctl->full[s2]), 1) &&
+                           globaltimer_ns() - t0 < 20000000ull) {}
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer: the warp walks the loops in lockstep, lane 0 issues
+    } else if (warp == 1 || (warp == 15 && p.n_issuers == 2)) {
+        // ---------------- MMA issuer(s): the warp walks the loops in lockstep, lane 0 issues. With two issuers, issuer i
+        // takes the CTA's tiles i, i + 2, ..., reads ring i and owns the accumulator buffers i*acc_per .. + acc_per - 1.
         const uint32_t leader = lane == 0 ? 1u : 0u;
         const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
         const uint64_t bstep = B_MN ? 128ull : 2ull;
         const uint32_t b_lbo = B_MN ? 8192u : 16u;
         const int last_steps = (p.c_red - (p.k_chunks - 1) * kKC + 15) / 16;      // k-steps of a tap's last chunk
-        int s = 0, ph = 0, b = 0, aph = 0;
+        const int NI = p.n_issuers, issuer = warp == 1 ? 0 : 1;
+        const int SR = p.stages / NI, sbase = issuer * SR;
+        int s = 0, ph = 0, b = 0, aph = 0, nt = 0;
         bool ok = true;
         if (p.resident) ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort_flag, p.status, 8);
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int tile = blockIdx.x + issuer * (int)gridDim.x; tile < total_tiles && ok; tile += NI * (int)gridDim.x, ++nt) {
+            if (NI == 2) { b = p.acc_per == 2 ? issuer * 2 + (nt & 1) : issuer; aph = p.acc_per == 2 ? (nt >> 1) & 1 : nt & 1; }
             ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 7);
             if (!ok) break;
             tc_fence_after();
@@ -224,10 +236,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             uint32_t acc = 0u;
             for (int tap = 0; tap < p.taps && ok; ++tap) {
                 for (int kc = 0; kc < p.k_chunks; ++kc) {
-                    ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 2);
+                    ok = mbar_wait(smem_u32(&ctl->full[sbase + s]), ph, abort_flag, p.status, 2);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a_src = data_base + (uint32_t)s * stage_bytes;
+                    const uint32_t a_src = data_base + (uint32_t)(sbase + s) * stage_bytes;
                     const uint32_t b_src = p.resident ? w_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot : a_src + a_bytes;
                     // one descriptor per operand and stage; a k-step only moves the 14-bit start-address field
                     // (units of 16 bytes): +32 B inside a K-major row, +2048 B (16 rows) in an MN-major tile
@@ -241,12 +253,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         for (int k = 0; k < last_steps; ++k) umma_bf16_lead(d_tmem, ad0 + 2ull * k, bd0 + bstep * k, idesc, k ? 1u : acc, leader);
                     }
                     acc = 1u;
-                    umma_commit_lead(smem_u32(&ctl->empty[s]), leader);       // frees the stage when these MMAs have read it
-                    if (++s == p.stages) { s = 0; ph ^= 1; }
+                    umma_commit_lead(smem_u32(&ctl->empty[sbase + s]), leader);   // frees the stage when these MMAs have read it
+                    if (++s == SR) { s = 0; ph ^= 1; }
                 }
             }
             if (ok) umma_commit_lead(smem_u32(&ctl->acc_full[b]), leader);   // this tile's accumulator is complete
-            if (++b == p.epi_groups) { b = 0; aph ^= 1; }
+            if (NI == 1 && ++b == p.epi_groups) { b = 0; aph ^= 1; }
         }
     } else if (warp - 2 < 4 * p.epi_groups) {
         // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; group g drains accumulator buffer g,
@@ -256,7 +268,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         int tc = group, sl = 0;
         bool ok = true;
         for (int tile = blockIdx.x + group * gridDim.x; tile < total_tiles && ok; tile += G * gridDim.x, tc += G) {
-            const int b = group, aph = (tc / G) & 1;
+            int b = group, aph = (tc / G) & 1;
+            if (p.n_issuers == 2) {                     // G == 2: group g serves issuer g, whose nt-th tile this is
+                const int nt = tc >> 1;
+                b = p.acc_per == 2 ? group * 2 + (nt & 1) : group;
+                aph = p.acc_per == 2 ? (nt >> 1) & 1 : nt & 1;
+            }
             const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
             const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
             ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 3);
@@ -1270,9 +1287,21 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     const size_t staging = (size_t)p.epi_groups * 4 * kSlabs * 4096;
     const size_t w_all = (size_t)p.taps * p.k_chunks * b_bytes;
     p.resident = (p.n_tiles == 1 && w_all <= 64 * 1024 && per_cta >= 2) ? 1 : 0;
-    if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging + w_all, &smem);
-    else p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging, &smem);
-    p.tmem_cols = pow2_cols(p.epi_groups * p.BN);
+    p.n_issuers = 1; p.acc_per = 1;
+    if (p.resident && per_cta >= 4 && 2 * p.BN <= 512) {
+        // narrow tiles are bound by what one thread can issue: two issuer warps, two epilogue groups
+        p.n_issuers = 2;
+        p.epi_groups = 2;
+        p.acc_per = 4 * p.BN <= 512 ? 2 : 1;
+    }
+    const size_t staging2 = (size_t)p.epi_groups * 4 * kSlabs * 4096;
+    if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all, &smem);
+    else p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2, &smem);
+    if (p.n_issuers == 2) {
+        p.stages = p.stages / 2 * 2;
+        if (p.stages < 2) { p.n_issuers = 1; p.acc_per = 1; p.stages = 2; }
+    }
+    p.tmem_cols = pow2_cols((p.n_issuers == 2 ? 2 * p.acc_per : p.epi_groups) * p.BN);
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
