@@ -455,8 +455,8 @@ struct __align__(8) HCtl {
     int abort_flag;
 };
 
-// warp 0: TMA producer; warp 1 and warps 10..12: MMA issuers; warps 2..9: two groups of four epilogue warps
-constexpr int kHaloThreads = 416;
+// warp 0 (and 13): TMA producers; warp 1 and warps 10..12: MMA issuers; warps 2..9: two groups of four epilogue warps
+constexpr int kHaloThreads = 448;
 
 // Issuing one tcgen05.mma costs the issuing warp 50 to 100 cycles of instruction time, more than a narrow MMA (N <= 64)
 // takes to execute, so with a single issuer the tensor pipe of a small-channel layer idles most of the time. The
@@ -509,9 +509,14 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     grid_dependency_wait();              // nothing above touches global memory
     grid_launch_dependents();
 
-    if (warp == 0) {
+    // Streamed weights with two issuers: two complete pipelines (producer warp, A ring, B ring, issuer warp, accumulators),
+    // one per tile parity. Resident weights: one producer feeds every issuer's A ring.
+    const int n_prod = p.resident ? 1 : NI;
+    const int SB = p.stages_b / n_prod;                       // weight stages per pipeline
+    if (warp == 0 || (warp == 13 && n_prod == 2)) {
         if (lane == 0) {
-            // ---------------- TMA producer
+            // ---------------- TMA producer(s)
+            const int pid = warp == 0 ? 0 : 1;
             if (p.resident) {
                 // n_tiles == 1 here: the whole weight tensor of the layer, tap by tap and chunk by chunk, once
                 const uint32_t bar = smem_u32(&ctl->w_full);
@@ -524,8 +529,8 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
                     }
             }
-            int gb = 0, tc = 0;
-            for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tc) {
+            int gb = 0, tc = pid;
+            for (int tile = blockIdx.x + pid * (int)gridDim.x; tile < total_tiles && !*abort_flag; tile += n_prod * (int)gridDim.x, tc += n_prod) {
                 const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
                 const int img = m_tile / p.row_tiles, p0 = (m_tile - img * p.row_tiles) * p.nr;
                 const int n0 = n_tile * p.BN;
@@ -542,7 +547,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                     tma_load_4d(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, &tmA, bar, kc * kKC, p.lo_w, p0 + p.lo_h, img);
                     if (p.resident) continue;
                     for (int tap = 0; tap < p.taps; ++tap, ++gb) {
-                        const int sb = gb % p.stages_b, phb = (gb / p.stages_b) & 1;
+                        const int sb = pid * SB + gb % SB, phb = (gb / SB) & 1;
                         ok = mbar_wait(smem_u32(&ctl->empty_b[sb]), phb ^ 1, abort_flag, p.status, 12);
                         if (!ok) break;
                         const uint32_t bbar = smem_u32(&ctl->full_b[sb]);
@@ -555,7 +560,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                 }
                 if (!ok) break;
             }
-            if (*abort_flag) {       // bounded drain of the copies in flight before the shared memory is released
+            if (*abort_flag && pid == 0) {   // bounded drain of the copies in flight before the shared memory is released
                 const uint64_t t0 = globaltimer_ns();
                 for (int s = 0; s < p.stages_a; ++s)
                     while (!mbar_try_wait(smem_u32(&ctl->full_a[s]), 0) && !mbar_try_wait(smem_u32(&ctl->full_a[s]), 1) &&
@@ -611,7 +616,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                     }
                 } else {
                     for (int tap = 0; tap < p.taps; ++tap, ++gb) {
-                        const int sb = gb % p.stages_b, phb = (gb / p.stages_b) & 1;
+                        const int sb = issuer * SB + gb % SB, phb = (gb / SB) & 1;
                         ok = mbar_wait(smem_u32(&ctl->full_b[sb]), phb, abort_flag, p.status, 16);
                         if (!ok) break;
                         tc_fence_after();
@@ -1376,12 +1381,16 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     const size_t w_all = (size_t)h.n_taps * p.k_chunks * b_bytes;
     p.resident = (p.n_tiles == 1 && w_all + 2 * (size_t)p.a_alloc <= budget) ? 1 : 0;
     size_t left = budget - (p.resident ? w_all : 0);
+    bool two_pipes = false;
     if (!p.resident) {
         // ring: at least two A stages, the rest for weight stages (at least 3)
         p.stages_a = 2;
         if (left < 2 * (size_t)p.a_alloc + 3 * b_bytes) return PT_ERR_UNSUPPORTED;
         size_t sb = (left - 2 * (size_t)p.a_alloc) / b_bytes;
         p.stages_b = sb > kMaxStages ? kMaxStages : (int)sb;
+        // two pipelines (one per tile parity) when each can have three weight stages and the CTAs get several tiles
+        two_pipes = p.stages_b >= 6 && pt_ceil_div(p.N * p.row_tiles * p.n_tiles, c->sm_count) >= 2;
+        if (two_pipes) p.stages_b = p.stages_b / 2 * 2;
         left -= (size_t)p.stages_b * b_bytes;
         int sa = (int)(left / p.a_alloc);
         p.stages_a = sa > 4 ? 4 : sa;
@@ -1397,6 +1406,9 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     if (p.resident) {
         p.n_issuers = (p.stages_a >= 4 && 4 * p.BN <= 512) ? 4 : 2;
         p.acc_per = p.n_issuers * 2 * p.BN <= 512 ? 2 : 1;
+    } else if (two_pipes) {
+        p.n_issuers = 2;
+        p.acc_per = 4 * p.BN <= 512 ? 2 : 1;
     }
     p.stages_a = p.stages_a / p.n_issuers * p.n_issuers;
     p.tmem_cols = pow2_cols(p.n_issuers * p.acc_per * p.BN);
