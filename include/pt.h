@@ -59,6 +59,13 @@ const char *pt_status_string(pt_status s);
 pt_status pt_poll_device_status(pt_ctx *ctx, void *stream);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 uint64_t pt_launch_count(const pt_ctx *ctx);
+/* Upper bound on the CTAs (one per SM) a pt_conv_wgrad launch may use; 0 restores the default, all SMs. The weight gradient
+ * (Eq. 4) splits its reduction over the output pixels across CTAs, and the weight gradients of different layers are
+ * independent of each other: launches that leave SMs free can run side by side on several streams, which amortises their
+ * fixed cost (pipeline fill, partial-tile exchange). The setting changes the workspace pt_conv_workspace_bytes reports for
+ * PT_CONV_WGRAD, so set it before sizing workspaces; it has no effect on results beyond the summation order of the splits
+ * (still fixed for a given setting). PT_ERR_INVALID_ARG if max_ctas is negative. */
+pt_status pt_set_wgrad_cta_limit(pt_ctx *ctx, int max_ctas);
 
 /* ------------------------------------------------------------------------------------------
  * Convolutions (paper Sec. 2.1: convolution layers dominate training time; Eq. 4: weight gradient).

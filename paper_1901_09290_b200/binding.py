@@ -63,6 +63,7 @@ EXPORTS = {
     "pt_status_string": (c_char_p, [c_int32]),
     "pt_poll_device_status": (c_int32, [c_void_p, c_void_p]),
     "pt_launch_count": (c_uint64, [c_void_p]),
+    "pt_set_wgrad_cta_limit": (c_int32, [c_void_p, c_int32]),
     "pt_conv_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_conv_desc), c_int32]),
     "pt_conv_fwd": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_conv_dgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
@@ -138,6 +139,9 @@ class Context:
     def launch_count(self) -> int:
         return int(lib().pt_launch_count(self.handle))
 
+    def set_wgrad_cta_limit(self, max_ctas: int):
+        _check(lib().pt_set_wgrad_cta_limit(self.handle, int(max_ctas)), "pt_set_wgrad_cta_limit")
+
     def poll(self, stream=None):
         _check(lib().pt_poll_device_status(self.handle, _stream(stream)), "pt_poll_device_status")
 
@@ -145,6 +149,10 @@ class Context:
 def make_conv_desc(N, H, W, C, K, R, S, stride, pad, ldx=None, ldy=None, ldw=None, out_f32=0, algo=0) -> pt_conv_desc:
     p8 = lambda c: (c + 7) // 8 * 8
     return pt_conv_desc(N, H, W, C, K, R, S, stride, pad, ldx or p8(C), ldy or p8(K), ldw or p8(C), out_f32, algo)
+
+
+def pt_set_wgrad_cta_limit(ctx: Context, max_ctas: int):
+    ctx.set_wgrad_cta_limit(max_ctas)
 
 
 def pt_conv_workspace_bytes(ctx: Context, d: pt_conv_desc, which: int) -> int:

@@ -78,6 +78,13 @@ extern "C" pt_status pt_destroy(pt_ctx *c)
 
 extern "C" uint64_t pt_launch_count(const pt_ctx *c) { return c ? c->launches : 0; }
 
+extern "C" pt_status pt_set_wgrad_cta_limit(pt_ctx *c, int max_ctas)
+{
+    if (!c || max_ctas < 0) return PT_ERR_INVALID_ARG;
+    c->wgrad_ctas = max_ctas;
+    return PT_OK;
+}
+
 extern "C" pt_status pt_poll_device_status(pt_ctx *c, void *stream)
 {
     if (!c) return PT_ERR_INVALID_ARG;

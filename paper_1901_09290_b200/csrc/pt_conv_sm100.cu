@@ -1485,7 +1485,8 @@ int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     const int tpc = wgrad_taps_per_cta(d->R * d->S, bn);
     const int tiles = pt_ceil_div(d->K, 128) * n_tiles * pt_ceil_div(d->R * d->S, tpc);
     const long long npix = (long long)d->N * P * Q;
-    long long s = c->sm_count / tiles;                     // one CTA per SM, one wave
+    const int budget = (c->wgrad_ctas > 0 && c->wgrad_ctas < c->sm_count) ? c->wgrad_ctas : c->sm_count;
+    long long s = budget / tiles;                          // at most one CTA per SM, one wave
     const long long max_s = (npix + 255) / 256;          // at least four 64-pixel stages per split
     if (s > max_s) s = max_s;
     if (s < 1) s = 1;

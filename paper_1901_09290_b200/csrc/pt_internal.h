@@ -42,6 +42,7 @@ struct pt_ctx {
     unsigned int *d_sync = nullptr;     // zero-initialised, self-resetting arrival counters of the split weight gradient
     unsigned int sync_next = 0;         // ring position in d_sync
     uint64_t launches = 0;
+    int wgrad_ctas = 0;                 // CTA limit of a weight-gradient launch (0 = all SMs)
     // tcgen05 conv path
     void *encode_tiled = nullptr;       // cuTensorMapEncodeTiled
     void *encode_im2col = nullptr;      // cuTensorMapEncodeIm2col

@@ -74,8 +74,13 @@ class TrainStep:
     """
 
     def __init__(self, ctx: B.Context, dense_net: W.Net, counts: Sequence[int], kept, N: int, seed: int,
-                 algo: int = 0, host_inputs: bool = False, decoys: int = 2, device_rng: bool = True):
+                 algo: int = 0, host_inputs: bool = False, decoys: int = 2, device_rng: bool = True,
+                 wgrad_ctas: int = 74, wgrad_streams: int = 3):
         self.ctx, self.N, self.algo = ctx, N, algo
+        # weight gradients of different layers are independent: each launch is held to `wgrad_ctas` CTAs and the launches
+        # go round-robin to `wgrad_streams` streams, each with a workspace of its own
+        self.wgrad_ctas, self.wgrad_streams = wgrad_ctas, max(1, wgrad_streams)
+        ctx.set_wgrad_cta_limit(wgrad_ctas)
         self.dense_net = dense_net
         self.net = W.with_sizes(dense_net, counts)
         self.counts = list(counts)
@@ -115,6 +120,7 @@ class TrainStep:
             for which in range(3):
                 ws_bytes = max(ws_bytes, B.pt_conv_workspace_bytes(ctx, d, which))
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        self.ws_w = [torch.empty(ws_bytes, dtype=torch.uint8, device="cuda") for _ in range(self.wgrad_streams)]
         # e2e: the image batch arrives from pinned host memory every step
         l0 = self.net.layers[0]
         self.h_image = None
@@ -162,8 +168,8 @@ class TrainStep:
     def conv_dgrad(self, li, stream=None):
         B.pt_conv_dgrad(self.ctx, self.desc[li], self.dy[li], self.mp.wb[li], self.dx[li], self.ws, stream)
 
-    def conv_wgrad(self, li, stream=None):
-        B.pt_conv_wgrad(self.ctx, self.desc[li], self.x[li], self.dy[li], self.mp.g[li], self.ws, stream)
+    def conv_wgrad(self, li, stream=None, ws_index: int = 0):
+        B.pt_conv_wgrad(self.ctx, self.desc[li], self.x[li], self.dy[li], self.mp.g[li], self.ws_w[ws_index], stream)
 
     def lasso(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
         B.pt_group_lasso_sgd_step(self.ctx, self.mp.arr, lam, lr, mu, 0.0, self.mp.reg, self.mp.ws, stream)
@@ -190,19 +196,22 @@ class TrainStep:
                 out.append((first, d))
         return out
 
-    def train_two_streams(self):
-        """The same launches on three streams, following the network's own data dependencies: a layer's data gradient and
-        weight gradient only share their input dy_l (the weight gradients use the workspace, the data gradients do not),
-        and a block's projection shortcut is independent of the block's other convolutions in both directions."""
+    def train_two_streams(self, fwd: bool = True, dgrad: bool = True, wgrad: bool = True, lasso: bool = True):
+        """The same launches on several streams, following the network's own data dependencies: the weight gradient of a
+        layer needs only x_l and dy_l, so it starts when dy_l exists and runs beside the data gradients below it (round-robin
+        over the weight-gradient streams, each with its own workspace); a block's projection shortcut is independent of
+        the block's other convolutions in both directions. The flags select passes (used to time one pass as scheduled)."""
         main = torch.cuda.current_stream()
-        side, aux = self._side, self._aux
+        aux, ws = self._aux, self._wstreams
         n = len(self.net.layers)
         br = self._branches()
         fork_at = {f: d for f, d in br}          # before layer f: start shortcut d on the aux stream
         ds_set = {d for _, d in br}
-        for li in range(n):
+        forked = set()                           # streams that joined this launch sequence and must be joined back
+        for li in range(n if fwd else 0):
             if li in fork_at:
                 aux.wait_stream(main)
+                forked.add(aux)
                 self.conv_fwd(fork_at[li], aux)
             if li in ds_set:
                 main.wait_stream(aux)            # the block's output needs both branches
@@ -210,31 +219,48 @@ class TrainStep:
             self.conv_fwd(li, main)
         first_of = {d: f for f, d in br}
         join_after = None
+        wi = 0
         for li in range(n - 1, -1, -1):
             # dy_l exists once the data gradients above layer l are done: the weight gradient of layer l starts there, next
             # to the layer's own data gradient
-            side.wait_stream(main)
+            wk = wi % len(ws)
+            side = ws[wk]
+            wi += 1
+            if wgrad:
+                side.wait_stream(main)
+                forked.add(side)
+                self.conv_wgrad(li, side, wk)
+            if not dgrad:
+                continue
             if li in ds_set:
                 aux.wait_stream(main)            # both branches start from the gradient of the block's output
+                forked.add(aux)
                 if li > 0:
                     self.conv_dgrad(li, aux)
-                self.conv_wgrad(li, side)
                 join_after = first_of[li]
                 continue
             if li > 0:
                 self.conv_dgrad(li, main)
-            self.conv_wgrad(li, side)
             if join_after == li:
                 main.wait_stream(aux)            # the gradient of the block's input sums both branches
                 join_after = None
-        main.wait_stream(side)
-        main.wait_stream(aux)
-        self.lasso(main)
+        for w in forked:
+            main.wait_stream(w)
+        if lasso:
+            self.lasso(main)
+
+    def capture_pass(self, kind: str):
+        """A CUDA graph of one pass kind ("fwd", "dgrad", "wgrad") with the stream assignment it has inside the step."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.train_two_streams(fwd=kind == "fwd", dgrad=kind == "dgrad", wgrad=kind == "wgrad", lasso=False)
+        return g
 
     def build_graph(self, two_streams: bool = True):
         """Captures the training part of the step (every launch after the reconfiguration's host sync) into a CUDA graph.
         Call after at least one eager step, so that every table and kernel attribute is already set up."""
         self._side = torch.cuda.Stream()
+        self._wstreams = [self._side] + [torch.cuda.Stream() for _ in range(self.wgrad_streams - 1)]
         self._aux = torch.cuda.Stream()
         l0 = self.ctx.launch_count()
         self.graph = torch.cuda.CUDAGraph()

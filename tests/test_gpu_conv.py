@@ -94,6 +94,22 @@ def test_wgrad_is_run_to_run_identical():
     assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("limit", [1, 7, 37])
+def test_wgrad_with_a_cta_limit(limit):
+    """The weight gradient may be held to fewer CTAs (to run beside other kernels): same result class, bounded by the limit."""
+    c = Hh.ctx()
+    try:
+        B.pt_set_wgrad_cta_limit(c, limit)
+        for (N, H, C, K, R) in [(4, 14, 93, 77, 3), (8, 28, 130, 70, 1), (3, 16, 11, 27, 3)]:
+            x, w, dy, pad = _case(N, H, H, C, K, R, 1, W.BASE_SEED + 31 + limit)
+            dw = Hh.run_conv_all(N, H, H, C, K, R, 1, pad, x, w, dy, algo=2)[2]
+            Hh.check_conv(dw, C, oracle.conv_wgrad(x.numpy(), dy.numpy(), R, R, 1, pad), what=f"wgrad limit {limit}")
+        with pytest.raises(B.PtError):
+            B.pt_set_wgrad_cta_limit(c, -1)
+    finally:
+        B.pt_set_wgrad_cta_limit(c, 0)
+
+
 def test_invalid_arguments_are_rejected_before_launch():
     c = Hh.ctx()
     buf = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
