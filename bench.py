@@ -24,6 +24,9 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum over the launches of each conv pass in one step of the default workload
+# (one ncu capture, 1 pass per launch; the summary and the command are in profiles/step_launch_list_resnet50_keep060_b64.txt)
+NCU_DRAM_BYTES = {"fwd": 1.140e9, "dgrad": 1.113e9, "wgrad": 2.123e9}   # incl. the stem layout kernels
 METRIC = "pruned ResNet-50 train-step conv TFLOP/s (useful FLOPs / whole step)"
 UNIT = "TFLOP/s"
 
@@ -396,7 +399,11 @@ def run_ours(args):
         "reconf_gbs": ts.reconf_bytes() / (phase["reconfigure"] * 1e-3) / 1e9,
         "roofline": {"kernel": f"conv_{dom} (all {n_dom} launches of a step, as the step schedules them)", "bound": "tensor",
                      "achieved": dom_flops / dom_t / 1e12, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": dom_flops / dom_t / tc_peak, "traffic": None, "peak_source": pk["source"] + " sustained bf16"},
+                     "frac": dom_flops / dom_t / tc_peak,
+                     # DRAM bytes of the pass's launches in one ncu capture of the default workload (profiles/step_launch_list_*)
+                     "traffic": NCU_DRAM_BYTES.get(dom) if (args.keep is None and args.batch == 64 and args.algo == 0) else None,
+                     "algorithmic_bytes": sum(ts.layer_bytes(li, which_id[dom]) for li in range(nL) if not (dom == "dgrad" and li == 0)),
+                     "peak_source": pk["source"] + " sustained bf16"},
     }
     if rank == 0:
         if args.per_layer:
