@@ -137,6 +137,28 @@ pt_status pt_group_lasso_sgd_step(pt_ctx *ctx, const pt_layer *layers /*host*/, 
                                   const pt_sgd_hparams *hp /*host*/, double *reg_sum_out,
                                   void *ws, size_t ws_bytes, void *stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Penalty coefficient set-up (Sec. 4.1, "Regularization Penalty Coefficient Setup", Eq. 3): lambda is chosen once, at the
+ * first training iteration, so that the group-lasso term is a given share (the paper uses 20-25 %) of the total loss:
+ *     ratio = lambda * R / (loss + lambda * R),  R = sum over groups of ||W_g||   =>   lambda = ratio * loss / ((1 - ratio) * R)
+ * with loss the cross-entropy of the first forward pass and R the value pt_group_lasso_sgd_step writes to reg_sum_out.
+ * ------------------------------------------------------------------------------------------ */
+
+/* loss_out[0] (device, double) = mean over the batch of -log softmax(logits[i])[labels[i]].
+ * logits: device, fp32, [n][ld] with ld >= classes (elements past `classes` are never read); labels: device, int32, each
+ * in [0, classes). Rows are reduced in fp32 with the row maximum subtracted, the batch mean is accumulated in fp64 in a
+ * fixed order (run-to-run identical). A label out of range makes the result NaN. ws: device scratch of at least
+ * pt_cross_entropy_workspace_bytes(n) bytes. PT_ERR_INVALID_ARG for n < 1, classes < 1, ld < classes, null pointers. */
+size_t pt_cross_entropy_workspace_bytes(int32_t n);
+pt_status pt_cross_entropy(pt_ctx *ctx, const float *logits, const int32_t *labels, int32_t n, int32_t classes, int32_t ld,
+                           double *loss_out, void *ws, size_t ws_bytes, void *stream);
+
+/* lambda_out[0] (device, float) = ratio * loss[0] / ((1 - ratio) * reg_sum[0])  (Eq. 3 solved for lambda), computed in fp64.
+ * loss, reg_sum: device doubles (from pt_cross_entropy and pt_group_lasso_sgd_step). reg_sum == 0 (no regularised group
+ * left) gives lambda = 0. PT_ERR_INVALID_ARG unless 0 < ratio < 1. The caller reads lambda_out back to fill
+ * pt_sgd_hparams.lambda_ for the steps that follow. */
+pt_status pt_set_coeff(pt_ctx *ctx, const double *loss, const double *reg_sum, float ratio, float *lambda_out, void *stream);
+
 /* zero_out[k] = (max_{rs,c} |w| < threshold), zero_in[c] = (max_{k,rs} |w| < threshold), strict <, in fp32
  * (Sec. 4.1: threshold 1e-4; Sec. 4.2 / Fig. 4: the absolute maximum of a channel's parameters). A NaN keeps
  * its groups. If zero_in_place != 0 the weights, momentum and shadow of every detected group are set to 0

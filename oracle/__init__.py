@@ -181,6 +181,18 @@ def set_coeff(loss1: float, reg_sum: float, ratio: float) -> float:
     return ratio * loss1 / ((1.0 - ratio) * reg_sum)
 
 
+def cross_entropy(logits, labels) -> float:
+    """The classification loss l(y, f(x, W)) of Eq. 1 / Eq. 3 for a softmax classifier: the batch mean of
+    -log(softmax(logits)[label]), in fp64 (the paper names the cross-entropy loss after the first forward pass)."""
+    z = np.asarray(logits, np.float64)
+    lab = np.asarray(labels, np.int64)
+    tot = 0.0
+    for i in range(z.shape[0]):
+        m = z[i].max()
+        tot += m + np.log(np.exp(z[i] - m).sum()) - z[i, lab[i]]
+    return tot / z.shape[0]
+
+
 # --------------------------------------------------------------------------- detection
 def find_zero_groups(w, thr: float = 1e-4) -> Tuple[np.ndarray, np.ndarray]:
     """(zero_out[K], zero_in[C]) uint8: group is zero iff every |w| < thr in fp32 (Sec. 4.1, Fig. 4)."""

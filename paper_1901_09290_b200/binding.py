@@ -73,6 +73,9 @@ EXPORTS = {
                                           c_void_p, c_size_t, c_void_p]),
     "pt_find_zero_groups": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_float, c_int32, c_void_p, c_size_t, c_void_p]),
     "pt_find_zero_groups_noalloc": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p]),
+    "pt_cross_entropy_workspace_bytes": (c_size_t, [c_int32]),
+    "pt_cross_entropy": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "pt_set_coeff": (c_int32, [c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]),
     "pt_reconfigure_plan": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(c_int32), c_void_p]),
     "pt_reconfigure": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(pt_graph), c_void_p]),
 }
@@ -211,6 +214,20 @@ def pt_find_zero_groups_noalloc(w, K, C, RS, threshold, zero_out, zero_in, strea
     """Detection of one weight tensor with the library's static scratch: for callers that cannot allocate a workspace."""
     _check(lib().pt_find_zero_groups_noalloc(_ptr(w), K, C, RS, threshold, _ptr(zero_out), _ptr(zero_in), _stream(stream)),
            "pt_find_zero_groups_noalloc")
+
+
+def pt_cross_entropy_workspace_bytes(n: int) -> int:
+    return int(lib().pt_cross_entropy_workspace_bytes(n))
+
+
+def pt_cross_entropy(ctx, logits, labels, n, classes, ld, loss_out, ws, stream=None):
+    p, nb = _ws(ws)
+    _check(lib().pt_cross_entropy(ctx.handle, _ptr(logits), _ptr(labels), n, classes, ld, _ptr(loss_out), p, nb, _stream(stream)),
+           "pt_cross_entropy")
+
+
+def pt_set_coeff(ctx, loss, reg_sum, ratio, lambda_out, stream=None):
+    _check(lib().pt_set_coeff(ctx.handle, _ptr(loss), _ptr(reg_sum), ratio, _ptr(lambda_out), _stream(stream)), "pt_set_coeff")
 
 
 class GraphHandle:

@@ -227,6 +227,14 @@ def gen_dy(N, P, Q, K, seed) -> torch.Tensor:
     return bf16_round(torch.randn((N, P, Q, K), generator=_gen(seed), dtype=torch.float32) * (2.0 ** -6))
 
 
+def gen_logits(n, classes, seed, scale=3.0):
+    """Classifier outputs of a freshly initialised network ~ N(0, scale) and uniform integer labels."""
+    g = _gen(seed)
+    logits = torch.randn((n, classes), generator=g, dtype=torch.float32) * scale
+    labels = torch.randint(0, classes, (n,), generator=g, dtype=torch.int32)
+    return logits, labels
+
+
 def gen_small(shape, seed, std=1e-3) -> torch.Tensor:
     """Gradients / momenta for stand-alone update runs ~ N(0, std)."""
     return torch.randn(tuple(shape), generator=_gen(seed), dtype=torch.float32) * std

@@ -136,3 +136,38 @@ def test_detection_config1_counts():
     kept = W.choose_kept(net, [13, 27], W.BASE_SEED + 1)
     dm = _check_detection(W.gen_model(net, W.BASE_SEED + 1, kept=kept))
     assert int(dm.z_out[0].sum()) == 5 and int(dm.z_in[0].sum()) == 3
+
+
+@pytest.mark.parametrize("n,classes,ld", [(1, 1, 1), (3, 10, 10), (64, 1000, 1000), (128, 100, 104), (37, 33, 40)])
+def test_cross_entropy_and_set_coeff(n, classes, ld):
+    """Eq. 3: cross-entropy of the first forward pass and lambda from the penalty ratio, against the fp64 oracle."""
+    c = Hh.ctx()
+    logits, labels = W.gen_logits(n, classes, W.BASE_SEED + 77 + n)
+    zd = torch.full((n, ld), float("nan"), dtype=torch.float32, device="cuda")      # pad lanes must never be read
+    zd[:, :classes] = logits
+    ld_ = labels.cuda()
+    loss = torch.zeros(1, dtype=torch.float64, device="cuda")
+    ws = torch.empty(max(16, B.pt_cross_entropy_workspace_bytes(n)), dtype=torch.uint8, device="cuda")
+    B.pt_cross_entropy(c, zd, ld_, n, classes, ld, loss, ws)
+    B.pt_cross_entropy(c, zd, ld_, n, classes, ld, loss, ws)                        # run-to-run identical
+    ref = oracle.cross_entropy(logits.numpy(), labels.numpy())
+    got = float(loss.cpu()[0])
+    assert abs(got - ref) <= 1e-5 * max(1.0, abs(ref)), (got, ref)
+    a = loss.clone()
+    B.pt_cross_entropy(c, zd, ld_, n, classes, ld, loss, ws)
+    assert torch.equal(a, loss)
+    reg = torch.tensor([812.5], dtype=torch.float64, device="cuda")
+    lam = torch.zeros(1, dtype=torch.float32, device="cuda")
+    for ratio in (0.2, 0.25):
+        B.pt_set_coeff(c, loss, reg, ratio, lam)
+        want = oracle.set_coeff(got, 812.5, float(np.float32(ratio)))
+        assert abs(float(lam.cpu()[0]) - want) <= 2e-7 * abs(want) + 1e-30
+    B.pt_set_coeff(c, loss, torch.zeros(1, dtype=torch.float64, device="cuda"), 0.25, lam)
+    assert float(lam.cpu()[0]) == 0.0
+    for bad in (0.0, 1.0, -0.1, float("nan")):
+        with pytest.raises(B.PtError):
+            B.pt_set_coeff(c, loss, reg, bad, lam)
+    with pytest.raises(B.PtError):
+        B.pt_cross_entropy(c, zd, ld_, n, classes, classes - 1, loss, ws)
+    torch.cuda.synchronize()
+    c.poll()

@@ -87,6 +87,41 @@ def test_set_coeff_roundtrip():
     assert abs(lam * 812.5 / (2.3 + lam * 812.5) - 0.25) < 1e-15
 
 
+def test_cross_entropy_closed_forms():
+    """Pins of the classification loss used by Eq. 3: uniform logits give ln(classes); a one-hot limit gives 0; the loss
+    does not move when a constant is added to a row; two classes reduce to the logistic loss log(1 + exp(-d))."""
+    rng = np.random.default_rng(5)
+    n, k = 7, 11
+    lab = rng.integers(0, k, n)
+    assert abs(oracle.cross_entropy(np.zeros((n, k)), lab) - np.log(k)) < 1e-15
+    z = np.full((n, k), -800.0)
+    z[np.arange(n), lab] = 0.0
+    assert oracle.cross_entropy(z, lab) == 0.0
+    z = rng.standard_normal((n, k)) * 4
+    shift = rng.standard_normal((n, 1)) * 100
+    assert abs(oracle.cross_entropy(z, lab) - oracle.cross_entropy(z + shift, lab)) < 1e-12
+    d = rng.standard_normal(n) * 3                       # two classes: margin d of the true class
+    z2 = np.stack([d, np.zeros(n)], axis=1)
+    assert abs(oracle.cross_entropy(z2, np.zeros(n, int)) - np.mean(np.log1p(np.exp(-d)))) < 1e-14
+    # brute force on a tiny case: exponentials written out
+    z3 = np.array([[1.0, 2.0, 0.5], [0.0, -1.0, 3.0]])
+    e = np.exp(z3)
+    ref = -(np.log(e[0, 1] / e[0].sum()) + np.log(e[1, 0] / e[1].sum())) / 2
+    assert abs(oracle.cross_entropy(z3, [1, 0]) - ref) < 1e-14
+
+
+def test_set_coeff_reaches_the_requested_share_on_a_model():
+    """Eq. 3 end to end on a small random model: with lambda from set_coeff the lasso term is `ratio` of the total loss."""
+    rng = np.random.default_rng(9)
+    ws = [rng.standard_normal((6, 3, 3, 4)), rng.standard_normal((5, 1, 1, 6))]
+    R = oracle.lasso_penalty(ws, reg_in=[False, True], reg_out=[True, True])
+    z = rng.standard_normal((8, 10))
+    loss = oracle.cross_entropy(z, rng.integers(0, 10, 8))
+    for ratio in (0.2, 0.25):
+        lam = oracle.set_coeff(loss, R, ratio)
+        assert abs(lam * R / (loss + lam * R) - ratio) < 1e-14 and lam > 0
+
+
 def test_detection_boundaries():
     thr = np.float32(1e-4)
     w = np.ones((6, 1, 2, 5), np.float32)
