@@ -270,6 +270,64 @@ def conv_flops(N, H, W, C, K, R, S, stride, pad) -> int:
     return 2 * N * P * Q * K * C * R * S
 
 
+# --------------------------------------------------------------------------- feature normalisation (Sec. 2.1)
+def bn_relu_fwd(x, gamma, beta, eps: float = 1e-5, residual=None, relu: bool = True):
+    """Training-mode batch normalisation of x [N][H][W][C] followed by the residual add and the ReLU of a ResNet block.
+
+    Sec. 2.1: the normalisation layer computes each channel's mean and variance over the mini-batch and the feature map
+    and normalises with them; gamma and beta are the per-channel scale and shift that the compaction carries along
+    (Sec. 4.2). Per channel c, over the M = N*H*W positions:
+        mean = sum(x)/M,  var = sum((x - mean)^2)/M,  xhat = (x - mean)/sqrt(var + eps),
+        z = gamma*xhat + beta (+ residual),  y = max(z, 0) if relu else z.
+    Returns y, mean, invstd = 1/sqrt(var + eps), var (biased), all fp64."""
+    x = np.asarray(x, np.float64)
+    N, H, W, C = x.shape
+    M = N * H * W
+    y = np.empty_like(x)
+    mean = np.empty(C)
+    var = np.empty(C)
+    for c in range(C):
+        xc = x[..., c]
+        mean[c] = xc.sum() / M
+        var[c] = ((xc - mean[c]) ** 2).sum() / M
+        z = gamma[c] * (xc - mean[c]) / np.sqrt(var[c] + eps) + beta[c]
+        if residual is not None:
+            z = z + np.asarray(residual, np.float64)[..., c]
+        y[..., c] = np.maximum(z, 0.0) if relu else z
+    return y, mean, 1.0 / np.sqrt(var + eps), var
+
+
+def bn_running_stats(running_mean, running_var, mean, var, M: int, momentum: float = 0.1):
+    """The moving statistics a normalisation layer keeps for inference (the vectors the compaction gathers, Sec. 4.2):
+    r <- (1 - momentum)*r + momentum*batch statistic, with the unbiased variance var*M/(M-1) (M > 1)."""
+    rm = (1.0 - momentum) * np.asarray(running_mean, np.float64) + momentum * mean
+    rv = (1.0 - momentum) * np.asarray(running_var, np.float64) + momentum * var * (M / (M - 1.0) if M > 1 else 1.0)
+    return rm, rv
+
+
+def bn_relu_bwd(x, y, dy, gamma, mean, invstd, relu: bool = True):
+    """Back-propagation through y = relu(gamma*xhat + beta + residual) with the batch statistics of the forward pass.
+
+    dz = dy where the ReLU passed (y > 0), else 0; the residual branch receives dz unchanged;
+        dbeta = sum(dz),  dgamma = sum(dz*xhat),
+        dx = gamma*invstd/M * (M*dz - dbeta - xhat*dgamma)      (mean and variance depend on every position)
+    Returns dx, dresidual, dgamma, dbeta (fp64)."""
+    x = np.asarray(x, np.float64)
+    dy = np.asarray(dy, np.float64)
+    N, H, W, C = x.shape
+    M = N * H * W
+    dz = dy * (np.asarray(y, np.float64) > 0) if relu else dy.copy()
+    dx = np.empty_like(x)
+    dgamma = np.empty(C)
+    dbeta = np.empty(C)
+    for c in range(C):
+        xhat = (x[..., c] - mean[c]) * invstd[c]
+        dbeta[c] = dz[..., c].sum()
+        dgamma[c] = (dz[..., c] * xhat).sum()
+        dx[..., c] = gamma[c] * invstd[c] / M * (M * dz[..., c] - dbeta[c] - xhat * dgamma[c])
+    return dx, dz, dgamma, dbeta
+
+
 # --------------------------------------------------------------------------- toy network (invariant only)
 def bn_affine(y, gamma, beta, mean, var, eps=1e-5):
     """Inference-form batch norm with given running statistics, per output channel."""
