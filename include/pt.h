@@ -138,6 +138,44 @@ pt_status pt_group_lasso_sgd_step(pt_ctx *ctx, const pt_layer *layers /*host*/, 
                                   void *ws, size_t ws_bytes, void *stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Feature normalisation (Sec. 2.1: batch normalisation layers take about 30 % of CNN training time and are bound by memory
+ * bandwidth because they read their input several times) with the residual add and ReLU of a ResNet block fused in.
+ * Activations are NHWC bf16 with channel pitch ld, exactly as the convolutions read and write them; C is the CURRENT
+ * (pruned, possibly ragged) channel count. Per channel, over the M = N*H*W positions:
+ *     mean = sum(x)/M, var = sum((x-mean)^2)/M, xhat = (x-mean)/sqrt(var+eps), z = gamma*xhat + beta (+ residual),
+ *     y = relu ? max(z, 0) : z;   running <- (1-momentum)*running + momentum*(mean | var*M/(M-1)).
+ * Backward (dz = dy where y > 0, or dy without ReLU):
+ *     dbeta = sum(dz), dgamma = sum(dz*xhat), dx = gamma/sqrt(var+eps)/M * (M*dz - dbeta - xhat*dgamma), dresidual = dz.
+ * All pointers are device pointers; x, y, residual, dy, dx, dresidual are 16-byte aligned [N][H][W][ld] bf16 tensors whose
+ * pad lanes (channel >= C) are read but never used, and are written as zeros in the outputs. Statistics, gamma, beta and
+ * their gradients are fp32 vectors of C elements. Sums are combined in a fixed order (run-to-run identical).
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    int32_t N, H, W, C;
+    int32_t ld;        /* channel pitch (elements, multiple of 8, >= C, <= 2048) */
+    float eps;         /* >= 0 */
+    float momentum;    /* of the moving statistics, in [0, 1] */
+    int32_t relu;      /* 0 / 1 */
+} pt_bn_desc;
+
+/* Bytes of workspace both calls need for this descriptor (partial sums of the reduction blocks). */
+size_t pt_bn_workspace_bytes(const pt_ctx *ctx, const pt_bn_desc *d);
+
+/* y = relu(gamma*xhat + beta + residual). residual may be NULL. running_mean / running_var: both NULL (not kept) or both
+ * given (updated in place). save_mean, save_invstd (C floats each) receive the batch statistics the backward pass needs.
+ * PT_ERR_INVALID_ARG for bad sizes, pitches, alignment or missing pointers; PT_ERR_UNSUPPORTED for ld > 2048;
+ * PT_ERR_WORKSPACE if ws is too small. */
+pt_status pt_bn_relu_fwd(pt_ctx *ctx, const pt_bn_desc *d, const void *x, const void *residual, const float *gamma,
+                         const float *beta, float *running_mean, float *running_var, float *save_mean, float *save_invstd,
+                         void *y, void *ws, size_t ws_bytes, void *stream);
+
+/* Gradients of the call above. y is the forward output (only its sign is used, and only with relu = 1; may be NULL
+ * otherwise); dresidual may be NULL when the block has no residual input. */
+pt_status pt_bn_relu_bwd(pt_ctx *ctx, const pt_bn_desc *d, const void *x, const void *y, const void *dy, const float *gamma,
+                         const float *save_mean, const float *save_invstd, void *dx, void *dresidual, float *dgamma,
+                         float *dbeta, void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
  * Penalty coefficient set-up (Sec. 4.1, "Regularization Penalty Coefficient Setup", Eq. 3): lambda is chosen once, at the
  * first training iteration, so that the group-lasso term is a given share (the paper uses 20-25 %) of the total loss:
  *     ratio = lambda * R / (loss + lambda * R),  R = sum over groups of ||W_g||   =>   lambda = ratio * loss / ((1 - ratio) * R)

@@ -44,6 +44,11 @@ class pt_sgd_hparams(Structure):
     _fields_ = [("lambda_", c_float), ("lr", c_float), ("momentum", c_float), ("weight_decay", c_float)]
 
 
+class pt_bn_desc(Structure):
+    _fields_ = [("N", c_int32), ("H", c_int32), ("W", c_int32), ("C", c_int32), ("ld", c_int32),
+                ("eps", c_float), ("momentum", c_float), ("relu", c_int32)]
+
+
 class pt_space(Structure):
     _fields_ = [("size", c_int32), ("fixed", c_uint8)]
 
@@ -73,6 +78,9 @@ EXPORTS = {
                                           c_void_p, c_size_t, c_void_p]),
     "pt_find_zero_groups": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_float, c_int32, c_void_p, c_size_t, c_void_p]),
     "pt_find_zero_groups_noalloc": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p]),
+    "pt_bn_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_bn_desc)]),
+    "pt_bn_relu_fwd": (c_int32, [c_void_p, POINTER(pt_bn_desc)] + [c_void_p] * 9 + [c_void_p, c_size_t, c_void_p]),
+    "pt_bn_relu_bwd": (c_int32, [c_void_p, POINTER(pt_bn_desc)] + [c_void_p] * 10 + [c_void_p, c_size_t, c_void_p]),
     "pt_cross_entropy_workspace_bytes": (c_size_t, [c_int32]),
     "pt_cross_entropy": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_set_coeff": (c_int32, [c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]),
@@ -214,6 +222,27 @@ def pt_find_zero_groups_noalloc(w, K, C, RS, threshold, zero_out, zero_in, strea
     """Detection of one weight tensor with the library's static scratch: for callers that cannot allocate a workspace."""
     _check(lib().pt_find_zero_groups_noalloc(_ptr(w), K, C, RS, threshold, _ptr(zero_out), _ptr(zero_in), _stream(stream)),
            "pt_find_zero_groups_noalloc")
+
+
+def make_bn_desc(N, H, W, C, ld=None, eps=1e-5, momentum=0.1, relu=True) -> pt_bn_desc:
+    return pt_bn_desc(N, H, W, C, ld or (C + 7) // 8 * 8, eps, momentum, int(bool(relu)))
+
+
+def pt_bn_workspace_bytes(ctx, d: pt_bn_desc) -> int:
+    return int(lib().pt_bn_workspace_bytes(ctx.handle, byref(d)))
+
+
+def pt_bn_relu_fwd(ctx, d, x, residual, gamma, beta, running_mean, running_var, save_mean, save_invstd, y, ws, stream=None):
+    p, n = _ws(ws)
+    _check(lib().pt_bn_relu_fwd(ctx.handle, byref(d), _ptr(x), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(running_mean),
+                                _ptr(running_var), _ptr(save_mean), _ptr(save_invstd), _ptr(y), p, n, _stream(stream)),
+           "pt_bn_relu_fwd")
+
+
+def pt_bn_relu_bwd(ctx, d, x, y, dy, gamma, save_mean, save_invstd, dx, dresidual, dgamma, dbeta, ws, stream=None):
+    p, n = _ws(ws)
+    _check(lib().pt_bn_relu_bwd(ctx.handle, byref(d), _ptr(x), _ptr(y), _ptr(dy), _ptr(gamma), _ptr(save_mean), _ptr(save_invstd),
+                                _ptr(dx), _ptr(dresidual), _ptr(dgamma), _ptr(dbeta), p, n, _stream(stream)), "pt_bn_relu_bwd")
 
 
 def pt_cross_entropy_workspace_bytes(n: int) -> int:

@@ -2,6 +2,7 @@
 
     python -m paper_1901_09290_b200.layerbench --layer s1b1.c3 --passes fwd,dgrad,wgrad --iters 20
     python -m paper_1901_09290_b200.layerbench --shape 64,56,36,143,1,1 --passes fwd      # N,H,C,K,R,stride
+    python -m paper_1901_09290_b200.layerbench --bn 64,56,143                              # batch norm + ReLU + residual: N,H,C
 
 It is also the small case ncu captures are taken on.
 """
@@ -26,7 +27,10 @@ def main():
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--algo", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true", help="time eager launches (includes host launch cost)")
+    ap.add_argument("--bn", default=None, help="N,H,C: time pt_bn_relu_fwd / pt_bn_relu_bwd instead of a convolution")
     args = ap.parse_args()
+    if args.bn:
+        return bn_main(args)
     if args.shape:
         N, H, C, K, R, stride = [int(t) for t in args.shape.split(",")]
         name = args.shape
@@ -84,6 +88,50 @@ def main():
         us = e0.elapsed_time(e1) * 1e3 / args.iters
         by = act + K * C * R * R * (4 if ps == "wgrad" else 2)
         out[ps] = {"us": round(us, 2), "tflops": round(flops / us / 1e6, 1), "gbs": round(by / us / 1e3, 1)}
+    ctx.poll()
+    print(json.dumps(out))
+
+
+def bn_main(args):
+    """Batch norm + residual + ReLU on one activation tensor: device time and algorithmic GB/s (every tensor counted once:
+    forward x, residual, y = 6 B per element; backward x, y, dy, dx, dresidual = 10 B per element)."""
+    N, H, C = [int(t) for t in args.bn.split(",")]
+    ld = W.pad16(C)
+    ctx = B.Context(0)
+    d = B.make_bn_desc(N, H, H, C, ld)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    mk = lambda: torch.randn((N, H, H, ld), generator=g, device="cuda").to(torch.bfloat16)
+    sets = [tuple(mk() for _ in range(7)) for _ in range(args.sets)]
+    gamma, beta = torch.ones(C, device="cuda"), torch.zeros(C, device="cuda")
+    rm, rv = torch.zeros(C, device="cuda"), torch.ones(C, device="cuda")
+    sm, si, dg, db = (torch.empty(C, device="cuda") for _ in range(4))
+    ws = torch.empty(max(16, B.pt_bn_workspace_bytes(ctx, d)), dtype=torch.uint8, device="cuda")
+    elems = N * H * H * C
+    out = {"bn": args.bn, "ld": ld}
+    for ps in ("fwd", "bwd"):
+        def run(i):
+            x, r, y, dy, dx, dr, _ = sets[i % len(sets)]
+            if ps == "fwd":
+                B.pt_bn_relu_fwd(ctx, d, x, r, gamma, beta, rm, rv, sm, si, y, ws)
+            else:
+                B.pt_bn_relu_bwd(ctx, d, x, y, dy, gamma, sm, si, dx, dr, dg, db, ws)
+        for i in range(3):
+            run(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            for i in range(args.iters):
+                run(i)
+        gr.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        gr.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / args.iters
+        by = elems * (6 if ps == "fwd" else 10)
+        out[ps] = {"us": round(us, 2), "gbs": round(by / us / 1e3, 1)}
     ctx.poll()
     print(json.dumps(out))
 
