@@ -72,37 +72,37 @@ __global__ void __launch_bounds__(kBnThreads) bn_reduce_kernel(const BnP p, cons
         }
         const long long m0 = (long long)blockIdx.x * p.chunk;
         const long long m1 = m0 + p.chunk < p.M ? m0 + p.chunk : p.M;
-        for (long long m = m0 + pr; m < m1; m += 2 * p.ppb) {
-            const long long mb = m + p.ppb;
-            const bool two = mb < m1;
-            const size_t ia = (size_t)m * p.LV + cv, ib = (size_t)mb * p.LV + cv;
-            float xa[8], xb[8];
-            const uint4 va = x[ia];
-            uint4 vb = va;
-            if (two) vb = x[ib];
-            if (MODE == 0) {
-                unpack8(va, xa);
-                unpack8(vb, xb);
+        constexpr int U = MODE == 0 ? 4 : 2;          // pixels per iteration: all their loads are issued before any arithmetic
+        for (long long m = m0 + pr; m < m1; m += (long long)U * p.ppb) {
+            uint4 vx[U], vg[U], vy[U];
+            bool live[U];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float da = xa[j] - piv[j], db = two ? xb[j] - piv[j] : 0.f;
-                    a0[j] += da; a1[j] += da * da;
-                    a0[j] += db; a1[j] += db * db;
-                }
-            } else {
-                const uint4 ga = dy[ia], ya = y[ia];
-                uint4 gb = ga, yb = ya;
-                if (two) { gb = dy[ib]; yb = y[ib]; }
-                float da[8], db[8], fa[8], fb[8];
-                unpack8(va, xa); unpack8(vb, xb);
-                unpack8(ga, da); unpack8(gb, db);
-                unpack8(ya, fa); unpack8(yb, fb);
+            for (int u = 0; u < U; ++u) {
+                const long long mu_ = m + (long long)u * p.ppb;
+                live[u] = mu_ < m1;
+                const size_t i = (size_t)(live[u] ? mu_ : m) * p.LV + cv;
+                vx[u] = x[i];
+                if (MODE == 1) { vg[u] = dy[i]; vy[u] = y[i]; }
+            }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float za = (!p.relu || fa[j] > 0.f) ? da[j] : 0.f;
-                    const float zb = two ? ((!p.relu || fb[j] > 0.f) ? db[j] : 0.f) : 0.f;
-                    a0[j] += za; a1[j] += za * ((xa[j] - mu[j]) * is[j]);
-                    a0[j] += zb; a1[j] += zb * ((xb[j] - mu[j]) * is[j]);
+            for (int u = 0; u < U; ++u) {
+                float xv[8];
+                unpack8(vx[u], xv);
+                if (MODE == 0) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float dd = live[u] ? xv[j] - piv[j] : 0.f;
+                        a0[j] += dd; a1[j] += dd * dd;
+                    }
+                } else {
+                    float dv[8], fv[8];
+                    unpack8(vg[u], dv);
+                    unpack8(vy[u], fv);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float z = (live[u] && (!p.relu || fv[j] > 0.f)) ? dv[j] : 0.f;
+                        a0[j] += z; a1[j] += z * ((xv[j] - mu[j]) * is[j]);
+                    }
                 }
             }
         }
