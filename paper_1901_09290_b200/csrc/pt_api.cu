@@ -65,6 +65,11 @@ extern "C" pt_status pt_destroy(pt_ctx *c)
     if (!c) return PT_OK;
     (void)cudaSetDevice(c->device);
     if (c->upload_done) cudaEventDestroy(c->upload_done);
+    for (int i = 0; i < 3; ++i) {
+        if (c->fork_stream[i]) cudaStreamDestroy(c->fork_stream[i]);
+        if (c->join_ev[i]) cudaEventDestroy(c->join_ev[i]);
+    }
+    if (c->fork_ev) cudaEventDestroy(c->fork_ev);
     if (c->d_status) cudaFree(c->d_status);
     if (c->h_status) cudaFreeHost(c->h_status);
     if (c->d_arena) cudaFree(c->d_arena);

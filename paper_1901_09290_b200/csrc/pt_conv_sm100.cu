@@ -1618,11 +1618,30 @@ pt_status dgrad_stride2_halo(pt_ctx *c, const pt_conv_desc *d, int P, int Q, con
     // pixel-linear tiles of the im2col kernel do better
     if (d->R * d->S == 1 && (d->H / 2) * (d->W / 2) < 64) return PT_ERR_UNSUPPORTED;
     if (any_empty) PT_CUDA_OK(cudaMemsetAsync(dx, 0, (size_t)d->N * d->H * d->W * d->ldx * 2, st));
-    for (int i = 0; i < n_launch; ++i) {
-        pt_status r = launch_halo<true>(c, d, hs[i], w, dx, st);
-        if (r != PT_OK) return r == PT_ERR_UNSUPPORTED && i == 0 && !any_empty ? r : (r == PT_ERR_UNSUPPORTED ? PT_ERR_CUDA : r);
+    // The parity classes write disjoint pixels of dx and read the same inputs: launches 1.. go to the context's helper
+    // streams (forked from and joined back to the caller's stream by events) so that their fills and drains overlap.
+    if (n_launch > 1 && !c->fork_ev) {
+        bool ok = cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < 3 && ok; ++i)
+            ok = cudaStreamCreateWithFlags(&c->fork_stream[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->join_ev[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { (void)cudaGetLastError(); return PT_ERR_CUDA; }
     }
-    return PT_OK;
+    if (n_launch > 1) PT_CUDA_OK(cudaEventRecord(c->fork_ev, st));
+    pt_status first = PT_OK;
+    for (int i = 0; i < n_launch; ++i) {
+        cudaStream_t si = i == 0 ? st : c->fork_stream[i - 1];
+        if (i > 0) PT_CUDA_OK(cudaStreamWaitEvent(si, c->fork_ev, 0));
+        pt_status r = launch_halo<true>(c, d, hs[i], w, dx, si);
+        if (i > 0) {                                   // join even after a failure, so that a capture stays well formed
+            PT_CUDA_OK(cudaEventRecord(c->join_ev[i - 1], si));
+            PT_CUDA_OK(cudaStreamWaitEvent(st, c->join_ev[i - 1], 0));
+        }
+        if (r != PT_OK && first == PT_OK)
+            first = (r == PT_ERR_UNSUPPORTED && i == 0 && !any_empty) ? r : (r == PT_ERR_UNSUPPORTED ? PT_ERR_CUDA : r);
+        if (first != PT_OK && i == 0) return first;    // nothing forked yet
+    }
+    return first;
 }
 
 }  // namespace

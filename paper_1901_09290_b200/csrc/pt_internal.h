@@ -43,6 +43,10 @@ struct pt_ctx {
     unsigned int sync_next = 0;         // ring position in d_sync
     uint64_t launches = 0;
     int wgrad_ctas = 0;                 // CTA limit of a weight-gradient launch (0 = all SMs)
+    // Helper streams for independent launches inside one call (the parity classes of a stride-2 data gradient): the caller's
+    // stream forks to them and joins them back through events, which a stream capture records as graph edges.
+    cudaStream_t fork_stream[3] = {nullptr, nullptr, nullptr};
+    cudaEvent_t fork_ev = nullptr, join_ev[3] = {nullptr, nullptr, nullptr};
     // tcgen05 conv path
     void *encode_tiled = nullptr;       // cuTensorMapEncodeTiled
     void *encode_im2col = nullptr;      // cuTensorMapEncodeIm2col
