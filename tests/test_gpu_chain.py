@@ -1,0 +1,149 @@
+"""A chained residual block through the C ABI -- conv, batch norm, ReLU, shortcut, residual add, and the whole backward pass
+down to the weight gradients -- against the same composition of the oracle's functions. Every tensor the CUDA path stores
+in bf16 is rounded to bf16 at the same place on the oracle side (a storage conversion, not arithmetic)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_09290_b200 import binding as B
+from paper_1901_09290_b200 import workloads as W
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+
+def _r(a):
+    return oracle.round_bf16(np.asarray(a, np.float32)).astype(np.float64)
+
+
+def _dev(a, ld):
+    return Hh.to_dev_padded(torch.from_numpy(np.asarray(a, np.float32)), ld)
+
+
+def _rel(got, ref):
+    return np.linalg.norm((got - ref).ravel()) / max(np.linalg.norm(ref.ravel()), 1e-300)
+
+
+class _Conv:
+    def __init__(self, N, H, C, K, R, seed):
+        self.N, self.H, self.C, self.K, self.R, self.pad = N, H, C, K, R, R // 2
+        self.w = W.bf16_round(W.gen_weight(K, R, R, C, seed)).numpy()
+        self.d = B.make_conv_desc(N, H, H, C, K, R, R, 1, self.pad, W.pad8(C), W.pad8(K), W.pad8(C))
+        self.wd = _dev(self.w, W.pad8(C))
+
+    def ws(self, which):
+        return Hh.conv_ws(self.d, which)
+
+
+class _Bn:
+    def __init__(self, N, H, C, relu, seed):
+        g = torch.Generator().manual_seed(seed)
+        self.gamma = (torch.rand(C, generator=g) + 0.5).numpy().astype(np.float64)
+        self.beta = (torch.rand(C, generator=g) - 0.5).numpy().astype(np.float64)
+        self.C, self.relu = C, relu
+        self.d = B.make_bn_desc(N, H, H, C, W.pad8(C), 1e-5, 0.1, relu)
+        self.gd, self.bd = torch.from_numpy(self.gamma).float().cuda(), torch.from_numpy(self.beta).float().cuda()
+        self.sm, self.si = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
+        self.dg, self.db = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
+        self.ws = torch.empty(max(16, B.pt_bn_workspace_bytes(Hh.ctx(), self.d)), dtype=torch.uint8, device="cuda")
+
+
+def test_chained_bottleneck_block_forward_and_backward():
+    c = Hh.ctx()
+    N, H = 4, 12
+    C0, C1, C2, C3 = 27, 19, 13, 44                       # ragged counts, as after pruning
+    seed = W.BASE_SEED + 4100
+    x0 = _r(W.gen_act(N, H, H, C0, seed).numpy())
+    G = _r(W.gen_dy(N, H, H, C3, seed + 1).numpy() * 64)
+    c1, c2, c3, ds = _Conv(N, H, C0, C1, 1, seed + 2), _Conv(N, H, C1, C2, 3, seed + 3), _Conv(N, H, C2, C3, 1, seed + 4), _Conv(N, H, C0, C3, 1, seed + 5)
+    b1, b2, b3, bs = _Bn(N, H, C1, True, seed + 6), _Bn(N, H, C2, True, seed + 7), _Bn(N, H, C3, True, seed + 8), _Bn(N, H, C3, False, seed + 9)
+
+    # ---------------- oracle: the block written out, bf16 storage rounding where the CUDA path stores bf16
+    def o_conv(cv, x):
+        return _r(oracle.conv_fwd(x.astype(np.float32), cv.w, 1, cv.pad))
+
+    def o_bn(bn, y, res=None):
+        a, mean, invstd, _ = oracle.bn_relu_fwd(y, bn.gamma, bn.beta, 1e-5, res, bn.relu)
+        return _r(a), mean.astype(np.float32).astype(np.float64), invstd.astype(np.float32).astype(np.float64)
+
+    y1 = o_conv(c1, x0); a1, m1, i1 = o_bn(b1, y1)
+    y2 = o_conv(c2, a1); a2, m2, i2 = o_bn(b2, y2)
+    y3 = o_conv(c3, a2)
+    ys = o_conv(ds, x0); r, ms, is_ = o_bn(bs, ys)
+    out, m3, i3 = o_bn(b3, y3, r)
+
+    def o_bn_bwd(bn, y, a, da, mean, invstd):
+        dx, dres, dg, db = oracle.bn_relu_bwd(y, a, da, bn.gamma, mean, invstd, bn.relu)
+        return _r(dx), _r(dres), dg, db
+
+    dy3, dr, dg3, db3 = o_bn_bwd(b3, y3, out, G, m3, i3)
+    dys, _, dgs, dbs = o_bn_bwd(bs, ys, r, dr, ms, is_)
+    dw3 = oracle.conv_wgrad(a2.astype(np.float32), dy3.astype(np.float32), 1, 1, 1, 0)
+    dws = oracle.conv_wgrad(x0.astype(np.float32), dys.astype(np.float32), 1, 1, 1, 0)
+    da2 = _r(oracle.conv_dgrad(dy3.astype(np.float32), c3.w, H, H, 1, 0))
+    dy2, _, dg2, db2 = o_bn_bwd(b2, y2, a2, da2, m2, i2)
+    dw2 = oracle.conv_wgrad(a1.astype(np.float32), dy2.astype(np.float32), 3, 3, 1, 1)
+    da1 = _r(oracle.conv_dgrad(dy2.astype(np.float32), c2.w, H, H, 1, 1))
+    dy1, _, dg1, db1 = o_bn_bwd(b1, y1, a1, da1, m1, i1)
+    dw1 = oracle.conv_wgrad(x0.astype(np.float32), dy1.astype(np.float32), 1, 1, 1, 0)
+
+    # ---------------- the same block through the C ABI
+    def buf(C):
+        return torch.zeros((N, H, H, W.pad8(C)), dtype=torch.bfloat16, device="cuda")
+
+    def g_conv(cv, x):
+        y = buf(cv.K)
+        B.pt_conv_fwd(c, cv.d, x, cv.wd, y, cv.ws(B.PT_CONV_FWD))
+        return y
+
+    def g_bn(bn, y, res=None):
+        a = buf(bn.C)
+        B.pt_bn_relu_fwd(c, bn.d, y, res, bn.gd, bn.bd, None, None, bn.sm, bn.si, a, bn.ws)
+        return a
+
+    x0d = _dev(x0, W.pad8(C0))
+    gy1 = g_conv(c1, x0d); ga1 = g_bn(b1, gy1)
+    gy2 = g_conv(c2, ga1); ga2 = g_bn(b2, gy2)
+    gy3 = g_conv(c3, ga2)
+    gys = g_conv(ds, x0d); gr = g_bn(bs, gys)
+    gout = g_bn(b3, gy3, gr)
+
+    def g_bn_bwd(bn, y, a, da, want_res):
+        dx, dres = buf(bn.C), (buf(bn.C) if want_res else None)
+        B.pt_bn_relu_bwd(c, bn.d, y, a, da, bn.gd, bn.sm, bn.si, dx, dres, bn.dg, bn.db, bn.ws)
+        return dx, dres
+
+    def g_wgrad(cv, x, dy):
+        dw = torch.empty((cv.K, cv.R, cv.R, cv.C), dtype=torch.float32, device="cuda")
+        B.pt_conv_wgrad(c, cv.d, x, dy, dw, cv.ws(B.PT_CONV_WGRAD))
+        return dw
+
+    def g_dgrad(cv, dy):
+        dx = buf(cv.C)
+        B.pt_conv_dgrad(c, cv.d, dy, cv.wd, dx, cv.ws(B.PT_CONV_DGRAD))
+        return dx
+
+    Gd = _dev(G, W.pad8(C3))
+    gdy3, gdr = g_bn_bwd(b3, gy3, gout, Gd, True)
+    gdys, _ = g_bn_bwd(bs, gys, gr, gdr, False)
+    gdw3, gdws = g_wgrad(c3, ga2, gdy3), g_wgrad(ds, x0d, gdys)
+    gda2 = g_dgrad(c3, gdy3)
+    gdy2, _ = g_bn_bwd(b2, gy2, ga2, gda2, False)
+    gdw2 = g_wgrad(c2, ga1, gdy2)
+    gda1 = g_dgrad(c2, gdy2)
+    gdy1, _ = g_bn_bwd(b1, gy1, ga1, gda1, False)
+    gdw1 = g_wgrad(c1, x0d, gdy1)
+    torch.cuda.synchronize()
+    c.poll()
+
+    # ---------------- compare. Rounding differences compound along the chain and may flip a ReLU decision at isolated
+    # near-zero elements, so the bound is on relative Frobenius errors: tight at the front, looser at the far end.
+    f = lambda t, C: t.float().cpu().numpy()[..., :C].astype(np.float64)
+    assert _rel(f(gout, C3), out) < 5e-3
+    assert _rel(f(gdy3, C3), dy3) < 1e-2 and _rel(f(gdr, C3), dr) < 1e-2
+    for got, ref, nm in ((gdw3, dw3, "c3"), (gdws, dws, "ds"), (gdw2, dw2, "c2"), (gdw1, dw1, "c1")):
+        assert _rel(got.cpu().numpy().astype(np.float64), ref) < 2e-2, nm
+    for bn, dg, db, nm in ((b3, dg3, db3, "bn3"), (bs, dgs, dbs, "bn_ds"), (b2, dg2, db2, "bn2"), (b1, dg1, db1, "bn1")):
+        assert _rel(bn.dg.cpu().numpy().astype(np.float64), dg) < 2e-2, nm
+        assert _rel(bn.db.cpu().numpy().astype(np.float64), db) < 2e-2, nm
