@@ -840,6 +840,18 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
             if (is_dy) my_bytes = second ? a_bytes : 8192u;
             else my_bytes = (uint32_t)((n_x - xp + 3) / 4) * 8192u;
             int q = pix_beg % p.Qd, t = pix_beg / p.Qd, pp = t % p.Pd, n = t / p.Pd;   // first pixel of the stage
+            // a stage advances 64 pixels = dn images + dp rows + dq columns: carried without divisions in the loop
+            const int dn = 64 / (p.Pd * p.Qd), rem64 = 64 - dn * p.Pd * p.Qd, dp = rem64 / p.Qd, dq = rem64 - dp * p.Qd;
+            // this warp's x boxes (at most two per stage: tpc * BN/64 <= 8 boxes over four warps): tap and channel block of each
+            int n_mine = 0, box_dst[2] = {0, 0}, box_c[2] = {0, 0};
+            uint16_t box_sw[2] = {0, 0}, box_sh[2] = {0, 0};
+            if (!is_dy)
+                for (int j = xp; j < n_x && n_mine < 2; j += 4, ++n_mine) {
+                    const int tt = j / (int)nb_b, nb = j - tt * (int)nb_b;
+                    const int r = (tap0 + tt) / p.S;
+                    box_dst[n_mine] = j * 8192; box_c[n_mine] = c0 + nb * 64;
+                    box_sh[n_mine] = (uint16_t)r; box_sw[n_mine] = (uint16_t)((tap0 + tt) - r * p.S);
+                }
             int s = 0, ph = 0, issued = 0;
             for (int it = 0; it < iters; ++it) {
                 if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 4)) break;
@@ -851,14 +863,12 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                     tma_load_2d(a_dst, &tmDy, bar, k0, pix);
                     if (second) tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
                 } else {
-                    for (int j = xp; j < n_x; j += 4) {
-                        const int tt = j / (int)nb_b, nb = j - tt * (int)nb_b;
-                        const int r = (tap0 + tt) / p.S, sft = (tap0 + tt) - r * p.S;
-                        tma_load_im2col_4d(b_dst + (uint32_t)j * 8192u, &tmX, bar, c0 + nb * 64, q * p.stride + p.lo_w,
-                                           pp * p.stride + p.lo_h, n, (uint16_t)sft, (uint16_t)r);
-                    }
-                    q += 64;                                          // the next stage starts 64 pixels further on
-                    while (q >= p.Qd) { q -= p.Qd; if (++pp == p.Pd) { pp = 0; ++n; } }
+                    const int w = q * p.stride + p.lo_w, h = pp * p.stride + p.lo_h;
+                    tma_load_im2col_4d(b_dst + (uint32_t)box_dst[0], &tmX, bar, box_c[0], w, h, n, box_sw[0], box_sh[0]);
+                    if (n_mine > 1) tma_load_im2col_4d(b_dst + (uint32_t)box_dst[1], &tmX, bar, box_c[1], w, h, n, box_sw[1], box_sh[1]);
+                    q += dq; pp += dp; n += dn;                       // the next stage starts 64 pixels further on
+                    if (q >= p.Qd) { q -= p.Qd; ++pp; }
+                    if (pp >= p.Pd) { pp -= p.Pd; ++n; }
                 }
                 issued = it + 1;
                 if (++s == p.stages) { s = 0; ph ^= 1; }
