@@ -10,6 +10,10 @@
 //   stem_* kernels     space-to-depth layout kernels of the few-channel stride-2 stem.
 // Ragged channel counts are handled by the TMA unit (true extents in the tensor maps: zero-fill on load, clipping on
 // store) and by skipping the 16-wide k-steps past the last valid channel.
+// Issue is spread over warps in all three kernels: one thread spends ~200 cycles per TMA instruction and 50-100 per
+// tcgen05.mma, more than a narrow MMA takes to run, so operands are loaded by several producer warps and, where
+// independent accumulators exist, MMAs are issued by up to four warps, each with its own ring and TMEM buffers.
+// The kernels are launched with programmatic stream serialization (griddepcontrol.wait after the prologue).
 // Every wait is bounded; on expiry the CTA records PT_DEV_TIMEOUT in the status word, drains its copies and exits.
 #include "pt_internal.h"
 #include "pt_sm100_ptx.cuh"
@@ -92,7 +96,6 @@ struct __align__(8) PCtl {
 };
 
 constexpr uint32_t kSlabs = 2;                          // staging slabs per epilogue warp (TMA stores in flight)
-constexpr int kMaxEpiGroups = 3;                        // epilogue warp groups (4 warps each) working on different 64-channel chunks
 
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... The TMA ring runs continuously across
 // tiles. The accumulator has G = 2 or 3 buffers in TMEM and buffer b has its own group of four epilogue warps, so the
@@ -970,7 +973,7 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                 if (warp == 2) WTRACE(4);
                 named_barrier(1, 256);
                 // ---- (2) every split CTA of this tile is resident (the grid is at most one CTA per SM): wait for all of them
-                unsigned int *arrived = p.sync + 2 * blockIdx.x, *reduced = arrived + 1;
+                unsigned int *arrived = p.sync + 2 * blockIdx.x;
                 if (gtid == 0) {
                     atomicAdd(arrived, 1u);
                     const uint64_t t0 = globaltimer_ns();
@@ -1299,7 +1302,6 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     if (per_cta < p.epi_groups) p.epi_groups = per_cta < 2 ? 2 : per_cta;
     // Small weights (one channel tile, all taps x chunks within 64 KB) stay resident: the ring then carries A tiles only and
     // holds more of them, which is what an activation-bound layer needs to cover the memory latency.
-    const size_t staging = (size_t)p.epi_groups * 4 * kSlabs * 4096;
     const size_t w_all = (size_t)p.taps * p.k_chunks * b_bytes;
     p.resident = (p.n_tiles == 1 && w_all <= 64 * 1024 && per_cta >= 2) ? 1 : 0;
     p.n_issuers = 1; p.acc_per = 1;
