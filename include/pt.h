@@ -197,6 +197,17 @@ pt_status pt_cross_entropy(pt_ctx *ctx, const float *logits, const int32_t *labe
  * pt_sgd_hparams.lambda_ for the steps that follow. */
 pt_status pt_set_coeff(pt_ctx *ctx, const double *loss, const double *reg_sum, float ratio, float *lambda_out, void *stream);
 
+/* The same step in two calls, for callers that want the group norms out of the way early: the norms depend on the weights
+ * only (Algorithm 1 evaluates GroupLassoReg on W_i, the weights the forward pass used), not on the gradients, so
+ * pt_group_lasso_norms may run on another stream while the backward pass is still producing g. It fills sumsq_out /
+ * sumsq_in, reg_sum_out (optional) and the inverse norms kept in ws; pt_group_lasso_sgd_apply then performs the update
+ * from them. Contract: same layers array, same ws, and the weights unchanged between the two calls; the pair computes
+ * bit for bit what pt_group_lasso_sgd_step computes. (g may be NULL in the layers given to pt_group_lasso_norms.) */
+pt_status pt_group_lasso_norms(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers, double *reg_sum_out,
+                               void *ws, size_t ws_bytes, void *stream);
+pt_status pt_group_lasso_sgd_apply(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers,
+                                   const pt_sgd_hparams *hp /*host*/, void *ws, size_t ws_bytes, void *stream);
+
 /* zero_out[k] = (max_{rs,c} |w| < threshold), zero_in[c] = (max_{k,rs} |w| < threshold), strict <, in fp32
  * (Sec. 4.1: threshold 1e-4; Sec. 4.2 / Fig. 4: the absolute maximum of a channel's parameters). A NaN keeps
  * its groups. If zero_in_place != 0 the weights, momentum and shadow of every detected group are set to 0

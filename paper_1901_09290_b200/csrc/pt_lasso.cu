@@ -390,15 +390,16 @@ extern "C" size_t pt_group_lasso_workspace_bytes(const pt_ctx *c, const pt_layer
     return t.ws.total;
 }
 
-extern "C" pt_status pt_group_lasso_sgd_step(pt_ctx *c, const pt_layer *layers, int32_t n, const pt_sgd_hparams *hp,
-                                             double *reg_sum_out, void *ws, size_t ws_bytes, void *stream)
+// phases: 1 = group norms (partial sums, finish, regulariser value), 2 = parameter update from the norms in the workspace
+static pt_status lasso_phases(pt_ctx *c, const pt_layer *layers, int32_t n, const pt_sgd_hparams *hp, double *reg_sum_out, void *ws,
+                              size_t ws_bytes, void *stream, int phases)
 {
-    if (!c || !hp) return PT_ERR_INVALID_ARG;
+    if (!c || ((phases & 2) && !hp)) return PT_ERR_INVALID_ARG;
     Tables t;
     pt_status s = build_tables(layers, n, &t);
     if (s != PT_OK) return s;
     for (int i = 0; i < n; ++i)
-        if (!layers[i].g || !layers[i].sumsq_out || !layers[i].sumsq_in) return PT_ERR_INVALID_ARG;
+        if (((phases & 2) && !layers[i].g) || !layers[i].sumsq_out || !layers[i].sumsq_in) return PT_ERR_INVALID_ARG;
     if (!ws || ws_bytes < t.ws.total || ((uintptr_t)ws & 255)) return PT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     const LayerDev *dl; const Chunk *dc; const FinishJob *dj;
@@ -409,15 +410,37 @@ extern "C" pt_status pt_group_lasso_sgd_step(pt_ctx *c, const pt_layer *layers, 
     float *inv_out = (float *)(b + t.ws.inv_out), *inv_in = (float *)(b + t.ws.inv_in);
     double *layer_reg = (double *)(b + t.ws.layer_reg);
     const unsigned nch = (unsigned)t.chunks.size();
-    norms_partial_kernel<<<nch, kThreads, 0, st>>>(dl, dc, linesum, colpart);
-    const int nj = (int)t.jobs.size();
-    norms_finish_kernel<<<nj, kThreads, 0, st>>>(dl, dj, linesum, colpart, inv_out, inv_in, layer_reg);
-    c->launches += 2;
-    if (reg_sum_out) { reg_total_kernel<<<1, 32, 0, st>>>(layer_reg, nj, reg_sum_out); c->launches += 1; }
-    update_kernel<<<nch, kThreads, 0, st>>>(dl, dc, inv_out, inv_in, *hp);
-    c->launches += 1;
+    if (phases & 1) {
+        norms_partial_kernel<<<nch, kThreads, 0, st>>>(dl, dc, linesum, colpart);
+        const int nj = (int)t.jobs.size();
+        norms_finish_kernel<<<nj, kThreads, 0, st>>>(dl, dj, linesum, colpart, inv_out, inv_in, layer_reg);
+        c->launches += 2;
+        if (reg_sum_out) { reg_total_kernel<<<1, 32, 0, st>>>(layer_reg, nj, reg_sum_out); c->launches += 1; }
+    }
+    if (phases & 2) {
+        update_kernel<<<nch, kThreads, 0, st>>>(dl, dc, inv_out, inv_in, *hp);
+        c->launches += 1;
+    }
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
+}
+
+extern "C" pt_status pt_group_lasso_sgd_step(pt_ctx *c, const pt_layer *layers, int32_t n, const pt_sgd_hparams *hp,
+                                             double *reg_sum_out, void *ws, size_t ws_bytes, void *stream)
+{
+    return lasso_phases(c, layers, n, hp, reg_sum_out, ws, ws_bytes, stream, 3);
+}
+
+extern "C" pt_status pt_group_lasso_norms(pt_ctx *c, const pt_layer *layers, int32_t n, double *reg_sum_out, void *ws,
+                                          size_t ws_bytes, void *stream)
+{
+    return lasso_phases(c, layers, n, nullptr, reg_sum_out, ws, ws_bytes, stream, 1);
+}
+
+extern "C" pt_status pt_group_lasso_sgd_apply(pt_ctx *c, const pt_layer *layers, int32_t n, const pt_sgd_hparams *hp, void *ws,
+                                              size_t ws_bytes, void *stream)
+{
+    return lasso_phases(c, layers, n, hp, nullptr, ws, ws_bytes, stream, 2);
 }
 
 extern "C" pt_status pt_find_zero_groups(pt_ctx *c, const pt_layer *layers, int32_t n, float threshold,

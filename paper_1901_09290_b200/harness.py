@@ -174,6 +174,12 @@ class TrainStep:
     def lasso(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
         B.pt_group_lasso_sgd_step(self.ctx, self.mp.arr, lam, lr, mu, 0.0, self.mp.reg, self.mp.ws, stream)
 
+    def lasso_norms(self, stream=None):
+        B.pt_group_lasso_norms(self.ctx, self.mp.arr, self.mp.reg, self.mp.ws, stream)
+
+    def lasso_apply(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
+        B.pt_group_lasso_sgd_apply(self.ctx, self.mp.arr, lam, lr, mu, 0.0, self.mp.ws, stream)
+
     def train(self, stream=None):
         n = len(self.net.layers)
         for li in range(n):
@@ -208,6 +214,12 @@ class TrainStep:
         fork_at = {f: d for f, d in br}          # before layer f: start shortcut d on the aux stream
         ds_set = {d for _, d in br}
         forked = set()                           # streams that joined this launch sequence and must be joined back
+        if lasso and fwd:
+            # the group norms need the weights only (GroupLassoReg(W_i) of Algorithm 1): they run beside the forward pass
+            nstream = ws[-1]
+            nstream.wait_stream(main)
+            forked.add(nstream)
+            self.lasso_norms(nstream)
         for li in range(n if fwd else 0):
             if li in fork_at:
                 aux.wait_stream(main)
@@ -247,7 +259,10 @@ class TrainStep:
         for w in forked:
             main.wait_stream(w)
         if lasso:
-            self.lasso(main)
+            if fwd:
+                self.lasso_apply(main)
+            else:
+                self.lasso(main)
 
     def capture_pass(self, kind: str):
         """A CUDA graph of one pass kind ("fwd", "dgrad", "wgrad") with the stream assignment it has inside the step."""

@@ -76,6 +76,26 @@ def test_step_is_run_to_run_identical_and_table_cache_reuploads():
         assert torch.equal(x, y)
 
 
+def test_step_in_two_calls_equals_the_single_call():
+    """pt_group_lasso_norms (on another stream, before the gradients exist) + pt_group_lasso_sgd_apply == pt_group_lasso_sgd_step."""
+    net = W.resnet32()
+    kept = W.choose_kept(net, W.random_keep(net, W.BASE_SEED + 6), W.BASE_SEED + 6)
+    model = W.gen_model(net, W.BASE_SEED + 6, kept=kept, decoys=1)
+    one = _check_step(model, 2e-4, 0.1, 0.9, 1e-4)          # single call, checked against the oracle
+    dm = DevModel(model)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    B.pt_group_lasso_norms(Hh.ctx(), dm.arr, dm.reg, dm.ws, side)
+    torch.cuda.current_stream().wait_stream(side)
+    B.pt_group_lasso_sgd_apply(Hh.ctx(), dm.arr, 2e-4, 0.1, 0.9, 1e-4, dm.ws)
+    torch.cuda.synchronize()
+    Hh.ctx().poll()
+    for li in range(len(model.net.layers)):
+        assert torch.equal(dm.w[li], one.w[li]) and torch.equal(dm.v[li], one.v[li]) and torch.equal(dm.wb[li].view(torch.int16), one.wb[li].view(torch.int16))
+        assert torch.equal(dm.sq_out[li], one.sq_out[li]) and torch.equal(dm.sq_in[li], one.sq_in[li])
+    assert dm.reg.item() == one.reg.item()
+
+
 def test_step_resnet50_all_layers():
     net = W.resnet50()
     model = W.gen_model(net, W.BASE_SEED + 4)
