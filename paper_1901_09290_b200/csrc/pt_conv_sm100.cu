@@ -441,7 +441,10 @@ struct HaloP {
 };
 
 constexpr int kHaloMaxIssuers = 4;
-#ifdef PT_HALO_TRACE
+// Device-side timeline for tuning: a build with -DPT_DEVICE_TRACE makes CTA 0 stamp %globaltimer at the hand-over points of
+// each role (producer issue, accumulator free, operands landed, MMAs committed, epilogue start, store issued) and exports
+// pt_debug_halo_trace / pt_debug_wgrad_trace to read the stamps back. The normal build compiles the macros away.
+#ifdef PT_DEVICE_TRACE
 __device__ unsigned long long g_halo_trace[8][64];
 #define HTRACE(role, idx) do { if (blockIdx.x == 0 && (idx) < 64 && (threadIdx.x & 31) == 0) g_halo_trace[role][idx] = globaltimer_ns(); } while (0)
 #else
@@ -768,7 +771,7 @@ struct WgradP {
     unsigned int *status;
 };
 
-#ifdef PT_HALO_TRACE
+#ifdef PT_DEVICE_TRACE
 __device__ unsigned long long g_wg_trace[8][64];
 #define WTRACE(i) do { if (blockIdx.x == 0 && blockIdx.y < 64 && (threadIdx.x & 31) == 0) g_wg_trace[i][blockIdx.y] = globaltimer_ns(); } while (0)
 #else
@@ -1868,7 +1871,7 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
     return PT_OK;
 }
 
-#ifdef PT_HALO_TRACE
+#ifdef PT_DEVICE_TRACE
 extern "C" int pt_debug_wgrad_trace(unsigned long long *host_out)
 {
     return (int)cudaMemcpyFromSymbol(host_out, g_wg_trace, sizeof(unsigned long long) * 8 * 64);
