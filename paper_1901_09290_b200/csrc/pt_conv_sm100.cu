@@ -1129,8 +1129,10 @@ StemPlan stem_plan(const pt_conv_desc *d)
     return s;
 }
 
-__global__ void stem_s2d_x_kernel(const __nv_bfloat16 *__restrict__ x, __nv_bfloat16 *__restrict__ xs, int N, int H, int W, int C,
-                                  int Hs, int Ws, int Wp, int pl)
+// CT = channel count as a compile-time constant (1..4): the 16 output lanes are then plain registers
+template <int CT>
+__global__ void __launch_bounds__(256) stem_s2d_x_kernel_t(const __nv_bfloat16 *__restrict__ x, __nv_bfloat16 *__restrict__ xs, int N, int H,
+                                                           int W, int Hs, int Ws, int Wp, int pl)
 {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t total = (size_t)N * Hs * Wp;
@@ -1138,22 +1140,36 @@ __global__ void stem_s2d_x_kernel(const __nv_bfloat16 *__restrict__ x, __nv_bflo
     const int jp = (int)(idx % Wp);
     const size_t t = idx / Wp;
     const int i = (int)(t % Hs), n = (int)(t / Hs);
-    __align__(16) __nv_bfloat16 o[16];
+    __align__(16) unsigned short o[16];
 #pragma unroll
-    for (int e = 0; e < 16; ++e) o[e] = __float2bfloat16_rn(0.f);
+    for (int e = 0; e < 16; ++e) o[e] = 0;
     const int j = jp - pl;
     if (j >= 0 && j < Ws) {
+        uint4 px[4];
+#pragma unroll
+        for (int ab = 0; ab < 4; ++ab)          // the four loads go out together
+            px[ab] = __ldg(reinterpret_cast<const uint4 *>(x + ((size_t)(n * H + 2 * i + (ab >> 1)) * W + 2 * j + (ab & 1)) * 8));
 #pragma unroll
         for (int ab = 0; ab < 4; ++ab) {
-            const int a = ab >> 1, b = ab & 1;
-            const uint4 px = *reinterpret_cast<const uint4 *>(x + ((size_t)(n * H + 2 * i + a) * W + 2 * j + b) * 8);
-            const __nv_bfloat16 *pe = reinterpret_cast<const __nv_bfloat16 *>(&px);
-            for (int c = 0; c < C; ++c) o[ab * C + c] = pe[c];
+            const unsigned short *pe = reinterpret_cast<const unsigned short *>(&px[ab]);
+#pragma unroll
+            for (int c = 0; c < CT; ++c) o[ab * CT + c] = pe[c];
         }
     }
     uint4 *dst = reinterpret_cast<uint4 *>(xs + idx * 16);
     dst[0] = *reinterpret_cast<uint4 *>(&o[0]);
     dst[1] = *reinterpret_cast<uint4 *>(&o[8]);
+}
+
+void stem_s2d_x_kernel_launch(unsigned blocks, cudaStream_t st, const __nv_bfloat16 *x, __nv_bfloat16 *xs, int N, int H, int W, int C,
+                              int Hs, int Ws, int Wp, int pl)
+{
+    switch (C) {
+    case 1: stem_s2d_x_kernel_t<1><<<blocks, 256, 0, st>>>(x, xs, N, H, W, Hs, Ws, Wp, pl); break;
+    case 2: stem_s2d_x_kernel_t<2><<<blocks, 256, 0, st>>>(x, xs, N, H, W, Hs, Ws, Wp, pl); break;
+    case 3: stem_s2d_x_kernel_t<3><<<blocks, 256, 0, st>>>(x, xs, N, H, W, Hs, Ws, Wp, pl); break;
+    default: stem_s2d_x_kernel_t<4><<<blocks, 256, 0, st>>>(x, xs, N, H, W, Hs, Ws, Wp, pl); break;
+    }
 }
 
 // w2[k][u][v*16 + (a*2+b)*C + c] = w[k][2u+a-off][2v+b-off][c]  (0 where the tap falls outside the filter)
@@ -1706,8 +1722,8 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
             char *part = wsb + sp.xs_bytes + pt_align_up(sp.w2_elems * 4, 1024);
             const pt_conv_desc v = stem_virtual_desc(d, sp);
             const size_t tot = (size_t)d->N * sp.Hs * sp.Wp;
-            stem_s2d_x_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)a, xs, d->N, d->H, d->W, d->C, sp.Hs,
-                                                                          sp.Ws, sp.Wp, sp.pl);
+            stem_s2d_x_kernel_launch((unsigned)((tot + 255) / 256), st, (const __nv_bfloat16 *)a, xs, d->N, d->H, d->W, d->C, sp.Hs, sp.Ws,
+                                     sp.Wp, sp.pl);
             c->launches += 1;
             CUtensorMap tmX;
             const int up_h = (sp.P - 1) - sp.pl - (sp.Hs - 1);
@@ -1735,8 +1751,8 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         char *wsb = (char *)ws;
         __nv_bfloat16 *xs = (__nv_bfloat16 *)wsb, *w2 = (__nv_bfloat16 *)(wsb + sp.xs_bytes);
         const size_t tot = (size_t)d->N * sp.Hs * sp.Wp;
-        stem_s2d_x_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)a, xs, d->N, d->H, d->W, d->C, sp.Hs, sp.Ws,
-                                                                      sp.Wp, sp.pl);
+        stem_s2d_x_kernel_launch((unsigned)((tot + 255) / 256), st, (const __nv_bfloat16 *)a, xs, d->N, d->H, d->W, d->C, sp.Hs, sp.Ws, sp.Wp,
+                                 sp.pl);
         stem_s2d_w_kernel<<<(unsigned)((sp.w2_elems + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)b, w2, d->K, d->R, d->S, d->C, d->ldw,
                                                                               sp.U, sp.V, sp.off);
         c->launches += 2;
