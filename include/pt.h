@@ -176,6 +176,26 @@ pt_status pt_bn_relu_bwd(pt_ctx *ctx, const pt_bn_desc *d, const void *x, const 
                          float *dbeta, void *ws, size_t ws_bytes, void *stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Dynamic mini-batch adjustment (Sec. 4.3; Algorithm 1, "UpdateMiniBatch(system_memory, Net)"): after every reconfiguration
+ * the memory one training iteration needs is re-evaluated for the smaller network, the mini-batch grows in steps of a
+ * granularity (the paper uses 32 samples per GPU) as far as the device memory allows, and the learning rate grows by the
+ * same ratio. Host-side arithmetic only; no device is touched.
+ * The memory model is this library's own buffers (the paper gives none): per parameter fp32 weight, gradient and momentum
+ * plus the bf16 shadow (14 bytes, pitch padding included for the shadow); per sample and per convolution the bf16 input
+ * and output activations and their two gradients, at the channel pitch the tensors are stored with (multiple of 8).
+ * ------------------------------------------------------------------------------------------ */
+typedef struct { int32_t H, W, C, K, R, S, stride, pad; } pt_layer_shape;   /* CURRENT (pruned) sizes of one convolution */
+
+/* Bytes one iteration needs at mini-batch `batch` (0 if an argument is invalid). */
+size_t pt_training_memory_bytes(const pt_layer_shape *layers /*host*/, int32_t n_layers, int32_t batch);
+
+/* new_batch = cur_batch + granularity * g with the largest g >= 0 whose memory fits capacity_bytes (the mini-batch never
+ * shrinks: if even cur_batch does not fit, it is returned unchanged); new_lr = cur_lr * new_batch / cur_batch.
+ * PT_ERR_INVALID_ARG for cur_batch < 1, granularity < 1, bad shapes or null pointers. */
+pt_status pt_update_mini_batch(const pt_layer_shape *layers /*host*/, int32_t n_layers, size_t capacity_bytes, int32_t cur_batch,
+                               float cur_lr, int32_t granularity, int32_t *new_batch /*host*/, float *new_lr /*host*/);
+
+/* ------------------------------------------------------------------------------------------
  * Penalty coefficient set-up (Sec. 4.1, "Regularization Penalty Coefficient Setup", Eq. 3): lambda is chosen once, at the
  * first training iteration, so that the group-lasso term is a given share (the paper uses 20-25 %) of the total loss:
  *     ratio = lambda * R / (loss + lambda * R),  R = sum over groups of ||W_g||   =>   lambda = ratio * loss / ((1 - ratio) * R)

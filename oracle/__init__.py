@@ -270,6 +270,31 @@ def conv_flops(N, H, W, C, K, R, S, stride, pad) -> int:
     return 2 * N * P * Q * K * C * R * S
 
 
+# --------------------------------------------------------------------------- dynamic mini-batch adjustment (Sec. 4.3)
+def training_memory_bytes(shapes, batch: int) -> int:
+    """Memory one training iteration needs (Sec. 4.3: the "memory context volume of a training iteration"), as the sum
+    over the convolutions (H, W, C, K, R, S, stride, pad) of: the parameters' fp32 weight, gradient and momentum and their
+    bf16 shadow; and, per sample, the layer's input and output in bf16 together with the gradients of both. Channel
+    pitches are the channel counts rounded up to 8, as the tensors are stored."""
+    pad8 = lambda c: -(-c // 8) * 8
+    tot = 0
+    for (H, W, C, K, R, S, stride, pad) in shapes:
+        P, Q = out_dim(H, R, stride, pad), out_dim(W, S, stride, pad)
+        tot += K * R * S * C * (4 + 4 + 4) + K * R * S * pad8(C) * 2
+        tot += batch * 2 * 2 * (H * W * pad8(C) + P * Q * pad8(K))
+    return tot
+
+
+def update_mini_batch(shapes, capacity_bytes: int, cur_batch: int, cur_lr: float, granularity: int = 32):
+    """Algorithm 1, UpdateMiniBatch(system_memory, Net): the largest mini-batch cur_batch + g*granularity (g >= 0) whose
+    iteration still fits the device memory, found by stepping; the learning rate grows by the same ratio (Sec. 4.3)."""
+    nb = cur_batch
+    if training_memory_bytes(shapes, cur_batch) <= capacity_bytes:
+        while training_memory_bytes(shapes, nb + granularity) <= capacity_bytes:
+            nb += granularity
+    return nb, cur_lr * nb / cur_batch
+
+
 # --------------------------------------------------------------------------- feature normalisation (Sec. 2.1)
 def bn_relu_fwd(x, gamma, beta, eps: float = 1e-5, residual=None, relu: bool = True):
     """Training-mode batch normalisation of x [N][H][W][C] followed by the residual add and the ReLU of a ResNet block.

@@ -49,6 +49,10 @@ class pt_bn_desc(Structure):
                 ("eps", c_float), ("momentum", c_float), ("relu", c_int32)]
 
 
+class pt_layer_shape(Structure):
+    _fields_ = [(n, c_int32) for n in ("H", "W", "C", "K", "R", "S", "stride", "pad")]
+
+
 class pt_space(Structure):
     _fields_ = [("size", c_int32), ("fixed", c_uint8)]
 
@@ -83,6 +87,8 @@ EXPORTS = {
     "pt_bn_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_bn_desc)]),
     "pt_bn_relu_fwd": (c_int32, [c_void_p, POINTER(pt_bn_desc)] + [c_void_p] * 9 + [c_void_p, c_size_t, c_void_p]),
     "pt_bn_relu_bwd": (c_int32, [c_void_p, POINTER(pt_bn_desc)] + [c_void_p] * 10 + [c_void_p, c_size_t, c_void_p]),
+    "pt_training_memory_bytes": (c_size_t, [POINTER(pt_layer_shape), c_int32, c_int32]),
+    "pt_update_mini_batch": (c_int32, [POINTER(pt_layer_shape), c_int32, c_size_t, c_int32, c_float, c_int32, POINTER(c_int32), POINTER(c_float)]),
     "pt_cross_entropy_workspace_bytes": (c_size_t, [c_int32]),
     "pt_cross_entropy": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_set_coeff": (c_int32, [c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]),
@@ -258,6 +264,25 @@ def pt_bn_relu_bwd(ctx, d, x, y, dy, gamma, save_mean, save_invstd, dx, dresidua
     p, n = _ws(ws)
     _check(lib().pt_bn_relu_bwd(ctx.handle, byref(d), _ptr(x), _ptr(y), _ptr(dy), _ptr(gamma), _ptr(save_mean), _ptr(save_invstd),
                                 _ptr(dx), _ptr(dresidual), _ptr(dgamma), _ptr(dbeta), p, n, _stream(stream)), "pt_bn_relu_bwd")
+
+
+def shape_array(shapes) -> "ctypes.Array":
+    """shapes: iterable of (H, W, C, K, R, S, stride, pad)."""
+    shapes = list(shapes)
+    return (pt_layer_shape * len(shapes))(*[pt_layer_shape(*[int(v) for v in t]) for t in shapes])
+
+
+def pt_training_memory_bytes(shapes, batch: int) -> int:
+    arr = shape_array(shapes)
+    return int(lib().pt_training_memory_bytes(arr, len(arr), batch))
+
+
+def pt_update_mini_batch(shapes, capacity_bytes: int, cur_batch: int, cur_lr: float, granularity: int = 32):
+    arr = shape_array(shapes)
+    nb, nl = c_int32(), c_float()
+    _check(lib().pt_update_mini_batch(arr, len(arr), capacity_bytes, cur_batch, cur_lr, granularity, byref(nb), byref(nl)),
+           "pt_update_mini_batch")
+    return nb.value, nl.value
 
 
 def pt_cross_entropy_workspace_bytes(n: int) -> int:

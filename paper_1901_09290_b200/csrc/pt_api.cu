@@ -201,3 +201,54 @@ extern "C" pt_status pt_conv_wgrad(pt_ctx *c, const pt_conv_desc *d, const void 
 {
     return conv_dispatch(c, d, PT_CONV_WGRAD, x, dy, dw, ws, ws_bytes, stream);
 }
+
+// ------------------------------------------------------------------ dynamic mini-batch adjustment (Sec. 4.3), host arithmetic
+static bool shape_ok(const pt_layer_shape &l)
+{
+    return l.H > 0 && l.W > 0 && l.C > 0 && l.K > 0 && l.R > 0 && l.S > 0 && l.stride > 0 && l.pad >= 0 &&
+           pt_out_dim(l.H, l.R, l.stride, l.pad) > 0 && pt_out_dim(l.W, l.S, l.stride, l.pad) > 0;
+}
+
+static void memory_terms(const pt_layer_shape *layers, int32_t n, size_t *fixed, size_t *per_sample)
+{
+    size_t f = 0, a = 0;
+    for (int i = 0; i < n; ++i) {
+        const pt_layer_shape &l = layers[i];
+        const size_t P = (size_t)pt_out_dim(l.H, l.R, l.stride, l.pad), Q = (size_t)pt_out_dim(l.W, l.S, l.stride, l.pad);
+        const size_t ldc = pt_align_up((size_t)l.C, 8), ldk = pt_align_up((size_t)l.K, 8);
+        f += (size_t)l.K * l.R * l.S * l.C * 12 + (size_t)l.K * l.R * l.S * ldc * 2;     // w, g, v fp32; bf16 shadow at its pitch
+        a += ((size_t)l.H * l.W * ldc + P * Q * ldk) * 2 * 2;                             // x, dx, y, dy in bf16
+    }
+    *fixed = f;
+    *per_sample = a;
+}
+
+extern "C" size_t pt_training_memory_bytes(const pt_layer_shape *layers, int32_t n, int32_t batch)
+{
+    if (!layers || n < 1 || batch < 1) return 0;
+    for (int i = 0; i < n; ++i)
+        if (!shape_ok(layers[i])) return 0;
+    size_t f, a;
+    memory_terms(layers, n, &f, &a);
+    return f + a * (size_t)batch;
+}
+
+extern "C" pt_status pt_update_mini_batch(const pt_layer_shape *layers, int32_t n, size_t capacity_bytes, int32_t cur_batch,
+                                          float cur_lr, int32_t granularity, int32_t *new_batch, float *new_lr)
+{
+    if (!layers || n < 1 || cur_batch < 1 || granularity < 1 || !new_batch || !new_lr) return PT_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i)
+        if (!shape_ok(layers[i])) return PT_ERR_INVALID_ARG;
+    size_t f, a;
+    memory_terms(layers, n, &f, &a);
+    int32_t nb = cur_batch;
+    const size_t now = f + a * (size_t)cur_batch;
+    if (now <= capacity_bytes) {
+        const size_t steps = (capacity_bytes - now) / (a * (size_t)granularity);
+        const size_t cap_steps = (size_t)(0x7fffffff - cur_batch) / (size_t)granularity;
+        nb = cur_batch + (int32_t)(steps < cap_steps ? steps : cap_steps) * granularity;
+    }
+    *new_batch = nb;
+    *new_lr = (float)((double)cur_lr * (double)nb / (double)cur_batch);
+    return PT_OK;
+}
