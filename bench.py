@@ -210,7 +210,12 @@ def run_ours(args):
     pk = peaks()
     ctx = B.Context(local)
     net, counts, kept, seed, name = workload(args)
-    ts = harness.TrainStep(ctx, net, counts, kept, args.batch, seed + 17 * rank, algo=args.algo, host_inputs=True)
+    # N > 1 default: independent replicas (no data-path collective). --data-parallel: every rank holds the same model (same
+    # seed; the synthetic batch is then the same too, which the timing does not depend on) and the weight gradients are
+    # averaged by one NCCL all-reduce before the update.
+    dp = world > 1 and args.data_parallel
+    ts = harness.TrainStep(ctx, net, counts, kept, args.batch, seed + (0 if dp else 17 * rank), algo=args.algo, host_inputs=True,
+                           world=world if dp else 1)
     flops = ts.conv_flops()
     tot_flops = sum(flops.values())
     stream = torch.cuda.current_stream()
@@ -374,7 +379,8 @@ def run_ours(args):
         "config": {"workload": name, "batch_per_gpu": args.batch, "image": 224, "conv_layers": nL,
                    "kept_params": ts.mp.n_params(), "dense_params": ts.md.n_params(),
                    "useful_conv_flops_per_step": tot_flops, "l2": "inputs larger than L2 (per-layer activations 20-400 MB, ~6 GB per step)",
-                   "parallelism": "independent data-parallel replicas, no collective" if world > 1 else "1 GPU",
+                   "parallelism": ("data parallel: one NCCL all-reduce (mean) of the weight gradients per step" if dp else
+                                   "independent data-parallel replicas, no collective") if world > 1 else "1 GPU",
                    "algo": args.algo,
                    "launch": "eager" if args.no_graph else ("CUDA graph replay after the reconfiguration's host sync; "
                                                             + ("1 stream" if args.one_stream else f"streams along the network's data dependencies: dgrad chain, projection shortcuts beside their blocks, wgrads round-robin on {ts.wgrad_streams} streams at <= {ts.wgrad_ctas} CTAs each"))},
@@ -431,6 +437,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--data-parallel", action="store_true",
+                    help="N > 1: average the weight gradients over the ranks with one NCCL all-reduce per step (default: replicas)")
     ap.add_argument("--keep", type=float, default=None, help="uniform keep ratio instead of the seeded per-space draw")
     ap.add_argument("--algo", type=int, default=0)
     ap.add_argument("--per-layer", default=None, help="write the per-layer table (JSON) here")

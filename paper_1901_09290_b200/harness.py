@@ -23,7 +23,15 @@ class DeviceModel:
         self.net = model.net
         self.w = [t.clone().cuda() for t in model.w]
         self.v = [t.clone().cuda() for t in model.v]
-        self.g = [t.clone().cuda() for t in model.g]
+        # the weight gradients of all layers are views of one flat buffer: a data-parallel run reduces them in one collective
+        al = lambda n: (n + 63) // 64 * 64                  # every view starts on a 256-byte boundary
+        self.g_flat = torch.zeros(sum(al(t.numel()) for t in model.g), dtype=torch.float32, device="cuda")
+        self.g, off = [], 0
+        for t in model.g:
+            v = self.g_flat[off:off + t.numel()].view(t.shape)
+            v.copy_(t)
+            self.g.append(v)
+            off += al(t.numel())
         self.bn = [[b.clone().cuda() for b in bb] for bb in model.bn]
         self.wb, self.sq_out, self.sq_in, self.z_out, self.z_in, self.layers = [], [], [], [], [], []
         for li, l in enumerate(self.net.layers):
@@ -64,6 +72,21 @@ def empty_model(net: W.Net, fill: float = 0.0) -> W.Model:
                    [[torch.full((l.K,), fill) for _ in range(4)] for l in net.layers])
 
 
+def allreduce_mean(flat: torch.Tensor, world: int):
+    """The one exchange of a data-parallel step (Sec. 2.2, data parallelism: the partial weight gradients of all GPUs are
+    reduced, then used to update the weights): the mean of the ranks' gradient buffers, in place, in one collective over
+    the flat buffer whose size shrinks as the model is pruned. NCCL averages inside the collective; gloo (CPU tests) sums
+    and the division follows."""
+    import torch.distributed as dist
+    if world <= 1:
+        return
+    if flat.is_cuda:
+        dist.all_reduce(flat, op=dist.ReduceOp.AVG)
+    else:
+        dist.all_reduce(flat, op=dist.ReduceOp.SUM)
+        flat.div_(world)
+
+
 class TrainStep:
     """The hot path on one GPU for one network: reconfiguration of a dense-shaped model with embedded zero
     groups into the pruned model, then the pruned model's conv training step (every layer's forward, then data and
@@ -75,8 +98,9 @@ class TrainStep:
 
     def __init__(self, ctx: B.Context, dense_net: W.Net, counts: Sequence[int], kept, N: int, seed: int,
                  algo: int = 0, host_inputs: bool = False, decoys: int = 2, device_rng: bool = True,
-                 wgrad_ctas: int = 74, wgrad_streams: int = 3):
+                 wgrad_ctas: int = 74, wgrad_streams: int = 3, world: int = 1):
         self.ctx, self.N, self.algo = ctx, N, algo
+        self.world = world          # > 1: data parallel, the weight gradients are averaged over the ranks before the update
         # weight gradients of different layers are independent: each launch is held to `wgrad_ctas` CTAs and the launches
         # go round-robin to `wgrad_streams` streams, each with a workspace of its own
         self.wgrad_ctas, self.wgrad_streams = wgrad_ctas, max(1, wgrad_streams)
@@ -188,6 +212,8 @@ class TrainStep:
             if li > 0:
                 self.conv_dgrad(li, stream)
             self.conv_wgrad(li, stream)
+        if self.world > 1:
+            allreduce_mean(self.mp.g_flat, self.world)
         self.lasso(stream)
 
     def _branches(self):
@@ -279,8 +305,12 @@ class TrainStep:
         self._aux = torch.cuda.Stream()
         l0 = self.ctx.launch_count()
         self.graph = torch.cuda.CUDAGraph()
+        self._graph_has_update = self.world <= 1
         with torch.cuda.graph(self.graph):
-            if two_streams:
+            if self.world > 1:
+                # data parallel: the graph ends with the weight gradients; the collective and the update follow it eagerly
+                self.train_two_streams(lasso=False)
+            elif two_streams:
                 self.train_two_streams()
             else:
                 self.train()
@@ -291,6 +321,9 @@ class TrainStep:
         self.reconfigure(stream)
         if getattr(self, "graph", None) is not None:
             self.graph.replay()
+            if not self._graph_has_update:
+                allreduce_mean(self.mp.g_flat, self.world)       # the one exchange of a data-parallel step
+                self.lasso(stream)
         else:
             self.train(stream)
 

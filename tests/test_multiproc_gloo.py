@@ -35,6 +35,28 @@ def test_two_gloo_ranks_take_the_max_time_and_sum_the_work():
             assert abs(value - 2 * 2.0e12 / (15.0e-3 / 4) / 1e12) < 1e-9   # both ranks' FLOPs over that time, TFLOP/s
 
 
+def _allreduce_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    from paper_1901_09290_b200 import harness
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    g = torch.arange(1000, dtype=torch.float32) * (rank + 1)        # rank r holds (r + 1) * [0, 1, 2, ...]
+    harness.allreduce_mean(g, world)
+    out[rank] = g.clone()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_average_the_flat_gradient_buffer():
+    """The one exchange of a data-parallel step: every rank ends with the mean of the ranks' gradient buffers."""
+    world, port = 2, 29733
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_allreduce_worker, args=(world, port, out), nprocs=world, join=True)
+        want = torch.arange(1000, dtype=torch.float32) * 1.5
+        for rank in range(world):
+            assert torch.equal(out[rank], want)
+
+
 def test_single_rank_is_the_identity():
     sys.path.insert(0, ROOT)
     import bench
