@@ -765,6 +765,18 @@ struct WgradP {
     int splits;
     int Pd, Qd, stride, lo_h, lo_w, S;
     int stages, tmem_cols;
+    // row-block form (stride-1 filters with several taps): a stage is `nr` output rows of one image
+    int nr, Wp, RB;         // rows per unit, row pitch of both staged tiles in pixels (Q + S - 1), units per image
+    int units, units_per_split;
+    int ksteps;             // 16-pixel MMA steps per unit: ceil(nr * Wp / 16)
+    int nb_a;               // 64-channel dy boxes per stage (1 when K <= 64)
+    int lo_span;            // R - 1: extra rows of the x halo box
+    int pair;               // row-block form, C <= 64: the M side of an MMA is TWO taps x 64 input channels of the x tile
+                            // (the second tap is the first one shifted: the operand's 64-element block stride is that shift)
+                            // and the N side is the output channels; accumulator lanes = (tap, c), columns = k
+    int apc;                // accumulators per CTA (= tpc, or tpc / 2 in the paired form)
+    int acc_cols;           // columns of one accumulator (= BN, or the padded K in the paired form)
+    unsigned a_box, b_box;  // bytes reserved per dy box and per x box (multiples of 1024)
     float *out;             // dw
     float *partial;         // splits > 1: workspace [blockIdx.x][tap in group][split][128][BN] fp32
     unsigned int *sync;     // splits > 1: two zeroed counters per blockIdx.x (arrived, reduced); left zero again at exit
@@ -777,6 +789,215 @@ __device__ unsigned long long g_wg_trace[8][64];
 #else
 #define WTRACE(i) do { } while (0)
 #endif
+// Everything after the main loop of a weight-gradient kernel: the accumulators leave TMEM (directly to dw, or as this
+// split's partial tile), the splits of a tile meet, and every CTA sums its share of the tile over the splits.
+// `ring_bytes` of shared memory at `data_base` are free by then and serve as staging.
+__device__ __forceinline__ void wgrad_finish(const WgradP &p, const CUtensorMap &tmP, Ctl *ctl, uint32_t data_base, uint32_t tmem_base,
+                                             int ntap, int tap0, int k0, int c0, int split, int iters, uint32_t ring_bytes, int n_acc, int acc_cols)
+{
+    volatile int *abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp >= 1) {
+        // ---------------- epilogue: the four epilogue warps and, once they are done issuing, the four issuer warps; a warp
+        // may read the TMEM lanes of quarter warp % 4, so each quarter has two warps, which take alternate 32-column chunks
+        const int quarter = warp & 3, wset = (warp >= 2 && warp < 6) ? 0 : 1;
+        bool ok = true;
+        if (iters > 0) ok = mbar_wait(smem_u32(&ctl->accum), 0, abort_flag, p.status, 6);
+        if (warp == 2) WTRACE(3);
+        tc_fence_after();
+        if (ok) {
+            const int k = k0 + quarter * 32 + lane;
+            const bool row_ok = k < p.K;
+            (void)row_ok;
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            if (p.splits > 1) {
+                // ---- (1) this CTA's fp32 partial tile goes to the workspace through swizzled staging + TMA stores
+                const int gtid = (warp - 1) * 32 + lane;
+                int sl = 0, ci = 0;
+                for (int tt = 0; tt < n_acc; ++tt)
+                for (int cc = 0; cc < acc_cols; cc += 32, ++ci) {
+                    if ((ci & 1) != wset) continue;
+                    sl ^= 1;
+                    const uint32_t slab = data_base + (uint32_t)((wset * 4 + quarter) * 2 + sl) * 4096u;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                    uint32_t lo[16], hi[16];
+                    if (iters > 0) {
+                        tmem_ld16(lane_addr + (uint32_t)(tt * acc_cols + cc), lo);
+                        if (cc + 16 < acc_cols) tmem_ld16(lane_addr + (uint32_t)(tt * acc_cols + cc) + 16u, hi);
+                        tmem_ld_wait();
+                    }
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        if (iters <= 0) lo[e] = 0u;
+                        if (iters <= 0 || cc + 16 >= acc_cols) hi[e] = 0u;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t *src = j < 4 ? &lo[4 * j] : &hi[4 * (j - 4)];
+                        const uint32_t addr = slab + (uint32_t)lane * 128u + (((uint32_t)j ^ ((uint32_t)lane & 7u)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(src[0]), "r"(src[1]), "r"(src[2]), "r"(src[3])
+                                     : "memory");
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmP, slab, cc, (((int)blockIdx.x * p.apc + tt) * p.splits + split) * 128 + quarter * 32);
+                        tma_store_commit();
+                    }
+                }
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // the writes have completed
+                __threadfence();
+                if (warp == 2) WTRACE(4);
+                named_barrier(1, 256);
+                // ---- (2) every split CTA of this tile is resident (the grid is at most one CTA per SM): wait for all of them
+                unsigned int *arrived = p.sync + 2 * blockIdx.x;
+                if (gtid == 0) {
+                    atomicAdd(arrived, 1u);
+                    const uint64_t t0 = globaltimer_ns();
+                    while (atomicAdd(arrived, 0u) < (unsigned)p.splits) {
+                        if (*abort_flag) break;
+                        if (globaltimer_ns() - t0 > 2000000000ull) { record_timeout(p.status, 8); *abort_flag = 1; break; }
+                        __nanosleep(64);
+                    }
+                }
+                named_barrier(1, 256);
+                if (warp == 2) WTRACE(5);
+            } else if (p.pair) {
+                // lanes are (tap of the pair, input channel), columns are output channels: for one column a warp's lanes
+                // write consecutive floats of dw
+                const int l = quarter * 32 + lane, c = l & 63;
+                int ci = 0;
+                for (int tt = 0; tt < n_acc; ++tt)
+                for (int cc = 0; cc < acc_cols; cc += 16, ++ci) {
+                    if ((ci & 1) != wset) continue;
+                    const int tap = tap0 + 2 * tt + (l >> 6);
+                    uint32_t v[16];
+                    if (iters > 0) {
+                        tmem_ld16(lane_addr + (uint32_t)(tt * acc_cols + cc), v);
+                        tmem_ld_wait();
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) v[e] = 0u;
+                    }
+                    if (c >= p.C || tap >= tap0 + ntap) continue;
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        if (cc + e < p.K) p.out[((size_t)(cc + e) * p.taps + tap) * p.C + c] = __uint_as_float(v[e]);
+                }
+            } else {
+            float *obase = p.out;
+            // The stages are free once the accumulator is complete: each warp transposes its 32 x 32 blocks through
+            // a padded shared-memory square so that a warp writes 32 consecutive floats of one dw row at a time.
+            const uint32_t sq = data_base + (uint32_t)(wset * 4 + quarter) * (32u * 33u * 4u);
+            int ci = 0;
+            for (int tt = 0; tt < n_acc; ++tt)
+            for (int cc = 0; cc < acc_cols; cc += 32, ++ci) {
+                if ((ci & 1) != wset) continue;
+                const int tap = tap0 + tt;
+                uint32_t v[32];
+                if (iters > 0) {
+                    uint32_t lo[16], hi[16];
+                    tmem_ld16(lane_addr + (uint32_t)(tt * acc_cols + cc), lo);
+                    if (cc + 16 < acc_cols) tmem_ld16(lane_addr + (uint32_t)(tt * acc_cols + cc) + 16u, hi);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) { v[e] = lo[e]; v[16 + e] = (cc + 16 < acc_cols) ? hi[e] : 0u; }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = 0u;
+                }
+                __syncwarp();
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(sq + (uint32_t)(lane * 33 + e) * 4u), "r"(v[e]) : "memory");
+                __syncwarp();
+                const int col = c0 + cc + lane;
+                for (int rr = 0; rr < 32; ++rr) {
+                    const int kk = k0 + quarter * 32 + rr;
+                    if (kk >= p.K) break;
+                    uint32_t t;
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(t) : "r"(sq + (uint32_t)(rr * 33 + lane) * 4u) : "memory");
+                    if (col < p.C && cc + lane < p.BN) obase[((size_t)kk * p.taps + tap) * p.C + col] = __uint_as_float(t);
+                }
+            }
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (p.splits > 1 && !*abort_flag) {
+        // ---- (3) all threads: this CTA sums its share of the tile's elements over the splits
+        __threadfence();
+        // Work items are (tap, row, 4-column group) of the real rows of the CTA's tiles, dealt out evenly to the split CTAs.
+        // The partial tiles sit in L2; what costs time is a chain of dependent loads, so every thread first issues the
+        // asynchronous 16-byte copies of its items for ALL splits into the (now idle) stage memory, and only then are the
+        // copies summed from shared memory in ascending split order: deterministic, whichever CTA does the work.
+        const int rows_real = p.pair ? 128 : min(128, p.K - k0);
+        const int ngrp = acc_cols / 4;                               // float4 groups per row (a multiple of 16 columns)
+        const int items = rows_real * ngrp;
+        const int total = n_acc * items;
+        const int per_cta = (total + p.splits - 1) / p.splits;
+        const int it_beg = split * per_cta, it_end = min(total, it_beg + per_cta);
+        const size_t zstride = (size_t)128 * acc_cols;
+        const float *pbase = p.partial + (size_t)blockIdx.x * p.apc * p.splits * zstride;
+        const int cap = (int)(((size_t)ring_bytes) / ((size_t)p.splits * 16));   // items the stage memory holds
+        for (int c_beg = it_beg; c_beg < it_end; c_beg += cap) {
+            const int n_chunk = min(cap, it_end - c_beg);
+            for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
+                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
+                const float *src = pbase + (size_t)tt * p.splits * zstride + (size_t)item * 4;
+                uint32_t dst = data_base + (uint32_t)i * 16u;
+                for (int z = 0; z < p.splits; ++z, src += zstride, dst += (uint32_t)n_chunk * 16u)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            __syncthreads();
+            for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
+                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
+                const int r = item / ngrp, col = (item - r * ngrp) * 4;
+                if (!p.pair && c0 + col >= p.C) continue;
+                float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                uint32_t a = data_base + (uint32_t)i * 16u;
+                for (int z = 0; z < p.splits; ++z, a += (uint32_t)n_chunk * 16u) {
+                    float4 t;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "r"(a) : "memory");
+                    sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+                }
+                if (p.pair) {
+                    // row = (tap of the pair, input channel), columns = output channels
+                    const int tap = tap0 + 2 * tt + (r >> 6), c = r & 63;
+                    if (c < p.C && tap < tap0 + ntap) {
+                        const float v4[4] = {sum.x, sum.y, sum.z, sum.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (col + e < p.K) p.out[((size_t)(col + e) * p.taps + tap) * p.C + c] = v4[e];
+                    }
+                    continue;
+                }
+                float *dst = p.out + ((size_t)(k0 + r) * p.taps + tap0 + tt) * p.C + c0 + col;
+                const int nv = min(4, p.C - (c0 + col));
+                dst[0] = sum.x;
+                if (nv > 1) dst[1] = sum.y;
+                if (nv > 2) dst[2] = sum.z;
+                if (nv > 3) dst[3] = sum.w;
+            }
+            __syncthreads();
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) WTRACE(6);
+        if (threadIdx.x == 0) {
+            unsigned int *arrived = p.sync + 2 * blockIdx.x, *reduced = arrived + 1;
+            __threadfence();
+            if (atomicAdd(reduced, 1u) == (unsigned)p.splits - 1u) {          // last one out clears the counters
+                *arrived = 0u;
+                *reduced = 0u;
+                __threadfence();
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_constant__ CUtensorMap tmDy,
                                                               const __grid_constant__ CUtensorMap tmX,
                                                               const __grid_constant__ CUtensorMap tmP, const WgradP p)
@@ -922,172 +1143,160 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
         if (ok) umma_commit_lead(smem_u32(&ctl->accum), leader);
         if (warp == 1) WTRACE(2);
     }
-    if (warp >= 1) {
-        // ---------------- epilogue: the four epilogue warps and, once they are done issuing, the four issuer warps; a warp
-        // may read the TMEM lanes of quarter warp % 4, so each quarter has two warps, which take alternate 32-column chunks
-        const int quarter = warp & 3, wset = (warp >= 2 && warp < 6) ? 0 : 1;
-        bool ok = true;
-        if (iters > 0) ok = mbar_wait(smem_u32(&ctl->accum), 0, abort_flag, p.status, 6);
-        if (warp == 2) WTRACE(3);
+    wgrad_finish(p, tmP, ctl, data_base, tmem_base, ntap, tap0, k0, c0, split, iters, (uint32_t)p.stages * stage_bytes, ntap, p.BN);
+    if (warp == 1) {
         tc_fence_after();
-        if (ok) {
-            const int k = k0 + quarter * 32 + lane;
-            const bool row_ok = k < p.K;
-            (void)row_ok;
-            const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-            if (p.splits > 1) {
-                // ---- (1) this CTA's fp32 partial tile goes to the workspace through swizzled staging + TMA stores
-                const int gtid = (warp - 1) * 32 + lane;
-                int sl = 0, ci = 0;
-                for (int tt = 0; tt < ntap; ++tt)
-                for (int cc = 0; cc < p.BN; cc += 32, ++ci) {
-                    if ((ci & 1) != wset) continue;
-                    sl ^= 1;
-                    const uint32_t slab = data_base + (uint32_t)((wset * 4 + quarter) * 2 + sl) * 4096u;
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    __syncwarp();
-                    uint32_t lo[16], hi[16];
-                    if (iters > 0) {
-                        tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc), lo);
-                        if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc) + 16u, hi);
-                        tmem_ld_wait();
-                    }
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        if (iters <= 0) lo[e] = 0u;
-                        if (iters <= 0 || cc + 16 >= p.BN) hi[e] = 0u;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t *src = j < 4 ? &lo[4 * j] : &hi[4 * (j - 4)];
-                        const uint32_t addr = slab + (uint32_t)lane * 128u + (((uint32_t)j ^ ((uint32_t)lane & 7u)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(src[0]), "r"(src[1]), "r"(src[2]), "r"(src[3])
-                                     : "memory");
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tmP, slab, cc, (((int)blockIdx.x * p.tpc + tt) * p.splits + split) * 128 + quarter * 32);
-                        tma_store_commit();
-                    }
-                }
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // the writes have completed
-                __threadfence();
-                if (warp == 2) WTRACE(4);
-                named_barrier(1, 256);
-                // ---- (2) every split CTA of this tile is resident (the grid is at most one CTA per SM): wait for all of them
-                unsigned int *arrived = p.sync + 2 * blockIdx.x;
-                if (gtid == 0) {
-                    atomicAdd(arrived, 1u);
-                    const uint64_t t0 = globaltimer_ns();
-                    while (atomicAdd(arrived, 0u) < (unsigned)p.splits) {
-                        if (*abort_flag) break;
-                        if (globaltimer_ns() - t0 > 2000000000ull) { record_timeout(p.status, 8); *abort_flag = 1; break; }
-                        __nanosleep(64);
-                    }
-                }
-                named_barrier(1, 256);
-                if (warp == 2) WTRACE(5);
-            } else {
-            float *obase = p.out;
-            // The stages are free once the accumulator is complete: each warp transposes its 32 x 32 blocks through
-            // a padded shared-memory square so that a warp writes 32 consecutive floats of one dw row at a time.
-            const uint32_t sq = data_base + (uint32_t)(wset * 4 + quarter) * (32u * 33u * 4u);
-            int ci = 0;
-            for (int tt = 0; tt < ntap; ++tt)
-            for (int cc = 0; cc < p.BN; cc += 32, ++ci) {
-                if ((ci & 1) != wset) continue;
-                const int tap = tap0 + tt;
-                uint32_t v[32];
-                if (iters > 0) {
-                    uint32_t lo[16], hi[16];
-                    tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc), lo);
-                    if (cc + 16 < p.BN) tmem_ld16(lane_addr + (uint32_t)(tt * p.BN + cc) + 16u, hi);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) { v[e] = lo[e]; v[16 + e] = (cc + 16 < p.BN) ? hi[e] : 0u; }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = 0u;
-                }
-                __syncwarp();
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(sq + (uint32_t)(lane * 33 + e) * 4u), "r"(v[e]) : "memory");
-                __syncwarp();
-                const int col = c0 + cc + lane;
-                for (int rr = 0; rr < 32; ++rr) {
-                    const int kk = k0 + quarter * 32 + rr;
-                    if (kk >= p.K) break;
-                    uint32_t t;
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(t) : "r"(sq + (uint32_t)(rr * 33 + lane) * 4u) : "memory");
-                    if (col < p.C && cc + lane < p.BN) obase[((size_t)kk * p.taps + tap) * p.C + col] = __uint_as_float(t);
-                }
-            }
-            }
-        }
-        tc_fence_before();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
+}
+
+// Row-block form of the weight gradient for stride-1 filters with several taps and at most 64 input channels. A stage is
+// one unit = `nr` output rows of one image: dy as a box of nr rows x Wp columns (the columns past Q and the rows past P
+// are zero-filled by the TMA unit) and x as the halo box of nr + R - 1 rows x Wp columns starting at (-pad, -pad) of the
+// unit, both with one 128-byte swizzle row per pixel. Pixel m = i * Wp + j of the dy box pairs with pixel
+// m + r * Wp + s of the x box for tap (r, s), so every tap reads the SAME staged x tile through an operand descriptor
+// whose start is shifted by r * Wp + s rows: x crosses the memory system once per unit instead of once per tap. Where
+// j + s runs past the row the dy factor is a zero column. Rows past the boxes (up to the 16-pixel step) are zeroed once
+// and never written again.
+//   The x tile is the M side of the MMA and carries TWO taps: M rows 0..63 are the 64 channel lanes at the first tap's
+// shift, rows 64..127 the same lanes at the second tap's shift (the descriptor's 64-element block stride is the
+// difference of the shifts). The N side is dy's output channels. An accumulator therefore holds dw^T of a pair of taps:
+// lanes = (tap, c), columns = k -- half the MMAs of the one-tap-per-accumulator form, and none of the 128 rows wasted
+// when K is small.
+__global__ void __launch_bounds__(kThreads) conv_wgrad_rows_kernel(const __grid_constant__ CUtensorMap tmDy,
+                                                                   const __grid_constant__ CUtensorMap tmX,
+                                                                   const __grid_constant__ CUtensorMap tmP, const WgradP p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw);
+    const uint32_t smem_base = smem_u32(smem_raw);
+    const uint32_t data_base = (smem_base + (uint32_t)sizeof(Ctl) + 1023u) & ~1023u;
+    const uint32_t nb_b = (uint32_t)((p.BN + 63) / 64);
+    const uint32_t a_bytes = (uint32_t)p.nb_a * p.a_box;
+    const uint32_t stage_bytes = a_bytes + nb_b * p.b_box;
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int bx = blockIdx.x;
+    const int n_tile = bx % p.n_tiles; bx /= p.n_tiles;
+    const int m_tile = bx % p.m_tiles; bx /= p.m_tiles;
+    const int tap0 = bx * p.tpc;
+    const int ntap = min(p.tpc, p.taps - tap0);
+    const int split = blockIdx.y;
+    const int k0 = m_tile * 128, c0 = n_tile * p.BN;
+    const int u_beg = split * p.units_per_split;
+    const int u_end = min(p.units, u_beg + p.units_per_split);
+    const int iters = u_end > u_beg ? u_end - u_beg : 0;
+    const int n_acc = (ntap + 1) / 2;                                 // accumulators: one per pair of taps
+    const int NI = n_acc < 4 ? n_acc : 4;                             // MMA issuer warps in use: pairs i, i + NI, ...
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 2u);                   // the dy producer and the x producer
+            mbar_init(smem_u32(&ctl->empty[s]), (uint32_t)NI);
+        }
+        mbar_init(smem_u32(&ctl->accum), (uint32_t)NI);
+        ctl->abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tmDy);
+        prefetch_tmap(&tmX);
+    }
+    // the ring starts as zeros: the rows between the end of a box and the end of the last 16-pixel step are read by the
+    // MMAs (times zero) and must be finite
+    for (uint32_t off = threadIdx.x * 16u; off < (uint32_t)p.stages * stage_bytes; off += kThreads * 16u)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(data_base + off), "r"(0u) : "memory");
+    fence_proxy_async();
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
     __syncthreads();
-    if (p.splits > 1 && !*abort_flag) {
-        // ---- (3) all threads: this CTA sums its share of the tile's elements over the splits
-        __threadfence();
-        // Work items are (tap, row, 4-column group) of the real rows of the CTA's tiles, dealt out evenly to the split CTAs.
-        // The partial tiles sit in L2; what costs time is a chain of dependent loads, so every thread first issues the
-        // asynchronous 16-byte copies of its items for ALL splits into the (now idle) stage memory, and only then are the
-        // copies summed from shared memory in ascending split order: deterministic, whichever CTA does the work.
-        const int rows_real = min(128, p.K - k0);
-        const int ngrp = p.BN / 4;                                   // float4 groups per row (BN is a multiple of 16)
-        const int items = rows_real * ngrp;
-        const int total = ntap * items;
-        const int per_cta = (total + p.splits - 1) / p.splits;
-        const int it_beg = split * per_cta, it_end = min(total, it_beg + per_cta);
-        const size_t zstride = (size_t)128 * p.BN;
-        const float *pbase = p.partial + (size_t)blockIdx.x * p.tpc * p.splits * zstride;
-        const int cap = (int)(((size_t)p.stages * stage_bytes) / ((size_t)p.splits * 16));   // items the stage memory holds
-        for (int c_beg = it_beg; c_beg < it_end; c_beg += cap) {
-            const int n_chunk = min(cap, it_end - c_beg);
-            for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
-                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
-                const float *src = pbase + (size_t)tt * p.splits * zstride + (size_t)item * 4;
-                uint32_t dst = data_base + (uint32_t)i * 16u;
-                for (int z = 0; z < p.splits; ++z, src += zstride, dst += (uint32_t)n_chunk * 16u)
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-            }
-            asm volatile("cp.async.wait_all;" ::: "memory");
-            __syncthreads();
-            for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
-                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
-                const int r = item / ngrp, col = (item - r * ngrp) * 4;
-                if (c0 + col >= p.C) continue;
-                float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-                uint32_t a = data_base + (uint32_t)i * 16u;
-                for (int z = 0; z < p.splits; ++z, a += (uint32_t)n_chunk * 16u) {
-                    float4 t;
-                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "r"(a) : "memory");
-                    sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const int issuer = warp == 1 ? 0 : warp - 5;                      // warps 6, 7, 8 -> issuers 1, 2, 3
+    grid_dependency_wait();              // nothing above touches global memory
+    grid_launch_dependents();
+    if (threadIdx.x == 0) WTRACE(0);
+
+    if (warp == 0 || warp == 2) {
+        if (lane == 0) {
+            // ---------------- producers: warp 0 brings the dy boxes of every unit, warp 2 the x halo boxes
+            const bool is_dy = warp == 0;
+            const int n_dy = p.nb_a;
+            const uint32_t my_bytes = is_dy ? (uint32_t)(n_dy * p.nr * p.Wp) * 128u
+                                            : nb_b * (uint32_t)((p.nr + p.lo_span) * p.Wp) * 128u;
+            int n = u_beg / p.RB, rb = u_beg - n * p.RB;
+            int s = 0, ph = 0, issued = 0;
+            for (int it = 0; it < iters; ++it) {
+                if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 4)) break;
+                const uint32_t bar = smem_u32(&ctl->full[s]);
+                const uint32_t a_dst = data_base + (uint32_t)s * stage_bytes, b_dst = a_dst + a_bytes;
+                mbar_arrive_expect_tx(bar, my_bytes);
+                const int p0 = rb * p.nr;
+                if (is_dy) {
+                    for (int b = 0; b < n_dy; ++b) tma_load_4d(a_dst + (uint32_t)b * p.a_box, &tmDy, bar, b * 64, 0, p0, n);
+                } else {
+                    for (uint32_t b = 0; b < nb_b; ++b)
+                        tma_load_4d(b_dst + b * p.b_box, &tmX, bar, c0 + (int)b * 64, p.lo_w, p0 + p.lo_h, n);
                 }
-                float *dst = p.out + ((size_t)(k0 + r) * p.taps + tap0 + tt) * p.C + c0 + col;
-                const int nv = min(4, p.C - (c0 + col));
-                dst[0] = sum.x;
-                if (nv > 1) dst[1] = sum.y;
-                if (nv > 2) dst[2] = sum.z;
-                if (nv > 3) dst[3] = sum.w;
+                if (++rb == p.RB) { rb = 0; ++n; }
+                issued = it + 1;
+                if (++s == p.stages) { s = 0; ph ^= 1; }
             }
-            __syncthreads();
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) WTRACE(6);
-        if (threadIdx.x == 0) {
-            unsigned int *arrived = p.sync + 2 * blockIdx.x, *reduced = arrived + 1;
-            __threadfence();
-            if (atomicAdd(reduced, 1u) == (unsigned)p.splits - 1u) {          // last one out clears the counters
-                *arrived = 0u;
-                *reduced = 0u;
-                __threadfence();
+            if (*abort_flag) {
+                for (int it = max(0, issued - p.stages); it < issued; ++it) {
+                    const int s2 = it % p.stages, ph2 = (it / p.stages) & 1;
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!mbar_try_wait(smem_u32(&ctl->full[s2]), ph2) && globaltimer_ns() - t0 < 20000000ull) {}
+                }
             }
         }
+        __syncwarp();
     }
+    if (warp == 1 || (warp >= 6 && issuer < NI)) {
+        // ---------------- MMA issuer `issuer`: the warp walks the loop in lockstep, lane 0 issues
+        const uint32_t leader = lane == 0 ? 1u : 0u;
+        const uint32_t idesc = make_idesc_bf16(128, p.acc_cols, 1, 1);
+        // this issuer's pairs (at most four: 16 accumulators of 32 columns fill the tensor memory): byte offset of the
+        // first tap's rows in the x tile and the distance to the second tap's rows
+        uint32_t tap_shift[4] = {0u, 0u, 0u, 0u}, tap_lbo[4] = {128u, 128u, 128u, 128u};
+        int n_mine = 0;
+        for (int a = issuer; a < n_acc && n_mine < 4; a += NI, ++n_mine) {
+            const int t0 = tap0 + 2 * a, r0 = t0 / p.S, sh0 = r0 * p.Wp + (t0 - r0 * p.S);
+            int sh1 = sh0 + 1;                                        // an odd last tap: the upper 64 lanes are not stored
+            if (2 * a + 1 < ntap) {
+                const int r1 = (t0 + 1) / p.S;
+                sh1 = r1 * p.Wp + (t0 + 1 - r1 * p.S);
+            }
+            tap_shift[n_mine] = (uint32_t)sh0 * 128u;
+            tap_lbo[n_mine] = (uint32_t)(sh1 - sh0) * 128u;
+        }
+        bool ok = true;
+        int s = 0, ph = 0;
+        for (int it = 0; it < iters && ok; ++it) {
+            ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status, 5);
+            if (!ok) break;
+            if (it == 0 && warp == 1) WTRACE(1);
+            tc_fence_after();
+            const uint32_t a_src = data_base + (uint32_t)s * stage_bytes, b_src = a_src + a_bytes;
+            const uint64_t dyd = make_desc(a_src, p.a_box, 1024u);
+            const uint32_t acc = it != 0 ? 1u : 0u;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (j >= n_mine) break;
+                const uint64_t xd = make_desc(b_src + tap_shift[j], tap_lbo[j], 1024u);
+                const uint32_t d_tmem = tmem_base + (uint32_t)((issuer + j * NI) * p.acc_cols);
+                umma_bf16_lead(d_tmem, xd, dyd, idesc, acc, leader);
+                for (int k = 1; k < p.ksteps; ++k) umma_bf16_lead(d_tmem, xd + 128ull * k, dyd + 128ull * k, idesc, 1u, leader);
+            }
+            umma_commit_lead(smem_u32(&ctl->empty[s]), leader);
+            if (++s == p.stages) { s = 0; ph ^= 1; }
+        }
+        if (ok) umma_commit_lead(smem_u32(&ctl->accum), leader);
+        if (warp == 1) WTRACE(2);
+    }
+    wgrad_finish(p, tmP, ctl, data_base, tmem_base, ntap, tap0, k0, c0, split, iters, (uint32_t)p.stages * stage_bytes, n_acc, p.acc_cols);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
@@ -1525,15 +1734,102 @@ int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     return (int)s;
 }
 
+// Plan of the row-block weight gradient (stride-1 filters with several taps); ok = 0 where the generic kernel is used.
+struct WgRows {
+    int ok;
+    int bn, n_tiles, m_tiles, tpc, tap_groups, apc, acc_cols;
+    int nr, Wp, RB, units, units_per_split, splits, ksteps, nb_a, stages;
+    unsigned a_box, b_box;
+    size_t stage_bytes, smem;
+};
+
+WgRows wgrad_rows_plan(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
+{
+    WgRows w;
+    memset(&w, 0, sizeof(w));
+    const int taps = d->R * d->S;
+    if (d->stride != 1 || taps < 2 || taps > kMaxTaps) return w;
+    w.Wp = Q + d->S - 1;
+    if (w.Wp > 256 || P < 1 || Q < 1) return w;
+    // paired form only: the x tile is the M side (two taps x 64 channel lanes), dy's output channels the N side
+    w.acc_cols = pt_ceil_div(d->K, 16) * 16;
+    if (d->C > 64 || w.acc_cols > 256) return w;
+    w.bn = tile_n(d->C, &w.n_tiles);
+    w.m_tiles = 1;
+    const int pairs = pt_ceil_div(taps, 2);
+    int t = 512 / w.acc_cols;
+    if (t > 16) t = 16;                                   // four issuer warps x four accumulators
+    if (t > pairs) t = pairs;
+    w.tap_groups = pt_ceil_div(pairs, t);
+    w.apc = pt_ceil_div(pairs, w.tap_groups);
+    w.tpc = 2 * w.apc;
+    w.tap_groups = pt_ceil_div(taps, w.tpc);
+    w.nb_a = pt_ceil_div(w.acc_cols, 64);
+    const int nb_b = 1;
+    // rows per unit: the least traffic per useful row (dy rows + x halo rows, the last unit of an image padded) times
+    // the MMA steps spent per useful pixel, among the sizes that leave at least two stages
+    double best = 1e30;
+    for (int nr = 1; nr <= P && nr + d->R - 1 <= 256; ++nr) {
+        const int ks = pt_ceil_div(nr * w.Wp, 16);
+        const size_t a_box = (size_t)ks * 2048;
+        const size_t b_box = pt_align_up(((size_t)(d->R - 1) * w.Wp + d->S + (size_t)ks * 16) * 128, 1024);
+        const size_t stage = w.nb_a * a_box + nb_b * b_box;
+        const int st = (int)((220 * 1024 - 2048) / stage);
+        if (st < 2) break;
+        const int rb = pt_ceil_div(P, nr);
+        const double traffic = (double)(w.nb_a * nr + nb_b * (nr + d->R - 1)) * rb / P;
+        const double steps = (double)ks * 16 * rb / ((double)P * w.Wp);
+        const double cost = traffic * steps;
+        if (cost < best) {
+            best = cost;
+            w.nr = nr; w.ksteps = ks; w.a_box = (unsigned)a_box; w.b_box = (unsigned)b_box;
+            w.stages = st > kMaxStages ? kMaxStages : st;
+            w.stage_bytes = stage;
+        }
+    }
+    if (w.nr == 0) return w;
+    w.RB = pt_ceil_div(P, w.nr);
+    w.units = d->N * w.RB;
+    const int tiles = w.m_tiles * w.n_tiles * w.tap_groups;
+    const int budget = (c->wgrad_ctas > 0 && c->wgrad_ctas < c->sm_count) ? c->wgrad_ctas : c->sm_count;
+    int s = budget / tiles;                                // at most one CTA per SM, one wave
+    if (s > w.units / 2) s = w.units / 2;                  // at least two units per split
+    if (s < 1) s = 1;
+    if (s > 512) s = 512;
+    w.units_per_split = pt_ceil_div(w.units, s);
+    w.splits = pt_ceil_div(w.units, w.units_per_split);
+    if (w.stages > w.units_per_split && w.units_per_split >= 2) w.stages = w.units_per_split;
+    w.smem = 2048 + (size_t)w.stages * w.stage_bytes;
+    if (w.smem < 2048 + 8 * 2 * 4096) w.smem = 2048 + 8 * 2 * 4096;    // the epilogue's staging slabs reuse the ring
+    w.ok = 1;
+    return w;
+}
+
 // Workspace of the split weight gradient: one padded 128 x BN fp32 tile per (tile, split).
 size_t wgrad_partial_bytes(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
 {
+    const WgRows wr = wgrad_rows_plan(c, d, P, Q);
+    if (wr.ok)
+        return wr.splits <= 1 ? 0 : (size_t)wr.tap_groups * wr.apc * wr.splits * 128 * wr.acc_cols * sizeof(float);
     const int s = wgrad_splits(c, d, P, Q);
     if (s <= 1) return 0;
     int n_tiles;
     const int bn = tile_n(d->C, &n_tiles);
     const int tpc = wgrad_taps_per_cta(d->R * d->S, bn);
     return (size_t)n_tiles * pt_ceil_div(d->K, 128) * pt_ceil_div(d->R * d->S, tpc) * tpc * s * 128 * bn * sizeof(float);
+}
+
+// The splits' fp32 partial tiles as a 2-D tensor (BN columns, rows): box 32 x 32, 128-byte swizzle.
+bool make_partial_map(const pt_ctx *c, CUtensorMap *tm, void *ws, int bn, size_t rows)
+{
+    if (!c->encode_tiled) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)bn, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)bn * 4};
+    cuuint32_t box[2] = {32, 32}, estr[2] = {1, 1};
+    CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ws, dims, strides, box, estr,
+                                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
 }
 
 // Launches the weight-gradient kernel for a problem whose x operand is described by `tmX` (64 pixels x 64 channels boxes).
@@ -1547,6 +1843,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     p.m_tiles = pt_ceil_div(d->K, 128);
     p.tpc = wgrad_taps_per_cta(p.taps, p.BN);
     p.tap_groups = pt_ceil_div(p.taps, p.tpc);
+    p.apc = p.tpc; p.acc_cols = p.BN;
     p.npix = d->N * P * Q;
     p.splits = wgrad_splits(c, d, P, Q);
     p.pix_per_split = pt_ceil_div(pt_ceil_div(p.npix, p.splits), 64) * 64;
@@ -1567,13 +1864,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
         if (c->sync_next + 2 * gx > 16384) c->sync_next = 0;
         p.sync = c->d_sync + c->sync_next;
         c->sync_next += 2 * gx;
-        cuuint64_t dims[2] = {(cuuint64_t)p.BN, (cuuint64_t)gx * p.tpc * p.splits * 128};
-        cuuint64_t strides[1] = {(cuuint64_t)p.BN * 4};
-        cuuint32_t box[2] = {32, 32}, estr[2] = {1, 1};
-        CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmP, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ws, dims, strides, box, estr,
-                                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                                      CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+        if (!make_partial_map(c, &tmP, ws, p.BN, (size_t)gx * p.tpc * p.splits * 128)) return PT_ERR_CUDA;
     }
     // A: dy as a 2-D tensor (K channels, N*P*Q pixels), box 64 channels x 64 pixels
     if (!c->encode_tiled) return PT_ERR_CUDA;
@@ -1598,6 +1889,55 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     }
     dim3 grid((unsigned)gx, (unsigned)p.splits);
     PT_CUDA_OK(launch_pdl(conv_wgrad_kernel, grid, dim3(kThreads), smem, st, tmA, tmX, tmP, p));
+    c->launches += 1;
+    PT_CUDA_OK(cudaGetLastError());
+    return PT_OK;
+}
+
+// Launches the row-block weight-gradient kernel; PT_ERR_UNSUPPORTED (nothing launched) where the plan declines the shape.
+pt_status run_wgrad_rows(pt_ctx *c, const pt_conv_desc *d, int P, int Q, const void *x, const void *dy, float *out, void *ws,
+                         size_t ws_bytes, cudaStream_t st)
+{
+    const WgRows wr = wgrad_rows_plan(c, d, P, Q);
+    if (!wr.ok || !c->encode_tiled) return PT_ERR_UNSUPPORTED;
+    WgradP p;
+    memset(&p, 0, sizeof(p));
+    p.K = d->K; p.C = d->C; p.taps = d->R * d->S; p.S = d->S;
+    p.BN = wr.bn; p.n_tiles = wr.n_tiles; p.m_tiles = wr.m_tiles;
+    p.tpc = wr.tpc; p.tap_groups = wr.tap_groups;
+    p.pair = 1; p.apc = wr.apc; p.acc_cols = wr.acc_cols;
+    p.npix = d->N * P * Q;
+    p.splits = wr.splits;
+    p.Pd = P; p.Qd = Q; p.stride = 1; p.lo_h = -d->pad; p.lo_w = -d->pad;
+    p.nr = wr.nr; p.Wp = wr.Wp; p.RB = wr.RB; p.units = wr.units; p.units_per_split = wr.units_per_split;
+    p.ksteps = wr.ksteps; p.nb_a = wr.nb_a; p.lo_span = d->R - 1; p.a_box = wr.a_box; p.b_box = wr.b_box;
+    p.stages = wr.stages;
+    p.tmem_cols = pow2_cols(p.apc * p.acc_cols);
+    p.status = c->d_status;
+    p.out = out;
+    const int gx = p.n_tiles * p.m_tiles * p.tap_groups;
+    CUtensorMap tmP, tmA, tmX;
+    memset(&tmP, 0, sizeof(tmP));
+    if (p.splits > 1) {
+        const size_t need = (size_t)gx * p.apc * p.splits * 128 * p.acc_cols * sizeof(float);
+        if (!ws || ws_bytes < need) return PT_ERR_WORKSPACE;
+        p.partial = (float *)ws;
+        if (2 * gx > 8192) return PT_ERR_UNSUPPORTED;
+        if (c->sync_next + 2 * gx > 16384) c->sync_next = 0;
+        p.sync = c->d_sync + c->sync_next;
+        c->sync_next += 2 * gx;
+        if (!make_partial_map(c, &tmP, ws, p.acc_cols, (size_t)gx * p.apc * p.splits * 128)) return PT_ERR_CUDA;
+    }
+    // dy: box of nr rows x Wp columns (Wp > Q: the extra columns are out of bounds and read as zeros); x: the halo box
+    if (!make_halo_in_map(c, &tmA, dy, d->K, Q, P, d->N, d->ldy, wr.Wp, wr.nr)) return PT_ERR_UNSUPPORTED;
+    if (!make_halo_in_map(c, &tmX, x, d->C, d->W, d->H, d->N, d->ldx, wr.Wp, wr.nr + d->R - 1)) return PT_ERR_UNSUPPORTED;
+    static bool attr_set = false;
+    if (!attr_set) {
+        PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        attr_set = true;
+    }
+    dim3 grid((unsigned)gx, (unsigned)p.splits);
+    PT_CUDA_OK(launch_pdl(conv_wgrad_rows_kernel, grid, dim3(kThreads), wr.smem, st, tmA, tmX, tmP, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
@@ -1735,6 +2075,10 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
             c->launches += 1;
             PT_CUDA_OK(cudaGetLastError());
             return PT_OK;
+        }
+        {
+            const pt_status r = run_wgrad_rows(c, d, P, Q, a, b, (float *)out, ws, ws_bytes, st);
+            if (r != PT_ERR_UNSUPPORTED) return r;
         }
         CUtensorMap tmX;
         const int up_w = (Q - 1) * d->stride - d->pad - (d->W - 1), up_h = (P - 1) * d->stride - d->pad - (d->H - 1);

@@ -26,6 +26,7 @@ def main():
     ap.add_argument("--sets", type=int, default=4, help="rotating buffer sets (footprint larger than L2)")
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--algo", type=int, default=0)
+    ap.add_argument("--wgrad-ctas", type=int, default=0, help="CTA limit of the weight-gradient kernels (0 = one per SM)")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches (includes host launch cost)")
     ap.add_argument("--bn", default=None, help="N,H,C: time pt_bn_relu_fwd / pt_bn_relu_bwd instead of a convolution")
     args = ap.parse_args()
@@ -43,6 +44,8 @@ def main():
     pad = R // 2
     P = (H + 2 * pad - R) // stride + 1
     ctx = B.Context(0)
+    if args.wgrad_ctas:
+        ctx.set_wgrad_cta_limit(args.wgrad_ctas)
     d = B.make_conv_desc(N, H, H, C, K, R, R, stride, pad, 8 if C <= 4 else W.pad16(C), W.pad16(K), algo=args.algo)
     g = torch.Generator(device="cuda").manual_seed(1)
     sets = []

@@ -86,6 +86,31 @@ def test_config3_pruned_bottleneck(algo):
         Hh.check_conv(dw, l.C, oracle.conv_wgrad(x.numpy(), dy.numpy(), l.R, l.R, l.stride, pad), what=l.name + " wgrad")
 
 
+# (N, H, W, C, K, R, pad): stride-1 filters with several taps and at most 64 input channels -- the weight gradient that
+# stages row blocks and pairs taps: two dy boxes (K > 64), several tap groups with an odd last one (K = 200), 25 taps,
+# a wide image, an even filter, padding 0 and padding larger than (R - 1) / 2
+ROW_BLOCK = [
+    (3, 12, 12, 20, 100, 3, 1), (2, 10, 14, 64, 200, 3, 1), (2, 9, 9, 6, 10, 5, 2), (1, 8, 120, 9, 12, 3, 1),
+    (2, 11, 11, 13, 21, 3, 0), (2, 7, 7, 5, 9, 3, 2), (2, 6, 6, 33, 40, 2, 0), (64, 20, 20, 38, 38, 3, 1),
+]
+
+
+@pytest.mark.parametrize("shape", ROW_BLOCK)
+def test_row_block_weight_gradient(shape):
+    N, H, Wd, C, K, R, pad = shape
+    seed = W.BASE_SEED + 41
+    x = W.gen_act(N, H, Wd, C, seed)
+    w = W.bf16_round(W.gen_weight(K, R, R, C, seed + 1))
+    P, Q = H + 2 * pad - R + 1, Wd + 2 * pad - R + 1
+    dy = W.gen_dy(N, P, Q, K, seed + 2)
+    y, dx, dw, _ = Hh.run_conv_all(N, H, Wd, C, K, R, 1, pad, x, w, dy, algo=2)
+    Hh.check_conv(dw, C, oracle.conv_wgrad(x.numpy(), dy.numpy(), R, R, 1, pad), what="wgrad")
+    Hh.check_conv(y, K, oracle.conv_fwd(x.numpy(), w.numpy(), 1, pad), what="fwd")
+    Hh.check_conv(dx, C, oracle.conv_dgrad(dy.numpy(), w.numpy(), H, Wd, 1, pad), what="dgrad")
+    again = Hh.run_conv_all(N, H, Wd, C, K, R, 1, pad, x, w, dy, algo=2)[2]
+    assert torch.equal(dw, again)
+
+
 def test_wgrad_is_run_to_run_identical():
     N, H, C, K, R = 4, 14, 27, 19, 3
     x, w, dy, pad = _case(N, H, H, C, K, R, 1, W.BASE_SEED + 5)
