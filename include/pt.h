@@ -55,7 +55,9 @@ typedef struct pt_ctx pt_ctx;  /* opaque: device id, SM count, status word, tabl
 pt_status pt_create(pt_ctx **ctx, int device);
 pt_status pt_destroy(pt_ctx *ctx);
 const char *pt_status_string(pt_status s);
-/* Synchronises `stream`, reads and clears the device status word. PT_OK if no kernel recorded an error. */
+/* Synchronises `stream`, reads and clears the device status word. PT_OK if no kernel recorded an error; PT_ERR_TIMEOUT for
+ * an expired device-side wait; PT_ERR_INVALID_ARG for a channel index outside its tensor (pt_channel_gather /
+ * pt_channel_scatter_add skip such an entry). */
 pt_status pt_poll_device_status(pt_ctx *ctx, void *stream);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 uint64_t pt_launch_count(const pt_ctx *ctx);
@@ -281,6 +283,36 @@ pt_status pt_reconfigure_plan(pt_ctx *ctx, const pt_graph *g, int32_t *new2old, 
  * new_g must have the same topology, and each space size equal to the count pt_reconfigure_plan returned.
  * Layers whose new K or C is 0 are skipped. */
 pt_status pt_reconfigure(pt_ctx *ctx, const pt_graph *old_g, const int32_t *new2old, const pt_graph *new_g, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Channel gating (Sec. 4.2: gating layers on each residual branch gather the dense channels at the branch's entry and scatter
+ * them back at the merge point, so that every convolution of the branch works on dense channels only; the paper measured it
+ * against channel union and found the tensor reshaping too costly). Tensors are NHWC bf16 with a channel pitch that is a
+ * multiple of 8, 16-byte aligned, given as [npix][ld] with npix = N*H*W; all pointers are device pointers.
+ * The gradient of the gather is the scatter-add (into the node's gradient) and the gradient of the scatter-add is the
+ * gather, so these two calls serve the forward and the backward pass.
+ * ------------------------------------------------------------------------------------------ */
+
+/* idx[0..count) = the positions i < n with zero_flags[i] == 0, ascending (the dense channels of a group-mask produced by
+ * pt_find_zero_groups); idx[count..n) = -1; *count (device) = their number. One small launch, no synchronisation. */
+pt_status pt_dense_channel_list(pt_ctx *ctx, const uint8_t *zero_flags, int32_t n, int32_t *idx, int32_t *count, void *stream);
+
+/* dst[p][j] = src[p][idx[j]] for j < n_sel; dst's pad lanes (n_sel <= j < ld_dst) are written as zeros. src has c_src
+ * channels at pitch ld_src. idx (device, n_sel entries, each in [0, c_src)) may be in any order and may repeat.
+ * PT_ERR_INVALID_ARG for null pointers, pitches that are not multiples of 8 or smaller than the channel counts, misaligned
+ * tensors; PT_ERR_UNSUPPORTED for ld_dst > 4096. An out-of-range index is skipped (the lane reads as zero) and reported by
+ * pt_poll_device_status. */
+pt_status pt_channel_gather(pt_ctx *ctx, const void *src, int32_t ld_src, int32_t c_src, const int32_t *idx, int32_t n_sel,
+                            void *dst, int32_t ld_dst, int64_t npix, void *stream);
+
+/* node_out[p][c] = act(node_in[p][c] + b), c < c_node, where b = branch[p][j] if idx[j] == c for some j < n_sel, else 0;
+ * act = max(., 0) if relu, identity otherwise; the sum is formed in fp32 and rounded once to bf16 (nearest even); pad lanes
+ * of node_out are written as zeros. node_in may be NULL (read as zeros) and may be the same tensor as node_out. idx holds
+ * n_sel DISTINCT channels of the node, in any order.
+ * Errors as for pt_channel_gather (PT_ERR_UNSUPPORTED for ld_node > 4096). */
+pt_status pt_channel_scatter_add(pt_ctx *ctx, const void *branch, int32_t ld_branch, const int32_t *idx, int32_t n_sel,
+                                 const void *node_in, void *node_out, int32_t ld_node, int32_t c_node, int64_t npix,
+                                 int32_t relu, void *stream);
 
 #ifdef __cplusplus
 }

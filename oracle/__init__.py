@@ -353,6 +353,65 @@ def bn_relu_bwd(x, y, dy, gamma, mean, invstd, relu: bool = True):
     return dx, dz, dgamma, dbeta
 
 
+# --------------------------------------------------------------------------- channel gating (Sec. 4.2)
+def dense_channel_list(zero_flags) -> np.ndarray:
+    """Ascending positions of the groups that are NOT sparsified: the "dense channel indices" a gating layer gathers
+    and scatters (Sec. 4.2)."""
+    out = []
+    for i, z in enumerate(np.asarray(zero_flags)):
+        if not z:
+            out.append(i)
+    return np.asarray(out, dtype=np.int32)
+
+
+def channel_gather(x, idx) -> np.ndarray:
+    """Gate at the entry of a residual branch (Sec. 4.2): the branch's first convolution sees only the listed channels
+    of the node tensor x [N][H][W][C]: out[..., j] = x[..., idx[j]]."""
+    x = np.asarray(x)
+    out = np.empty(x.shape[:-1] + (len(idx),), x.dtype)
+    for j, c in enumerate(idx):
+        out[..., j] = x[..., int(c)]
+    return out
+
+
+def channel_scatter_add(branch, idx, node=None, c_node: Optional[int] = None, relu: bool = False) -> np.ndarray:
+    """Gate at the merge point (Sec. 4.2): channel j of the branch output goes back to position idx[j] of the node, where
+    it is added to what the node holds (the short-cut); every other channel of the node passes through unchanged.
+    The paper fixes no precision; the tensors are bf16 and the sum decides a rounding, so, as in the CUDA path, the
+    sum is formed in fp32 and rounded once to bf16 (returned as the fp32 value of that bf16)."""
+    branch = np.asarray(branch, np.float32)
+    if node is None:
+        node = np.zeros(branch.shape[:-1] + (int(c_node),), np.float32)
+    out = np.array(node, dtype=np.float32, copy=True)
+    for j, c in enumerate(idx):
+        out[..., int(c)] = out[..., int(c)] + branch[..., j]
+    if relu:
+        out = np.maximum(out, np.float32(0))
+    return round_bf16(out)
+
+
+def gating_channel_counts(graph: Graph, zero_out: Sequence[np.ndarray], zero_in: Sequence[np.ndarray],
+                          keep: Sequence[np.ndarray]) -> List[Tuple[int, int]]:
+    """(input channels, output channels) every convolution works on under channel gating (Sec. 4.2).
+
+    A space shared by several branches (more than one writer or more than one reader: the node of a residual stage)
+    keeps the union of dense channels, `keep`, but every convolution reading it is gated down to ITS OWN dense input
+    channels and every convolution writing it to ITS OWN dense output channels. A private space between two adjacent
+    layers has no gate: both sides use the kept channels."""
+    writers = [0] * len(graph.sizes)
+    readers = [0] * len(graph.sizes)
+    for isp, osp in graph.layers:
+        readers[isp] += 1
+        writers[osp] += 1
+    shared = [(writers[s] > 1 or readers[s] > 1) and not graph.fixed[s] for s in range(len(graph.sizes))]
+    out = []
+    for li, (isp, osp) in enumerate(graph.layers):
+        c = sum(1 for j in keep[isp] if not zero_in[li][j]) if shared[isp] else len(keep[isp])
+        k = sum(1 for j in keep[osp] if not zero_out[li][j]) if shared[osp] else len(keep[osp])
+        out.append((c, k))
+    return out
+
+
 # --------------------------------------------------------------------------- toy network (invariant only)
 def bn_affine(y, gamma, beta, mean, var, eps=1e-5):
     """Inference-form batch norm with given running statistics, per output channel."""

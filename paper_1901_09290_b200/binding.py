@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import (POINTER, Structure, byref, c_char_p, c_double, c_float, c_int32, c_size_t, c_uint8, c_uint64,
+from ctypes import (POINTER, c_int64, Structure, byref, c_char_p, c_double, c_float, c_int32, c_size_t, c_uint8, c_uint64,
                     c_void_p)
 from typing import List, Optional, Sequence
 
@@ -92,6 +92,10 @@ EXPORTS = {
     "pt_cross_entropy_workspace_bytes": (c_size_t, [c_int32]),
     "pt_cross_entropy": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_set_coeff": (c_int32, [c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]),
+    "pt_dense_channel_list": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p]),
+    "pt_channel_gather": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p]),
+    "pt_channel_scatter_add": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32, c_int64,
+                                         c_int32, c_void_p]),
     "pt_reconfigure_plan": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(c_int32), c_void_p]),
     "pt_reconfigure": (c_int32, [c_void_p, POINTER(pt_graph), c_void_p, POINTER(pt_graph), c_void_p]),
 }
@@ -297,6 +301,20 @@ def pt_cross_entropy(ctx, logits, labels, n, classes, ld, loss_out, ws, stream=N
 
 def pt_set_coeff(ctx, loss, reg_sum, ratio, lambda_out, stream=None):
     _check(lib().pt_set_coeff(ctx.handle, _ptr(loss), _ptr(reg_sum), ratio, _ptr(lambda_out), _stream(stream)), "pt_set_coeff")
+
+
+def pt_dense_channel_list(ctx, zero_flags, n, idx, count, stream=None):
+    _check(lib().pt_dense_channel_list(ctx.handle, _ptr(zero_flags), n, _ptr(idx), _ptr(count), _stream(stream)), "pt_dense_channel_list")
+
+
+def pt_channel_gather(ctx, src, ld_src, c_src, idx, n_sel, dst, ld_dst, npix, stream=None):
+    _check(lib().pt_channel_gather(ctx.handle, _ptr(src), ld_src, c_src, _ptr(idx), n_sel, _ptr(dst), ld_dst, npix, _stream(stream)),
+           "pt_channel_gather")
+
+
+def pt_channel_scatter_add(ctx, branch, ld_branch, idx, n_sel, node_in, node_out, ld_node, c_node, npix, relu, stream=None):
+    _check(lib().pt_channel_scatter_add(ctx.handle, _ptr(branch), ld_branch, _ptr(idx), n_sel, _ptr(node_in),
+                                        _ptr(node_out), ld_node, c_node, npix, 1 if relu else 0, _stream(stream)), "pt_channel_scatter_add")
 
 
 class GraphHandle:

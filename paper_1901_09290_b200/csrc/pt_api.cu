@@ -100,7 +100,7 @@ extern "C" pt_status pt_poll_device_status(pt_ctx *c, void *stream)
     if (code != PT_DEV_OK) {
         PT_CUDA_OK(cudaMemsetAsync(c->d_status, 0, 16, st));
         PT_CUDA_OK(cudaStreamSynchronize(st));
-        return code == PT_DEV_TIMEOUT ? PT_ERR_TIMEOUT : PT_ERR_CUDA;
+        return code == PT_DEV_TIMEOUT ? PT_ERR_TIMEOUT : code == PT_DEV_BAD_INDEX ? PT_ERR_INVALID_ARG : PT_ERR_CUDA;
     }
     return PT_OK;
 }

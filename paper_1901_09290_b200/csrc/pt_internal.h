@@ -15,7 +15,7 @@
     } while (0)
 
 // Device status word layout: [0] = first error code recorded (0 = none), [1] = detail (where), [2..3] spare.
-enum { PT_DEV_OK = 0, PT_DEV_TIMEOUT = 1 };
+enum { PT_DEV_OK = 0, PT_DEV_TIMEOUT = 1, PT_DEV_BAD_INDEX = 2 };
 
 struct pt_region {              // one cached table in the arena
     size_t off = 0, cap = 0;    // byte range inside the arena

@@ -29,7 +29,10 @@ def main():
     ap.add_argument("--wgrad-ctas", type=int, default=0, help="CTA limit of the weight-gradient kernels (0 = one per SM)")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches (includes host launch cost)")
     ap.add_argument("--bn", default=None, help="N,H,C: time pt_bn_relu_fwd / pt_bn_relu_bwd instead of a convolution")
+    ap.add_argument("--gate", default=None, help="N,H,C,S: time pt_channel_gather / pt_channel_scatter_add of S of a node's C channels")
     args = ap.parse_args()
+    if args.gate:
+        return gate_main(args)
     if args.bn:
         return bn_main(args)
     if args.shape:
@@ -134,6 +137,46 @@ def bn_main(args):
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) * 1e3 / args.iters
         by = elems * (6 if ps == "fwd" else 10)
+        out[ps] = {"us": round(us, 2), "gbs": round(by / us / 1e3, 1)}
+    ctx.poll()
+    print(json.dumps(out))
+
+
+def gate_main(args):
+    """Channel gating on one node tensor: device time and GB/s of the bytes that must move (gather: the selected channels
+    in and out, 4 B per selected element; scatter-add: node in, branch in, node out)."""
+    N, H, C, S = [int(t) for t in args.gate.split(",")]
+    ld_n, ld_s = W.pad8(C), W.pad8(S)
+    npix = N * H * H
+    ctx = B.Context(0)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    idx = torch.sort(torch.randperm(C, generator=g, device="cuda")[:S])[0].to(torch.int32)
+    mk = lambda ld: torch.randn((npix, ld), generator=g, device="cuda").to(torch.bfloat16)
+    sets = [(mk(ld_n), mk(ld_s), mk(ld_n)) for _ in range(args.sets)]
+    out = {"gate": args.gate}
+    for ps in ("gather", "scatter_add"):
+        def run(i):
+            node, br, res = sets[i % len(sets)]
+            if ps == "gather":
+                B.pt_channel_gather(ctx, node, ld_n, C, idx, S, br, ld_s, npix)
+            else:
+                B.pt_channel_scatter_add(ctx, br, ld_s, idx, S, node, res, ld_n, C, npix, 1)
+        for i in range(3):
+            run(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            for i in range(args.iters):
+                run(i)
+        gr.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        gr.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / args.iters
+        by = npix * (4 * S if ps == "gather" else 4 * C + 2 * S)
         out[ps] = {"us": round(us, 2), "gbs": round(by / us / 1e3, 1)}
     ctx.poll()
     print(json.dumps(out))

@@ -127,6 +127,25 @@ def bottleneck_stage3(H: int = 28) -> Net:
     return b.net
 
 
+def vgg(depth: int = 16, image: int = 32) -> Net:
+    """Plain VGG-style stack (Tab. 1 trains VGG-11 and VGG-13 on CIFAR): 3x3 stride-1 convolutions in five groups of
+    64..512 channels, a 2x2 pooling (not on the path) halving the map after each group, no short-cuts, so every channel
+    space has one writer and one reader. Batch normalisation after every convolution, hence no conv bias."""
+    cfg = {11: (1, 1, 2, 2, 2), 13: (2, 2, 2, 2, 2), 16: (2, 2, 3, 3, 3)}[depth]
+    b = _Builder(f"vgg{depth}")
+    prev = b.space("img", 3, fixed=True, stage=0)
+    H, inC, n = image, 3, 0
+    n_total = sum(cfg)
+    for gi, (reps, width) in enumerate(zip(cfg, (64, 128, 256, 512, 512))):
+        for _ in range(reps):
+            n += 1
+            sp = b.space(f"a{n}", width, fixed=(n == n_total), stage=gi + 1)
+            b.conv(f"conv{n}", inC, width, 3, 1, H, prev, sp)
+            prev, inC = sp, width
+        H = max(1, H // 2)
+    return b.net
+
+
 def single_layer(C=16, K=32, R=3, H=16, stride=1) -> Net:
     """One conv as a 2-space graph: the layer is the only reader of its input space and the
     only writer of its output space."""
@@ -194,6 +213,30 @@ def choose_kept(net: Net, kept_counts: Sequence[int], seed: int) -> List[np.ndar
     for s, k in zip(net.space_sizes, kept_counts):
         out.append(np.sort(g.permutation(s)[:k]).astype(np.int32))
     return out
+
+
+def per_layer_zero_masks(net: Net, kept_counts: Sequence[int], seed: int, extra: float = 0.1):
+    """(zero_out[layer], zero_in[layer]) uint8 masks with sparsity that differs between the convolutions sharing a space,
+    as learned sparsity does (Sec. 4.2: each later residual path adds new information to the shared node). Every space
+    gets a common core of kept_counts[s] dense channels; in a space with several members each member additionally keeps
+    each remaining channel with probability `extra`, independently. Private spaces (one writer, one reader) share the core
+    exactly."""
+    g = np.random.default_rng(seed)
+    cores = choose_kept(net, kept_counts, seed + 1)
+    zo = [np.ones(l.K, np.uint8) for l in net.layers]
+    zi = [np.ones(l.C, np.uint8) for l in net.layers]
+    for s, size in enumerate(net.space_sizes):
+        members = [(li, "out") for li, l in enumerate(net.layers) if l.out_space == s] + \
+                  [(li, "in") for li, l in enumerate(net.layers) if l.in_space == s]
+        shared = sum(1 for _, sd in members if sd == "out") > 1 or sum(1 for _, sd in members if sd == "in") > 1
+        for li, side in members:
+            m = zo[li] if side == "out" else zi[li]
+            m[cores[s]] = 0
+            if net.space_fixed[s]:
+                m[:] = 0
+            elif shared and extra > 0:
+                m[g.random(size) < extra] = 0
+    return zo, zi
 
 
 # --------------------------------------------------------------------------- tensors
