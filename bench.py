@@ -86,12 +86,19 @@ class ClockSampler:
 
 def workload(args):
     from paper_1901_09290_b200 import workloads as W
-    net = W.resnet50()
     seed = W.BASE_SEED + 4
-    if args.keep is not None:
+    if args.net != "resnet50":
+        # the paper's CIFAR models (Tab. 1) as extra workloads; the default and the headline stay the ImageNet ResNet-50
+        net = W.resnet32() if args.net == "resnet32" else W.vgg(int(args.net[3:]))
+        keep = 0.6 if args.keep is None else args.keep
+        counts = W.uniform_keep(net, keep)
+        name = f"{args.net}-32x32-uniform-keep-{keep:g}"
+    elif args.keep is not None:
+        net = W.resnet50()
         counts = W.uniform_keep(net, args.keep)
         name = f"resnet50-uniform-keep-{args.keep:g}"
     else:
+        net = W.resnet50()
         counts = W.staged_keep_to_flops(net, seed, 0.60)
         name = "resnet50-224-53conv-keep-drawn-to-0.60-flops"
     kept = W.choose_kept(net, counts, seed)
@@ -215,7 +222,7 @@ def run_ours(args):
     # averaged by one NCCL all-reduce before the update.
     dp = world > 1 and args.data_parallel
     ts = harness.TrainStep(ctx, net, counts, kept, args.batch, seed + (0 if dp else 17 * rank), algo=args.algo, host_inputs=True,
-                           world=world if dp else 1)
+                           world=world if dp else 1, wgrad_ctas=args.wgrad_ctas, wgrad_streams=args.wgrad_streams)
     flops = ts.conv_flops()
     tot_flops = sum(flops.values())
     stream = torch.cuda.current_stream()
@@ -407,7 +414,7 @@ def run_ours(args):
                      "achieved": dom_flops / dom_t / 1e12, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": dom_flops / dom_t / tc_peak,
                      # DRAM bytes of the pass's launches in one ncu capture of the default workload (profiles/step_launch_list_*)
-                     "traffic": NCU_DRAM_BYTES.get(dom) if (args.keep is None and args.batch == 64 and args.algo == 0) else None,
+                     "traffic": NCU_DRAM_BYTES.get(dom) if (args.net == "resnet50" and args.keep is None and args.batch == 64 and args.algo == 0) else None,
                      "algorithmic_bytes": sum(ts.layer_bytes(li, which_id[dom]) for li in range(nL) if not (dom == "dgrad" and li == 0)),
                      "peak_source": pk["source"] + " sustained bf16"},
     }
@@ -440,6 +447,11 @@ def main():
     ap.add_argument("--data-parallel", action="store_true",
                     help="N > 1: average the weight gradients over the ranks with one NCCL all-reduce per step (default: replicas)")
     ap.add_argument("--keep", type=float, default=None, help="uniform keep ratio instead of the seeded per-space draw")
+    ap.add_argument("--net", default="resnet50", choices=["resnet50", "resnet32", "vgg11", "vgg13", "vgg16"],
+                    help="shape table; resnet50 (224x224) is the headline workload, the others are the paper's 32x32 CIFAR models")
+    ap.add_argument("--wgrad-ctas", type=int, default=49, help="CTA limit of a weight-gradient launch")
+    ap.add_argument("--wgrad-streams", type=int, default=3,
+                    help="streams the weight gradients go round-robin on; streams x CTA limit must not exceed the SM count")
     ap.add_argument("--algo", type=int, default=0)
     ap.add_argument("--per-layer", default=None, help="write the per-layer table (JSON) here")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -66,7 +66,11 @@ uint64_t pt_launch_count(const pt_ctx *ctx);
  * independent of each other: launches that leave SMs free can run side by side on several streams, which amortises their
  * fixed cost (pipeline fill, partial-tile exchange). The setting changes the workspace pt_conv_workspace_bytes reports for
  * PT_CONV_WGRAD, so set it before sizing workspaces; it has no effect on results beyond the summation order of the splits
- * (still fixed for a given setting). PT_ERR_INVALID_ARG if max_ctas is negative. */
+ * (still fixed for a given setting). PT_ERR_INVALID_ARG if max_ctas is negative.
+ * The CTAs of a split launch wait (bounded) for one another and occupy an SM each, so all of them must be able to be on
+ * the device at once: a caller that keeps weight-gradient launches in flight on S streams sets a limit L with
+ * S * L <= the SM count. Beyond that the launches may starve each other until a wait expires (PT_ERR_TIMEOUT at the next
+ * pt_poll_device_status; nothing hangs). */
 pt_status pt_set_wgrad_cta_limit(pt_ctx *ctx, int max_ctas);
 
 /* ------------------------------------------------------------------------------------------

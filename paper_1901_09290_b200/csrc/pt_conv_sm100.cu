@@ -1712,6 +1712,12 @@ void halo_spec_stride1(const pt_conv_desc *d, HaloSpec *h, const void *src, int 
     h->oH = P; h->oW = Q; h->o_step = 1; h->o_h0 = 0; h->o_w0 = 0;
 }
 
+// A CTA of a split weight gradient holds its tensor memory while it waits for the other splits of its tile. Two such CTAs
+// on one SM could block each other's tensor-memory allocation (the second allocation waits for columns the first one
+// frees only after a CTA that cannot start has arrived), so a split launch asks for more than half of an SM's shared
+// memory: at most one of them per SM, whatever else runs beside it (kernels that wait for nobody always finish).
+constexpr size_t kSplitSmemFloor = 116 * 1024;
+
 // Taps handled by one weight-gradient CTA: they share the dy tile and get one TMEM accumulator of BN columns each.
 // Bounded by the 512 TMEM columns and by a stage of 16 KB (dy) + taps x BN/64 x 8 KB (x) staying at or below 48 KB, so
 // that at least four pipeline stages fit (measured: with two stages the kernel is slower than with one tap per CTA);
@@ -1891,6 +1897,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
     const size_t stage = 2 * 8192 + (size_t)p.tpc * pt_ceil_div(p.BN, 64) * 8192;
     p.stages = pick_stages(stage, pt_ceil_div(p.pix_per_split, 64), 0, &smem);
     if (smem < 2048 + 8 * 2 * 4096) smem = 2048 + 8 * 2 * 4096;        // the epilogue's staging slabs reuse the stage memory
+    if (p.splits > 1 && smem < kSplitSmemFloor) smem = kSplitSmemFloor;
     static bool attr_set = false;
     if (!attr_set) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
@@ -1946,7 +1953,8 @@ pt_status run_wgrad_rows(pt_ctx *c, const pt_conv_desc *d, int P, int Q, const v
         attr_set = true;
     }
     dim3 grid((unsigned)gx, (unsigned)p.splits);
-    PT_CUDA_OK(launch_pdl(conv_wgrad_rows_kernel, grid, dim3(kThreads), wr.smem, st, tmA, tmX, tmP, p));
+    const size_t smem = (p.splits > 1 && wr.smem < kSplitSmemFloor) ? kSplitSmemFloor : wr.smem;
+    PT_CUDA_OK(launch_pdl(conv_wgrad_rows_kernel, grid, dim3(kThreads), smem, st, tmA, tmX, tmP, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;

@@ -127,11 +127,13 @@ class TrainStep:
 
     def __init__(self, ctx: B.Context, dense_net: W.Net, counts: Sequence[int], kept, N: int, seed: int,
                  algo: int = 0, host_inputs: bool = False, decoys: int = 2, device_rng: bool = True,
-                 wgrad_ctas: int = 74, wgrad_streams: int = 3, world: int = 1):
+                 wgrad_ctas: int = 49, wgrad_streams: int = 3, world: int = 1):
         self.ctx, self.N, self.algo = ctx, N, algo
         self.world = world          # > 1: data parallel, the weight gradients are averaged over the ranks before the update
         # weight gradients of different layers are independent: each launch is held to `wgrad_ctas` CTAs and the launches
-        # go round-robin to `wgrad_streams` streams, each with a workspace of its own
+        # go round-robin to `wgrad_streams` streams, each with a workspace of its own. The CTAs of a split weight gradient
+        # wait for one another, one per SM, so streams x limit stays within the SM count (3 x 49 <= 148): every launch
+        # that can be in flight then fits on the device together, whatever order the hardware picks its CTAs in.
         self.wgrad_ctas, self.wgrad_streams = wgrad_ctas, max(1, wgrad_streams)
         ctx.set_wgrad_cta_limit(wgrad_ctas)
         self.dense_net = dense_net

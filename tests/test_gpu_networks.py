@@ -41,6 +41,46 @@ def test_config2_resnet32_every_layer_batch128():
         _full_layer_check(l, 128, W.layer_seed(2, li), li == 0)
 
 
+def test_vgg13_plain_stack_every_layer_batch32():
+    """The paper's second model family (Tab. 1: VGG on CIFAR): a plain 3x3 stack without short-cuts, pruned."""
+    net = W.vgg(13)
+    counts = W.random_keep(net, W.BASE_SEED + 8)
+    pruned = W.with_sizes(net, counts)
+    for li, l in enumerate(pruned.layers):
+        _full_layer_check(l, 32, W.layer_seed(8, li), li == 0)
+
+
+def test_vgg11_training_step_on_a_network_without_shortcuts():
+    """The multi-stream, graph-replayed step on a plain stack: every weight gradient equals the single call on the same
+    buffers, and the last layer's outputs agree with the oracle on the weights the step started from."""
+    ctx = Hh.ctx()
+    net = W.vgg(11)
+    seed = W.BASE_SEED + 8
+    counts = W.uniform_keep(net, 0.6)
+    kept = W.choose_kept(net, counts, seed)
+    ts = harness.TrainStep(ctx, net, counts, kept, 16, seed, host_inputs=False, device_rng=True)
+    ts.step()
+    torch.cuda.synchronize()
+    ts.build_graph(two_streams=True)
+    li = len(net.layers) - 1
+    l = ts.net.layers[li]
+    ts.step()
+    torch.cuda.synchronize()
+    ctx.poll()
+    # every step re-gathers the pruned model from the dense one before it trains: those are the weights the convs saw
+    w_before = oracle.gather_weight(ts.md.wb[li][..., :net.layers[li].C].float().cpu().numpy(), kept[l.out_space], kept[l.in_space])
+    x = ts.x[li][..., :l.C].float().cpu().numpy()
+    dy = ts.dy[li][..., :l.K].float().cpu().numpy()
+    Hh.check_conv(ts.y[li], l.K, oracle.conv_fwd(x, w_before, l.stride, l.pad), what="vgg fwd")
+    Hh.check_conv(ts.dx[li], l.C, oracle.conv_dgrad(dy, w_before, l.H, l.H, l.stride, l.pad), what="vgg dgrad")
+    for i in range(len(net.layers)):
+        g_step = ts.mp.g[i].clone()
+        ts.conv_wgrad(i)
+        torch.cuda.synchronize()
+        assert torch.equal(g_step, ts.mp.g[i]), net.layers[i].name
+    Hh.check_conv(ts.mp.g[li], l.C, oracle.conv_wgrad(x, dy, l.R, l.R, l.stride, l.pad), what="vgg wgrad")
+
+
 def test_config4_resnet50_every_layer_batch2():
     net = W.resnet50()
     counts = W.staged_keep_to_flops(net, W.BASE_SEED + 4)

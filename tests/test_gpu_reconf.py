@@ -117,6 +117,18 @@ def test_resnet32_union_with_decoys():
         assert keep[s].tolist() == kept[s].tolist()
 
 
+def test_vgg16_plain_stack_reconfiguration():
+    """No shared node anywhere: every space has one writer and one reader, and a channel goes only if both agree."""
+    net = W.vgg(16)
+    kept = W.choose_kept(net, W.random_keep(net, W.BASE_SEED + 8), W.BASE_SEED + 8)
+    model = W.gen_model(net, W.BASE_SEED + 8, kept=kept, decoys=2)
+    dm = DevModel(model)
+    dn, maps, sizes = reconfigure(dm)
+    keep = check_against_oracle(model, dm, dn, maps, sizes)
+    for s in range(len(kept)):
+        assert keep[s].tolist() == kept[s].tolist()
+
+
 def test_bottleneck_config3_counts():
     net = W.bottleneck_stage3()
     kept = W.choose_kept(net, [371, 93, 77], W.BASE_SEED + 3)
