@@ -431,6 +431,7 @@ struct HaloP {
     int a_box_bytes, a_alloc;            // bytes one A load brings / bytes reserved per A stage
     int stages_a, stages_b, resident;    // ring depths; resident: weights loaded once
     int n_issuers, acc_per;              // MMA issuer warps (each with its own A ring of stages_a / n_issuers stages); accumulators per issuer (1 or 2)
+    int row32;                           // 1: 16 channel lanes per pixel, 32-byte rows and swizzle (the space-to-depth stem): one MMA per tap
     int b_slot, b_rows, staging;         // bytes reserved per weight tile, rows a K-major weight box brings, bytes of an epilogue group's staging slab
     int tmem_cols, tma_store, out_f32, ld_out;
     int oH, oW, o_step, o_h0, o_w0;      // direct stores: raster (n, i, j) -> out[((n*oH + i*o_step + o_h0)*oW + j*o_step + o_w0)*ld_out]
@@ -441,6 +442,30 @@ struct HaloP {
 };
 
 constexpr int kHaloMaxIssuers = 4;
+
+// Coordinates of the tiles t0, t0 + D, t0 + 2D, ... of a halo launch, advanced without integer divisions (a division costs
+// a single issuing thread ~150 cycles, and the smallest tiles are only a few hundred cycles of work).
+struct TileWalk {
+    int n_tile, rt, img;          // channel tile, row tile within the image, image
+    int dn, d_rt, d_img, n_tiles, row_tiles;
+    __device__ __forceinline__ void init(int tile, int D, int n_tiles_, int row_tiles_)
+    {
+        n_tiles = n_tiles_; row_tiles = row_tiles_;
+        n_tile = tile % n_tiles;
+        const int m_tile = tile / n_tiles;
+        img = m_tile / row_tiles; rt = m_tile - img * row_tiles;
+        dn = D % n_tiles;
+        const int dm = D / n_tiles;
+        d_img = dm / row_tiles; d_rt = dm - d_img * row_tiles;
+    }
+    __device__ __forceinline__ void next()
+    {
+        n_tile += dn;
+        rt += d_rt; img += d_img;
+        if (n_tile >= n_tiles) { n_tile -= n_tiles; ++rt; }
+        while (rt >= row_tiles) { rt -= row_tiles; ++img; }
+    }
+};
 // Device-side timeline for tuning: a build with -DPT_DEVICE_TRACE makes CTA 0 stamp %globaltimer at the hand-over points of
 // each role (producer issue, accumulator free, operands landed, MMAs committed, epilogue start, store issued) and exports
 // pt_debug_halo_trace / pt_debug_wgrad_trace to read the stamps back. The normal build compiles the macros away.
@@ -480,7 +505,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     const uint32_t staging_base = (smem_base + (uint32_t)sizeof(HCtl) + 1023u) & ~1023u;
     const uint32_t b_base = staging_base + 2u * (uint32_t)p.staging;
     // bytes one weight tile brings: a K-major tile only holds the rows (output channels) that exist
-    const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.b_rows * 128u;
+    const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.b_rows * (p.row32 ? 32u : 128u);
     const uint32_t b_slot = (uint32_t)p.b_slot;
     const uint32_t n_bslots = p.resident ? (uint32_t)(p.taps * p.k_chunks) : (uint32_t)p.stages_b;
     const uint32_t a_base = b_base + n_bslots * b_slot;
@@ -502,7 +527,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         prefetch_tmap(&tmB);
         if (p.tma_store) prefetch_tmap(&tmC);
     }
-    if (threadIdx.x < p.taps) ctl->tap_aoff[threadIdx.x] = (uint32_t)(p.tap_oh[threadIdx.x] * p.Wp + p.tap_ow[threadIdx.x]) * 8u;
+    if (threadIdx.x < p.taps) ctl->tap_aoff[threadIdx.x] = (uint32_t)(p.tap_oh[threadIdx.x] * p.Wp + p.tap_ow[threadIdx.x]) * (p.row32 ? 2u : 8u);
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), (uint32_t)p.tmem_cols);
         tmem_relinquish();
@@ -535,25 +560,32 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
                     }
             }
-            int gb = 0, tc = pid;
+            int tc = pid;
+            TileWalk tw;
+            tw.init((int)blockIdx.x + pid * (int)gridDim.x, n_prod * (int)gridDim.x, p.n_tiles, p.row_tiles);
+            // ring = tc % NI; every ring has carried (tc / NI) * k_chunks chunks before its tile of this round: position and
+            // phase of that count in a ring of SR stages, advanced per round
+            int ring = pid % NI, base_pos = 0, base_ph = 0;
+            const int kdiv = p.k_chunks / SR, kmod = p.k_chunks - kdiv * SR;
+            int sb_pos = 0, sb_ph = 0;                         // position in this pipeline's weight ring
             for (int tile = blockIdx.x + pid * (int)gridDim.x; tile < total_tiles && !*abort_flag; tile += n_prod * (int)gridDim.x, tc += n_prod) {
-                const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
-                const int img = m_tile / p.row_tiles, p0 = (m_tile - img * p.row_tiles) * p.nr;
-                const int n0 = n_tile * p.BN;
-                const int ring = tc % NI;
-                int cnt = (tc / NI) * p.k_chunks;              // chunks this ring has carried before this tile
+                const int img = tw.img, p0 = tw.rt * p.nr;
+                const int n0 = tw.n_tile * p.BN;
                 bool ok = true;
-                for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++cnt) {
-                    const int sa = ring * SR + cnt % SR, pha = (cnt / SR) & 1;
-                    ok = mbar_wait(smem_u32(&ctl->empty_a[sa]), pha ^ 1, abort_flag, p.status, 11);
+                int pos = base_pos, pha = base_ph;
+                for (int kc = 0; kc < p.k_chunks && ok; ++kc) {
+                    const int sa = ring * SR + pos, ph_use = pha;
+                    if (++pos == SR) { pos = 0; pha ^= 1; }
+                    ok = mbar_wait(smem_u32(&ctl->empty_a[sa]), ph_use ^ 1, abort_flag, p.status, 11);
                     if (!ok) break;
                     const uint32_t bar = smem_u32(&ctl->full_a[sa]);
                     HTRACE(0, tc);
                     mbar_arrive_expect_tx(bar, (uint32_t)p.a_box_bytes);
                     tma_load_4d(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, &tmA, bar, kc * kKC, p.lo_w, p0 + p.lo_h, img);
                     if (p.resident) continue;
-                    for (int tap = 0; tap < p.taps; ++tap, ++gb) {
-                        const int sb = pid * SB + gb % SB, phb = (gb / SB) & 1;
+                    for (int tap = 0; tap < p.taps; ++tap) {
+                        const int sb = pid * SB + sb_pos, phb = sb_ph;
+                        if (++sb_pos == SB) { sb_pos = 0; sb_ph ^= 1; }
                         ok = mbar_wait(smem_u32(&ctl->empty_b[sb]), phb ^ 1, abort_flag, p.status, 12);
                         if (!ok) break;
                         const uint32_t bbar = smem_u32(&ctl->full_b[sb]);
@@ -565,6 +597,15 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                     }
                 }
                 if (!ok) break;
+                tw.next();
+                ring += n_prod;
+                while (ring >= NI) {                           // next round: every ring has carried k_chunks more
+                    ring -= NI;
+                    base_pos += kmod;
+                    int wraps = kdiv;
+                    if (base_pos >= SR) { base_pos -= SR; ++wraps; }
+                    base_ph ^= wraps & 1;
+                }
             }
             if (*abort_flag && pid == 0) {   // bounded drain of the copies in flight before the shared memory is released
                 const uint64_t t0 = globaltimer_ns();
@@ -579,7 +620,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         const uint32_t idesc = make_idesc_bf16(kBM, p.BN, 0, B_MN ? 1 : 0);
         const uint64_t bstep = B_MN ? 128ull : 2ull;
         const uint32_t b_lbo = B_MN ? 8192u : 16u;
-        int gb = 0;
+        int sb_pos = 0, sb_ph = 0;                            // position in this issuer's weight ring
         int s_loc = 0, pha = 0;                               // position in this issuer's A ring
         bool ok = true;
         if (p.resident) ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort_flag, p.status, 13);
@@ -604,7 +645,16 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                 const int rem = p.c_red - kc * kKC;
                 const int ksteps = rem >= kKC ? 4 : (rem + 15) / 16;
                 const uint64_t abase = make_desc(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, 16u, 1024u);
-                if (p.resident) {
+                if (p.row32) {
+                    // 32-byte rows: a pixel's 16 lanes are one K step, so a tap is a single MMA on the row-shifted tile
+                    const uint64_t a32 = make_desc_sw32(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, 256u);
+                    uint64_t b32 = make_desc_sw32(b_base, 256u);
+                    const uint64_t b_tap_step = (uint64_t)(b_slot >> 4);
+                    for (int tap = 0; tap < p.taps; ++tap, b32 += b_tap_step) {
+                        umma_bf16_lead(d_tmem, a32 + ctl->tap_aoff[tap], b32, idesc, accumulate, leader);
+                        accumulate = 1u;
+                    }
+                } else if (p.resident) {
                     // every tap is the same A tile read through a descriptor that starts (r*Wp + s) rows further on
                     uint64_t bd0 = make_desc(b_base + (uint32_t)kc * b_slot, b_lbo, 1024u);
                     const uint64_t b_tap_step = (uint64_t)(((uint32_t)p.k_chunks * b_slot) >> 4);
@@ -621,8 +671,9 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         }
                     }
                 } else {
-                    for (int tap = 0; tap < p.taps; ++tap, ++gb) {
-                        const int sb = issuer * SB + gb % SB, phb = (gb / SB) & 1;
+                    for (int tap = 0; tap < p.taps; ++tap) {
+                        const int sb = issuer * SB + sb_pos, phb = sb_ph;
+                        if (++sb_pos == SB) { sb_pos = 0; sb_ph ^= 1; }
                         ok = mbar_wait(smem_u32(&ctl->full_b[sb]), phb, abort_flag, p.status, 16);
                         if (!ok) break;
                         tc_fence_after();
@@ -646,17 +697,17 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         const int gtid = (warp - 2 - group * 4) * 32 + lane;         // 0..127 within the group
         const uint32_t slab = staging_base + (uint32_t)group * (uint32_t)p.staging;
         bool ok = true;
-        const int step = NI == 1 ? 1 : 2;                     // one issuer: the groups alternate tiles like its two buffers
-        for (int tc = group; ok; tc += 2) {
+        const int ni_shift = NI == 4 ? 2 : NI == 2 ? 1 : 0;   // NI is 1, 2 or 4
+        TileWalk tw;
+        tw.init((int)blockIdx.x + group * (int)gridDim.x, 2 * (int)gridDim.x, p.n_tiles, p.row_tiles);
+        for (int tc = group; ok; tc += 2, tw.next()) {
             const int tile = blockIdx.x + tc * (int)gridDim.x;
             if (tile >= total_tiles) break;
             // tile tc is the nt-th tile of issuer tc % NI (NI is 1 or even, so a group always serves the same issuers)
-            const int iss = NI == 1 ? 0 : tc % NI, nt = NI == 1 ? tc : tc / NI;
+            const int iss = tc & (NI - 1), nt = tc >> ni_shift;
             const int b = p.acc_per == 2 ? iss * 2 + (nt & 1) : iss, aph = p.acc_per == 2 ? (nt >> 1) & 1 : nt & 1;
-            (void)step;
-            const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
-            const int img = m_tile / p.row_tiles, p0 = (m_tile - img * p.row_tiles) * p.nr;
-            const int n0 = n_tile * p.BN;
+            const int img = tw.img, p0 = tw.rt * p.nr;
+            const int n0 = tw.n_tile * p.BN;
             ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 17);
             if (!ok) break;
             if (gtid == 0) HTRACE(4, tc);
@@ -1569,14 +1620,16 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
 }
 
 // Source activations as a tiled 4-D tensor (C, W, H, N): box 64 channels x box_w x box_h x 1 (the halo tile).
-bool make_halo_in_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, int W, int H, int N, int ld, int box_w, int box_h)
+// `lanes` = 64 (128-byte rows and swizzle) or 16 (32-byte rows and swizzle).
+bool make_halo_in_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, int W, int H, int N, int ld, int box_w, int box_h,
+                      int lanes = kKC)
 {
     if (!c->encode_tiled || box_w > 256 || box_h > 256) return false;
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
     cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)W * ld * 2, (cuuint64_t)H * W * ld * 2};
-    cuuint32_t box[4] = {(cuuint32_t)kKC, (cuuint32_t)box_w, (cuuint32_t)box_h, 1}, estr[4] = {1, 1, 1, 1};
+    cuuint32_t box[4] = {(cuuint32_t)lanes, (cuuint32_t)box_w, (cuuint32_t)box_h, 1}, estr[4] = {1, 1, 1, 1};
     CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box,
-                                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, lanes == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -1591,6 +1644,7 @@ struct HaloSpec {
     int tap_oh[kMaxTaps], tap_ow[kMaxTaps], tap_wt[kMaxTaps];
     int n_cols, ld_out;                              // output channels and pitch
     int oH, oW, o_step, o_h0, o_w0;                  // output view: raster (i, j) -> pixel (i*o_step + o_h0, j*o_step + o_w0) of oH x oW
+    int row32, w_taps;                               // 16-lane pixels (32-byte rows); taps per output channel in the weight tensor
 };
 
 template <bool B_MN>
@@ -1606,6 +1660,9 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     p.n_cols = h.n_cols;
     p.BN = tile_n(h.n_cols, &p.n_tiles);
     p.c_red = h.Cs; p.k_chunks = pt_ceil_div(h.Cs, kKC); p.taps = h.n_taps;
+    p.row32 = h.row32 ? 1 : 0;
+    const int row_bytes = h.row32 ? 32 : 128;
+    if (h.row32 && (B_MN || h.Cs != 16)) return PT_ERR_UNSUPPORTED;
     p.lo_h = h.lo_h; p.lo_w = h.lo_w;
     for (int t = 0; t < h.n_taps; ++t) {
         p.tap_oh[t] = (unsigned char)h.tap_oh[t]; p.tap_ow[t] = (unsigned char)h.tap_ow[t];
@@ -1613,16 +1670,16 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     }
     const int box_h = p.nr + h.span_h - 1;
     if (box_h > 256) return PT_ERR_UNSUPPORTED;
-    p.a_box_bytes = box_h * Wp * 128;
+    p.a_box_bytes = box_h * Wp * row_bytes;
     // The M = 128 MMAs of the last tap read up to this many rows; the rows past the box only feed raster positions that
     // are never stored, so consecutive A stages may overlap there (and a tail pad follows the last stage).
     const int need_rows = 128 + (h.span_h - 1) * Wp + h.span_w - 1;
     p.a_alloc = (int)pt_align_up((size_t)p.a_box_bytes, 1024);
-    const size_t a_tail = need_rows * 128 > p.a_alloc ? pt_align_up((size_t)need_rows * 128 - p.a_alloc, 1024) : 0;
+    const size_t a_tail = need_rows * row_bytes > p.a_alloc ? pt_align_up((size_t)need_rows * row_bytes - p.a_alloc, 1024) : 0;
     // a K-major weight box only brings the output channels that exist (in whole 8-row swizzle atoms); the MMA still reads
     // BN rows, the rest from whatever follows in shared memory: columns that are never stored
     p.b_rows = (int)pt_align_up((size_t)(p.BN < h.n_cols ? p.BN : h.n_cols), 8);
-    const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : (size_t)p.b_rows * 128;
+    const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : (size_t)p.b_rows * row_bytes;
     p.b_slot = (int)b_bytes;
     // epilogue staging: one slab of the tile's raster rows x 128 bytes per group (direct-store launches use none)
     p.staging = d->out_f32 ? 0 : (int)pt_align_up((size_t)(p.nr * Wp < 128 ? p.nr * Wp : 128) * 128, 1024);
@@ -1667,8 +1724,21 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     p.status = c->d_status;
     CUtensorMap tmA, tmB, tmC;
     memset(&tmC, 0, sizeof(tmC));
-    if (!make_halo_in_map(c, &tmA, h.src, h.Cs, h.Ws, h.Hs, d->N, h.lds, Wp, box_h)) return PT_ERR_CUDA;
-    if (!make_weight_map(c, &tmB, w, d->C, d->R * d->S, d->K, d->ldw, B_MN ? kKC : p.b_rows)) return PT_ERR_CUDA;
+    if (h.row32) {
+        if (!p.resident) return PT_ERR_UNSUPPORTED;
+        if (!make_halo_in_map(c, &tmA, h.src, h.Cs, h.Ws, h.Hs, d->N, h.lds, Wp, box_h, 16)) return PT_ERR_CUDA;
+        // weights [K][w_taps][16]: one 32-byte row per output channel and tap
+        cuuint64_t dims[3] = {16, (cuuint64_t)h.w_taps, (cuuint64_t)h.n_cols};
+        cuuint64_t strides[2] = {32, (cuuint64_t)h.w_taps * 32};
+        cuuint32_t box[3] = {16, 1, (cuuint32_t)p.b_rows}, estr[3] = {1, 1, 1};
+        CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w), dims, strides, box,
+                                                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
+                                                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+    } else {
+        if (!make_halo_in_map(c, &tmA, h.src, h.Cs, h.Ws, h.Hs, d->N, h.lds, Wp, box_h)) return PT_ERR_CUDA;
+        if (!make_weight_map(c, &tmB, w, d->C, d->R * d->S, d->K, d->ldw, B_MN ? kKC : p.b_rows)) return PT_ERR_CUDA;
+    }
     if (p.tma_store) {
         // the output view as a 4-D tensor (channels, raster columns, raster rows, images); strided when o_step > 1
         const size_t es = 2;
@@ -2117,6 +2187,21 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         stem_s2d_w_kernel<<<(unsigned)((sp.w2_elems + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)b, w2, d->K, d->R, d->S, d->C, d->ldw,
                                                                               sp.U, sp.V, sp.off);
         c->launches += 2;
+        if (!d->out_f32) {
+            // row-block form on 32-byte pixels: the U x V taps are row shifts of one staged tile (each xs byte read once)
+            HaloSpec h;
+            memset(&h, 0, sizeof(h));
+            h.src = xs; h.Cs = 16; h.Ws = sp.Wp; h.Hs = sp.Hs; h.lds = 16;
+            h.P = sp.P; h.Q = sp.Q;
+            h.n_taps = sp.U * sp.V; h.span_h = sp.U; h.span_w = sp.V;
+            h.lo_h = -sp.pl; h.lo_w = 0;
+            for (int t = 0; t < h.n_taps; ++t) { h.tap_oh[t] = t / sp.V; h.tap_ow[t] = t % sp.V; h.tap_wt[t] = (t / sp.V) * 4 + t % sp.V; }
+            h.n_cols = d->K; h.ld_out = d->ldy;
+            h.oH = sp.P; h.oW = sp.Q; h.o_step = 1; h.o_h0 = 0; h.o_w0 = 0;
+            h.row32 = 1; h.w_taps = sp.U * 4;
+            const pt_status r = launch_halo<false>(c, d, h, w2, out, st);
+            if (r != PT_ERR_UNSUPPORTED) return r;
+        }
         p.M_total = d->N * sp.P * sp.Q;
         p.n_cols = d->K;
         p.BN = tile_n(d->K, &p.n_tiles);

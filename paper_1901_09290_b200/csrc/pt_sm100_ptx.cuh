@@ -174,6 +174,19 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
+// The same for the 32-byte swizzle, K-major only: rows of 32 B (16 bf16 along K: exactly one MMA K step), 8-row groups
+// `sbo_bytes` (256 for a dense tile) apart.
+__device__ __forceinline__ uint64_t make_desc_sw32(uint32_t saddr, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3ffffu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)6 << 61;      // SWIZZLE_32B
+    return d;
+}
+
 // Instruction descriptor: bf16 x bf16 -> fp32, M x N tile, operand majors (0 = K-major, 1 = MN-major).
 __host__ __device__ __forceinline__ uint32_t make_idesc_bf16(int M, int N, int a_mn, int b_mn)
 {
