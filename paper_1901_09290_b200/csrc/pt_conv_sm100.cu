@@ -1587,7 +1587,7 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     // accumulator buffers = epilogue groups: three when 3 * BN fits the 512 TMEM columns, else two; narrow layers whose
     // CTAs get a single tile need no more than that
     p.epi_groups = 3 * p.BN <= 512 ? 3 : 2;
-    if (per_cta < p.epi_groups) p.epi_groups = per_cta < 2 ? 2 : per_cta;
+    if (per_cta < p.epi_groups) p.epi_groups = per_cta;           // a single tile per CTA: one group, and its staging goes to the ring
     // Small weights (one channel tile, all taps x chunks within 64 KB) stay resident: the ring then carries A tiles only and
     // holds more of them, which is what an activation-bound layer needs to cover the memory latency.
     const size_t w_all = (size_t)p.taps * p.k_chunks * b_bytes;
