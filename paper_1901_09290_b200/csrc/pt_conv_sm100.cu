@@ -70,6 +70,7 @@ struct GemmP {
     int resident;       // 1: every weight tile of the launch stays in shared memory (loaded once); the ring carries A only
     int n_issuers;      // 2 (resident weights only): two MMA issuer warps take alternate tiles, each with half of the ring's stages
     int acc_per;        // two issuers: accumulator buffers per issuer (1 or 2)
+    int alias_staging;  // 1: the CTA has a single tile; the epilogue's staging slabs lie in the (then idle) ring
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
@@ -113,7 +114,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     const uint32_t b_bytes = B_MN ? (uint32_t)((p.BN + 63) / 64) * 8192u : (uint32_t)p.BN * 128u;
     const uint32_t b_slot = (b_bytes + 1023u) & ~1023u;
     // resident weights: all taps x chunks sit in front of the ring, whose stages then hold an A tile only
-    const uint32_t w_base = staging_base + (uint32_t)p.epi_groups * 4u * kSlabs * 4096u;
+    // a CTA with a single tile stages its output in the ring, which is idle by then: no separate staging area
+    const uint32_t w_base = staging_base + (p.alias_staging ? 0u : (uint32_t)p.epi_groups * 4u * kSlabs * 4096u);
     const uint32_t stage_bytes = p.resident ? a_bytes : a_bytes + b_slot;
     const uint32_t data_base = w_base + (p.resident ? (uint32_t)(p.taps * p.k_chunks) * b_slot : 0u);
     volatile int *abort_flag = &ctl->abort_flag;
@@ -267,7 +269,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; group g drains accumulator buffer g,
         // i.e. the tiles tc = g, g + G, g + 2G, ... of this CTA
         const int quarter = warp & 3, group = (warp - 2) >> 2, G = p.epi_groups;
-        const uint32_t slab0 = staging_base + (uint32_t)(warp - 2) * (kSlabs * 4096u);
+        const uint32_t slab0 = (p.alias_staging ? data_base : staging_base) + (uint32_t)(warp - 2) * (kSlabs * 4096u);
         int tc = group, sl = 0;
         bool ok = true;
         for (int tile = blockIdx.x + group * gridDim.x; tile < total_tiles && ok; tile += G * gridDim.x, tc += G) {
@@ -1599,7 +1601,10 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
         p.epi_groups = 2;
         p.acc_per = 4 * p.BN <= 512 ? 2 : 1;
     }
-    const size_t staging2 = (size_t)p.epi_groups * 4 * kSlabs * 4096;
+    // one tile per CTA and streamed weights: the output is staged in the ring (all of its stages have been consumed when the
+    // accumulator is complete), which leaves room for one more stage
+    p.alias_staging = (per_cta == 1 && !p.resident) ? 1 : 0;
+    const size_t staging2 = p.alias_staging ? 0 : (size_t)p.epi_groups * 4 * kSlabs * 4096;
     if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all, &smem);
     else p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2, &smem);
     if (p.n_issuers == 2) {
