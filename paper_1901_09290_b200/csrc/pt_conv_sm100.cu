@@ -123,10 +123,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int iters = p.taps * p.k_chunks;
     const int total_tiles = p.m_tiles * p.n_tiles;
+    // streamed MN-major weight tiles are one 8 KB box per 64 columns: with several boxes per stage a second producer warp
+    // (warp 15, otherwise idle without resident weights) issues every other one
+    const int nb_b = (p.BN + 63) / 64;
+    const bool two_b = B_MN && !p.resident && nb_b > 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), p.resident ? 1 : 2);   // the A producer and, with streamed weights, the B producer
+            mbar_init(smem_u32(&ctl->full[s]), p.resident ? 1 : (two_b ? 3 : 2));   // the A producer and, with streamed weights, the B producer(s)
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->w_full), 1);
@@ -151,12 +155,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     grid_dependency_wait();              // nothing above touches global memory
     grid_launch_dependents();
 
-    if (warp == 0 || warp == 14) {
+    if (warp == 0 || warp == 14 || (warp == 15 && two_b)) {
         if (lane == 0) {
             // ---------------- TMA producers: warp 0 brings the A tile of every stage, warp 14 the B tile (issuing a TMA
             // instruction costs its thread about 200 cycles, so the two operands are issued side by side)
             const bool is_a = warp == 0;
-            const uint32_t my_bytes = is_a ? a_bytes : b_bytes;
+            const int bsel = warp == 15 ? 1 : 0, nbp = two_b ? 2 : 1;         // this B producer's boxes: bsel, bsel + nbp, ...
+            const uint32_t my_bytes = is_a ? a_bytes : (two_b ? (uint32_t)((nb_b + 1 - bsel) / 2) * 8192u : b_bytes);
             int s = 0, ph = 0, issued = 0;   // stage-ring position, continuous across tiles
             int s1 = 0, ph1 = 0;             // position in the second issuer's ring
             const int SR = p.stages / p.n_issuers;
@@ -201,7 +206,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         } else if (!B_MN) {
                             tma_load_3d(b_dst, &tmB, bar, kc * kKC, wtap, n0);
                         } else {
-                            for (int nb = 0; nb < (p.BN + 63) / 64; ++nb)
+                            for (int nb = bsel; nb < nb_b; nb += nbp)
                                 tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
                         }
                         ++issued;
