@@ -286,6 +286,43 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             }
             const int n_tile = tile % p.n_tiles, m_tile = tile / p.n_tiles;
             const int m0 = m_tile * kBM, n0 = n_tile * p.BN;
+            // direct stores: this thread's raster pixel and where it lands in the output view
+            const int m = m0 + quarter * 32 + lane;
+            const bool row_ok = !p.tma_store && m < p.M_total;
+            size_t row_off = 0;
+            int cell_h = 0, cell_w = 0, img = 0;
+            if (row_ok) {
+                const int j = m % p.Qd, t = m / p.Qd, i = t % p.Pd;
+                img = t / p.Pd;
+                cell_h = i * p.o_step;
+                cell_w = j * p.o_step;
+                row_off = ((size_t)(img * p.oH + cell_h + p.o_h0) * p.oW + cell_w + p.o_w0) * (size_t)p.ld_out;
+            }
+            if (!p.tma_store && p.zero_mask && n_tile == 0) {
+                // stride-2 data gradient: the pixels of each 2x2 cell that no tap reaches are zeros. They do not depend on the
+                // accumulator, so the warp writes them (a row at a time, lanes on consecutive 16-byte pieces) while the
+                // main loop is still running
+                for (int r = 0; r < 32; ++r) {
+                    if (!__shfl_sync(0xffffffffu, row_ok ? 1 : 0, r)) continue;
+                    const int ch_ = __shfl_sync(0xffffffffu, cell_h, r), cw_ = __shfl_sync(0xffffffffu, cell_w, r);
+                    const int im_ = __shfl_sync(0xffffffffu, img, r);
+                    for (int ab = 0; ab < 4; ++ab) {
+                        if (!((p.zero_mask >> ab) & 1)) continue;
+                        const int hh = ch_ + (ab >> 1), ww = cw_ + (ab & 1);
+                        if (hh >= p.oH || ww >= p.oW) continue;
+                        const size_t off = ((size_t)(im_ * p.oH + hh) * p.oW + ww) * (size_t)p.ld_out;
+                        if (p.out_f32) {
+                            float *o = (float *)p.out + off;
+                            for (int e = lane; e < p.n_cols; e += 32) o[e] = 0.f;
+                        } else {
+                            __nv_bfloat16 *o = (__nv_bfloat16 *)p.out + off;
+                            const int whole = p.n_cols & ~7;
+                            for (int e = lane * 8; e < whole; e += 256) *reinterpret_cast<uint4 *>(o + e) = make_uint4(0, 0, 0, 0);
+                            if (lane < p.n_cols - whole) o[whole + lane] = __float2bfloat16_rn(0.f);
+                        }
+                    }
+                }
+            }
             ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 3);
             if (!ok) break;
             tc_fence_after();
@@ -338,17 +375,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                 continue;
             }
             // ---- direct stores (fp32 outputs, strided stride-2 data-gradient outputs)
-            const int m = m0 + quarter * 32 + lane;
-            const bool row_ok = m < p.M_total;
-            size_t row_off = 0;
-            int cell_h = 0, cell_w = 0, img = 0;
-            if (row_ok) {
-                const int j = m % p.Qd, t = m / p.Qd, i = t % p.Pd;
-                img = t / p.Pd;
-                cell_h = i * p.o_step;
-                cell_w = j * p.o_step;
-                row_off = ((size_t)(img * p.oH + cell_h + p.o_h0) * p.oW + cell_w + p.o_w0) * (size_t)p.ld_out;
-            }
             for (int c0 = 0; c0 < p.BN; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld16(lane_addr + (uint32_t)c0, v);
@@ -389,24 +415,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         } else {
                             for (int e = 8 * g; e < nvalid; ++e) o[e] = __float2bfloat16_rn(__uint_as_float(v[e]));
                         }
-                    }
-                }
-            }
-            // stride-2 data gradient: pixels of this 2x2 cell that no tap reaches are written as zeros here
-            if (row_ok && p.zero_mask && n_tile == 0) {
-                for (int ab = 0; ab < 4; ++ab) {
-                    if (!((p.zero_mask >> ab) & 1)) continue;
-                    const int hh = cell_h + (ab >> 1), ww = cell_w + (ab & 1);
-                    if (hh >= p.oH || ww >= p.oW) continue;
-                    const size_t off = ((size_t)(img * p.oH + hh) * p.oW + ww) * (size_t)p.ld_out;
-                    if (p.out_f32) {
-                        float *o = (float *)p.out + off;
-                        for (int e = 0; e < p.n_cols; ++e) o[e] = 0.f;
-                    } else {
-                        __nv_bfloat16 *o = (__nv_bfloat16 *)p.out + off;
-                        int e = 0;
-                        for (; e + 8 <= p.n_cols; e += 8) *reinterpret_cast<uint4 *>(o + e) = make_uint4(0, 0, 0, 0);
-                        for (; e < p.n_cols; ++e) o[e] = __float2bfloat16_rn(0.f);
                     }
                 }
             }
