@@ -1536,14 +1536,29 @@ bool make_weight_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, 
 // 64 (the TMA-store chunk) chosen to waste the fewest padded columns.
 int tile_n(int cols, int *n_tiles, int m_tiles = 1 << 30, int sms = 0)
 {
-    (void)m_tiles; (void)sms;
-    if (cols <= 256) { *n_tiles = 1; return pt_ceil_div(cols, 16) * 16; }
-    int best = 256, best_pad = 1 << 30;
-    for (int bn = 256; bn >= 128; bn -= 64) {
-        int pad = pt_ceil_div(cols, bn) * bn;
-        if (pad < best_pad) { best_pad = pad; best = bn; }
+    int best = 256;
+    if (cols <= 256) {
+        *n_tiles = 1;
+        best = pt_ceil_div(cols, 16) * 16;
+    } else {
+        int best_pad = 1 << 30;
+        for (int bn = 256; bn >= 128; bn -= 64) {
+            int pad = pt_ceil_div(cols, bn) * bn;
+            if (pad < best_pad) { best_pad = pad; best = bn; }
+        }
+        *n_tiles = pt_ceil_div(cols, best);
     }
-    *n_tiles = pt_ceil_div(cols, best);
+    if (sms <= 0 || m_tiles >= sms) return best;
+    // Few pixel tiles (the 7x7 maps): a CTA's time is what it streams per reduction stage -- the 16 KB activation tile plus
+    // bn x 128 bytes of weights -- times the waves of tiles. Narrower channel tiles put more SMs to work and cut the weight
+    // bytes per CTA; the activation tile is then read by more CTAs, from L2. Taken when the estimate drops by 10 % or more.
+    long long cost0 = (long long)pt_ceil_div(m_tiles * *n_tiles, sms) * (16 * 1024 + (long long)pt_ceil_div(best, 64) * 8192);
+    for (int bn = 192; bn >= 64; bn -= 64) {
+        if (bn >= best) continue;
+        const int nt = pt_ceil_div(cols, bn);
+        const long long cost = (long long)pt_ceil_div(m_tiles * nt, sms) * (16 * 1024 + (long long)bn * 128);
+        if (cost * 10 <= cost0 * 9) { cost0 = cost; best = bn; *n_tiles = nt; }
+    }
     return best;
 }
 
