@@ -1854,7 +1854,7 @@ int wgrad_splits(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     return (int)s;
 }
 
-// Plan of the row-block weight gradient (stride-1 filters with several taps); ok = 0 where the generic kernel is used.
+// Plan of the row-block weight gradient (stride-1 filters with at most 64 input channels); ok = 0 where the generic kernel is used.
 struct WgRows {
     int ok;
     int bn, n_tiles, m_tiles, tpc, tap_groups, apc, acc_cols;
@@ -1868,7 +1868,11 @@ WgRows wgrad_rows_plan(const pt_ctx *c, const pt_conv_desc *d, int P, int Q)
     WgRows w;
     memset(&w, 0, sizeof(w));
     const int taps = d->R * d->S;
-    if (d->stride != 1 || taps < 2 || taps > kMaxTaps) return w;
+    if (d->stride != 1 || taps > kMaxTaps) return w;
+    // a 1x1 filter has no halo to save, but the orientation (x on the M side, all of dy's channels on the N side: one tile
+    // where the generic kernel needs two for K > 128) and the plain tiled loads (no im2col boxes on 96-byte pixel pitches)
+    // still pay on large maps (56x56, 59 -> 143: 53 -> 31 us at 49 CTAs); small maps have too few units to split
+    if (taps < 2 && P * Q < 784) return w;
     w.Wp = Q + d->S - 1;
     if (w.Wp > 256 || P < 1 || Q < 1) return w;
     // paired form only: the x tile is the M side (two taps x 64 channel lanes), dy's output channels the N side

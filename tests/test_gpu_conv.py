@@ -92,6 +92,8 @@ def test_config3_pruned_bottleneck(algo):
 ROW_BLOCK = [
     (3, 12, 12, 20, 100, 3, 1), (2, 10, 14, 64, 200, 3, 1), (2, 9, 9, 6, 10, 5, 2), (1, 8, 120, 9, 12, 3, 1),
     (2, 11, 11, 13, 21, 3, 0), (2, 7, 7, 5, 9, 3, 2), (2, 6, 6, 33, 40, 2, 0), (64, 20, 20, 38, 38, 3, 1),
+    # 1x1 filters on large maps take the same kernel (single tap, K > 128 in one tile)
+    (3, 30, 30, 59, 143, 1, 0), (2, 28, 28, 7, 19, 1, 0), (2, 40, 33, 64, 250, 1, 0),
 ]
 
 
