@@ -830,6 +830,7 @@ struct WgradP {
     int pix_per_split;      // multiple of 64
     int splits;
     int Pd, Qd, stride, lo_h, lo_w, S;
+    int x_tiled;            // 1: 1x1 stride-1 filter without padding: x is a plain 2-D (channels, pixels) tiled map
     int stages, tmem_cols;
     // row-block form (stride-1 filters with several taps): a stage is `nr` output rows of one image
     int nr, Wp, RB;         // rows per unit, row pitch of both staged tiles in pixels (Q + S - 1), units per image
@@ -1157,8 +1158,14 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                     if (second) tma_load_2d(a_dst + 8192u, &tmDy, bar, k0 + 64, pix);
                 } else {
                     const int w = q * p.stride + p.lo_w, h = pp * p.stride + p.lo_h;
-                    tma_load_im2col_4d(b_dst + (uint32_t)box_dst[0], &tmX, bar, box_c[0], w, h, n, box_sw[0], box_sh[0]);
-                    if (n_mine > 1) tma_load_im2col_4d(b_dst + (uint32_t)box_dst[1], &tmX, bar, box_c[1], w, h, n, box_sw[1], box_sh[1]);
+                    if (p.x_tiled) {
+                        const int pix = pix_beg + it * 64;
+                        tma_load_2d(b_dst + (uint32_t)box_dst[0], &tmX, bar, box_c[0], pix);
+                        if (n_mine > 1) tma_load_2d(b_dst + (uint32_t)box_dst[1], &tmX, bar, box_c[1], pix);
+                    } else {
+                        tma_load_im2col_4d(b_dst + (uint32_t)box_dst[0], &tmX, bar, box_c[0], w, h, n, box_sw[0], box_sh[0]);
+                        if (n_mine > 1) tma_load_im2col_4d(b_dst + (uint32_t)box_dst[1], &tmX, bar, box_c[1], w, h, n, box_sw[1], box_sh[1]);
+                    }
                     q += dq; pp += dp; n += dn;                       // the next stage starts 64 pixels further on
                     if (q >= p.Qd) { q -= p.Qd; ++pp; }
                     if (pp >= p.Pd) { pp -= p.Pd; ++n; }
@@ -1958,10 +1965,11 @@ bool make_partial_map(const pt_ctx *c, CUtensorMap *tm, void *ws, int bn, size_t
 
 // Launches the weight-gradient kernel for a problem whose x operand is described by `tmX` (64 pixels x 64 channels boxes).
 pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, int lo_h, int lo_w, const CUtensorMap &tmX,
-                    const void *dy, float *out, void *ws, size_t ws_bytes, cudaStream_t st)
+                    const void *dy, float *out, void *ws, size_t ws_bytes, cudaStream_t st, bool x_tiled = false)
 {
     WgradP p;
     memset(&p, 0, sizeof(p));
+    p.x_tiled = x_tiled ? 1 : 0;
     p.K = d->K; p.C = d->C; p.taps = d->R * d->S; p.S = d->S;
     p.BN = tile_n(d->C, &p.n_tiles);
     p.m_tiles = pt_ceil_div(d->K, 128);
@@ -2223,8 +2231,11 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         }
         CUtensorMap tmX;
         const int up_w = (Q - 1) * d->stride - d->pad - (d->W - 1), up_h = (P - 1) * d->stride - d->pad - (d->H - 1);
-        if (!make_im2col_map(c, &tmX, a, d->C, d->W, d->H, d->N, d->ldx, -d->pad, -d->pad, up_w, up_h, d->stride, 64)) return PT_ERR_CUDA;
-        return run_wgrad(c, d, P, Q, d->stride, -d->pad, -d->pad, tmX, b, (float *)out, ws, ws_bytes, st);
+        const bool plain = d->R == 1 && d->S == 1 && d->stride == 1 && d->pad == 0;     // pixels of x and dy coincide
+        if (plain) {
+            if (!make_act2d_map(c, &tmX, a, d->C, (long long)d->N * d->H * d->W, d->ldx, 64)) return PT_ERR_CUDA;
+        } else if (!make_im2col_map(c, &tmX, a, d->C, d->W, d->H, d->N, d->ldx, -d->pad, -d->pad, up_w, up_h, d->stride, 64)) return PT_ERR_CUDA;
+        return run_wgrad(c, d, P, Q, d->stride, -d->pad, -d->pad, tmX, b, (float *)out, ws, ws_bytes, st, plain);
     }
 
     GemmP p;
