@@ -4,9 +4,12 @@
 //                      128 pixels x 64 channels, K-major (fwd) or MN-major (dgrad) weight tiles from the same bf16 shadow,
 //                      double/triple-buffered fp32 accumulators in TMEM, TMA-store epilogue.
 //   conv_halo_kernel   stride-1 RxS fwd/dgrad and the parities of a stride-2 dgrad: one halo tile per 64-channel chunk,
-//                      filter taps as row-shifted UMMA descriptors of that tile.
+//                      filter taps as row-shifted UMMA descriptors of that tile; a 32-byte-pixel mode (16 lanes per
+//                      position, 32-byte swizzle, one MMA per tap) runs the space-to-depth stem.
 //   conv_wgrad_kernel  weight gradient: both operands MN-major, reduction over pixels split across CTAs, partial tiles
 //                      summed in-kernel in a fixed order.
+//   conv_wgrad_rows_kernel  weight gradient of stride-1 layers with at most 64 input channels: row blocks of x staged
+//                      once, taps as row-shifted descriptors, two taps per MMA on the M side; same finish phase.
 //   stem_* kernels     space-to-depth layout kernels of the few-channel stride-2 stem.
 // Ragged channel counts are handled by the TMA unit (true extents in the tensor maps: zero-fill on load, clipping on
 // store) and by skipping the 16-wide k-steps past the last valid channel.
