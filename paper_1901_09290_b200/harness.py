@@ -348,8 +348,10 @@ class TrainStep:
         self.graph_launches = self.ctx.launch_count() - l0
         return self.graph
 
-    def step(self, stream=None):
+    def step(self, stream=None, before_train=None):
         self.reconfigure(stream)
+        if before_train is not None:
+            torch.cuda.current_stream().wait_event(before_train)     # e.g. the image batch has reached the stem's input
         if getattr(self, "graph", None) is not None:
             self.graph.replay()
             if not self._graph_has_update:
@@ -362,30 +364,26 @@ class TrainStep:
         """The same step with the image batch copied from pinned host memory and the regulariser value read back.
 
         The host-to-device copy runs on a copy stream into a staging buffer, so the copy of the next step's batch
-        overlaps this step's kernels (one copy per step; the first call issues its own). The step itself starts with a
-        device-to-device move of the staged batch into the stem's input."""
+        overlaps this step's kernels (one copy per step; the first call issues its own). The device-to-device move of the
+        staged batch into the stem's input runs on the copy stream too, beside the reconfiguration (which does not touch
+        the activations); the training part of the step waits for it."""
         main = torch.cuda.current_stream()
         if getattr(self, "_copy_stream", None) is None:
             self._copy_stream = torch.cuda.Stream()
             self._x_stage = torch.empty_like(self.x[0])
             self._ev_copied = torch.cuda.Event()
-            self._ev_free = torch.cuda.Event()
+            self._ev_placed = torch.cuda.Event()
             self._prefetched = False
         cs = self._copy_stream
-        if not self._prefetched:
-            cs.wait_stream(main)
-            with torch.cuda.stream(cs):
+        cs.wait_stream(main)                             # the previous step has finished reading the stem's input
+        with torch.cuda.stream(cs):
+            if not self._prefetched:
                 self._x_stage.copy_(self.h_image, non_blocking=True)
-                self._ev_copied.record(cs)
-        main.wait_event(self._ev_copied)
-        self.x[0].copy_(self._x_stage, non_blocking=True)
-        self._ev_free.record(main)
-        cs.wait_event(self._ev_free)
-        with torch.cuda.stream(cs):                      # the next step's batch
-            self._x_stage.copy_(self.h_image, non_blocking=True)
-            self._ev_copied.record(cs)
+            self.x[0].copy_(self._x_stage, non_blocking=True)
+            self._ev_placed.record(cs)
+            self._x_stage.copy_(self.h_image, non_blocking=True)     # the next step's batch
         self._prefetched = True
-        self.step(stream)
+        self.step(stream, before_train=self._ev_placed)
         self.h_reg.copy_(self.mp.reg, non_blocking=True)
 
     def e2e_bytes(self):
