@@ -233,6 +233,13 @@ pt_status pt_group_lasso_norms(pt_ctx *ctx, const pt_layer *layers /*host*/, int
                                void *ws, size_t ws_bytes, void *stream);
 pt_status pt_group_lasso_sgd_apply(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers,
                                    const pt_sgd_hparams *hp /*host*/, void *ws, size_t ws_bytes, void *stream);
+/* The update of layers [first, first + count) only, from the norms pt_group_lasso_norms left in ws (same layers array, same
+ * ws). A layer's update needs its own gradient and nothing else, so a caller can apply it as soon as that gradient exists
+ * (on the stream that produced it) instead of after the whole backward pass. Calls covering every layer exactly once compute
+ * bit for bit what pt_group_lasso_sgd_apply computes. PT_ERR_INVALID_ARG for a range outside [0, n_layers). */
+pt_status pt_group_lasso_sgd_apply_layers(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers, int32_t first,
+                                          int32_t count, const pt_sgd_hparams *hp /*host*/, void *ws, size_t ws_bytes,
+                                          void *stream);
 
 /* zero_out[k] = (max_{rs,c} |w| < threshold), zero_in[c] = (max_{k,rs} |w| < threshold), strict <, in fp32
  * (Sec. 4.1: threshold 1e-4; Sec. 4.2 / Fig. 4: the absolute maximum of a channel's parameters). A NaN keeps

@@ -82,6 +82,8 @@ EXPORTS = {
                                           c_void_p, c_size_t, c_void_p]),
     "pt_group_lasso_norms": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_group_lasso_sgd_apply": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, POINTER(pt_sgd_hparams), c_void_p, c_size_t, c_void_p]),
+    "pt_group_lasso_sgd_apply_layers": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_int32, c_int32, POINTER(pt_sgd_hparams), c_void_p,
+                                                  c_size_t, c_void_p]),
     "pt_find_zero_groups": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_float, c_int32, c_void_p, c_size_t, c_void_p]),
     "pt_find_zero_groups_noalloc": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p]),
     "pt_bn_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_bn_desc)]),
@@ -234,6 +236,14 @@ def pt_group_lasso_sgd_apply(ctx, layers, lam, lr, momentum, weight_decay=0.0, w
     hp = pt_sgd_hparams(lam, lr, momentum, weight_decay)
     p, n = _ws(ws)
     _check(lib().pt_group_lasso_sgd_apply(ctx.handle, arr, len(arr), byref(hp), p, n, _stream(stream)), "pt_group_lasso_sgd_apply")
+
+
+def pt_group_lasso_sgd_apply_layers(ctx, layers, first, count, lam, lr, momentum, weight_decay=0.0, ws=None, stream=None):
+    arr = layers if not isinstance(layers, (list, tuple)) else layer_array(layers)
+    hp = pt_sgd_hparams(lam, lr, momentum, weight_decay)
+    p, n = _ws(ws)
+    _check(lib().pt_group_lasso_sgd_apply_layers(ctx.handle, arr, len(arr), first, count, byref(hp), p, n, _stream(stream)),
+           "pt_group_lasso_sgd_apply_layers")
 
 
 def pt_find_zero_groups(ctx, layers, threshold=1e-4, zero_in_place=False, ws=None, stream=None):

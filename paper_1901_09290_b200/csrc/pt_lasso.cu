@@ -391,10 +391,12 @@ extern "C" size_t pt_group_lasso_workspace_bytes(const pt_ctx *c, const pt_layer
 }
 
 // phases: 1 = group norms (partial sums, finish, regulariser value), 2 = parameter update from the norms in the workspace
+// The update may be restricted to layers [first, first + count) (count < 0: all): the chunk table is ordered by layer.
 static pt_status lasso_phases(pt_ctx *c, const pt_layer *layers, int32_t n, const pt_sgd_hparams *hp, double *reg_sum_out, void *ws,
-                              size_t ws_bytes, void *stream, int phases)
+                              size_t ws_bytes, void *stream, int phases, int first = 0, int count = -1)
 {
     if (!c || ((phases & 2) && !hp)) return PT_ERR_INVALID_ARG;
+    if (count >= 0 && (first < 0 || first + count > n)) return PT_ERR_INVALID_ARG;
     Tables t;
     pt_status s = build_tables(layers, n, &t);
     if (s != PT_OK) return s;
@@ -418,8 +420,16 @@ static pt_status lasso_phases(pt_ctx *c, const pt_layer *layers, int32_t n, cons
         if (reg_sum_out) { reg_total_kernel<<<1, 32, 0, st>>>(layer_reg, nj, reg_sum_out); c->launches += 1; }
     }
     if (phases & 2) {
-        update_kernel<<<nch, kThreads, 0, st>>>(dl, dc, inv_out, inv_in, *hp);
-        c->launches += 1;
+        unsigned c0 = 0, c1 = nch;
+        if (count >= 0) {
+            c0 = nch; c1 = 0;
+            for (unsigned i = 0; i < nch; ++i)
+                if (t.chunks[i].layer >= first && t.chunks[i].layer < first + count) { c0 = i < c0 ? i : c0; c1 = i + 1; }
+        }
+        if (c1 > c0) {
+            update_kernel<<<c1 - c0, kThreads, 0, st>>>(dl, dc + c0, inv_out, inv_in, *hp);
+            c->launches += 1;
+        }
     }
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
@@ -441,6 +451,13 @@ extern "C" pt_status pt_group_lasso_sgd_apply(pt_ctx *c, const pt_layer *layers,
                                               size_t ws_bytes, void *stream)
 {
     return lasso_phases(c, layers, n, hp, nullptr, ws, ws_bytes, stream, 2);
+}
+
+extern "C" pt_status pt_group_lasso_sgd_apply_layers(pt_ctx *c, const pt_layer *layers, int32_t n, int32_t first, int32_t count,
+                                                     const pt_sgd_hparams *hp, void *ws, size_t ws_bytes, void *stream)
+{
+    if (count < 0) return PT_ERR_INVALID_ARG;
+    return lasso_phases(c, layers, n, hp, nullptr, ws, ws_bytes, stream, 2, first, count);
 }
 
 extern "C" pt_status pt_find_zero_groups(pt_ctx *c, const pt_layer *layers, int32_t n, float threshold,

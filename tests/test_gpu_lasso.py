@@ -96,6 +96,28 @@ def test_step_in_two_calls_equals_the_single_call():
     assert dm.reg.item() == one.reg.item()
 
 
+def test_apply_by_layer_ranges_equals_the_single_call():
+    """pt_group_lasso_sgd_apply_layers over ranges that cover every layer once == pt_group_lasso_sgd_apply, bit for bit."""
+    net = W.resnet32()
+    model = W.gen_model(net, W.BASE_SEED + 7, kept=W.choose_kept(net, W.random_keep(net, W.BASE_SEED + 7), W.BASE_SEED + 7))
+    one = DevModel(model)
+    B.pt_group_lasso_norms(Hh.ctx(), one.arr, one.reg, one.ws)
+    B.pt_group_lasso_sgd_apply(Hh.ctx(), one.arr, 2e-4, 0.1, 0.9, 1e-4, one.ws)
+    dm = DevModel(model)
+    B.pt_group_lasso_norms(Hh.ctx(), dm.arr, dm.reg, dm.ws)
+    n = len(net.layers)
+    for first, count in [(20, n - 20), (0, 1), (7, 13), (1, 6), (5, 0)]:      # any order; an empty range is a no-op
+        B.pt_group_lasso_sgd_apply_layers(Hh.ctx(), dm.arr, first, count, 2e-4, 0.1, 0.9, 1e-4, dm.ws)
+    torch.cuda.synchronize()
+    Hh.ctx().poll()
+    for li in range(n):
+        assert torch.equal(dm.w[li], one.w[li]) and torch.equal(dm.v[li], one.v[li]), net.layers[li].name
+        assert torch.equal(dm.wb[li].view(torch.int16), one.wb[li].view(torch.int16))
+    for bad in [(-1, 2), (n, 1), (3, n)]:
+        with pytest.raises(B.PtError):
+            B.pt_group_lasso_sgd_apply_layers(Hh.ctx(), dm.arr, bad[0], bad[1], 2e-4, 0.1, 0.9, 1e-4, dm.ws)
+
+
 def test_step_resnet50_all_layers():
     net = W.resnet50()
     model = W.gen_model(net, W.BASE_SEED + 4)
