@@ -174,6 +174,14 @@ class TrainStep:
             self.dx.append(torch.empty((N, l.H, l.H, ldx), dtype=torch.bfloat16, device="cuda") if li > 0 else None)
             for which in range(3):
                 ws_bytes = max(ws_bytes, B.pt_conv_workspace_bytes(ctx, d, which))
+        # The last weight gradients of the backward pass (the stem's and its two predecessors in launch order) have nothing
+        # left to run beside: instead of three equal shares, the SMs are divided in proportion to their estimated work, so
+        # that they end together. The three shares still sum to the SM count, as every three consecutive launches must.
+        self.wgrad_limit = self._tail_limits() if (wgrad_streams == 3 and wgrad_ctas * 3 <= 148 and len(self.net.layers) >= 4) else {}
+        for li, lim in self.wgrad_limit.items():
+            ctx.set_wgrad_cta_limit(lim)
+            ws_bytes = max(ws_bytes, B.pt_conv_workspace_bytes(ctx, self.desc[li], 2))
+        ctx.set_wgrad_cta_limit(wgrad_ctas)
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
         self.ws_w = [torch.empty(ws_bytes, dtype=torch.uint8, device="cuda") for _ in range(self.wgrad_streams)]
         # e2e: the image batch arrives from pinned host memory every step
@@ -182,6 +190,35 @@ class TrainStep:
         if host_inputs:
             self.h_image = self.x[0].cpu().pin_memory()
         self.h_reg = torch.zeros(1, dtype=torch.float64).pin_memory()
+
+    def _wgrad_work(self, li: int) -> float:
+        """Rough device time (us on one SM) of a layer's weight gradient: the larger of its MMA count at 55+ cycles each
+        and its tensor bytes at the ~35 GB/s one SM pulls; only ratios between layers are used."""
+        l = self.net.layers[li]
+        px = self.N * l.P * l.P
+        taps = l.R * l.R
+        if l.stride == 2 and l.C <= 4:                       # space-to-depth stem: (R+1)/2 vertical taps of 64 lanes
+            mmas = px / 16 * ((l.R + 1) // 2)
+            cyc = 55
+        elif l.stride == 1 and l.C <= 64:                    # row-block kernel: two taps per MMA, N = K
+            mmas = px / 16 * ((taps + 1) // 2)
+            cyc = max(55, W.pad16(l.K) // 2 + 8)
+        else:
+            bn = min(256, W.pad16(l.C))
+            mmas = px / 16 * taps * -(-l.K // 128) * -(-l.C // bn)
+            cyc = max(55, bn // 2 + 8)
+        t_mma = mmas * cyc / 1.9e3
+        t_mem = (self.N * l.H * l.H * W.pad16(l.C) + px * W.pad16(l.K)) * 2 / 35e3
+        return max(t_mma, t_mem)
+
+    def _tail_limits(self) -> Dict[int, int]:
+        tail = [2, 1, 0]                                     # launch order of the last three weight gradients
+        work = [self._wgrad_work(li) for li in tail]
+        tot = sum(work)
+        lim = [max(16, int(148 * w / tot)) for w in work]
+        while sum(lim) > 148:
+            lim[lim.index(max(lim))] -= 1
+        return {li: v for li, v in zip(tail, lim)}
 
     # ---- sizes used for reporting
     def conv_flops(self) -> Dict[str, int]:
@@ -224,7 +261,12 @@ class TrainStep:
         B.pt_conv_dgrad(self.ctx, self.desc[li], self.dy[li], self.mp.wb[li], self.dx[li], self.ws, stream)
 
     def conv_wgrad(self, li, stream=None, ws_index: int = 0):
+        lim = self.wgrad_limit.get(li)
+        if lim is not None:
+            self.ctx.set_wgrad_cta_limit(lim)
         B.pt_conv_wgrad(self.ctx, self.desc[li], self.x[li], self.dy[li], self.mp.g[li], self.ws_w[ws_index], stream)
+        if lim is not None:
+            self.ctx.set_wgrad_cta_limit(self.wgrad_ctas)
 
     def lasso(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
         B.pt_group_lasso_sgd_step(self.ctx, self.mp.arr, lam, lr, mu, 0.0, self.mp.reg, self.mp.ws, stream)
