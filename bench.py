@@ -26,7 +26,7 @@ sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum over the launches of each conv pass in one step of the default workload
 # (one ncu capture, 1 pass per launch; the summary and the command are in profiles/step_launch_list_resnet50_keep060_b64.txt)
-NCU_DRAM_BYTES = {"fwd": 1.103e9, "dgrad": 1.101e9, "wgrad": 2.121e9}   # incl. the stem layout kernels
+NCU_DRAM_BYTES = {"fwd": 1.102e9, "dgrad": 1.101e9, "wgrad": 2.122e9}   # incl. the stem layout kernels
 METRIC = "pruned ResNet-50 train-step conv TFLOP/s (useful FLOPs / whole step)"
 UNIT = "TFLOP/s"
 
