@@ -91,6 +91,12 @@ enum { PT_CONV_FWD = 0, PT_CONV_DGRAD = 1, PT_CONV_WGRAD = 2 };
 
 /* Bytes of caller-provided workspace the given pass needs for this descriptor (0 = none). */
 size_t pt_conv_workspace_bytes(const pt_ctx *ctx, const pt_conv_desc *d, int which);
+/* CTAs pt_conv_wgrad launches for this descriptor at the context's current limit (pt_set_wgrad_cta_limit): tiles x splits,
+ * splits being the largest count that keeps the product within the limit (at least 1: a descriptor with more tiles than
+ * the limit runs unsplit). *waits (optional) = 1 if those CTAs wait for one another (splits > 1), which is what the
+ * co-residency rule of pt_set_wgrad_cta_limit is about. Lets a caller choose per-launch limits that waste no SMs.
+ * 0 if the tcgen05 kernels do not take the descriptor. */
+int32_t pt_conv_wgrad_ctas(const pt_ctx *ctx, const pt_conv_desc *d, int32_t *waits);
 
 /* y[n,p,q,k] = sum_{r,s,c} x[n, p*stride-pad+r, q*stride-pad+s, c] * w[k,r,s,c], zero outside the image.
  * x: bf16 [N][H][W][ldx]; w: bf16 shadow [K][R][S][ldw]; y: [N][P][Q][ldy] bf16 or fp32. fp32 accumulation. */

@@ -73,6 +73,7 @@ EXPORTS = {
     "pt_poll_device_status": (c_int32, [c_void_p, c_void_p]),
     "pt_launch_count": (c_uint64, [c_void_p]),
     "pt_set_wgrad_cta_limit": (c_int32, [c_void_p, c_int32]),
+    "pt_conv_wgrad_ctas": (c_int32, [c_void_p, POINTER(pt_conv_desc), POINTER(c_int32)]),
     "pt_conv_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_conv_desc), c_int32]),
     "pt_conv_fwd": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_conv_dgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
@@ -307,6 +308,13 @@ def pt_cross_entropy(ctx, logits, labels, n, classes, ld, loss_out, ws, stream=N
     p, nb = _ws(ws)
     _check(lib().pt_cross_entropy(ctx.handle, _ptr(logits), _ptr(labels), n, classes, ld, _ptr(loss_out), p, nb, _stream(stream)),
            "pt_cross_entropy")
+
+
+def pt_conv_wgrad_ctas(ctx, d):
+    """(CTAs of the weight-gradient launch at the current limit, whether they wait for one another)."""
+    w = c_int32(0)
+    n = int(lib().pt_conv_wgrad_ctas(ctx.handle, byref(d), byref(w)))
+    return n, bool(w.value)
 
 
 def pt_set_coeff(ctx, loss, reg_sum, ratio, lambda_out, stream=None):

@@ -164,6 +164,18 @@ extern "C" size_t pt_conv_workspace_bytes(const pt_ctx *c, const pt_conv_desc *d
     return a > b ? a : b;
 }
 
+extern "C" int32_t pt_conv_wgrad_ctas(const pt_ctx *c, const pt_conv_desc *d, int32_t *waits)
+{
+    int P, Q;
+    if (waits) *waits = 0;
+    if (pt_conv_validate(c, d, &P, &Q) != PT_OK) return 0;
+    if (d->algo == 1 || !pt_sm100_conv_supported(c, d, PT_CONV_WGRAD)) return 0;
+    int w = 0;
+    const int n = pt_sm100_wgrad_ctas(c, d, &w);
+    if (waits) *waits = w;
+    return n;
+}
+
 static pt_status conv_dispatch(pt_ctx *c, const pt_conv_desc *d, int which, const void *a, const void *b, void *out,
                                void *ws, size_t ws_bytes, void *stream)
 {

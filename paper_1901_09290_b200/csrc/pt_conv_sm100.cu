@@ -2186,6 +2186,29 @@ static pt_conv_desc stem_virtual_desc(const pt_conv_desc *d, const StemPlan &sp)
     return v;
 }
 
+// CTAs the weight gradient of `d` launches at the context's current CTA limit: tiles x splits; *waits = 1 if they wait for
+// one another (splits > 1).
+int pt_sm100_wgrad_ctas(const pt_ctx *c, const pt_conv_desc *d, int *waits)
+{
+    const StemPlan sp = stem_plan(d);
+    pt_conv_desc v = sp.ok ? stem_virtual_desc(d, sp) : *d;
+    const int P = sp.ok ? sp.P : pt_out_dim(d->H, d->R, d->stride, d->pad), Q = sp.ok ? sp.Q : pt_out_dim(d->W, d->S, d->stride, d->pad);
+    int tiles, splits;
+    const WgRows wr = sp.ok ? WgRows() : wgrad_rows_plan(c, &v, P, Q);
+    if (!sp.ok && wr.ok) {
+        tiles = wr.n_tiles * wr.m_tiles * wr.tap_groups;
+        splits = wr.splits;
+    } else {
+        int n_tiles;
+        const int bn = tile_n(v.C, &n_tiles);
+        const int tpc = wgrad_taps_per_cta(v.R * v.S, bn);
+        tiles = pt_ceil_div(v.K, 128) * n_tiles * pt_ceil_div(v.R * v.S, tpc);
+        splits = wgrad_splits(c, &v, P, Q);
+    }
+    if (waits) *waits = splits > 1 ? 1 : 0;
+    return tiles * splits;
+}
+
 size_t pt_sm100_conv_workspace(const pt_ctx *c, const pt_conv_desc *d, int which)
 {
     const StemPlan sp = stem_plan(d);

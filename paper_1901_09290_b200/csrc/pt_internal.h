@@ -79,3 +79,4 @@ bool pt_sm100_conv_supported(const pt_ctx *ctx, const pt_conv_desc *d, int which
 pt_status pt_sm100_conv(pt_ctx *ctx, const pt_conv_desc *d, int which, const void *a, const void *b, void *out,
                         void *ws, size_t ws_bytes, cudaStream_t st);
 size_t pt_sm100_conv_workspace(const pt_ctx *ctx, const pt_conv_desc *d, int which);
+int pt_sm100_wgrad_ctas(const pt_ctx *ctx, const pt_conv_desc *d, int *waits);

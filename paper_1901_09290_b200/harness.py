@@ -174,10 +174,9 @@ class TrainStep:
             self.dx.append(torch.empty((N, l.H, l.H, ldx), dtype=torch.bfloat16, device="cuda") if li > 0 else None)
             for which in range(3):
                 ws_bytes = max(ws_bytes, B.pt_conv_workspace_bytes(ctx, d, which))
-        # The last weight gradients of the backward pass (the stem's and its two predecessors in launch order) have nothing
-        # left to run beside: instead of three equal shares, the SMs are divided in proportion to their estimated work, so
-        # that they end together. The three shares still sum to the SM count, as every three consecutive launches must.
-        self.wgrad_limit = self._tail_limits() if (wgrad_streams == 3 and wgrad_ctas * 3 <= 148 and len(self.net.layers) >= 4) else {}
+        # Per-launch CTA limits: whole multiples of each layer's tiles (no idle share of a budget), larger for the layers
+        # with more work, every three consecutive launches within the SM count (see _wgrad_limits)
+        self.wgrad_limit = self._wgrad_limits() if (wgrad_streams == 3 and wgrad_ctas * 3 <= 148 and len(self.net.layers) >= 4) else {}
         for li, lim in self.wgrad_limit.items():
             ctx.set_wgrad_cta_limit(lim)
             ws_bytes = max(ws_bytes, B.pt_conv_workspace_bytes(ctx, self.desc[li], 2))
@@ -211,14 +210,60 @@ class TrainStep:
         t_mem = (self.N * l.H * l.H * W.pad16(l.C) + px * W.pad16(l.K)) * 2 / 35e3
         return max(t_mma, t_mem)
 
-    def _tail_limits(self) -> Dict[int, int]:
-        tail = [2, 1, 0]                                     # launch order of the last three weight gradients
-        work = [self._wgrad_work(li) for li in tail]
-        tot = sum(work)
-        lim = [max(16, int(148 * w / tot)) for w in work]
-        while sum(lim) > 148:
-            lim[lim.index(max(lim))] -= 1
-        return {li: v for li, v in zip(tail, lim)}
+    def _wgrad_limits(self) -> Dict[int, int]:
+        """CTA limit of every weight-gradient launch. The launches go round-robin to three streams in reverse layer order,
+        so any three consecutive ones can be in flight together and their CTAs (which wait for one another) must fit on
+        the device at once. Within that constraint the limits minimise the sum over launches of work / CTAs (dynamic
+        programme over the CTA counts each layer can actually use, as the library reports them), which gives the layers
+        with more work the larger shares and wastes no part of a share on a tile count that does not divide it. The
+        last three launches have nothing after them and end up sharing all SMs."""
+        sm = torch.cuda.get_device_properties(0).multi_processor_count
+        order = list(range(len(self.net.layers) - 1, -1, -1))
+        cands = []
+        for li in order:
+            seen = {}
+            for lim in range(16, min(sm, 128) + 1):
+                self.ctx.set_wgrad_cta_limit(lim)
+                ctas, waits = B.pt_conv_wgrad_ctas(self.ctx, self.desc[li])
+                if ctas <= 0:
+                    break
+                # an unsplit launch waits for nobody and may run in waves: it only counts as a fair share in the sums
+                room = ctas if waits else min(ctas, sm // 3)
+                if (ctas, room) not in seen and room <= sm:
+                    seen[(ctas, room)] = lim
+            cands.append([(room, lim, ctas) for (ctas, room), lim in sorted(seen.items())] or [(self.wgrad_ctas, self.wgrad_ctas, self.wgrad_ctas)])
+        self.ctx.set_wgrad_cta_limit(self.wgrad_ctas)
+        work = [self._wgrad_work(li) for li in order]
+        INF = float("inf")
+        # best[(a, b)] = (cost, choices) over the first i launches with the last two using cands[i-2][a], cands[i-1][b]
+        best = {(-1, -1): (0.0, [])}
+        for i, cs in enumerate(cands):
+            nxt = {}
+            for (a, b), (cost, path) in best.items():
+                ca = cands[i - 2][a][0] if a >= 0 else 0
+                cb = cands[i - 1][b][0] if b >= 0 else 0
+                for k, (room, _, ctas) in enumerate(cs):
+                    if ca + cb + room > sm:
+                        continue
+                    c2 = cost + work[i] / min(ctas, sm)
+                    key = (b, k)
+                    if c2 < nxt.get(key, (INF,))[0]:
+                        nxt[key] = (c2, path + [k])
+            if not nxt:                                    # cannot happen with the smallest candidates; keep the default
+                return {}
+            best = nxt
+        path = min(best.values(), key=lambda v: v[0])[1]
+        lim = {li: cands[i][k][1] for i, (li, k) in enumerate(zip(order, path))}
+        # the last three launches end the backward pass: what counts for them is that they finish together, i.e. shares in
+        # proportion to their work rather than to its square root
+        tail, wt = order[-3:], work[-3:]
+        share = [max(16, int(sm * w / sum(wt))) for w in wt]
+        while sum(share) > sm:
+            share[share.index(max(share))] -= 1
+        prev = [cands[i][path[i]][0] for i in (len(order) - 5, len(order) - 4)]
+        if prev[0] + prev[1] + share[0] <= sm and prev[1] + share[0] + share[1] <= sm:
+            lim.update({li: v for li, v in zip(tail, share)})
+        return lim
 
     # ---- sizes used for reporting
     def conv_flops(self) -> Dict[str, int]:
