@@ -134,6 +134,7 @@ class TrainStep:
         # go round-robin to `wgrad_streams` streams, each with a workspace of its own. The CTAs of a split weight gradient
         # wait for one another, one per SM, so streams x limit stays within the SM count (3 x 49 <= 148): every launch
         # that can be in flight then fits on the device together, whatever order the hardware picks its CTAs in.
+        # `wgrad_ctas` is the nominal share; _wgrad_limits() refines it per launch under the same constraint.
         self.wgrad_ctas, self.wgrad_streams = wgrad_ctas, max(1, wgrad_streams)
         ctx.set_wgrad_cta_limit(wgrad_ctas)
         self.dense_net = dense_net
