@@ -137,6 +137,29 @@ def test_wgrad_with_a_cta_limit(limit):
         B.pt_set_wgrad_cta_limit(c, 0)
 
 
+def test_wgrad_cta_query_follows_the_limit():
+    """pt_conv_wgrad_ctas reports tiles x splits at the current limit: never above a limit it can meet, whole multiples of
+    the tile count, and an unsplit launch (more tiles than the limit) is reported as not waiting."""
+    c = Hh.ctx()
+    try:
+        for (N, H, C, K, R, stride) in [(64, 14, 213, 242, 3, 1), (64, 56, 46, 59, 3, 1), (64, 28, 418, 113, 1, 1), (64, 7, 434, 495, 3, 1),
+                                        (64, 224, 3, 55, 7, 2)]:
+            d = B.make_conv_desc(N, H, H, C, K, R, R, stride, R // 2, 8 if C <= 4 else W.pad16(C), W.pad16(K))
+            B.pt_set_wgrad_cta_limit(c, 1)
+            tiles, waits = B.pt_conv_wgrad_ctas(c, d)
+            assert tiles >= 1 and not waits
+            prev = 0
+            for lim in (8, 24, 49, 74, 148):
+                B.pt_set_wgrad_cta_limit(c, lim)
+                n, waits = B.pt_conv_wgrad_ctas(c, d)
+                assert n % tiles == 0 and n >= prev
+                assert (n <= lim and waits == (n > tiles)) or (n == tiles and not waits)
+                prev = n
+        assert B.pt_conv_wgrad_ctas(c, B.make_conv_desc(2, 8, 8, 16, 16, 3, 3, 1, 1, algo=1)) == (0, False)
+    finally:
+        B.pt_set_wgrad_cta_limit(c, 0)
+
+
 def test_invalid_arguments_are_rejected_before_launch():
     c = Hh.ctx()
     buf = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
