@@ -94,6 +94,8 @@ ROW_BLOCK = [
     (2, 11, 11, 13, 21, 3, 0), (2, 7, 7, 5, 9, 3, 2), (2, 6, 6, 33, 40, 2, 0), (64, 20, 20, 38, 38, 3, 1),
     # 1x1 filters on large maps take the same kernel (single tap, K > 128 in one tile)
     (3, 30, 30, 59, 143, 1, 0), (2, 28, 28, 7, 19, 1, 0), (2, 40, 33, 64, 250, 1, 0),
+    # more than 64 input channels (the generic kernel): ragged channel tiles, 25 taps, a 28x28 map
+    (2, 14, 14, 93, 77, 3, 1), (2, 15, 16, 130, 40, 3, 1), (3, 14, 20, 213, 242, 3, 1), (2, 16, 16, 128, 100, 5, 2), (8, 28, 28, 113, 111, 3, 1),
 ]
 
 
