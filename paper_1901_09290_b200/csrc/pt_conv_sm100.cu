@@ -155,7 +155,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
-    grid_dependency_wait();              // nothing above touches global memory
+    // The weights are not written by the kernels that precede a convolution in a stream (those that trigger their dependents
+    // early are convolutions themselves), so the weight producers start loading at once; everybody else waits for the
+    // previous kernel's results here.
+    if (!(warp == 14 || (warp == 15 && two_b))) grid_dependency_wait();
     grid_launch_dependents();
 
     if (warp == 0 || warp == 14 || (warp == 15 && two_b)) {
@@ -555,7 +558,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int issuer = warp == 1 ? 0 : warp - 9;             // warps 10, 11, 12 -> issuers 1, 2, 3
-    grid_dependency_wait();              // nothing above touches global memory
+    if (!(warp == 0 && p.resident)) grid_dependency_wait();   // the producer first issues the resident weights (see below)
     grid_launch_dependents();
 
     // Streamed weights with two issuers: two complete pipelines (producer warp, A ring, B ring, issuer warp, accumulators),
@@ -577,6 +580,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         if (!B_MN) tma_load_3d(dst, &tmB, bar, kc * kKC, wtap, 0);
                         else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
                     }
+                grid_dependency_wait();          // the activations are the previous kernel's output
             }
             int tc = pid;
             TileWalk tw;
