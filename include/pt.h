@@ -98,6 +98,10 @@ size_t pt_conv_workspace_bytes(const pt_ctx *ctx, const pt_conv_desc *d, int whi
  * 0 if the tcgen05 kernels do not take the descriptor. */
 int32_t pt_conv_wgrad_ctas(const pt_ctx *ctx, const pt_conv_desc *d, int32_t *waits);
 
+/* Stream order: the three calls below are ordinary stream work. Their kernels are launched with programmatic stream
+ * serialization and read the WEIGHTS before waiting for the preceding kernel of the stream; that is invisible to callers
+ * because only kernels that release their dependents early can be overtaken, and the only such kernels are this library's
+ * convolutions, which never write weights. */
 /* y[n,p,q,k] = sum_{r,s,c} x[n, p*stride-pad+r, q*stride-pad+s, c] * w[k,r,s,c], zero outside the image.
  * x: bf16 [N][H][W][ldx]; w: bf16 shadow [K][R][S][ldw]; y: [N][P][Q][ldy] bf16 or fp32. fp32 accumulation. */
 pt_status pt_conv_fwd(pt_ctx *ctx, const pt_conv_desc *d, const void *x, const void *w, void *y,

@@ -2282,6 +2282,8 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         stem_s2d_w_kernel<<<(unsigned)((sp.w2_elems + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)b, w2, d->K, d->R, d->S, d->C, d->ldw,
                                                                               sp.U, sp.V, sp.off);
         c->launches += 2;
+        // (plain launches: the convolution below loads w2 before its dependency wait, which is safe because stem_s2d_w_kernel
+        // does not release its dependents before it has completed)
         if (!d->out_f32) {
             // row-block form on 32-byte pixels: the U x V taps are row shifts of one staged tile (each xs byte read once)
             HaloSpec h;
