@@ -863,6 +863,16 @@ __device__ unsigned long long g_wg_trace[8][64];
 #else
 #define WTRACE(i) do { } while (0)
 #endif
+// n / d for 0 <= n < 2^22 and a divisor known per kernel: float reciprocal plus one correction step (an integer division
+// costs ~40 instructions, and the reduction below does two per 16-byte item).
+__device__ __forceinline__ int fast_div(int n, int d, float inv_d)
+{
+    int q = __float2int_rz(__int2float_rn(n) * inv_d);
+    if ((q + 1) * d <= n) ++q;
+    if (q * d > n) --q;
+    return q;
+}
+
 // Everything after the main loop of a weight-gradient kernel: the accumulators leave TMEM (directly to dw, or as this
 // split's partial tile), the splits of a tile meet, and every CTA sums its share of the tile over the splits.
 // `ring_bytes` of shared memory at `data_base` are free by then and serve as staging.
@@ -1016,10 +1026,11 @@ __device__ __forceinline__ void wgrad_finish(const WgradP &p, const CUtensorMap 
         const size_t zstride = (size_t)128 * acc_cols;
         const float *pbase = p.partial + (size_t)blockIdx.x * p.apc * p.splits * zstride;
         const int cap = (int)(((size_t)ring_bytes) / ((size_t)p.splits * 16));   // items the stage memory holds
+        const float inv_items = 1.0f / (float)items, inv_ngrp = 1.0f / (float)ngrp;
         for (int c_beg = it_beg; c_beg < it_end; c_beg += cap) {
             const int n_chunk = min(cap, it_end - c_beg);
             for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
-                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
+                const int idx = c_beg + i, tt = fast_div(idx, items, inv_items), item = idx - tt * items;
                 const float *src = pbase + (size_t)tt * p.splits * zstride + (size_t)item * 4;
                 uint32_t dst = data_base + (uint32_t)i * 16u;
                 for (int z = 0; z < p.splits; ++z, src += zstride, dst += (uint32_t)n_chunk * 16u)
@@ -1028,8 +1039,8 @@ __device__ __forceinline__ void wgrad_finish(const WgradP &p, const CUtensorMap 
             asm volatile("cp.async.wait_all;" ::: "memory");
             __syncthreads();
             for (int i = threadIdx.x; i < n_chunk; i += kThreads) {
-                const int idx = c_beg + i, tt = idx / items, item = idx - tt * items;
-                const int r = item / ngrp, col = (item - r * ngrp) * 4;
+                const int idx = c_beg + i, tt = fast_div(idx, items, inv_items), item = idx - tt * items;
+                const int r = fast_div(item, ngrp, inv_ngrp), col = (item - r * ngrp) * 4;
                 if (!p.pair && c0 + col >= p.C) continue;
                 float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
                 uint32_t a = data_base + (uint32_t)i * 16u;
@@ -1051,6 +1062,15 @@ __device__ __forceinline__ void wgrad_finish(const WgradP &p, const CUtensorMap 
                 }
                 float *dst = p.out + ((size_t)(k0 + r) * p.taps + tap0 + tt) * p.C + c0 + col;
                 const int nv = min(4, p.C - (c0 + col));
+                if (nv == 4 && ((uintptr_t)dst & 15) == 0) {
+                    *reinterpret_cast<float4 *>(dst) = sum;           // a dw row starts on a 16-byte boundary only if C allows it
+                    continue;
+                }
+                if (nv == 4 && ((uintptr_t)dst & 7) == 0) {
+                    reinterpret_cast<float2 *>(dst)[0] = make_float2(sum.x, sum.y);
+                    reinterpret_cast<float2 *>(dst)[1] = make_float2(sum.z, sum.w);
+                    continue;
+                }
                 dst[0] = sum.x;
                 if (nv > 1) dst[1] = sum.y;
                 if (nv > 2) dst[2] = sum.z;
