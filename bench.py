@@ -381,7 +381,8 @@ def run_ours(args):
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 operands, f32 accumulate (convs); f32 (lasso/SGD); u8/i32 (detection, compaction)",
+        "dtype": "bf16",
+        "arithmetic": "bf16 operands, f32 accumulate (convs); f32 (lasso/SGD); u8/i32 (detection, compaction)",
         "data": "synthetic",
         "config": {"workload": name, "batch_per_gpu": args.batch, "image": 224, "conv_layers": nL,
                    "kept_params": ts.mp.n_params(), "dense_params": ts.md.n_params(),
