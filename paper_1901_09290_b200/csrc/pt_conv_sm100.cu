@@ -751,6 +751,15 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         if (g >= groups || m >= p.nr * p.Wp) break;   // the slab only holds the tile's raster rows
+                        // accumulator columns past the channel count come from weight rows that were never loaded (whatever
+                        // follows the tile in shared memory); those that the store still covers (the pad lanes up to the next
+                        // multiple of 16) are written as zeros
+                        const int cbase = n0 + ch * 64 + g * 16;
+                        if (cbase + 16 > p.n_cols) {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e)
+                                if (cbase + e >= p.n_cols) v[g][e] = 0u;
+                        }
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 0]), __uint_as_float(v[g][8 * h + 1]));

@@ -115,6 +115,28 @@ def test_row_block_weight_gradient(shape):
     assert torch.equal(dw, again)
 
 
+@pytest.mark.parametrize("shape", [(2, 16, 16, 20, 36, 3, 1), (2, 14, 14, 37, 70, 3, 1), (2, 8, 8, 7, 33, 1, 1), (2, 16, 16, 41, 20, 3, 2)])
+def test_pad_lanes_up_to_a_multiple_of_16_are_zero(shape):
+    """With channel pitches that are multiples of 16 (as the training harness uses) the bf16 outputs are stored in whole
+    32-byte sectors: the pad lanes receive zeros, never stale accumulator columns."""
+    N, H, Wd, C, K, R, stride = shape
+    pad = R // 2
+    x, w, dy, _ = _case(N, H, Wd, C, K, R, stride, seed=W.BASE_SEED + 23)
+    ldx, ldy, ldw = W.pad16(C), W.pad16(K), W.pad8(C)
+    d = B.make_conv_desc(N, H, Wd, C, K, R, R, stride, pad, ldx, ldy, ldw, 0, 2)
+    P, Q = (H + 2 * pad - R) // stride + 1, (Wd + 2 * pad - R) // stride + 1
+    xd, wd, dyd = Hh.to_dev_padded(x, ldx), Hh.to_dev_padded(w, ldw), Hh.to_dev_padded(dy, ldy)
+    y = Hh.out_buffer((N, P, Q), K, ldy, 0)
+    dx = Hh.out_buffer((N, H, Wd), C, ldx, 0)
+    B.pt_conv_fwd(Hh.ctx(), d, xd, wd, y, Hh.conv_ws(d, B.PT_CONV_FWD))
+    B.pt_conv_dgrad(Hh.ctx(), d, dyd, wd, dx, Hh.conv_ws(d, B.PT_CONV_DGRAD))
+    torch.cuda.synchronize()
+    Hh.ctx().poll()
+    Hh.check_conv(y, K, oracle.conv_fwd(x.numpy(), w.numpy(), stride, pad), what="fwd")
+    Hh.check_conv(dx, C, oracle.conv_dgrad(dy.numpy(), w.numpy(), H, Wd, stride, pad), what="dgrad")
+    assert torch.all(y[..., K:] == 0) and torch.all(dx[..., C:] == 0)
+
+
 def test_wgrad_is_run_to_run_identical():
     N, H, C, K, R = 4, 14, 27, 19, 3
     x, w, dy, pad = _case(N, H, H, C, K, R, 1, W.BASE_SEED + 5)
