@@ -751,15 +751,6 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         if (g >= groups || m >= p.nr * p.Wp) break;   // the slab only holds the tile's raster rows
-                        // accumulator columns past the channel count come from weight rows that were never loaded (whatever
-                        // follows the tile in shared memory); those that the store still covers (the pad lanes up to the next
-                        // multiple of 16) are written as zeros
-                        const int cbase = n0 + ch * 64 + g * 16;
-                        if (cbase + 16 > p.n_cols) {
-#pragma unroll
-                            for (int e = 0; e < 16; ++e)
-                                if (cbase + e >= p.n_cols) v[g][e] = 0u;
-                        }
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(v[g][8 * h + 0]), __uint_as_float(v[g][8 * h + 1]));
@@ -1753,9 +1744,11 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     const int need_rows = 128 + (h.span_h - 1) * Wp + h.span_w - 1;
     p.a_alloc = (int)pt_align_up((size_t)p.a_box_bytes, 1024);
     const size_t a_tail = need_rows * row_bytes > p.a_alloc ? pt_align_up((size_t)need_rows * row_bytes - p.a_alloc, 1024) : 0;
-    // a K-major weight box only brings the output channels that exist (in whole 8-row swizzle atoms); the MMA still reads
-    // BN rows, the rest from whatever follows in shared memory: columns that are never stored
-    p.b_rows = (int)pt_align_up((size_t)(p.BN < h.n_cols ? p.BN : h.n_cols), 8);
+    // a K-major weight box brings the output channels that exist rounded up to 16 (the rows past the count are zero-filled
+    // by the TMA unit): exactly the columns the output map covers, so the pad lanes it writes are zeros; the MMA may still
+    // read up to BN rows, the rest from whatever follows in shared memory: columns that are never stored
+    p.b_rows = p.BN < h.n_cols ? p.BN : pt_ceil_div(h.n_cols, 16) * 16;
+    if (p.b_rows > p.BN) p.b_rows = p.BN;
     const size_t b_bytes = B_MN ? (size_t)pt_ceil_div(p.BN, 64) * 8192 : (size_t)p.b_rows * row_bytes;
     p.b_slot = (int)b_bytes;
     // epilogue staging: one slab of the tile's raster rows x 128 bytes per group (direct-store launches use none)
