@@ -21,9 +21,11 @@
  * Physical layouts
  *   activations x, y, dy, dx : [N][H][W][ld]   bf16 (or fp32 outputs when out_f32 = 1), channels
  *                              innermost, channel pitch ld >= channels, ld a multiple of 8 elements.
- *                              Pad lanes (channel index >= channels) are never read. Outputs may get zeros
- *                              written into the pad lanes that share the last 16-byte granule with valid
- *                              channels (an effect of the TMA store); other pad lanes are left untouched.
+ *                              Pad lanes (channel index >= channels) are never read. bf16 outputs may get zeros
+ *                              written into the pad lanes up to the next multiple of 16 channels where the pitch has
+ *                              room for them (whole 32-byte sectors are stored: a half-written sector costs a
+ *                              read-modify-write in the memory system), else up to the end of the last 16-byte
+ *                              granule; other pad lanes are left untouched.
  *   master weights w, momentum v, gradient g/dw : [K][R][S][C] fp32, dense (no pitch).
  *   bf16 weight shadow       : [K][R][S][ldw]  bf16, ldw >= C, ldw a multiple of 8.
  *   Output size: P = floor((H + 2*pad - R)/stride) + 1, Q likewise from W and S.
