@@ -86,6 +86,23 @@ def test_config3_pruned_bottleneck(algo):
         Hh.check_conv(dw, l.C, oracle.conv_wgrad(x.numpy(), dy.numpy(), l.R, l.R, l.stride, pad), what=l.name + " wgrad")
 
 
+# (N, H, W, C, K, R, stride): stride-2 weight gradients with few input channels (the generic kernel and the stem path):
+# odd and even tap groups, K above and below 64, 5x5 and 7x7 stems
+STRIDED_SMALL_C = [
+    (2, 16, 16, 20, 36, 3, 2), (2, 18, 18, 64, 128, 3, 2), (3, 16, 16, 7, 70, 5, 2), (2, 32, 32, 3, 16, 7, 2), (2, 12, 12, 1, 9, 5, 2),
+    (4, 20, 20, 33, 100, 2, 2),
+]
+
+
+@pytest.mark.parametrize("shape", STRIDED_SMALL_C)
+def test_strided_weight_gradient_with_few_input_channels(shape):
+    N, H, Wd, C, K, R, stride = shape
+    x, w, dy, pad = _case(N, H, Wd, C, K, R, stride, seed=W.BASE_SEED + 53)
+    dw = Hh.run_conv_all(N, H, Wd, C, K, R, stride, pad, x, w, dy, algo=2)[2]
+    Hh.check_conv(dw, C, oracle.conv_wgrad(x.numpy(), dy.numpy(), R, R, stride, pad), what="wgrad")
+    assert torch.equal(dw, Hh.run_conv_all(N, H, Wd, C, K, R, stride, pad, x, w, dy, algo=2)[2])
+
+
 # (N, H, W, C, K, R, pad): stride-1 filters with several taps and at most 64 input channels -- the weight gradient that
 # stages row blocks and pairs taps: two dy boxes (K > 64), several tap groups with an odd last one (K = 200), 25 taps,
 # a wide image, an even filter, padding 0 and padding larger than (R - 1) / 2
