@@ -143,3 +143,37 @@ def test_config4_full_size_sampled_batch64():
 @pytest.mark.parametrize("keep,N", [(0.3, 256), (0.6, 128), (1.0, 64)])
 def test_config5_sweep_points_sampled(keep, N):
     _sampled_step_check(keep, N, [0, 2, 12, 26, 45], n_samples=2048)
+
+
+def test_end_to_end_step_delivers_each_host_batch_one_step_later():
+    """The end-to-end step copies the NEXT batch from pinned host memory while the current one trains: the stem must see
+    batch k during call k + 1 (the first call brings its own), bit for bit, and the step's results must follow it."""
+    ctx = Hh.ctx()
+    net = W.vgg(11)
+    seed = W.BASE_SEED + 9
+    counts = W.uniform_keep(net, 0.6)
+    kept = W.choose_kept(net, counts, seed)
+    ts = harness.TrainStep(ctx, net, counts, kept, 16, seed, host_inputs=True, device_rng=True)
+    ts.step()
+    torch.cuda.synchronize()
+    ts.build_graph(two_streams=True)
+    g = torch.Generator().manual_seed(seed)
+    batches = [torch.randn(ts.h_image.shape, generator=g).to(ts.h_image.dtype) for _ in range(3)]
+    l0 = ts.net.layers[0]
+    ts.h_image.copy_(batches[0])
+    ts.step_e2e()                                   # trains on batch 0 (its own copy), stages batch 0 again
+    torch.cuda.synchronize()
+    assert torch.equal(ts.x[0].cpu(), batches[0])
+    ts.h_image.copy_(batches[1])                    # too late for the copy already made: call 2 still sees batch 0
+    ts.step_e2e()
+    torch.cuda.synchronize()
+    assert torch.equal(ts.x[0].cpu(), batches[0])
+    ts.h_image.copy_(batches[2])
+    ts.step_e2e()                                   # sees batch 1, staged during call 2
+    torch.cuda.synchronize()
+    ctx.poll()
+    assert torch.equal(ts.x[0].cpu(), batches[1])
+    w0 = oracle.gather_weight(ts.md.wb[0][..., :net.layers[0].C].float().cpu().numpy(), kept[l0.out_space], kept[l0.in_space])
+    x0 = batches[1][..., :l0.C].float().numpy()
+    Hh.check_conv(ts.y[0], l0.K, oracle.conv_fwd(x0, w0, l0.stride, l0.pad), what="e2e stem fwd")
+    assert float(ts.h_reg[0]) == float(ts.mp.reg.cpu()[0]) and float(ts.h_reg[0]) > 0
