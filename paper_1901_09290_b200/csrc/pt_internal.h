@@ -38,6 +38,11 @@ struct pt_ctx {
     // different callers must not evict each other: the lasso step and the detection have their own slot sets.
     pt_region lasso_tab[3], detect_tab[2], graph_tab, gather_tab;
     int lasso_next = 0, detect_next = 0;
+    // pt_reconfigure: the argument bytes the gather table in `gather_tab` was built from, and its launch shape. A call with
+    // the same arguments (every reconfiguration of a fixed pair of models) launches straight from the cached table.
+    std::vector<char> gather_args;
+    unsigned gather_chunks = 0;
+    size_t gather_jobs_bytes = 0;
     int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan
     unsigned int *d_sync = nullptr;     // zero-initialised, self-resetting arrival counters of the split weight gradient
     unsigned int sync_next = 0;         // ring position in d_sync

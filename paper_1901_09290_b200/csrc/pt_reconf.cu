@@ -177,12 +177,34 @@ extern "C" pt_status pt_reconfigure_plan(pt_ctx *c, const pt_graph *g, int32_t *
 
 extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t *new2old, const pt_graph *ng, void *stream)
 {
-    if (!c || !new2old) return PT_ERR_INVALID_ARG;
+    if (!c || !new2old || !og || !ng) return PT_ERR_INVALID_ARG;
+    if (!og->spaces || !og->layers || !og->links || !ng->spaces || !ng->layers || !ng->links) return PT_ERR_INVALID_ARG;
+    if (og->n_spaces <= 0 || og->n_layers <= 0 || og->n_spaces != ng->n_spaces || og->n_layers != ng->n_layers) return PT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    // The table below depends on the arguments only (shapes, pointers, the map's address), not on what the buffers hold:
+    // this call sits right behind the host synchronisation of the plan, so a repeated reconfiguration skips the rebuild.
+    std::vector<char> args;
+    {
+        const size_t ns = (size_t)og->n_spaces * sizeof(pt_space), nl = (size_t)og->n_layers * sizeof(pt_layer);
+        const size_t nk = (size_t)og->n_layers * sizeof(pt_layer_link);
+        args.resize(2 * (ns + nl + nk) + sizeof(new2old));
+        char *a = args.data();
+        memcpy(a, og->spaces, ns); a += ns; memcpy(a, ng->spaces, ns); a += ns;
+        memcpy(a, og->layers, nl); a += nl; memcpy(a, ng->layers, nl); a += nl;
+        memcpy(a, og->links, nk); a += nk; memcpy(a, ng->links, nk); a += nk;
+        memcpy(a, &new2old, sizeof(new2old));
+    }
+    if (c->gather_tab.valid && c->gather_chunks && args == c->gather_args) {
+        const char *dev = c->d_arena + c->gather_tab.off;
+        gather_kernel<<<c->gather_chunks, 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + c->gather_jobs_bytes));
+        c->launches += 1;
+        PT_CUDA_OK(cudaGetLastError());
+        return PT_OK;
+    }
     pt_status s = check_graph(og);
     if (s != PT_OK) return s;
     s = check_graph(ng);
     if (s != PT_OK) return s;
-    if (og->n_spaces != ng->n_spaces || og->n_layers != ng->n_layers) return PT_ERR_INVALID_ARG;
     std::vector<int> map_off(og->n_spaces);
     long long off = 0;
     for (int i = 0; i < og->n_spaces; ++i) {
@@ -230,12 +252,15 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
     std::vector<char> buf(jb + cb, 0);
     memcpy(buf.data(), jobs.data(), jobs.size() * sizeof(GatherJob));
     memcpy(buf.data() + jb, chunks.data(), cb);
-    cudaStream_t st = (cudaStream_t)stream;
     char *dev = nullptr;
+    c->gather_chunks = 0;
     s = pt_upload_table(c, &c->gather_tab, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
     gather_kernel<<<(unsigned)chunks.size(), 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + jb));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
+    c->gather_args.swap(args);
+    c->gather_chunks = (unsigned)chunks.size();
+    c->gather_jobs_bytes = jb;
     return PT_OK;
 }
