@@ -452,6 +452,7 @@ struct HaloP {
     int a_box_bytes, a_alloc;            // bytes one A load brings / bytes reserved per A stage
     int stages_a, stages_b, resident;    // ring depths; resident: weights loaded once
     int n_issuers, acc_per;              // MMA issuer warps (each with its own A ring of stages_a / n_issuers stages); accumulators per issuer (1 or 2)
+    int shared_b;                        // two pipelines fed by ONE weight stream: a stage is read by both issuers (their tiles of a round)
     int row32;                           // 1: 16 channel lanes per pixel, 32-byte rows and swizzle (the space-to-depth stem): one MMA per tap
     int b_slot, b_rows, staging;         // bytes reserved per weight tile, rows a K-major weight box brings, bytes of an epilogue group's staging slab
     int tmem_cols, tma_store, out_f32, ld_out;
@@ -508,7 +509,7 @@ struct __align__(8) HCtl {
 };
 
 // warp 0 (and 13): TMA producers; warp 1 and warps 10..12: MMA issuers; warps 2..9: two groups of four epilogue warps
-constexpr int kHaloThreads = 448;
+constexpr int kHaloThreads = 512;
 
 // Issuing one tcgen05.mma costs the issuing warp 50 to 100 cycles of instruction time, more than a narrow MMA (N <= 64)
 // takes to execute, so with a single issuer the tensor pipe of a small-channel layer idles most of the time. The
@@ -539,7 +540,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages_a; ++s) { mbar_init(smem_u32(&ctl->full_a[s]), 1); mbar_init(smem_u32(&ctl->empty_a[s]), 1); }
-        for (int s = 0; s < p.stages_b; ++s) { mbar_init(smem_u32(&ctl->full_b[s]), 1); mbar_init(smem_u32(&ctl->empty_b[s]), 1); }
+        for (int s = 0; s < p.stages_b; ++s) { mbar_init(smem_u32(&ctl->full_b[s]), 1); mbar_init(smem_u32(&ctl->empty_b[s]), p.shared_b ? 2 : 1); }
         mbar_init(smem_u32(&ctl->w_full), 1);
         for (int b = 0; b < 2 * kHaloMaxIssuers; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 4); }
         ctl->abort_flag = 0;
@@ -558,17 +559,26 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int issuer = warp == 1 ? 0 : warp - 9;             // warps 10, 11, 12 -> issuers 1, 2, 3
-    if (!(warp == 0 && p.resident)) grid_dependency_wait();   // the producer first issues the resident weights (see below)
+    // the weight producers do not read the previous kernel's output: resident weights are issued first and the wait follows
+    // them (below); the producers of streamed weights never need it
+    if (!(warp == 0 || (warp == 13 && !p.resident))) grid_dependency_wait();
     grid_launch_dependents();
 
     // Streamed weights with two issuers: two complete pipelines (producer warp, A ring, B ring, issuer warp, accumulators),
     // one per tile parity. Resident weights: one producer feeds every issuer's A ring.
+    // With `shared_b` the two pipelines read the same weight stages: the tiles of a round (blockIdx.x + 2r*grid and + (2r+1)*grid)
+    // use the same weights, so one stream through the whole ring feeds both issuers, half the bytes and twice the depth.
     const int n_prod = p.resident ? 1 : NI;
-    const int SB = p.stages_b / n_prod;                       // weight stages per pipeline
-    if (warp == 0 || (warp == 13 && n_prod == 2)) {
+    const int SB = p.shared_b ? p.stages_b : p.stages_b / n_prod;     // weight stages per weight stream
+    // Streamed weights: the activation boxes have a producer warp of their own per pipeline (14, 15), so that the next tile's
+    // boxes go out as soon as their stage is free instead of behind the weight loads of the current tile, which wait for the
+    // MMAs (the next tile's activations used to be issued only when the current tile was nearly done: ~4 us per tile exposed).
+    const bool a_warp = !p.resident && (warp == 14 || (warp == 15 && n_prod == 2));
+    if (warp == 0 || (warp == 13 && n_prod == 2 && !p.shared_b) || a_warp) {
         if (lane == 0) {
             // ---------------- TMA producer(s)
-            const int pid = warp == 0 ? 0 : 1;
+            const int pid = (warp == 0 || warp == 14) ? 0 : 1;
+            const bool a_role = a_warp || p.resident, b_role = !a_warp && !p.resident;
             if (p.resident) {
                 // n_tiles == 1 here: the whole weight tensor of the layer, tap by tap and chunk by chunk, once
                 const uint32_t bar = smem_u32(&ctl->w_full);
@@ -598,15 +608,17 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                 for (int kc = 0; kc < p.k_chunks && ok; ++kc) {
                     const int sa = ring * SR + pos, ph_use = pha;
                     if (++pos == SR) { pos = 0; pha ^= 1; }
-                    ok = mbar_wait(smem_u32(&ctl->empty_a[sa]), ph_use ^ 1, abort_flag, p.status, 11);
-                    if (!ok) break;
-                    const uint32_t bar = smem_u32(&ctl->full_a[sa]);
-                    HTRACE(0, tc);
-                    mbar_arrive_expect_tx(bar, (uint32_t)p.a_box_bytes);
-                    tma_load_4d(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, &tmA, bar, kc * kKC, p.lo_w, p0 + p.lo_h, img);
-                    if (p.resident) continue;
+                    if (a_role) {
+                        ok = mbar_wait(smem_u32(&ctl->empty_a[sa]), ph_use ^ 1, abort_flag, p.status, 11);
+                        if (!ok) break;
+                        const uint32_t bar = smem_u32(&ctl->full_a[sa]);
+                        HTRACE(0, tc);
+                        mbar_arrive_expect_tx(bar, (uint32_t)p.a_box_bytes);
+                        tma_load_4d(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, &tmA, bar, kc * kKC, p.lo_w, p0 + p.lo_h, img);
+                    }
+                    if (!b_role) continue;
                     for (int tap = 0; tap < p.taps; ++tap) {
-                        const int sb = pid * SB + sb_pos, phb = sb_ph;
+                        const int sb = (p.shared_b ? 0 : pid * SB) + sb_pos, phb = sb_ph;
                         if (++sb_pos == SB) { sb_pos = 0; sb_ph ^= 1; }
                         ok = mbar_wait(smem_u32(&ctl->empty_b[sb]), phb ^ 1, abort_flag, p.status, 12);
                         if (!ok) break;
@@ -629,7 +641,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                     base_ph ^= wraps & 1;
                 }
             }
-            if (*abort_flag && pid == 0) {   // bounded drain of the copies in flight before the shared memory is released
+            if (*abort_flag && pid == 0 && a_role) {   // bounded drain of the copies in flight before the shared memory is released
                 const uint64_t t0 = globaltimer_ns();
                 for (int s = 0; s < p.stages_a; ++s)
                     while (!mbar_try_wait(smem_u32(&ctl->full_a[s]), 0) && !mbar_try_wait(smem_u32(&ctl->full_a[s]), 1) &&
@@ -649,7 +661,19 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         int nt = 0;                                           // tiles this issuer has started
         for (int tc = issuer; ok; tc += NI, ++nt) {
             const int tile = blockIdx.x + tc * (int)gridDim.x;
-            if (tile >= total_tiles) break;
+            if (tile >= total_tiles) {
+                // shared weight stream: the other issuer may still have a tile in this round; its stages need this issuer's
+                // release too, given in step with the stream
+                if (p.shared_b && issuer == 1 && tile - (int)gridDim.x < total_tiles) {
+                    for (int i = 0; i < p.k_chunks * p.taps && ok; ++i) {
+                        const int sb = sb_pos, phb = sb_ph;
+                        if (++sb_pos == SB) { sb_pos = 0; sb_ph ^= 1; }
+                        ok = mbar_wait(smem_u32(&ctl->full_b[sb]), phb, abort_flag, p.status, 16);
+                        if (ok && lane == 0) mbar_arrive(smem_u32(&ctl->empty_b[sb]));
+                    }
+                }
+                break;
+            }
             // accumulator buffers issuer*acc_per .. +acc_per-1, used in turn
             const int b = p.acc_per == 2 ? issuer * 2 + (nt & 1) : issuer, aph = p.acc_per == 2 ? (nt >> 1) & 1 : nt & 1;
             ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), aph ^ 1, abort_flag, p.status, 14);
@@ -694,7 +718,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                     }
                 } else {
                     for (int tap = 0; tap < p.taps; ++tap) {
-                        const int sb = issuer * SB + sb_pos, phb = sb_ph;
+                        const int sb = (p.shared_b ? 0 : issuer * SB) + sb_pos, phb = sb_ph;
                         if (++sb_pos == SB) { sb_pos = 0; sb_ph ^= 1; }
                         ok = mbar_wait(smem_u32(&ctl->full_b[sb]), phb, abort_flag, p.status, 16);
                         if (!ok) break;
@@ -1785,6 +1809,7 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     } else if (two_pipes) {
         p.n_issuers = 2;
         p.acc_per = 4 * p.BN <= 512 ? 2 : 1;
+        p.shared_b = p.n_tiles == 1 ? 1 : 0;          // the tiles of a round then use the same weight columns
     }
     p.stages_a = p.stages_a / p.n_issuers * p.n_issuers;
     p.tmem_cols = pow2_cols(p.n_issuers * p.acc_per * p.BN);
