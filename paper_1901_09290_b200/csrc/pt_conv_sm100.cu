@@ -1791,6 +1791,15 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
         // two pipelines (one per tile parity) when each can have three weight stages and the CTAs get several tiles
         two_pipes = p.stages_b >= 6 && pt_ceil_div(p.N * p.row_tiles * p.n_tiles, c->sm_count) >= 2;
         if (two_pipes) p.stages_b = p.stages_b / 2 * 2;
+        // Two pipelines on one weight stream (a single channel tile): every chunk of both tiles should have an activation stage
+        // of its own -- a chunk that waits for the previous chunk's MMAs to free its stage exposes a DRAM round trip per tile
+        // (28x28, 69 -> 93 channels, MN-major weights: two stages against four, 30 -> 22 us) -- as long as four weight stages
+        // remain for the shared stream.
+        const int want_a = 2 * p.k_chunks > 4 ? 4 : 2 * p.k_chunks;
+        if (two_pipes && p.n_tiles == 1 && left >= (size_t)want_a * p.a_alloc + 4 * b_bytes) {
+            const size_t sb2 = (left - (size_t)want_a * p.a_alloc) / b_bytes;
+            if ((size_t)p.stages_b > sb2) p.stages_b = (int)sb2;
+        }
         left -= (size_t)p.stages_b * b_bytes;
         int sa = (int)(left / p.a_alloc);
         p.stages_a = sa > 4 ? 4 : sa;
