@@ -508,7 +508,8 @@ struct __align__(8) HCtl {
     int abort_flag;
 };
 
-// warp 0 (and 13): TMA producers; warp 1 and warps 10..12: MMA issuers; warps 2..9: two groups of four epilogue warps
+// warp 0 (and 13): TMA producers (weights; with resident weights warp 0 also brings the activations); warps 14, 15: activation
+// producers of the streamed-weight pipelines; warp 1 and warps 10..12: MMA issuers; warps 2..9: two groups of four epilogue warps
 constexpr int kHaloThreads = 512;
 
 // Issuing one tcgen05.mma costs the issuing warp 50 to 100 cycles of instruction time, more than a narrow MMA (N <= 64)
