@@ -42,6 +42,7 @@ struct WsLayout {
 constexpr int kThreads = 256;
 constexpr int kUnroll = 8;                // lines in flight per thread
 constexpr int kSweeps = 4;                // unrolled sweeps per chunk: every block does the same number of iterations
+constexpr int kUpdateSplit = 2;           // blocks per chunk in the update kernel
 
 // Eight per-lane values (one per line) are reduced over the 32 lanes with 9 shuffles instead of 40: three
 // halving exchanges leave lane l with the partial of line (l >> 2) & 7 over its 4-lane group's share, two more
@@ -188,7 +189,10 @@ __global__ void __launch_bounds__(kThreads) update_kernel(const LayerDev *__rest
                                                           const float *__restrict__ inv_out,
                                                           const float *__restrict__ inv_in, pt_sgd_hparams hp)
 {
-    const Chunk ch = chunks[blockIdx.x];
+    // kUpdateSplit blocks share a chunk (alternate sweeps): the update has no per-chunk results to combine, and the finer
+    // grain wastes less of the last wave
+    const Chunk ch = chunks[blockIdx.x / kUpdateSplit];
+    const int sub = blockIdx.x % kUpdateSplit;
     const LayerDev L = layers[ch.layer];
     const int TX = 1 << L.tx_log2, TY = kThreads >> L.tx_log2;
     const int tx = threadIdx.x & (TX - 1), ty = threadIdx.x >> L.tx_log2;
@@ -196,7 +200,7 @@ __global__ void __launch_bounds__(kThreads) update_kernel(const LayerDev *__rest
     if (c >= L.C) return;
     const float ci = inv_in[L.c_off + c];
     const float *io = inv_out + L.k_off;
-    for (int l = ty; l < ch.nlines; l += kUnroll * TY) {
+    for (int l = ty + sub * kUnroll * TY; l < ch.nlines; l += kUpdateSplit * kUnroll * TY) {
         float w[kUnroll], g[kUnroll], v[kUnroll], ko[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
@@ -427,7 +431,7 @@ static pt_status lasso_phases(pt_ctx *c, const pt_layer *layers, int32_t n, cons
                 if (t.chunks[i].layer >= first && t.chunks[i].layer < first + count) { c0 = i < c0 ? i : c0; c1 = i + 1; }
         }
         if (c1 > c0) {
-            update_kernel<<<c1 - c0, kThreads, 0, st>>>(dl, dc + c0, inv_out, inv_in, *hp);
+            update_kernel<<<(c1 - c0) * kUpdateSplit, kThreads, 0, st>>>(dl, dc + c0, inv_out, inv_in, *hp);
             c->launches += 1;
         }
     }
