@@ -1691,9 +1691,17 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     // one tile per CTA and streamed weights: the output is staged in the ring (all of its stages have been consumed when the
     // accumulator is complete), which leaves room for one more stage
     p.alias_staging = (per_cta == 1 && !p.resident) ? 1 : 0;
-    const size_t staging2 = p.alias_staging ? 0 : (size_t)p.epi_groups * 4 * kSlabs * 4096;
+    size_t staging2 = p.alias_staging ? 0 : (size_t)p.epi_groups * 4 * kSlabs * 4096;
     if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all, &smem);
-    else p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2, &smem);
+    else {
+        p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2, &smem);
+        if (p.stages < 4 && p.epi_groups == 3 && p.taps * p.k_chunks * per_cta >= 4) {
+            // a third epilogue group costs 32 KB of staging: with wide weight tiles that is the fourth pipeline stage
+            p.epi_groups = 2;
+            staging2 = (size_t)p.epi_groups * 4 * kSlabs * 4096;
+            p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2, &smem);
+        }
+    }
     if (p.n_issuers == 2) {
         p.stages = p.stages / 2 * 2;
         if (p.stages < 2) { p.n_issuers = 1; p.acc_per = 1; p.stages = 2; }
