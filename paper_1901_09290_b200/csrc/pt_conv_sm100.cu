@@ -101,6 +101,16 @@ struct __align__(8) PCtl {
 
 constexpr uint32_t kSlabs = 2;                          // staging slabs per epilogue warp (TMA stores in flight)
 
+// Device-side timeline of CTA 0 (a build with -DPT_DEVICE_TRACE; read back with pt_debug_gemm_trace): per pipeline stage in
+// issue order, when the A producer found it free / issued it, when the MMA issuer found it full / committed it; per tile, when
+// the epilogue got the accumulator and when it had issued its stores.
+#ifdef PT_DEVICE_TRACE
+__device__ unsigned long long g_gemm_trace[8][64];
+#define GTRACE(role, idx) do { if (blockIdx.x == 0 && (idx) < 64 && (threadIdx.x & 31) == 0) g_gemm_trace[role][idx] = globaltimer_ns(); } while (0)
+#else
+#define GTRACE(role, idx) do { } while (0)
+#endif
+
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... The TMA ring runs continuously across
 // tiles. The accumulator has G = 2 or 3 buffers in TMEM and buffer b has its own group of four epilogue warps, so the
 // loads and MMAs of the next tiles overlap the epilogues of the previous ones.
@@ -203,6 +213,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     for (int kc = 0; kc < p.k_chunks; ++kc) {
                         ok = mbar_wait(smem_u32(&ctl->empty[sbase + s]), ph ^ 1, abort_flag, p.status, 1);
                         if (!ok) break;
+                        if (is_a) GTRACE(0, issued); else if (warp == 14) GTRACE(2, issued);
                         const uint32_t bar = smem_u32(&ctl->full[sbase + s]);
                         const uint32_t a_dst = data_base + (uint32_t)(sbase + s) * stage_bytes, b_dst = a_dst + a_bytes;
                         mbar_arrive_expect_tx(bar, my_bytes);
@@ -215,6 +226,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                             for (int nb = bsel; nb < nb_b; nb += nbp)
                                 tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
                         }
+                        if (is_a) GTRACE(1, issued); else if (warp == 14) GTRACE(3, issued);
                         ++issued;
                         if (++s == SR) { s = 0; ph ^= 1; }
                     }
@@ -241,6 +253,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         const int NI = p.n_issuers, issuer = warp == 1 ? 0 : 1;
         const int SR = p.stages / NI, sbase = issuer * SR;
         int s = 0, ph = 0, b = 0, aph = 0, nt = 0;
+        int consumed = 0;
+        (void)consumed;
         bool ok = true;
         if (p.resident) ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort_flag, p.status, 8);
         for (int tile = blockIdx.x + issuer * (int)gridDim.x; tile < total_tiles && ok; tile += NI * (int)gridDim.x, ++nt) {
@@ -254,6 +268,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                 for (int kc = 0; kc < p.k_chunks; ++kc) {
                     ok = mbar_wait(smem_u32(&ctl->full[sbase + s]), ph, abort_flag, p.status, 2);
                     if (!ok) break;
+                    if (warp == 1) GTRACE(4, consumed);
                     tc_fence_after();
                     const uint32_t a_src = data_base + (uint32_t)(sbase + s) * stage_bytes;
                     const uint32_t b_src = p.resident ? w_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot : a_src + a_bytes;
@@ -270,6 +285,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     }
                     acc = 1u;
                     umma_commit_lead(smem_u32(&ctl->empty[sbase + s]), leader);   // frees the stage when these MMAs have read it
+                    if (warp == 1) GTRACE(5, consumed);
+                    ++consumed;
                     if (++s == SR) { s = 0; ph ^= 1; }
                 }
             }
@@ -331,6 +348,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             }
             ok = mbar_wait(smem_u32(&ctl->acc_full[b]), aph, abort_flag, p.status, 3);
             if (!ok) break;
+            if (quarter == 0) GTRACE(6, tc);
             tc_fence_after();
             const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.BN);
             if (p.tma_store) {
@@ -378,6 +396,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         tma_store_commit();
                     }
                 }
+                if (quarter == 0) GTRACE(7, tc);
                 continue;
             }
             // ---- direct stores (fp32 outputs, strided stride-2 data-gradient outputs)
@@ -490,7 +509,7 @@ struct TileWalk {
 };
 // Device-side timeline for tuning: a build with -DPT_DEVICE_TRACE makes CTA 0 stamp %globaltimer at the hand-over points of
 // each role (producer issue, accumulator free, operands landed, MMAs committed, epilogue start, store issued) and exports
-// pt_debug_halo_trace / pt_debug_wgrad_trace to read the stamps back. The normal build compiles the macros away.
+// pt_debug_halo_trace / pt_debug_wgrad_trace / pt_debug_gemm_trace to read the stamps back. The normal build compiles the macros away.
 #ifdef PT_DEVICE_TRACE
 __device__ unsigned long long g_halo_trace[8][64];
 #define HTRACE(role, idx) do { if (blockIdx.x == 0 && (idx) < 64 && (threadIdx.x & 31) == 0) g_halo_trace[role][idx] = globaltimer_ns(); } while (0)
@@ -2505,6 +2524,10 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
 extern "C" int pt_debug_wgrad_trace(unsigned long long *host_out)
 {
     return (int)cudaMemcpyFromSymbol(host_out, g_wg_trace, sizeof(unsigned long long) * 8 * 64);
+}
+extern "C" int pt_debug_gemm_trace(unsigned long long *host_out)
+{
+    return (int)cudaMemcpyFromSymbol(host_out, g_gemm_trace, sizeof(unsigned long long) * 8 * 64);
 }
 extern "C" int pt_debug_halo_trace(unsigned long long *host_out)
 {
