@@ -179,3 +179,55 @@ def test_empty_keep_set_and_second_reconfiguration():
         mc = mapsA[l.in_space][mapsB[l.in_space]]
         ref = oracle.gather_weight(m.w[li].numpy(), mk, mc)
         assert np.array_equal(dnB.w[li].cpu().numpy(), ref)
+
+
+def test_repeated_reconfiguration_reads_current_contents_and_rebuilds_for_new_arguments():
+    """A repeated call with the same arguments launches from the cached gather table: the table holds addresses and shapes
+    only, so the second call must carry over whatever the source buffers hold by then; a call with other destinations must
+    not reuse it."""
+    net = W.resnet32()
+    kept = W.choose_kept(net, W.random_keep(net, W.BASE_SEED + 12), W.BASE_SEED + 12)
+    model = W.gen_model(net, W.BASE_SEED + 12, kept=kept, decoys=1)
+    dm = DevModel(model)
+    dn, maps, sizes = reconfigure(dm)
+    check_against_oracle(model, dm, dn, maps, sizes)
+    c = Hh.ctx()
+    # same masks and maps; the kept entries of the source get new values (zero groups stay zero, so the plan stands)
+    new2old = torch.full((sum(net.space_sizes),), -1, dtype=torch.int32, device="cuda")
+    off = 0
+    for s, size in enumerate(net.space_sizes):
+        new2old[off:off + sizes[s]] = torch.from_numpy(maps[s]).cuda()
+        off += size
+    g_old, g_new = dm.graph(), dn.graph()
+    B.pt_reconfigure(c, g_old, new2old, g_new)          # builds the table for these arguments
+    for w in dm.w:
+        w.mul_(3.0)
+    for v in dm.v:
+        v.add_(0.25)
+    B.pt_reconfigure(c, g_old, new2old, g_new)          # same arguments: cached table, current contents
+    torch.cuda.synchronize()
+    c.poll()
+    for li, l in enumerate(net.layers):
+        mk, mc = maps[l.out_space], maps[l.in_space]
+        ref_w = oracle.gather_weight(dm.w[li].cpu().numpy(), mk, mc)
+        ref_v = oracle.gather_weight(dm.v[li].cpu().numpy(), mk, mc)
+        assert np.array_equal(dn.w[li].cpu().numpy().view(np.uint32), ref_w.view(np.uint32)), l.name
+        assert np.array_equal(dn.v[li].cpu().numpy().view(np.uint32), ref_v.view(np.uint32)), l.name
+    # other destinations: a fresh model of the same shapes must be filled, and the first one left as it is
+    snap = [w.clone() for w in dn.w]
+    for w in dm.w:
+        w.mul_(0.5)
+    new_net = W.with_sizes(net, sizes)
+    empty = W.Model(new_net, [torch.full((l.K, l.R, l.R, l.C), 7.0) for l in new_net.layers],
+                    [torch.full((l.K, l.R, l.R, l.C), 7.0) for l in new_net.layers],
+                    [torch.zeros((l.K, l.R, l.R, l.C)) for l in new_net.layers],
+                    [[torch.full((l.K,), 7.0) for _ in range(4)] for l in new_net.layers])
+    d2 = DevModel(empty)
+    B.pt_reconfigure(c, g_old, new2old, d2.graph())
+    torch.cuda.synchronize()
+    c.poll()
+    for li, l in enumerate(net.layers):
+        mk, mc = maps[l.out_space], maps[l.in_space]
+        ref_w = oracle.gather_weight(dm.w[li].cpu().numpy(), mk, mc)
+        assert np.array_equal(d2.w[li].cpu().numpy().view(np.uint32), ref_w.view(np.uint32)), l.name
+        assert torch.equal(dn.w[li], snap[li]), l.name
