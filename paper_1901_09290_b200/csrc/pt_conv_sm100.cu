@@ -1740,12 +1740,14 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
 
 // Source activations as a tiled 4-D tensor (C, W, H, N): box 64 channels x box_w x box_h x 1 (the halo tile).
 // `lanes` = 64 (128-byte rows and swizzle) or 16 (32-byte rows and swizzle).
+// `row_pixels` > 0: pixels between the starts of consecutive rows when that is not W (a padded row).
 bool make_halo_in_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, int W, int H, int N, int ld, int box_w, int box_h,
-                      int lanes = kKC)
+                      int lanes = kKC, int row_pixels = 0)
 {
     if (!c->encode_tiled || box_w > 256 || box_h > 256) return false;
+    const cuuint64_t rp = row_pixels > 0 ? (cuuint64_t)row_pixels : (cuuint64_t)W;
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
-    cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)W * ld * 2, (cuuint64_t)H * W * ld * 2};
+    cuuint64_t strides[3] = {(cuuint64_t)ld * 2, rp * ld * 2, (cuuint64_t)H * rp * ld * 2};
     cuuint32_t box[4] = {(cuuint32_t)lanes, (cuuint32_t)box_w, (cuuint32_t)box_h, 1}, estr[4] = {1, 1, 1, 1};
     CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box,
                                                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, lanes == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_128B,
@@ -2119,8 +2121,10 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
 }
 
 // Launches the row-block weight-gradient kernel; PT_ERR_UNSUPPORTED (nothing launched) where the plan declines the shape.
+// `x_row_pixels` > 0 and (lo_h, lo_w): x is a view whose rows are x_row_pixels apart and whose raster origin for tap (0, 0)
+// is at (lo_h, lo_w) instead of (-pad, -pad) -- the space-to-depth stem, whose "pixels" are overlapping 4-pixel windows.
 pt_status run_wgrad_rows(pt_ctx *c, const pt_conv_desc *d, int P, int Q, const void *x, const void *dy, float *out, void *ws,
-                         size_t ws_bytes, cudaStream_t st)
+                         size_t ws_bytes, cudaStream_t st, int x_row_pixels = 0, int lo_h = 0, int lo_w = 0)
 {
     const WgRows wr = wgrad_rows_plan(c, d, P, Q);
     if (!wr.ok || !c->encode_tiled) return PT_ERR_UNSUPPORTED;
@@ -2133,6 +2137,7 @@ pt_status run_wgrad_rows(pt_ctx *c, const pt_conv_desc *d, int P, int Q, const v
     p.npix = d->N * P * Q;
     p.splits = wr.splits;
     p.Pd = P; p.Qd = Q; p.stride = 1; p.lo_h = -d->pad; p.lo_w = -d->pad;
+    if (x_row_pixels > 0) { p.lo_h = lo_h; p.lo_w = lo_w; }
     p.nr = wr.nr; p.Wp = wr.Wp; p.RB = wr.RB; p.units = wr.units; p.units_per_split = wr.units_per_split;
     p.ksteps = wr.ksteps; p.nb_a = wr.nb_a; p.lo_span = d->R - 1; p.a_box = wr.a_box; p.b_box = wr.b_box;
     p.stages = wr.stages;
@@ -2154,7 +2159,7 @@ pt_status run_wgrad_rows(pt_ctx *c, const pt_conv_desc *d, int P, int Q, const v
     }
     // dy: box of nr rows x Wp columns (Wp > Q: the extra columns are out of bounds and read as zeros); x: the halo box
     if (!make_halo_in_map(c, &tmA, dy, d->K, Q, P, d->N, d->ldy, wr.Wp, wr.nr)) return PT_ERR_UNSUPPORTED;
-    if (!make_halo_in_map(c, &tmX, x, d->C, d->W, d->H, d->N, d->ldx, wr.Wp, wr.nr + d->R - 1)) return PT_ERR_UNSUPPORTED;
+    if (!make_halo_in_map(c, &tmX, x, d->C, d->W, d->H, d->N, d->ldx, wr.Wp, wr.nr + d->R - 1, kKC, x_row_pixels)) return PT_ERR_UNSUPPORTED;
     static bool attr_set = false;
     if (!attr_set) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_wgrad_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
@@ -2274,6 +2279,15 @@ static pt_conv_desc stem_virtual_desc(const pt_conv_desc *d, const StemPlan &sp)
     return v;
 }
 
+// The same for the row-block kernel: a stride-1 U x 1 filter over Q x Hs "pixels" of 64 lanes whose rows are Wp real pixels
+// (16 lanes each) apart; pixel j of a row is the window of real pixels j .. j+3.
+static pt_conv_desc stem_rows_desc(const pt_conv_desc *d, const StemPlan &sp)
+{
+    pt_conv_desc v = stem_virtual_desc(d, sp);
+    v.stride = 1; v.W = sp.Q; v.H = sp.Hs; v.ldx = 16;
+    return v;
+}
+
 // CTAs the weight gradient of `d` launches at the context's current CTA limit: tiles x splits; *waits = 1 if they wait for
 // one another (splits > 1).
 int pt_sm100_wgrad_ctas(const pt_ctx *c, const pt_conv_desc *d, int *waits)
@@ -2282,8 +2296,9 @@ int pt_sm100_wgrad_ctas(const pt_ctx *c, const pt_conv_desc *d, int *waits)
     pt_conv_desc v = sp.ok ? stem_virtual_desc(d, sp) : *d;
     const int P = sp.ok ? sp.P : pt_out_dim(d->H, d->R, d->stride, d->pad), Q = sp.ok ? sp.Q : pt_out_dim(d->W, d->S, d->stride, d->pad);
     int tiles, splits;
-    const WgRows wr = sp.ok ? WgRows() : wgrad_rows_plan(c, &v, P, Q);
-    if (!sp.ok && wr.ok) {
+    const pt_conv_desc vr = sp.ok ? stem_rows_desc(d, sp) : v;
+    const WgRows wr = wgrad_rows_plan(c, &vr, P, Q);
+    if (wr.ok) {
         tiles = wr.n_tiles * wr.m_tiles * wr.tap_groups;
         splits = wr.splits;
     } else {
@@ -2302,8 +2317,9 @@ size_t pt_sm100_conv_workspace(const pt_ctx *c, const pt_conv_desc *d, int which
     const StemPlan sp = stem_plan(d);
     if (sp.ok && which == PT_CONV_FWD) return sp.xs_bytes + pt_align_up(sp.w2_elems * 2, 1024);
     if (sp.ok && which == PT_CONV_WGRAD) {
-        const pt_conv_desc v = stem_virtual_desc(d, sp);
-        return sp.xs_bytes + pt_align_up(sp.w2_elems * 4, 1024) + wgrad_partial_bytes(c, &v, sp.P, sp.Q);
+        const pt_conv_desc v = stem_virtual_desc(d, sp), vr = stem_rows_desc(d, sp);
+        const size_t pa = wgrad_partial_bytes(c, &v, sp.P, sp.Q), pb = wgrad_partial_bytes(c, &vr, sp.P, sp.Q);
+        return sp.xs_bytes + pt_align_up(sp.w2_elems * 4, 1024) + (pa > pb ? pa : pb);
     }
     if (which != PT_CONV_WGRAD) return 0;
     const int P = pt_out_dim(d->H, d->R, d->stride, d->pad), Q = pt_out_dim(d->W, d->S, d->stride, d->pad);
@@ -2328,10 +2344,16 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
             stem_s2d_x_kernel_launch((unsigned)((tot + 255) / 256), st, (const __nv_bfloat16 *)a, xs, d->N, d->H, d->W, d->C, sp.Hs, sp.Ws,
                                      sp.Wp, sp.pl);
             c->launches += 1;
-            CUtensorMap tmX;
-            const int up_h = (sp.P - 1) - sp.pl - (sp.Hs - 1);
-            if (!make_im2col_map(c, &tmX, xs, 64, sp.Q, sp.Hs, d->N, 16, 0, -sp.pl, 0, up_h, 1, 64, sp.Wp)) return PT_ERR_CUDA;
-            pt_status r = run_wgrad(c, &v, sp.P, sp.Q, 1, -sp.pl, 0, tmX, b, dw2, part, ws_bytes - (size_t)(part - wsb), st);
+            // the row-block kernel first: the windows of a unit of rows are staged once for all U vertical taps and two taps share
+            // an MMA (M = 128 lanes where the generic kernel has 55 output channels on its M side)
+            const pt_conv_desc vr = stem_rows_desc(d, sp);
+            pt_status r = run_wgrad_rows(c, &vr, sp.P, sp.Q, xs, b, dw2, part, ws_bytes - (size_t)(part - wsb), st, sp.Wp, -sp.pl, 0);
+            if (r == PT_ERR_UNSUPPORTED) {
+                CUtensorMap tmX;
+                const int up_h = (sp.P - 1) - sp.pl - (sp.Hs - 1);
+                if (!make_im2col_map(c, &tmX, xs, 64, sp.Q, sp.Hs, d->N, 16, 0, -sp.pl, 0, up_h, 1, 64, sp.Wp)) return PT_ERR_CUDA;
+                r = run_wgrad(c, &v, sp.P, sp.Q, 1, -sp.pl, 0, tmX, b, dw2, part, ws_bytes - (size_t)(part - wsb), st);
+            }
             if (r != PT_OK) return r;
             const int n = d->K * d->R * d->S * d->C;
             stem_dw_back_kernel<<<(n + 255) / 256, 256, 0, st>>>(dw2, (float *)out, d->K, d->R, d->S, d->C, sp.U, sp.off);
