@@ -197,8 +197,8 @@ class TrainStep:
         l = self.net.layers[li]
         px = self.N * l.P * l.P
         taps = l.R * l.R
-        if l.stride == 2 and l.C <= 4:                       # space-to-depth stem: (R+1)/2 vertical taps of 64 lanes
-            mmas = px / 16 * ((l.R + 1) // 2)
+        if l.stride == 2 and l.C <= 4:                       # space-to-depth stem: (R+1)/2 vertical taps of 64 lanes, two per MMA
+            mmas = px / 16 * (((l.R + 1) // 2 + 1) // 2)
             cyc = 55
         elif l.stride == 1 and l.C <= 64:                    # row-block kernel: two taps per MMA, N = K
             mmas = px / 16 * ((taps + 1) // 2)
