@@ -234,7 +234,7 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         const int lines = n.K * n.RS;
         int TX = 32;
         while (TX < n.C && TX < 256) TX <<= 1;
-        const int per = (256 / TX) * kGatherUnroll * 4;      // equal trip counts for every block
+        const int per = (256 / TX) * kGatherUnroll * 3;      // equal trip counts for every block
         for (int l0 = 0; l0 < lines; l0 += per)
             for (int c0 = 0; c0 < n.C; c0 += TX) chunks.push_back(GatherChunk{job, l0, lines - l0 < per ? lines - l0 : per, c0});
         for (int b = 0; b < 4; ++b) {
