@@ -1819,7 +1819,9 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
         size_t sb = (left - 2 * (size_t)p.a_alloc) / b_bytes;
         p.stages_b = sb > kMaxStages ? kMaxStages : (int)sb;
         // two pipelines (one per tile parity) when each can have three weight stages and the CTAs get several tiles
-        two_pipes = p.stages_b >= 6 && pt_ceil_div(p.N * p.row_tiles * p.n_tiles, c->sm_count) >= 2;
+        // (a launch that shares the SMs with others has fewer CTAs, each with more tiles)
+        const int ctas_avail = (h.max_ctas > 0 && h.max_ctas < c->sm_count) ? h.max_ctas : c->sm_count;
+        two_pipes = p.stages_b >= 6 && pt_ceil_div(p.N * p.row_tiles * p.n_tiles, ctas_avail) >= 2;
         if (two_pipes) p.stages_b = p.stages_b / 2 * 2;
         // Two pipelines on one weight stream (a single channel tile): every chunk of both tiles should have an activation stage
         // of its own -- a chunk that waits for the previous chunk's MMAs to free its stage exposes a DRAM round trip per tile
