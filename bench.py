@@ -402,7 +402,7 @@ def run_ours(args):
                    "launch": "eager" if args.no_graph else ("CUDA graph replay after the reconfiguration's host sync; "
                                                             + ("1 stream" if args.one_stream else f"streams along the network's data dependencies: dgrad chain, projection shortcuts beside their blocks, wgrads round-robin on {ts.wgrad_streams} streams at <= {ts.wgrad_ctas} CTAs each" + (f" nominal; per-launch limits {min(ts.wgrad_limit.values())}..{max(ts.wgrad_limit.values())} CTAs from a work-per-CTA dynamic programme, every three consecutive launches within the SM count, the last three sharing the SMs as {[ts.wgrad_limit[k] for k in (2, 1, 0)]}" if ts.wgrad_limit else "")))},
         "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / args.steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "pipeline": "one pinned-host image copy per step on a copy stream, overlapping the previous step's kernels"},
+                "pipeline": "one pinned-host image copy per step on a copy stream into the other of two stem-input buffers (one CUDA graph per buffer), overlapping the current step's kernels"},
         "gpu_launches": launches,
         "clocks": clocks,
         "phases_ms": {"conv_fwd": conv_ms["fwd"], "conv_dgrad": conv_ms["dgrad"], "conv_wgrad": conv_ms["wgrad"],

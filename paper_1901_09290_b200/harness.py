@@ -422,6 +422,7 @@ class TrainStep:
         self._side = torch.cuda.Stream()
         self._wstreams = [self._side] + [torch.cuda.Stream() for _ in range(self.wgrad_streams - 1)]
         self._aux = torch.cuda.Stream()
+        self._graph_two = two_streams
         l0 = self.ctx.launch_count()
         self.graph = torch.cuda.CUDAGraph()
         self._graph_has_update = self.world <= 1
@@ -451,30 +452,37 @@ class TrainStep:
     def step_e2e(self, stream=None):
         """The same step with the image batch copied from pinned host memory and the regulariser value read back.
 
-        The host-to-device copy runs on a copy stream into a staging buffer, so the copy of the next step's batch
-        overlaps this step's kernels (one copy per step; the first call issues its own). The device-to-device move of the
-        staged batch into the stem's input runs on the copy stream too, beside the reconfiguration (which does not touch
-        the activations); the training part of the step waits for it. The copy of the next batch is enqueued AFTER this
-        step's launches: enqueued before them it delayed the step by ~55 us whatever its size (2.96 against 2.91 ms). The
-        host batch must stay untouched until that copy has run (the next call, or a synchronize)."""
+        The stem's input is double buffered: while a step reads one buffer, the next batch is copied from pinned host memory
+        into the other on a copy stream (one copy per step; the first call brings its own batch), and the next call trains
+        on that buffer -- with a CUDA graph of its own, captured on first use, because a graph holds the address of the
+        buffer its kernels read. Nothing is moved on the device. The copy of the next batch is enqueued AFTER this step's
+        launches: enqueued before them it delayed the step by ~55 us whatever its size. The host batch must stay untouched
+        until that copy has run (the next call, or a synchronize)."""
         main = torch.cuda.current_stream()
         if getattr(self, "_copy_stream", None) is None:
             self._copy_stream = torch.cuda.Stream()
-            self._x_stage = torch.empty_like(self.x[0])
-            self._ev_copied = torch.cuda.Event()
-            self._ev_placed = torch.cuda.Event()
-            self._prefetched = False
+            self._xbuf = [self.x[0], torch.empty_like(self.x[0])]
+            self._xgraph = [getattr(self, "graph", None), None]
+            self._ev_in = [torch.cuda.Event(), torch.cuda.Event()]
+            self._cur = 0
+            self._copy_stream.wait_stream(main)
+            with torch.cuda.stream(self._copy_stream):
+                self._xbuf[0].copy_(self.h_image, non_blocking=True)
+                self._ev_in[0].record(self._copy_stream)
         cs = self._copy_stream
-        cs.wait_stream(main)                             # the previous step has finished reading the stem's input
+        cur, nxt = self._cur, 1 - self._cur
+        self.x[0] = self._xbuf[cur]
+        if getattr(self, "graph", None) is not None:
+            if self._xgraph[cur] is None:
+                self.build_graph(self._graph_two)        # the launches that read this buffer
+                self._xgraph[cur] = self.graph
+            self.graph = self._xgraph[cur]
+        cs.wait_stream(main)                             # the previous step, the last reader of the other buffer, is done
+        self.step(stream, before_train=self._ev_in[cur])
         with torch.cuda.stream(cs):
-            if not self._prefetched:
-                self._x_stage.copy_(self.h_image, non_blocking=True)
-            self.x[0].copy_(self._x_stage, non_blocking=True)
-            self._ev_placed.record(cs)
-        self._prefetched = True
-        self.step(stream, before_train=self._ev_placed)
-        with torch.cuda.stream(cs):
-            self._x_stage.copy_(self.h_image, non_blocking=True)     # the next step's batch
+            self._xbuf[nxt].copy_(self.h_image, non_blocking=True)     # the next step's batch
+            self._ev_in[nxt].record(cs)
+        self._cur = nxt
         self.h_reg.copy_(self.mp.reg, non_blocking=True)
 
     def e2e_bytes(self):
