@@ -58,9 +58,21 @@ pt_status pt_create(pt_ctx **ctx, int device);
 pt_status pt_destroy(pt_ctx *ctx);
 const char *pt_status_string(pt_status s);
 /* Synchronises `stream`, reads and clears the device status word. PT_OK if no kernel recorded an error; PT_ERR_TIMEOUT for
- * an expired device-side wait; PT_ERR_INVALID_ARG for a channel index outside its tensor (pt_channel_gather /
- * pt_channel_scatter_add skip such an entry). */
+ * an expired device-side wait; PT_ERR_INVALID_ARG for a channel index outside its tensor (pt_channel_gather,
+ * pt_channel_scatter_add and pt_reconfigure skip such an entry). */
 pt_status pt_poll_device_status(pt_ctx *ctx, void *stream);
+/* Testing hooks for the bounded device-side waits (no counterpart in the paper). Every wait of a kernel on an mbarrier or on
+ * another CTA has a time limit (2 s); a wait that runs out makes its CTA record the time-out, drain the copies it issued,
+ * free its tensor memory and exit, and pt_poll_device_status then returns PT_ERR_TIMEOUT (and clears the arrival counters of
+ * the split weight gradients, which a kernel that gave up leaves behind). These two calls let a test reach that path without
+ * any fault: pt_test_set_wait_limit sets the limit for every context on the device (milliseconds; 0 restores 2 s; it
+ * synchronises), and pt_test_skip_next_arrive makes ONE later launch leave out one arrival, so that its waits run out:
+ *   which = 1: the next pt_conv_wgrad that splits its reduction over CTAs -- split 0 does not announce its partial tile;
+ *   which = 2: the next forward / data-gradient launch of the pixel-linear (GEMM-form) kernel -- the activation producer of
+ *              every CTA leaves out the first pipeline stage;   which = 0 disarms.
+ * The outputs of that launch are undefined. Not for production use. */
+pt_status pt_test_set_wait_limit(pt_ctx *ctx, uint32_t milliseconds);
+pt_status pt_test_skip_next_arrive(pt_ctx *ctx, int32_t which);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 uint64_t pt_launch_count(const pt_ctx *ctx);
 /* Upper bound on the CTAs (one per SM) a pt_conv_wgrad launch may use; 0 restores the default, all SMs. The weight gradient
@@ -232,7 +244,7 @@ pt_status pt_cross_entropy(pt_ctx *ctx, const float *logits, const int32_t *labe
 /* lambda_out[0] (device, float) = ratio * loss[0] / ((1 - ratio) * reg_sum[0])  (Eq. 3 solved for lambda), computed in fp64.
  * loss, reg_sum: device doubles (from pt_cross_entropy and pt_group_lasso_sgd_step). reg_sum == 0 (no regularised group
  * left) gives lambda = 0. PT_ERR_INVALID_ARG unless 0 < ratio < 1. The caller reads lambda_out back to fill
- * pt_sgd_hparams.lambda_ for the steps that follow. */
+ * pt_sgd_hparams.lambda for the steps that follow. */
 pt_status pt_set_coeff(pt_ctx *ctx, const double *loss, const double *reg_sum, float ratio, float *lambda_out, void *stream);
 
 /* The same step in two calls, for callers that want the group norms out of the way early: the norms depend on the weights
@@ -304,7 +316,9 @@ pt_status pt_reconfigure_plan(pt_ctx *ctx, const pt_graph *g, int32_t *new2old, 
  *   new.w[k',rs,c'] = old.w[new2old_out[k'], rs, new2old_in[c']]   (same for v and the bf16 shadow, bit for bit)
  *   new.bn[i][k']   = old.bn[i][new2old_out[k']]
  * new_g must have the same topology, and each space size equal to the count pt_reconfigure_plan returned.
- * Layers whose new K or C is 0 are skipped. */
+ * Layers whose new K or C is 0 are skipped. A new space larger than its planned count makes the gather meet the -1 padding of
+ * the map: such entries are skipped (the destination elements stay as they were) and pt_poll_device_status reports
+ * PT_ERR_INVALID_ARG. */
 pt_status pt_reconfigure(pt_ctx *ctx, const pt_graph *old_g, const int32_t *new2old, const pt_graph *new_g, void *stream);
 
 /* ------------------------------------------------------------------------------------------

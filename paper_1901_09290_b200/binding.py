@@ -72,6 +72,8 @@ EXPORTS = {
     "pt_status_string": (c_char_p, [c_int32]),
     "pt_poll_device_status": (c_int32, [c_void_p, c_void_p]),
     "pt_launch_count": (c_uint64, [c_void_p]),
+    "pt_test_set_wait_limit": (c_int32, [c_void_p, ctypes.c_uint32]),
+    "pt_test_skip_next_arrive": (c_int32, [c_void_p, c_int32]),
     "pt_set_wgrad_cta_limit": (c_int32, [c_void_p, c_int32]),
     "pt_conv_wgrad_ctas": (c_int32, [c_void_p, POINTER(pt_conv_desc), POINTER(c_int32)]),
     "pt_conv_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_conv_desc), c_int32]),
@@ -175,6 +177,14 @@ class Context:
 def make_conv_desc(N, H, W, C, K, R, S, stride, pad, ldx=None, ldy=None, ldw=None, out_f32=0, algo=0) -> pt_conv_desc:
     p8 = lambda c: (c + 7) // 8 * 8
     return pt_conv_desc(N, H, W, C, K, R, S, stride, pad, ldx or p8(C), ldy or p8(K), ldw or p8(C), out_f32, algo)
+
+
+def pt_test_set_wait_limit(ctx: Context, milliseconds: int):
+    _check(lib().pt_test_set_wait_limit(ctx.handle, milliseconds), "pt_test_set_wait_limit")
+
+
+def pt_test_skip_next_arrive(ctx: Context, which: int):
+    _check(lib().pt_test_skip_next_arrive(ctx.handle, which), "pt_test_skip_next_arrive")
 
 
 def pt_set_wgrad_cta_limit(ctx: Context, max_ctas: int):

@@ -3,6 +3,7 @@
 
 static const size_t kArenaBytes = 4u << 20;     // 4 MiB of tables
 static const size_t kSlotBytes = 512u << 10;    // eight slots of 512 KiB
+static const size_t kSyncWords = 16384;         // arrival counters of the split weight gradients
 
 extern "C" const char *pt_status_string(pt_status s)
 {
@@ -38,8 +39,8 @@ extern "C" pt_status pt_create(pt_ctx **out, int device)
               cudaMallocHost(&c->h_status, 16) == cudaSuccess && cudaMalloc(&c->d_arena, kArenaBytes) == cudaSuccess &&
               cudaMallocHost(&c->h_stage, kArenaBytes) == cudaSuccess &&
               cudaMallocHost(&c->h_counts, 65536 * sizeof(int32_t)) == cudaSuccess &&
-              cudaMalloc(&c->d_sync, 16384 * sizeof(unsigned int)) == cudaSuccess &&
-              cudaMemset(c->d_sync, 0, 16384 * sizeof(unsigned int)) == cudaSuccess &&
+              cudaMalloc(&c->d_sync, kSyncWords * sizeof(unsigned int)) == cudaSuccess &&
+              cudaMemset(c->d_sync, 0, kSyncWords * sizeof(unsigned int)) == cudaSuccess &&
               cudaEventCreateWithFlags(&c->upload_done, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); pt_destroy(c); return PT_ERR_CUDA; }
     size_t off = 0;
@@ -90,6 +91,20 @@ extern "C" pt_status pt_set_wgrad_cta_limit(pt_ctx *c, int max_ctas)
     return PT_OK;
 }
 
+extern "C" pt_status pt_test_set_wait_limit(pt_ctx *c, uint32_t milliseconds)
+{
+    if (!c) return PT_ERR_INVALID_ARG;
+    PT_CUDA_OK(cudaSetDevice(c->device));
+    return pt_sm100_set_wait_limit_ns(milliseconds ? (unsigned long long)milliseconds * 1000000ull : 2000000000ull, nullptr);
+}
+
+extern "C" pt_status pt_test_skip_next_arrive(pt_ctx *c, int32_t which)
+{
+    if (!c || which < 0 || which > 2) return PT_ERR_INVALID_ARG;
+    c->test_skip = which;
+    return PT_OK;
+}
+
 extern "C" pt_status pt_poll_device_status(pt_ctx *c, void *stream)
 {
     if (!c) return PT_ERR_INVALID_ARG;
@@ -99,6 +114,12 @@ extern "C" pt_status pt_poll_device_status(pt_ctx *c, void *stream)
     unsigned int code = c->h_status[0];
     if (code != PT_DEV_OK) {
         PT_CUDA_OK(cudaMemsetAsync(c->d_status, 0, 16, st));
+        if (code == PT_DEV_TIMEOUT) {
+            // A split weight gradient that gave up leaves its arrival counters non-zero (only the normal path resets them):
+            // clear the whole ring, or a later launch that gets the same slots would see its splits as already arrived.
+            PT_CUDA_OK(cudaMemsetAsync(c->d_sync, 0, kSyncWords * sizeof(unsigned int), st));
+            c->sync_next = 0;
+        }
         PT_CUDA_OK(cudaStreamSynchronize(st));
         return code == PT_DEV_TIMEOUT ? PT_ERR_TIMEOUT : code == PT_DEV_BAD_INDEX ? PT_ERR_INVALID_ARG : PT_ERR_CUDA;
     }

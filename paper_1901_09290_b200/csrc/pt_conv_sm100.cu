@@ -74,6 +74,7 @@ struct GemmP {
     int n_issuers;      // 2 (resident weights only): two MMA issuer warps take alternate tiles, each with half of the ring's stages
     int acc_per;        // two issuers: accumulator buffers per issuer (1 or 2)
     int alias_staging;  // 1: the CTA has a single tile; the epilogue's staging slabs lie in the (then idle) ring
+    int test_skip;      // test hook (pt_test_skip_next_arrive): the A producer leaves out the first stage of its first tile
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
@@ -216,6 +217,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         if (is_a) GTRACE(0, issued); else if (warp == 14) GTRACE(2, issued);
                         const uint32_t bar = smem_u32(&ctl->full[sbase + s]);
                         const uint32_t a_dst = data_base + (uint32_t)(sbase + s) * stage_bytes, b_dst = a_dst + a_bytes;
+                        if (is_a && p.test_skip && issued == 0) {         // test hook: this stage never becomes full
+                            ++issued;
+                            if (++s == SR) { s = 0; ph ^= 1; }
+                            continue;
+                        }
                         mbar_arrive_expect_tx(bar, my_bytes);
                         if (is_a) {
                             if (p.a_tiled) tma_load_2d(a_dst, &tmA, bar, kc * kKC, m0);
@@ -896,6 +902,7 @@ struct WgradP {
     int acc_cols;           // columns of one accumulator (= BN, or the padded K in the paired form)
     unsigned a_box, b_box;  // bytes reserved per dy box and per x box (multiples of 1024)
     float *out;             // dw
+    int test_skip;          // test hook (pt_test_skip_next_arrive): split 0 does not announce its partial tile
     float *partial;         // splits > 1: workspace [blockIdx.x][tap in group][split][128][BN] fp32
     unsigned int *sync;     // splits > 1: two zeroed counters per blockIdx.x (arrived, reduced); left zero again at exit
     unsigned int *status;
@@ -981,11 +988,12 @@ __device__ __forceinline__ void wgrad_finish(const WgradP &p, const CUtensorMap 
                 // ---- (2) every split CTA of this tile is resident (the grid is at most one CTA per SM): wait for all of them
                 unsigned int *arrived = p.sync + 2 * blockIdx.x;
                 if (gtid == 0) {
-                    atomicAdd(arrived, 1u);
+                    // (test hook: split 0 stays silent, so that every split of the tile runs into the bounded wait below)
+                    if (!(p.test_skip && split == 0)) atomicAdd(arrived, 1u);
                     const uint64_t t0 = globaltimer_ns();
                     while (atomicAdd(arrived, 0u) < (unsigned)p.splits) {
                         if (*abort_flag) break;
-                        if (globaltimer_ns() - t0 > 2000000000ull) { record_timeout(p.status, 8); *abort_flag = 1; break; }
+                        if (globaltimer_ns() - t0 > *(volatile unsigned long long *)&g_wait_limit_ns) { record_timeout(p.status, 8); *abort_flag = 1; break; }
                         __nanosleep(64);
                     }
                 }
@@ -1732,6 +1740,7 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
         attr_set[B_MN ? 1 : 0] = true;
     }
     const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
+    if (c->test_skip == 2) { p.test_skip = 1; c->test_skip = 0; }
     PT_CUDA_OK(launch_pdl(conv_gemm_kernel<B_MN>, dim3((unsigned)grid), dim3(kGemmThreads), smem, st, tmA, tmB, tmC, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
@@ -2116,6 +2125,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
         attr_set = true;
     }
     dim3 grid((unsigned)gx, (unsigned)p.splits);
+    if (c->test_skip == 1 && p.splits > 1) { p.test_skip = 1; c->test_skip = 0; }
     PT_CUDA_OK(launch_pdl(conv_wgrad_kernel, grid, dim3(kThreads), smem, st, tmA, tmX, tmP, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
@@ -2169,6 +2179,7 @@ pt_status run_wgrad_rows(pt_ctx *c, const pt_conv_desc *d, int P, int Q, const v
     }
     dim3 grid((unsigned)gx, (unsigned)p.splits);
     const size_t smem = (p.splits > 1 && wr.smem < kSplitSmemFloor) ? kSplitSmemFloor : wr.smem;
+    if (c->test_skip == 1 && p.splits > 1) { p.test_skip = 1; c->test_skip = 0; }
     PT_CUDA_OK(launch_pdl(conv_wgrad_rows_kernel, grid, dim3(kThreads), smem, st, tmA, tmX, tmP, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
@@ -2541,6 +2552,14 @@ pt_status pt_sm100_conv(pt_ctx *c, const pt_conv_desc *d, int which, const void 
         pt_status s = launch_gemm<true>(c, tmA, tmB, p, st);
         if (s != PT_OK) return s;
     }
+    return PT_OK;
+}
+
+// Sets the limit of the bounded device-side waits of this file's kernels (the variable lives in this translation unit).
+pt_status pt_sm100_set_wait_limit_ns(unsigned long long ns, cudaStream_t st)
+{
+    PT_CUDA_OK(cudaMemcpyToSymbolAsync(g_wait_limit_ns, &ns, sizeof(ns), 0, cudaMemcpyHostToDevice, st));
+    PT_CUDA_OK(cudaStreamSynchronize(st));
     return PT_OK;
 }
 

@@ -83,8 +83,8 @@ __device__ __forceinline__ float bf16_bits_to_float(unsigned short h) { return _
 // node_out[p][c] = act(node_in[p][c] + branch[p][j] where idx[j] == c), fp32 add, one rounding to bf16; 0 in the pad lanes.
 __global__ void __launch_bounds__(kGateThreads) scatter_add_kernel(const unsigned short *__restrict__ branch, int ld_b,
                                                                    const int *__restrict__ idx, int n_sel,
-                                                                   const unsigned short *__restrict__ node_in,
-                                                                   unsigned short *__restrict__ node_out, int ld_node, int c_node,
+                                                                   const unsigned short *node_in,
+                                                                   unsigned short *node_out, int ld_node, int c_node,
                                                                    long long npix, long long pix_per_block, int relu, unsigned int *status)
 {
     __shared__ short s_inv[kGateMax];
@@ -107,7 +107,8 @@ __global__ void __launch_bounds__(kGateThreads) scatter_add_kernel(const unsigne
     for (int it = threadIdx.x; it < items; it += kGateThreads) {
         const int p = it / groups, g = it - p * groups;
         uint4 in = make_uint4(0u, 0u, 0u, 0u);
-        if (i0) in = __ldg(reinterpret_cast<const uint4 *>(i0 + (size_t)p * ld_node + g * 8));
+        // node_in may be the tensor node_out (in-place merge): a plain load, not the read-only path, and no restrict
+        if (i0) in = *reinterpret_cast<const uint4 *>(i0 + (size_t)p * ld_node + g * 8);
         const unsigned short *ie = reinterpret_cast<const unsigned short *>(&in);
         const unsigned short *brow = b0 + (size_t)p * ld_b;
         __align__(16) unsigned short o[8];

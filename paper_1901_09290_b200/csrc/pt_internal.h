@@ -48,6 +48,7 @@ struct pt_ctx {
     unsigned int sync_next = 0;         // ring position in d_sync
     uint64_t launches = 0;
     int wgrad_ctas = 0;                 // CTA limit of a weight-gradient launch (0 = all SMs)
+    int test_skip = 0;                  // pt_test_skip_next_arrive: 1 = next split weight gradient, 2 = next fwd/dgrad GEMM-form launch
     // Helper streams for independent launches inside one call (the parity classes of a stride-2 data gradient): the caller's
     // stream forks to them and joins them back through events, which a stream capture records as graph edges.
     cudaStream_t fork_stream[3] = {nullptr, nullptr, nullptr};
@@ -85,3 +86,4 @@ pt_status pt_sm100_conv(pt_ctx *ctx, const pt_conv_desc *d, int which, const voi
                         void *ws, size_t ws_bytes, cudaStream_t st);
 size_t pt_sm100_conv_workspace(const pt_ctx *ctx, const pt_conv_desc *d, int which);
 int pt_sm100_wgrad_ctas(const pt_ctx *ctx, const pt_conv_desc *d, int *waits);
+pt_status pt_sm100_set_wait_limit_ns(unsigned long long ns, cudaStream_t st);

@@ -65,18 +65,30 @@ struct GatherJob {
     const int32_t *mapK, *mapC;
     int Kn, Cn, RS, Co, ldwo, ldwn;
     int kind;                  // 0 = weight tensors, 1 = per-channel vector
-    int pad_;
+    int Ko;                    // old number of output channels (range check of the map)
 };
 struct GatherChunk { int job, line0, nlines, col0; };
 
 constexpr int kGatherUnroll = 8;
 
-__global__ void __launch_bounds__(256) gather_kernel(const GatherJob *__restrict__ jobs, const GatherChunk *__restrict__ chunks)
+// A map entry outside the old tensor (a new graph larger than the plan's counts reads the -1 padding of the map) is skipped:
+// nothing is read or written for it, and the status word reports it (PT_ERR_INVALID_ARG at the next poll).
+__device__ __forceinline__ void bad_map_entry(unsigned int *status, unsigned int where)
+{
+    if (atomicCAS(&status[0], 0u, (unsigned)PT_DEV_BAD_INDEX) == 0u) status[1] = where;
+}
+
+__global__ void __launch_bounds__(256) gather_kernel(const GatherJob *__restrict__ jobs, const GatherChunk *__restrict__ chunks,
+                                                     unsigned int *status)
 {
     const GatherChunk ch = chunks[blockIdx.x];
     const GatherJob J = jobs[ch.job];
     if (J.kind == 1) {       // vector: nw[k'] = ow[mapK[k']]
-        for (int k = ch.line0 + threadIdx.x; k < ch.line0 + ch.nlines; k += blockDim.x) J.nw[k] = J.ow[J.mapK[k]];
+        for (int k = ch.line0 + threadIdx.x; k < ch.line0 + ch.nlines; k += blockDim.x) {
+            const int ko = J.mapK[k];
+            if (ko < 0 || ko >= J.Ko) { bad_map_entry(status, 50u); continue; }
+            J.nw[k] = J.ow[ko];
+        }
         return;
     }
     // Lines of the NEW tensor are (k', rs); a block covers a run of lines x up to 256 columns. Each thread owns one new
@@ -87,15 +99,21 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherJob *__restrict
     const int c = ch.col0 + tx;
     if (c >= J.Cn) return;
     const int co = J.mapC[c];
+    if (co < 0 || co >= J.Co) { bad_map_entry(status, 51u); return; }
     for (int l = ty; l < ch.nlines; l += kGatherUnroll * TY) {
         float w[kGatherUnroll], v[kGatherUnroll];
         __nv_bfloat16 h[kGatherUnroll];
+        bool okk[kGatherUnroll];
 #pragma unroll
         for (int u = 0; u < kGatherUnroll; ++u) {
             const int line = ch.line0 + l + u * TY;
+            okk[u] = false;
             if (l + u * TY < ch.nlines) {
                 const int kn = line / J.RS, rs = line - kn * J.RS;
-                const size_t oline = (size_t)J.mapK[kn] * J.RS + rs;
+                const int ko = J.mapK[kn];
+                if (ko < 0 || ko >= J.Ko) { bad_map_entry(status, 52u); continue; }
+                okk[u] = true;
+                const size_t oline = (size_t)ko * J.RS + rs;
                 w[u] = J.ow[oline * J.Co + co];
                 if (J.nv) v[u] = J.ov[oline * J.Co + co];
                 if (J.nwb) h[u] = J.owb[oline * J.ldwo + co];
@@ -104,7 +122,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherJob *__restrict
 #pragma unroll
         for (int u = 0; u < kGatherUnroll; ++u) {
             const int line = ch.line0 + l + u * TY;
-            if (l + u * TY < ch.nlines) {
+            if (okk[u]) {
                 const size_t dst = (size_t)line * J.Cn + c;
                 J.nw[dst] = w[u];
                 if (J.nv) J.nv[dst] = v[u];
@@ -196,7 +214,7 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
     }
     if (c->gather_tab.valid && c->gather_chunks && args == c->gather_args) {
         const char *dev = c->d_arena + c->gather_tab.off;
-        gather_kernel<<<c->gather_chunks, 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + c->gather_jobs_bytes));
+        gather_kernel<<<c->gather_chunks, 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + c->gather_jobs_bytes), c->d_status);
         c->launches += 1;
         PT_CUDA_OK(cudaGetLastError());
         return PT_OK;
@@ -227,7 +245,7 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         J.nw = n.w; J.nv = n.v; J.nwb = (__nv_bfloat16 *)n.w_bf16;
         J.mapK = new2old + map_off[ol.out_space];
         J.mapC = new2old + map_off[ol.in_space];
-        J.Kn = n.K; J.Cn = n.C; J.RS = n.RS; J.Co = o.C; J.ldwo = o.ldw; J.ldwn = n.ldw;
+        J.Kn = n.K; J.Cn = n.C; J.RS = n.RS; J.Co = o.C; J.Ko = o.K; J.ldwo = o.ldw; J.ldwn = n.ldw;
         J.kind = 0;
         const int job = (int)jobs.size();
         jobs.push_back(J);
@@ -242,7 +260,7 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
             if (!ol.bn[b]) return PT_ERR_INVALID_ARG;
             GatherJob V;
             memset(&V, 0, sizeof(V));
-            V.ow = ol.bn[b]; V.nw = nl.bn[b]; V.mapK = J.mapK; V.Kn = n.K; V.kind = 1;
+            V.ow = ol.bn[b]; V.nw = nl.bn[b]; V.mapK = J.mapK; V.Kn = n.K; V.Ko = o.K; V.kind = 1;
             chunks.push_back(GatherChunk{(int)jobs.size(), 0, n.K, 0});
             jobs.push_back(V);
         }
@@ -256,7 +274,7 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
     c->gather_chunks = 0;
     s = pt_upload_table(c, &c->gather_tab, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
-    gather_kernel<<<(unsigned)chunks.size(), 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + jb));
+    gather_kernel<<<(unsigned)chunks.size(), 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + jb), c->d_status);
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     c->gather_args.swap(args);

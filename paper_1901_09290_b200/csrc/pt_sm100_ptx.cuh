@@ -51,12 +51,15 @@ __device__ __forceinline__ void record_timeout(unsigned int *status, unsigned in
     if (atomicCAS(&status[0], 0u, 1u) == 0u) status[1] = where;
 }
 
-// Waits for the phase with the given parity to complete, for at most `limit_ns`. On expiry it
+// Limit of every bounded device-side wait, in nanoseconds (2 s unless pt_test_set_wait_limit changed it). It is read only
+// on the slow path of a wait (after 256 failed polls), never by a wait that succeeds at once.
+__device__ unsigned long long g_wait_limit_ns = 2000000000ull;
+
+// Waits for the phase with the given parity to complete, for at most g_wait_limit_ns. On expiry it
 // records the timeout, raises the CTA-wide abort flag and returns false; it also returns false
 // as soon as another thread has raised the flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          unsigned int *status, unsigned int where,
-                                          uint64_t limit_ns = 2000000000ull)
+                                          unsigned int *status, unsigned int where)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
@@ -64,7 +67,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     while (!mbar_try_wait(bar, parity)) {
         if ((++n & 0xffu) == 0u) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > limit_ns) {
+            if (globaltimer_ns() - t0 > *(volatile unsigned long long *)&g_wait_limit_ns) {
                 record_timeout(status, where);
                 *abort_flag = 1;
                 return false;

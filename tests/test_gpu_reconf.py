@@ -231,3 +231,42 @@ def test_repeated_reconfiguration_reads_current_contents_and_rebuilds_for_new_ar
         ref_w = oracle.gather_weight(dm.w[li].cpu().numpy(), mk, mc)
         assert np.array_equal(d2.w[li].cpu().numpy().view(np.uint32), ref_w.view(np.uint32)), l.name
         assert torch.equal(dn.w[li], snap[li]), l.name
+
+
+def test_new_graph_larger_than_the_plan_is_reported_and_reads_nothing_out_of_range():
+    """A destination model with one channel more than pt_reconfigure_plan counted makes the gather meet the -1 padding of
+    the keep map: the entry is skipped (guard values stay in place) and the next poll reports PT_ERR_INVALID_ARG."""
+    net = W.bottleneck_stage3(8)
+    kept = W.choose_kept(net, [300, 90, 70], W.BASE_SEED + 13)
+    model = W.gen_model(net, W.BASE_SEED + 13, kept=kept)
+    dm = DevModel(model)
+    c = Hh.ctx()
+    B.pt_find_zero_groups(c, dm.arr, 1e-4, False, dm.ws)
+    new2old = torch.full((sum(net.space_sizes),), -7, dtype=torch.int32, device="cuda")
+    sizes = B.pt_reconfigure_plan(c, dm.graph(), new2old)
+    assert sizes == [300, 90, 70]
+    bad = [sizes[0], sizes[1] + 1, sizes[2]]                      # one channel too many in the first internal space
+    bad_net = W.with_sizes(net, bad)
+    guard = 5555.0
+    empty = W.Model(bad_net, [torch.full((l.K, l.R, l.R, l.C), guard) for l in bad_net.layers],
+                    [torch.full((l.K, l.R, l.R, l.C), guard) for l in bad_net.layers],
+                    [torch.zeros((l.K, l.R, l.R, l.C)) for l in bad_net.layers],
+                    [[torch.full((l.K,), guard) for _ in range(4)] for l in bad_net.layers])
+    dn = DevModel(empty)
+    B.pt_reconfigure(c, dm.graph(), new2old, dn.graph())
+    torch.cuda.synchronize()
+    with pytest.raises(B.PtError) as e:
+        c.poll()
+    assert e.value.status == 1                                     # PT_ERR_INVALID_ARG
+    c.poll()
+    # layer 0 writes space 1: its extra output channel (index 90) kept the guard in w, v and the BN vectors; the valid part
+    # is the ordinary gather
+    l0 = bad_net.layers[0]
+    assert l0.K == 91
+    assert torch.all(dn.w[0][90] == guard) and torch.all(dn.v[0][90] == guard)
+    for b in range(4):
+        assert float(dn.bn[0][b][90]) == guard
+    ref = oracle.gather_weight(model.w[0].numpy(), kept[1], kept[0])
+    assert np.array_equal(dn.w[0][:90].cpu().numpy(), ref)
+    # layer 1 reads space 1: its extra input channel kept the guard
+    assert torch.all(dn.w[1][:, :, :, 90] == guard)
