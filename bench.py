@@ -24,9 +24,23 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum over the launches of each conv pass in one step of the default workload
-# (one ncu capture, 1 pass per launch; the summary and the command are in profiles/step_launch_list_resnet50_keep060_b64.txt)
-NCU_DRAM_BYTES = {"fwd": 1.102e9, "dgrad": 1.101e9, "wgrad": 2.122e9}   # incl. the stem layout kernels
+PROFILE_LAUNCH_LIST = os.path.join(ROOT, "profiles", "step_launch_list_resnet50_keep060_b64.txt")
+
+
+def ncu_pass_traffic(kind):
+    """dram__bytes_read.sum + dram__bytes_write.sum over the launches of one conv pass of the default workload, as the tracked
+    ncu summary records them (a line 'pass_dram_bytes fwd=... dgrad=... wgrad=...'); None if the summary has no such line.
+    A captured launch's writes mostly retire from the 126 MB L2 after it has ended, so the figure is dominated by reads."""
+    try:
+        for line in open(PROFILE_LAUNCH_LIST):
+            if line.startswith("# pass_dram_bytes"):
+                kv = dict(t.split("=") for t in line.split()[2:])
+                return float(kv[kind])
+    except Exception:
+        pass
+    return None
+
+
 METRIC = "pruned ResNet-50 train-step conv TFLOP/s (useful FLOPs / whole step)"
 UNIT = "TFLOP/s"
 
@@ -135,16 +149,13 @@ def oracle_step_sample(net_p, N_s, layer_ids, seed):
     return time.perf_counter() - t0, flops
 
 
-def pick_sample(net_p, budget_s, seed):
-    """Chooses every s-th layer at batch 1 so that one sample costs about budget_s seconds on this host."""
+CPU_SAMPLE_BATCH = 2          # both arms time the oracle on the same bounded sample: every layer of the workload at this batch
+
+
+def cpu_sample(net_p):
     ids = list(range(len(net_p.layers)))
-    t, f = oracle_step_sample(net_p, 1, [5], seed)          # calibration on one mid-size layer
-    rate = f / max(t, 1e-6)
-    full = sum(2 * l.P * l.P * l.K * l.C * l.R * l.R * (3 if i > 0 else 2) for i, l in enumerate(net_p.layers))
-    stride = 1
-    while full / stride / rate > budget_s and stride < len(ids):
-        stride += 1
-    return ids[::stride], stride
+    return ids, CPU_SAMPLE_BATCH, (f"batch {CPU_SAMPLE_BATCH}, all {len(ids)} layers of the workload: fwd+dgrad+wgrad+lasso+detection "
+                                   "per layer, as the oracle stands")
 
 
 def run_reference(args):
@@ -156,17 +167,15 @@ def run_reference(args):
     from paper_1901_09290_b200 import workloads as W
     net, counts, kept, seed, name = workload(args)
     net_p = W.with_sizes(net, counts)
-    per_step_budget = max(0.5, min(8.0, 150.0 / (args.steps + args.warmup)))
-    ids, stride = pick_sample(net_p, per_step_budget, seed)
+    ids, nb, sample = cpu_sample(net_p)
     for _ in range(args.warmup):
-        oracle_step_sample(net_p, 1, ids, seed)
+        oracle_step_sample(net_p, nb, ids, seed)
     T, F = 0.0, 0
     for _ in range(args.steps):
-        t, f = oracle_step_sample(net_p, 1, ids, seed)
+        t, f = oracle_step_sample(net_p, nb, ids, seed)
         T += t
         F += f
     val = F / T / 1e12
-    sample = f"batch 1 of {args.batch}, every {stride}-th of the 53 layers ({len(ids)} layers): fwd+dgrad+wgrad+lasso+detection"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": T / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -205,6 +214,10 @@ def run_ours(args):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE is {world}")
+    if local >= torch.cuda.device_count():
+        raise SystemExit(f"bench.py: rank {rank} needs GPU {local}, the machine has {torch.cuda.device_count()}")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -227,15 +240,26 @@ def run_ours(args):
     tot_flops = sum(flops.values())
     stream = torch.cuda.current_stream()
 
+    MIN_TIMED_S = 0.5
+
     def timed(fn, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
-            fn()
-        e1.record(stream)
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1), world)
+        """Device time of `steps` steps (max over ranks). The timed region is kept at or above half a second: the K requested
+        steps are repeated back to back r times inside one pair of events (r chosen from a first pass of K steps) and the
+        total is divided by r, so that a short K still gives a sustained-clock figure. Returns (ms for K steps, r)."""
+        def run(n):
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(n):
+                fn()
+            e1.record(stream)
+            barrier()
+            return max_over_ranks(e0.elapsed_time(e1), world)
+        first = run(steps)
+        r = max(1, int(MIN_TIMED_S * 1e3 / max(first, 1e-3)) + 1)
+        if r == 1:
+            return first, 1
+        return run(steps * r) / r, r
 
     if args.profile_steps:
         # a short run for profilers: one warm-up step, then the requested steps, nothing else
@@ -258,12 +282,14 @@ def run_ours(args):
     ctx.poll()
     l0 = ctx.launch_count()
     sampler = ClockSampler(local) if rank == 0 else None
-    ms = timed(ts.step, args.steps)
-    launches = (ctx.launch_count() - l0) + (args.steps * ts.graph_launches if getattr(ts, "graph", None) is not None else 0)
+    ms, reps_timed = timed(ts.step, args.steps)
+    n_timed = args.steps * (reps_timed + (1 if reps_timed > 1 else 0))      # steps run inside the timed regions (first pass + repeats)
+    per_step_launches = (ctx.launch_count() - l0) / max(1, n_timed) + (ts.graph_launches if getattr(ts, "graph", None) is not None else 0)
+    launches = int(round(per_step_launches * args.steps))
     # end-to-end: image batch from pinned host memory, regulariser value and new sizes read back, every step
     for _ in range(2):
         ts.step_e2e()
-    ms_e2e = timed(ts.step_e2e, args.steps)
+    ms_e2e, _ = timed(ts.step_e2e, args.steps)
     clocks = sampler.stop() if sampler else None
     ctx.poll()
 
@@ -271,7 +297,7 @@ def run_ours(args):
     nL = len(ts.net.layers)
     reps = max(2, min(5, args.steps))
     acc = {"fwd": [0.0] * nL, "dgrad": [0.0] * nL, "wgrad": [0.0] * nL}
-    phase = {"reconfigure": 0.0, "lasso": 0.0, "lasso_dense_model": 0.0}
+    phase = {}
 
     def ev_time(fn):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -333,21 +359,42 @@ def run_ours(args):
             b.record(stream)
             torch.cuda.synchronize()
             sched[kind] = a.elapsed_time(b) / reps
-    for _ in range(reps):
-        pend = [("reconfigure", ev_time(ts.reconfigure)), ("lasso", ev_time(ts.lasso))]
+    # Update and reconfiguration phases, each alone: replayed from a CUDA graph where the call has no host synchronisation
+    # (as the step launches it), with the L2 flushed before every repetition (in the step the convolutions in between do that)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def time_alone(fn, graph=True):
+        fn()
         torch.cuda.synchronize()
-        for kind, (a, b) in pend:
-            phase[kind] += a.elapsed_time(b) / reps
-    # the lasso step on the dense-shaped model (23.45 M parameters), timed alone
+        g = None
+        if graph:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+        tot = 0.0
+        for _ in range(reps):
+            flush.fill_(1)
+            a, b = ev_time(g.replay if g is not None else fn)
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b) / reps
+        return tot
+
     md = ts.md
-    g_saved = [w.clone() for w in md.w]
     v_saved = [v.clone() for v in md.v]
-    for _ in range(reps):
-        a, b = ev_time(lambda: B.pt_group_lasso_sgd_step(ctx, md.arr, 1e-4, 0.0, 0.9, 0.0, md.reg, md.ws))
-        torch.cuda.synchronize()
-        phase["lasso_dense_model"] += a.elapsed_time(b) / reps
-    for w, s in zip(md.v, v_saved):
-        w.copy_(s)
+    phase["reconfigure"] = time_alone(ts.reconfigure, graph=False)                      # contains the plan's host synchronisation
+    phase["detect"] = time_alone(lambda: B.pt_find_zero_groups(ctx, md.arr, 1e-4, False, md.ws))
+    phase["gather"] = time_alone(lambda: B.pt_reconfigure(ctx, md.graph(), ts.new2old, ts.mp.graph()))
+    phase["plan_incl_host_sync"] = time_alone(lambda: B.pt_reconfigure_plan(ctx, md.graph(), ts.new2old), graph=False)
+    phase["lasso"] = time_alone(ts.lasso)
+    ts.lasso_norms()
+    phase["lasso_carried"] = time_alone(ts.lasso_carried)
+    phase["lasso_dense_model"] = time_alone(lambda: B.pt_group_lasso_sgd_step(ctx, md.arr, 1e-4, 0.0, 0.9, 0.0, md.reg, md.ws))
+    B.pt_group_lasso_norms(ctx, md.arr, md.reg, md.ws)
+    phase["lasso_carried_dense_model"] = time_alone(lambda: B.pt_group_lasso_sgd_step_carried(ctx, md.arr, 1e-4, 0.0, 0.9, 0.0, md.reg, md.ws))
+    for w, sv in zip(md.v, v_saved):
+        w.copy_(sv)
+    del flush
+    ts.reconfigure()
     ctx.poll()
 
     which_id = {"fwd": 0, "dgrad": 1, "wgrad": 2}
@@ -377,6 +424,8 @@ def run_ours(args):
                      "pct_of_measured_sustained": 100 * sub_fl / sub_us * 1e12 / tc_peak if sub_us else None,
                      "best_layer_pct": max((100 * r["tflops"] * 1e12 / tc_peak for r in sub), default=None),
                      "timing": "fwd and dgrad launches whose FLOPs / tensor peak exceed their bytes / HBM rate, one after the other"}
+    floor_ms = {k: 1e3 * sum(max(2 * args.batch * l.P * l.P * l.K * l.C * l.R * l.R / tc_peak, ts.layer_bytes(li, which_id[k]) / bw_peak)
+                             for li, l in enumerate(ts.net.layers) if not (k == "dgrad" and li == 0)) for k in which_id}
     serial_ms = {k: sum(v) for k, v in acc.items()}           # launches of a pass one after the other
     conv_ms = sched if sched else serial_ms                     # passes as the step schedules them
     conv_total_ms = sum(conv_ms.values())
@@ -384,12 +433,14 @@ def run_ours(args):
     dom_flops = flops[dom]
     dom_t = conv_ms[dom] * 1e-3
     n_dom = nL - (1 if dom == "dgrad" else 0)
+    dom_bytes = sum(ts.layer_bytes(li, which_id[dom]) for li in range(nL) if not (dom == "dgrad" and li == 0))
     value = whole_job_value(tot_flops, world, ms, args.steps)
     e2e_val = whole_job_value(tot_flops, world, ms_e2e, args.steps)
     h2d, d2h = ts.e2e_bytes()
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms / args.steps, "timed_region": {"steps_per_pass": args.steps, "passes_averaged": reps_timed,
+                                                         "seconds": ms * reps_timed * 1e-3}, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16",
         "arithmetic": "bf16 operands, f32 accumulate (convs); f32 (lasso/SGD); u8/i32 (detection, compaction)",
         "data": "synthetic",
@@ -407,7 +458,7 @@ def run_ours(args):
         "clocks": clocks,
         "phases_ms": {"conv_fwd": conv_ms["fwd"], "conv_dgrad": conv_ms["dgrad"], "conv_wgrad": conv_ms["wgrad"],
                       "lasso_sgd_pruned": phase["lasso"], "detect_plan_compact": phase["reconfigure"],
-                      "lasso_sgd_dense_model": phase["lasso_dense_model"],
+                      "lasso_sgd_dense_model": phase["lasso_dense_model"], "lasso_sgd_carried_pruned": phase["lasso_carried"],
                       "note": "conv passes: each pass alone as the step schedules it (wgrads of different layers side by side)"
                               if sched else "conv passes: sum of the launches one after the other"},
         "phases_serial_ms": {"conv_fwd": serial_ms["fwd"], "conv_dgrad": serial_ms["dgrad"], "conv_wgrad": serial_ms["wgrad"]},
@@ -419,15 +470,32 @@ def run_ours(args):
         "per_layer_timing": timing_mode[0],
         "lasso_gbs": {"pruned_model": ts.lasso_bytes(ts.mp) / (phase["lasso"] * 1e-3) / 1e9,
                       "dense_model": ts.lasso_bytes(ts.md) / (phase["lasso_dense_model"] * 1e-3) / 1e9,
-                      "bytes_per_param": 26, "peak": pk["hbm_gbs"], "peak_source": pk["source"]},
+                      "bytes_per_param": 26,
+                      "carried_pruned_model": 22 * ts.mp.n_params() / (phase["lasso_carried"] * 1e-3) / 1e9,
+                      "carried_dense_model": 22 * ts.md.n_params() / (phase["lasso_carried_dense_model"] * 1e-3) / 1e9,
+                      "carried_bytes_per_param": 22, "peak": pk["hbm_gbs"], "peak_source": pk["source"]},
         "reconf_gbs": ts.reconf_bytes() / (phase["reconfigure"] * 1e-3) / 1e9,
-        "roofline": {"kernel": f"conv_{dom} (all {n_dom} launches of a step, as the step schedules them)", "bound": "tensor",
-                     "achieved": dom_flops / dom_t / 1e12, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": dom_flops / dom_t / tc_peak,
-                     # DRAM bytes of the pass's launches in one ncu capture of the default workload (profiles/step_launch_list_*)
-                     "traffic": NCU_DRAM_BYTES.get(dom) if (args.net == "resnet50" and args.keep is None and args.batch == 64 and args.algo == 0) else None,
-                     "algorithmic_bytes": sum(ts.layer_bytes(li, which_id[dom]) for li in range(nL) if not (dom == "dgrad" and li == 0)),
-                     "peak_source": pk["source"] + " sustained bf16"},
+        "reconf": {"whole_call_incl_host_sync_ms": phase["reconfigure"], "detect_ms": phase["detect"], "gather_ms": phase["gather"],
+                   "plan_incl_host_sync_ms": phase["plan_incl_host_sync"],
+                   "detect_gbs": 4 * ts.md.n_params() / (phase["detect"] * 1e-3) / 1e9,
+                   "gather_gbs": 18 * ts.mp.n_params() / (phase["gather"] * 1e-3) / 1e9,
+                   "kernels_gbs": ts.reconf_bytes() / ((phase["detect"] + phase["gather"]) * 1e-3) / 1e9},
+        "roofline": {"kernel": f"conv_{dom} (all {n_dom} launches of a step, as the step schedules them)",
+                     # the pass's own FLOPs and bytes decide which roof bounds it
+                     "bound": "tensor" if dom_flops / tc_peak > dom_bytes / bw_peak else "hbm",
+                     "achieved": (dom_flops / dom_t / 1e12) if dom_flops / tc_peak > dom_bytes / bw_peak else (dom_bytes / dom_t / 1e9),
+                     "peak": pk["bf16_tflops_sustained"] if dom_flops / tc_peak > dom_bytes / bw_peak else pk["hbm_gbs"],
+                     "unit": "TFLOP/s" if dom_flops / tc_peak > dom_bytes / bw_peak else "GB/s",
+                     # sum over the pass's layers of max(FLOPs / tensor peak, bytes / HBM rate), over the pass's scheduled time
+                     "frac": floor_ms[dom] / conv_ms[dom],
+                     "frac_all_passes": sum(floor_ms.values()) / conv_total_ms,
+                     "tensor_only": {"achieved_tflops": dom_flops / dom_t / 1e12, "frac_of_sustained_bf16": dom_flops / dom_t / tc_peak},
+                     "hbm_only": {"achieved_gbs": dom_bytes / dom_t / 1e9, "frac_of_copy_rate": dom_bytes / dom_t / bw_peak},
+                     "traffic": ncu_pass_traffic(dom) if (args.net == "resnet50" and args.keep is None and args.batch == 64 and args.algo == 0) else None,
+                     "traffic_note": "dram bytes of the pass's launches in the tracked ncu summary (profiles/); mostly reads: a launch's "
+                                     "writes retire from L2 after it has ended",
+                     "algorithmic_bytes": dom_bytes,
+                     "peak_source": pk["source"]},
     }
     if rank == 0:
         if args.per_layer:
@@ -436,13 +504,14 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             net_p = ts.net
-            ids, stride = pick_sample(net_p, 15.0, seed)
-            t1, f1 = oracle_step_sample(net_p, 1, ids, seed)
-            nb = max(1, min(8, int(12.0 / max(t1, 1e-3))))          # batch of the timed sample: about 10-20 s of CPU work
-            t, f = oracle_step_sample(net_p, nb, ids, seed) if nb > 1 else (t1, f1)
+            ids, nb, sample = cpu_sample(net_p)
+            oracle_step_sample(net_p, nb, ids[:4], seed)            # warm the thread pool
+            t, f, n_rep = 0.0, 0, 0
+            while t < 10.0 and n_rep < 8:                            # about 10-20 s of CPU work
+                t1, f1 = oracle_step_sample(net_p, nb, ids, seed)
+                t += t1; f += f1; n_rep += 1
             out["cpu_baseline"] = {"value": f / t / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                                   "sample": f"batch {nb} of {args.batch}, every {stride}-th of the 53 layers ({len(ids)} layers): "
-                                             f"fwd+dgrad+wgrad+lasso+detection, {t:.1f} s"}
+                                   "sample": f"{sample}; {n_rep} repetitions, {t:.1f} s"}
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -468,12 +537,40 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel eagerly instead of replaying a CUDA graph")
     ap.add_argument("--one-stream", action="store_true", help="capture the step on one stream (no dgrad/wgrad overlap)")
-    ap.add_argument("--profile-steps", type=int, default=0, help="run only this many steps after one warm-up (for ncu)")
+    ap.add_argument("--profile-steps", type=int, default=0,
+                    help="run only this many steps after one warm-up and print no timing: for a launch list (the one-pass "
+                         "gpu__time_duration capture); captures with more metrics belong on a small case (layerbench, --net resnet32)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher: start the N ranks here (one process per GPU, rendezvous on the loopback address)
+        spawn_ranks(args.gpus, _rank_main, (sys.argv[1:],))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
+
+
+def _rank_main(argv):
+    sys.argv = [sys.argv[0]] + list(argv)
+    main()
+
+
+def _spawn_entry(rank, world, port, fn, fn_args):
+    os.environ.update({"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world), "MASTER_ADDR": "127.0.0.1",
+                       "MASTER_PORT": str(port)})
+    fn(*fn_args)
+
+
+def spawn_ranks(n, fn, fn_args=()):
+    """Runs fn(*fn_args) in n processes with RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* set as a launcher would; raises if a
+    rank fails."""
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    mp.spawn(_spawn_entry, args=(n, port, fn, fn_args), nprocs=n, join=True)
 
 
 if __name__ == "__main__":

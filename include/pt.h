@@ -265,12 +265,31 @@ pt_status pt_group_lasso_sgd_apply_layers(pt_ctx *ctx, const pt_layer *layers /*
                                           int32_t count, const pt_sgd_hparams *hp /*host*/, void *ws, size_t ws_bytes,
                                           void *stream);
 
+/* The carried form of the step (Algorithm 1 evaluates GroupLassoReg on W_i: the sums of squares of W_{i+1} that step i + 1 needs
+ * can be taken while step i writes W_{i+1}): the update uses the 1/norm factors that ws already holds and, in the same pass
+ * over the weights, accumulates the sums of squares of the NEW weights -- and, with with_maxima != 0, the maxima of |w| that
+ * pt_find_zero_groups_carried reads (ask for them in the step before a reconfiguration) -- from which a short finish kernel
+ * rewrites the factors in ws, sumsq_out / sumsq_in (now those of the new weights) and the group maxima. A training loop then
+ * moves 22 bytes per parameter and step instead of 26. Contract: ws must hold the factors of the current weights -- left
+ * there by pt_group_lasso_norms or by the previous carried step on the same layers array and ws -- so call
+ * pt_group_lasso_norms again after anything else changed the weights (zeroing, reconfiguration, a load).
+ * reg_sum_next (device, optional) receives Eq. 2's sum for the NEW weights, i.e. the value the next iteration's loss uses.
+ * The result is bit for bit pt_group_lasso_sgd_step's when the factors in ws are those pt_group_lasso_norms computes. */
+pt_status pt_group_lasso_sgd_step_carried(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers,
+                                          const pt_sgd_hparams *hp /*host*/, int32_t with_maxima, double *reg_sum_next,
+                                          void *ws, size_t ws_bytes, void *stream);
+
 /* zero_out[k] = (max_{rs,c} |w| < threshold), zero_in[c] = (max_{k,rs} |w| < threshold), strict <, in fp32
  * (Sec. 4.1: threshold 1e-4; Sec. 4.2 / Fig. 4: the absolute maximum of a channel's parameters). A NaN keeps
  * its groups. If zero_in_place != 0 the weights, momentum and shadow of every detected group are set to 0
  * (the group sums of squares are then stale until the next pt_group_lasso_sgd_step recomputes them). */
 pt_status pt_find_zero_groups(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers, float threshold,
                               int32_t zero_in_place, void *ws, size_t ws_bytes, void *stream);
+/* The same masks without reading the weights: from the group maxima the last pt_group_lasso_sgd_step_carried on these layers
+ * (called with with_maxima != 0) and this ws left behind: the maxima of the weights that step wrote; max is order independent,
+ * so the masks are bit for bit those of pt_find_zero_groups. Valid only while the weights are unchanged since that step. */
+pt_status pt_find_zero_groups_carried(pt_ctx *ctx, const pt_layer *layers /*host*/, int32_t n_layers, float threshold,
+                                      int32_t zero_in_place, void *ws, size_t ws_bytes, void *stream);
 
 /* Zero-group detection of ONE weight tensor w[K][RS][C] without any allocation and without a workspace (no counterpart in
  * the paper: it exists for callers that may not allocate). It is for code that cannot call cudaMalloc: a host framework

@@ -88,6 +88,9 @@ EXPORTS = {
     "pt_group_lasso_sgd_apply_layers": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_int32, c_int32, POINTER(pt_sgd_hparams), c_void_p,
                                                   c_size_t, c_void_p]),
     "pt_find_zero_groups": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_float, c_int32, c_void_p, c_size_t, c_void_p]),
+    "pt_find_zero_groups_carried": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, c_float, c_int32, c_void_p, c_size_t, c_void_p]),
+    "pt_group_lasso_sgd_step_carried": (c_int32, [c_void_p, POINTER(pt_layer), c_int32, POINTER(pt_sgd_hparams), c_int32, c_void_p,
+                                                  c_void_p, c_size_t, c_void_p]),
     "pt_find_zero_groups_noalloc": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p]),
     "pt_bn_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_bn_desc)]),
     "pt_bn_relu_fwd": (c_int32, [c_void_p, POINTER(pt_bn_desc)] + [c_void_p] * 9 + [c_void_p, c_size_t, c_void_p]),
@@ -234,6 +237,23 @@ def pt_group_lasso_sgd_step(ctx, layers, lam, lr, momentum, weight_decay=0.0, re
     p, n = _ws(ws)
     _check(lib().pt_group_lasso_sgd_step(ctx.handle, arr, len(arr), byref(hp), _ptr(reg_sum_out), p, n, _stream(stream)),
            "pt_group_lasso_sgd_step")
+
+
+def pt_group_lasso_sgd_step_carried(ctx, layers, lam, lr, momentum, weight_decay=0.0, reg_sum_next=None, ws=None, stream=None,
+                                    with_maxima=False):
+    arr = layers if not isinstance(layers, (list, tuple)) else layer_array(layers)
+    hp = pt_sgd_hparams(lam, lr, momentum, weight_decay)
+    p, n = _ws(ws)
+    _check(lib().pt_group_lasso_sgd_step_carried(ctx.handle, arr, len(arr), byref(hp), int(bool(with_maxima)), _ptr(reg_sum_next), p, n,
+                                                 _stream(stream)),
+           "pt_group_lasso_sgd_step_carried")
+
+
+def pt_find_zero_groups_carried(ctx, layers, threshold=1e-4, zero_in_place=False, ws=None, stream=None):
+    arr = layers if not isinstance(layers, (list, tuple)) else layer_array(layers)
+    p, n = _ws(ws)
+    _check(lib().pt_find_zero_groups_carried(ctx.handle, arr, len(arr), threshold, int(bool(zero_in_place)), p, n, _stream(stream)),
+           "pt_find_zero_groups_carried")
 
 
 def pt_group_lasso_norms(ctx, layers, reg_sum_out=None, ws=None, stream=None):

@@ -1,4 +1,10 @@
-"""Builds the CUDA library in-tree: nvcc, sm_100a only, into paper_1901_09290_b200/libpt_b200.so."""
+"""Builds the CUDA library in-tree: nvcc, sm_100a only, into paper_1901_09290_b200/libpt_b200.so.
+
+``python -m paper_1901_09290_b200.build --trace`` (or ``build(trace=True)``) builds a second library,
+libpt_b200_trace.so, with -DPT_DEVICE_TRACE: CTA 0 of the convolution kernels then stamps %globaltimer at the hand-over
+points of its roles and the library exports pt_debug_gemm_trace / pt_debug_halo_trace / pt_debug_wgrad_trace, which copy
+the stamps (8 roles x 64 entries of nanoseconds) into a host array. It is a tuning aid; the product library never
+contains the hooks."""
 from __future__ import annotations
 
 import glob
@@ -26,14 +32,19 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+    if trace:
+        return _build(os.path.join(HERE, "libpt_b200_trace.so"), os.path.join(HERE, "build", "trace"), ["-DPT_DEVICE_TRACE"], verbose)
     if not force and not _stale():
         return LIB
+    return _build(LIB, os.path.join(HERE, "build"), [], verbose)
+
+
+def _build(lib: str, bdir: str, extra, verbose: bool) -> str:
     objs = []
     procs = []
-    bdir = os.path.join(HERE, "build")
     os.makedirs(bdir, exist_ok=True)
-    flags = [f for f in FLAGS if not f.startswith("--use_fast_math")]
+    flags = [f for f in FLAGS if not f.startswith("--use_fast_math")] + list(extra)
     for src in sources():
         obj = os.path.join(bdir, os.path.basename(src)[:-3] + ".o")
         cmd = [NVCC] + flags + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
@@ -47,11 +58,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB + ".tmp.%d" % os.getpid()
+    tmp = lib + ".tmp.%d" % os.getpid()
     subprocess.check_call([NVCC, "-shared", "-cudart", "static", "-o", tmp] + objs + ["-ldl", "-lpthread", "-lrt"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))

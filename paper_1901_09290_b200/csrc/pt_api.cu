@@ -38,7 +38,7 @@ extern "C" pt_status pt_create(pt_ctx **out, int device)
     bool ok = cudaMalloc(&c->d_status, 16) == cudaSuccess && cudaMemset(c->d_status, 0, 16) == cudaSuccess &&
               cudaMallocHost(&c->h_status, 16) == cudaSuccess && cudaMalloc(&c->d_arena, kArenaBytes) == cudaSuccess &&
               cudaMallocHost(&c->h_stage, kArenaBytes) == cudaSuccess &&
-              cudaMallocHost(&c->h_counts, 65536 * sizeof(int32_t)) == cudaSuccess &&
+              cudaMallocHost(&c->h_counts, (65536 + 16) * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&c->d_sync, kSyncWords * sizeof(unsigned int)) == cudaSuccess &&
               cudaMemset(c->d_sync, 0, kSyncWords * sizeof(unsigned int)) == cudaSuccess &&
               cudaEventCreateWithFlags(&c->upload_done, cudaEventDisableTiming) == cudaSuccess;

@@ -14,7 +14,8 @@
         if (e__ != cudaSuccess) { (void)cudaGetLastError(); return PT_ERR_CUDA; } \
     } while (0)
 
-// Device status word layout: [0] = first error code recorded (0 = none), [1] = detail (where), [2..3] spare.
+// Device status word layout: [0] = first error code recorded (0 = none), [1] = detail (where), [2] = ticket of the
+// keep-set scan (self-resetting), [3] spare.
 enum { PT_DEV_OK = 0, PT_DEV_TIMEOUT = 1, PT_DEV_BAD_INDEX = 2 };
 
 struct pt_region {              // one cached table in the arena
@@ -43,7 +44,8 @@ struct pt_ctx {
     std::vector<char> gather_args;
     unsigned gather_chunks = 0;
     size_t gather_jobs_bytes = 0;
-    int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan
+    int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan: [0] = flag the kernel raises, [16..] = counts
+    unsigned int plan_seq = 0;          // sequence number the next plan's flag carries
     unsigned int *d_sync = nullptr;     // zero-initialised, self-resetting arrival counters of the split weight gradient
     unsigned int sync_next = 0;         // ring position in d_sync
     uint64_t launches = 0;

@@ -2,6 +2,8 @@
 // rule, ascending keep maps by a block-wide scan, and the gather of the surviving weights,
 // momentum, bf16 shadow and BN vectors into the smaller dense model.
 #include "pt_internal.h"
+#include <atomic>
+#include <chrono>
 
 namespace {
 
@@ -13,10 +15,15 @@ struct SpaceDev {
 };
 struct MemberDev { const uint8_t *mask; };   // a writer's zero_out or a reader's zero_in (length = space size)
 
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // One block per space. keep[j] = fixed | OR_writers !zero_out[j] | OR_readers !zero_in[j].
+// The counts go straight to pinned host memory; the last block to finish (device ticket) then raises the host flag, so the
+// host learns the new sizes from one posted write instead of a copy and a stream synchronisation.
 __global__ void __launch_bounds__(1024) keep_scan_kernel(const SpaceDev *__restrict__ spaces,
                                                          const MemberDev *__restrict__ members,
-                                                         int32_t *__restrict__ new2old, int32_t *__restrict__ counts)
+                                                         int32_t *__restrict__ new2old, volatile int32_t *host_counts,
+                                                         volatile unsigned int *host_flag, unsigned int seq, unsigned int *ticket)
 {
     __shared__ int s_warp[32];
     __shared__ int s_base, s_tile;
@@ -24,13 +31,18 @@ __global__ void __launch_bounds__(1024) keep_scan_kernel(const SpaceDev *__restr
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
     if (threadIdx.x == 0) s_base = 0;
+    pdl_wait();                                  // the masks are the previous kernel's output
     __syncthreads();
     for (int j0 = 0; j0 < sp.size; j0 += blockDim.x) {
         const int j = j0 + threadIdx.x;
         int keep = 0;
         if (j < sp.size) {
             keep = sp.fixed;
-            for (int m = 0; m < sp.n_members && !keep; ++m) keep |= (members[sp.member0 + m].mask[j] == 0);
+            // all members' flags are fetched side by side (no early exit: the loads would form a dependent chain)
+            int dead = 1;
+#pragma unroll 4
+            for (int m = 0; m < sp.n_members; ++m) dead &= (members[sp.member0 + m].mask[j] != 0);
+            keep |= !dead;
         }
         const unsigned ball = __ballot_sync(0xffffffffu, keep);
         const int in_warp = __popc(ball & ((1u << lane) - 1u));
@@ -56,9 +68,22 @@ __global__ void __launch_bounds__(1024) keep_scan_kernel(const SpaceDev *__restr
     }
     const int total = s_base;
     for (int j = total + threadIdx.x; j < sp.size; j += blockDim.x) new2old[sp.map_off + j] = -1;
-    if (threadIdx.x == 0) counts[blockIdx.x] = total;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        host_counts[blockIdx.x] = total;
+        __threadfence_system();
+        if (atomicAdd(ticket, 1u) == gridDim.x - 1u) {
+            *ticket = 0u;
+            __threadfence_system();
+            *host_flag = seq;
+        }
+    }
 }
 
+// The gather walks the NEW tensor as one flat stream: a chunk is a run of whole lines (about 16K elements), thread t takes
+// elements t, t + 256, ... of it, so consecutive lanes read and write consecutive elements whatever the channel count. The
+// old line of every new line of the chunk and the old column of every new column sit in shared memory; a thread carries its
+// (line, column) along incrementally. Blocks are persistent and take equal shares of the chunk list.
 struct GatherJob {
     const float *ow, *ov; const __nv_bfloat16 *owb;
     float *nw, *nv; __nv_bfloat16 *nwb;
@@ -66,10 +91,14 @@ struct GatherJob {
     int Kn, Cn, RS, Co, ldwo, ldwn;
     int kind;                  // 0 = weight tensors, 1 = per-channel vector
     int Ko;                    // old number of output channels (range check of the map)
+    int lines, pad_;           // new tensor: Kn*RS lines
 };
-struct GatherChunk { int job, line0, nlines, col0; };
+struct GatherChunk { int job, line0, n_lines, pad; };
 
-constexpr int kGatherUnroll = 8;
+constexpr int kGThreads = 256;
+constexpr int kGMaxC = 4096;
+constexpr int kGMaxLines = 4096;
+constexpr int kGUnroll = 8;
 
 // A map entry outside the old tensor (a new graph larger than the plan's counts reads the -1 padding of the map) is skipped:
 // nothing is read or written for it, and the status word reports it (PT_ERR_INVALID_ARG at the next poll).
@@ -78,55 +107,85 @@ __device__ __forceinline__ void bad_map_entry(unsigned int *status, unsigned int
     if (atomicCAS(&status[0], 0u, (unsigned)PT_DEV_BAD_INDEX) == 0u) status[1] = where;
 }
 
-__global__ void __launch_bounds__(256) gather_kernel(const GatherJob *__restrict__ jobs, const GatherChunk *__restrict__ chunks,
-                                                     unsigned int *status)
+__global__ void __launch_bounds__(kGThreads, 4) gather_kernel(const GatherJob *__restrict__ jobs, const GatherChunk *__restrict__ chunks,
+                                                            int n_chunks, unsigned int *status)
 {
-    const GatherChunk ch = chunks[blockIdx.x];
-    const GatherJob J = jobs[ch.job];
-    if (J.kind == 1) {       // vector: nw[k'] = ow[mapK[k']]
-        for (int k = ch.line0 + threadIdx.x; k < ch.line0 + ch.nlines; k += blockDim.x) {
-            const int ko = J.mapK[k];
-            if (ko < 0 || ko >= J.Ko) { bad_map_entry(status, 50u); continue; }
-            J.nw[k] = J.ow[ko];
+    __shared__ int s_oline[kGMaxLines];          // old line of each new line of the chunk (-1: skipped)
+    __shared__ int s_co[kGMaxC];                 // old column of each new column (-1: skipped)
+    const int c_beg = (int)((long long)blockIdx.x * n_chunks / gridDim.x);
+    const int c_end = (int)((long long)(blockIdx.x + 1) * n_chunks / gridDim.x);
+    int cur_job = -1;
+    for (int ci = c_beg; ci < c_end; ++ci) {
+        const GatherChunk ch = chunks[ci];
+        const GatherJob J = jobs[ch.job];
+        if (J.kind == 1) {       // vector: nw[k'] = ow[mapK[k']]
+            for (int k = threadIdx.x; k < J.Kn; k += kGThreads) {
+                const int ko = J.mapK[k];
+                if (ko < 0 || ko >= J.Ko) { bad_map_entry(status, 50u); continue; }
+                J.nw[k] = J.ow[ko];
+            }
+            continue;
         }
-        return;
-    }
-    // Lines of the NEW tensor are (k', rs); a block covers a run of lines x up to 256 columns. Each thread owns one new
-    // column c' (its old column looked up once) and keeps four lines in flight; writes are coalesced, reads gathered.
-    int TX = 32;
-    while (TX < J.Cn && TX < 256) TX <<= 1;
-    const int TY = 256 / TX, tx = threadIdx.x % TX, ty = threadIdx.x / TX;
-    const int c = ch.col0 + tx;
-    if (c >= J.Cn) return;
-    const int co = J.mapC[c];
-    if (co < 0 || co >= J.Co) { bad_map_entry(status, 51u); return; }
-    for (int l = ty; l < ch.nlines; l += kGatherUnroll * TY) {
-        float w[kGatherUnroll], v[kGatherUnroll];
-        __nv_bfloat16 h[kGatherUnroll];
-        bool okk[kGatherUnroll];
-#pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u) {
-            const int line = ch.line0 + l + u * TY;
-            okk[u] = false;
-            if (l + u * TY < ch.nlines) {
-                const int kn = line / J.RS, rs = line - kn * J.RS;
-                const int ko = J.mapK[kn];
-                if (ko < 0 || ko >= J.Ko) { bad_map_entry(status, 52u); continue; }
-                okk[u] = true;
-                const size_t oline = (size_t)ko * J.RS + rs;
-                w[u] = J.ow[oline * J.Co + co];
-                if (J.nv) v[u] = J.ov[oline * J.Co + co];
-                if (J.nwb) h[u] = J.owb[oline * J.ldwo + co];
+        __syncthreads();                         // the previous chunk's tables are no longer read
+        if (ch.job != cur_job) {
+            cur_job = ch.job;
+            for (int c = threadIdx.x; c < J.Cn; c += kGThreads) {
+                int o = J.mapC[c];
+                if (o < 0 || o >= J.Co) { bad_map_entry(status, 51u); o = -1; }
+                s_co[c] = o;
             }
         }
+        for (int l = threadIdx.x; l < ch.n_lines; l += kGThreads) {
+            const int line = ch.line0 + l;
+            const int kn = line / J.RS, rs = line - kn * J.RS;
+            const int ko = J.mapK[kn];
+            int ol = -1;
+            if (ko < 0 || ko >= J.Ko) bad_map_entry(status, 52u);
+            else ol = ko * J.RS + rs;
+            s_oline[l] = ol;
+        }
+        __syncthreads();
+        // 32-bit element offsets throughout (the host checks that both tensors have fewer than 2^31 elements at their pitches)
+        const float *__restrict__ ow = J.ow;
+        const float *__restrict__ ov = J.ov;
+        const unsigned short *__restrict__ ob = reinterpret_cast<const unsigned short *>(J.owb);
+        float *__restrict__ nw = J.nw + (size_t)ch.line0 * J.Cn;
+        float *__restrict__ nv = J.nv ? J.nv + (size_t)ch.line0 * J.Cn : nullptr;
+        unsigned short *__restrict__ nb = J.nwb ? reinterpret_cast<unsigned short *>(J.nwb) + (size_t)ch.line0 * J.ldwn : nullptr;
+        const bool has_v = nv != nullptr, has_b = nb != nullptr;
+        const unsigned Co = (unsigned)J.Co, ldwo = (unsigned)J.ldwo, ldwn = (unsigned)J.ldwn;
+        const int Cn = J.Cn, total = ch.n_lines * Cn;
+        const int dl = kGThreads / Cn, dc = kGThreads - dl * Cn;                 // one step of 256 elements in (line, column)
+        int l = (int)threadIdx.x / Cn, c = (int)threadIdx.x - l * Cn;
+        for (int i0 = threadIdx.x; i0 < total; i0 += kGUnroll * kGThreads) {
+            float w[kGUnroll], v[kGUnroll];
+            unsigned short hb[kGUnroll];
+            int ll[kGUnroll], cc[kGUnroll];
+            bool ok[kGUnroll];
 #pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u) {
-            const int line = ch.line0 + l + u * TY;
-            if (okk[u]) {
-                const size_t dst = (size_t)line * J.Cn + c;
-                J.nw[dst] = w[u];
-                if (J.nv) J.nv[dst] = v[u];
-                if (J.nwb) J.nwb[(size_t)line * J.ldwn + c] = h[u];
+            for (int u = 0; u < kGUnroll; ++u) {
+                ll[u] = l; cc[u] = c;
+                ok[u] = false;
+                if (i0 + u * kGThreads < total) {
+                    const int ol = s_oline[l], co = s_co[c];
+                    if ((ol | co) >= 0) {
+                        ok[u] = true;
+                        const unsigned src = (unsigned)ol * Co + (unsigned)co;
+                        w[u] = ow[src];
+                        if (has_v) v[u] = ov[src];
+                        if (has_b) hb[u] = ob[(unsigned)ol * ldwo + (unsigned)co];
+                    }
+                }
+                l += dl; c += dc;
+                if (c >= Cn) { c -= Cn; ++l; }
+            }
+#pragma unroll
+            for (int u = 0; u < kGUnroll; ++u) {
+                if (!ok[u]) continue;
+                const unsigned idx = (unsigned)(i0 + u * kGThreads);
+                nw[idx] = w[u];
+                if (has_v) nv[idx] = v[u];
+                if (has_b) nb[(unsigned)ll[u] * ldwn + (unsigned)cc[u]] = hb[u];
             }
         }
     }
@@ -183,13 +242,42 @@ extern "C" pt_status pt_reconfigure_plan(pt_ctx *c, const pt_graph *g, int32_t *
     char *dev = nullptr;
     s = pt_upload_table(c, &c->graph_tab, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
-    int32_t *d_counts = (int32_t *)(dev + sb + mb);
-    keep_scan_kernel<<<g->n_spaces, 1024, 0, st>>>((const SpaceDev *)dev, (const MemberDev *)(dev + sb), new2old, d_counts);
+    // counts and flag live in pinned host memory the kernel writes directly: [0] = flag (sequence number), [16..] = counts
+    volatile unsigned int *flag = (volatile unsigned int *)c->h_counts;
+    volatile int32_t *counts = (volatile int32_t *)c->h_counts + 16;
+    const unsigned int seq = ++c->plan_seq;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)g->n_spaces); cfg.blockDim = dim3(1024); cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    PT_CUDA_OK(cudaLaunchKernelEx(&cfg, keep_scan_kernel, (const SpaceDev *)dev, (const MemberDev *)(dev + sb), new2old,
+                                  (volatile int32_t *)counts, (volatile unsigned int *)flag, seq, c->d_status + 2));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
-    PT_CUDA_OK(cudaMemcpyAsync(c->h_counts, d_counts, (size_t)g->n_spaces * 4, cudaMemcpyDeviceToHost, st));
-    PT_CUDA_OK(cudaStreamSynchronize(st));     // the documented synchronisation: the host needs the new sizes
-    memcpy(new_sizes, c->h_counts, (size_t)g->n_spaces * 4);
+    // The documented synchronisation: the host needs the new sizes. It waits for the kernel's flag (bounded), looking at the
+    // stream now and then so that an error upstream ends the wait.
+    {
+        const auto t0 = std::chrono::steady_clock::now();
+        unsigned spins = 0;
+        bool seen = false;
+        while (!(seen = (*flag == seq))) {
+            if ((++spins & 0x3fffu) == 0u) {
+                const cudaError_t q = cudaStreamQuery(st);
+                if (q == cudaSuccess) { seen = (*flag == seq); break; }
+                if (q != cudaErrorNotReady) { (void)cudaGetLastError(); return PT_ERR_CUDA; }
+                if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(30)) break;
+            }
+        }
+        if (!seen) {
+            PT_CUDA_OK(cudaStreamSynchronize(st));
+            if (*flag != seq) return PT_ERR_CUDA;
+        }
+    }
+    std::atomic_thread_fence(std::memory_order_acquire);
+    for (int i = 0; i < g->n_spaces; ++i) new_sizes[i] = counts[i];
     return PT_OK;
 }
 
@@ -214,7 +302,9 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
     }
     if (c->gather_tab.valid && c->gather_chunks && args == c->gather_args) {
         const char *dev = c->d_arena + c->gather_tab.off;
-        gather_kernel<<<c->gather_chunks, 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + c->gather_jobs_bytes), c->d_status);
+        const unsigned grid = c->gather_chunks < (unsigned)(4 * c->sm_count) ? c->gather_chunks : (unsigned)(4 * c->sm_count);
+        gather_kernel<<<grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + c->gather_jobs_bytes),
+                                                  (int)c->gather_chunks, c->d_status);
         c->launches += 1;
         PT_CUDA_OK(cudaGetLastError());
         return PT_OK;
@@ -239,6 +329,8 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         if (n.K == 0 || n.C == 0) continue;                 // a dead layer: nothing to carry over
         if (!o.w || !n.w || (n.v && !o.v) || (n.w_bf16 && !o.w_bf16)) return PT_ERR_INVALID_ARG;
         if (n.w_bf16 && (n.ldw < n.C || n.ldw % 8)) return PT_ERR_INVALID_ARG;
+        if (n.C > kGMaxC) return PT_ERR_UNSUPPORTED;
+        if ((long long)o.K * o.RS * (o.ldw > o.C ? o.ldw : o.C) >= (1ll << 31)) return PT_ERR_UNSUPPORTED;
         GatherJob J;
         memset(&J, 0, sizeof(J));
         J.ow = o.w; J.ov = o.v; J.owb = (const __nv_bfloat16 *)o.w_bf16;
@@ -247,21 +339,22 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         J.mapC = new2old + map_off[ol.in_space];
         J.Kn = n.K; J.Cn = n.C; J.RS = n.RS; J.Co = o.C; J.Ko = o.K; J.ldwo = o.ldw; J.ldwn = n.ldw;
         J.kind = 0;
+        J.lines = n.K * n.RS;
         const int job = (int)jobs.size();
         jobs.push_back(J);
-        const int lines = n.K * n.RS;
-        int TX = 32;
-        while (TX < n.C && TX < 256) TX <<= 1;
-        const int per = (256 / TX) * kGatherUnroll * 3;      // equal trip counts for every block
-        for (int l0 = 0; l0 < lines; l0 += per)
-            for (int c0 = 0; c0 < n.C; c0 += TX) chunks.push_back(GatherChunk{job, l0, lines - l0 < per ? lines - l0 : per, c0});
+        {
+            int per = 16384 / n.C;                       // whole lines, about 16K elements per chunk
+            if (per < 1) per = 1;
+            if (per > kGMaxLines) per = kGMaxLines;
+            for (int l0 = 0; l0 < J.lines; l0 += per) chunks.push_back(GatherChunk{job, l0, J.lines - l0 < per ? J.lines - l0 : per, 0});
+        }
         for (int b = 0; b < 4; ++b) {
             if (!nl.bn[b]) continue;
             if (!ol.bn[b]) return PT_ERR_INVALID_ARG;
             GatherJob V;
             memset(&V, 0, sizeof(V));
             V.ow = ol.bn[b]; V.nw = nl.bn[b]; V.mapK = J.mapK; V.Kn = n.K; V.Ko = o.K; V.kind = 1;
-            chunks.push_back(GatherChunk{(int)jobs.size(), 0, n.K, 0});
+            chunks.push_back(GatherChunk{(int)jobs.size(), 0, 0, 0});
             jobs.push_back(V);
         }
     }
@@ -274,7 +367,11 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
     c->gather_chunks = 0;
     s = pt_upload_table(c, &c->gather_tab, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
-    gather_kernel<<<(unsigned)chunks.size(), 256, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + jb), c->d_status);
+    {
+        const unsigned nchk = (unsigned)chunks.size();
+        const unsigned grid = nchk < (unsigned)(4 * c->sm_count) ? nchk : (unsigned)(4 * c->sm_count);
+        gather_kernel<<<grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + jb), (int)nchk, c->d_status);
+    }
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     c->gather_args.swap(args);

@@ -72,30 +72,6 @@ def empty_model(net: W.Net, fill: float = 0.0) -> W.Model:
                    [[torch.full((l.K,), fill) for _ in range(4)] for l in net.layers])
 
 
-def union_and_gating_counts(net: W.Net, zero_out, zero_in):
-    """Channel bookkeeping for the two reconfiguration mechanisms of Sec. 4.2, from per-layer zero-group masks (host logic,
-    no tensor data): returns (union_sizes per space, [(C, K) per layer under channel union], [(C, K) per layer under
-    channel gating]). Union keeps a channel of a space unless it is sparsified in every member; gating additionally
-    restricts every reader / writer of a space shared by several branches to its own dense channels."""
-    ns = len(net.space_sizes)
-    keep = [np.zeros(sz, bool) | bool(fx) for sz, fx in zip(net.space_sizes, net.space_fixed)]
-    n_w, n_r = [0] * ns, [0] * ns
-    for li, l in enumerate(net.layers):
-        keep[l.out_space] |= np.asarray(zero_out[li]) == 0
-        keep[l.in_space] |= np.asarray(zero_in[li]) == 0
-        n_w[l.out_space] += 1
-        n_r[l.in_space] += 1
-    shared = [(n_w[s] > 1 or n_r[s] > 1) and not net.space_fixed[s] for s in range(ns)]
-    sizes = [int(k.sum()) for k in keep]
-    union = [(sizes[l.in_space], sizes[l.out_space]) for l in net.layers]
-    gating = []
-    for li, l in enumerate(net.layers):
-        c = int((keep[l.in_space] & (np.asarray(zero_in[li]) == 0)).sum()) if shared[l.in_space] else sizes[l.in_space]
-        k = int((keep[l.out_space] & (np.asarray(zero_out[li]) == 0)).sum()) if shared[l.out_space] else sizes[l.out_space]
-        gating.append((c, k))
-    return sizes, union, gating
-
-
 def conv_macs(net: W.Net, counts) -> int:
     """Forward multiply-accumulates per image with the given (C, K) per layer."""
     return sum(l.P * l.P * k * c * l.R * l.R for l, (c, k) in zip(net.layers, counts))
@@ -316,6 +292,10 @@ class TrainStep:
 
     def lasso(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
         B.pt_group_lasso_sgd_step(self.ctx, self.mp.arr, lam, lr, mu, 0.0, self.mp.reg, self.mp.ws, stream)
+
+    def lasso_carried(self, stream=None, lam=1e-4, lr=0.1, mu=0.9, with_maxima=False):
+        """The step in its carried form: needs lasso_norms() (or a previous carried step) on the current weights."""
+        B.pt_group_lasso_sgd_step_carried(self.ctx, self.mp.arr, lam, lr, mu, 0.0, self.mp.reg, self.mp.ws, stream, with_maxima)
 
     def lasso_norms(self, stream=None):
         B.pt_group_lasso_norms(self.ctx, self.mp.arr, self.mp.reg, self.mp.ws, stream)

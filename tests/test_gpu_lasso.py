@@ -213,3 +213,93 @@ def test_cross_entropy_and_set_coeff(n, classes, ld):
         B.pt_cross_entropy(c, zd, ld_, n, classes, classes - 1, loss, ws)
     torch.cuda.synchronize()
     c.poll()
+
+
+def test_carried_steps_follow_the_oracle_chain_and_feed_the_detection():
+    """Two steps in the carried form (22 bytes per parameter: the norms of W_{i+1} are taken while step i writes it) against
+    two oracle steps; the sums the second step uses are those the first one left. Then the masks from the carried maxima
+    must be the oracle's brute-force masks of the GPU's own weights, and equal to the reading detection's, bit for bit."""
+    ctx = Hh.ctx()
+    net = W.resnet32()
+    kept = W.choose_kept(net, W.random_keep(net, W.BASE_SEED + 21), W.BASE_SEED + 21)
+    model = W.gen_model(net, W.BASE_SEED + 21, kept=kept, decoys=2)
+    lam, lr, mu, wd = 2e-3, 0.1, 0.9, 1e-4
+    dm = DevModel(model)
+    reg_next = torch.zeros(1, dtype=torch.float64, device="cuda")
+    B.pt_group_lasso_norms(ctx, dm.arr, dm.reg, dm.ws)
+    B.pt_group_lasso_sgd_step_carried(ctx, dm.arr, lam, lr, mu, wd, reg_next, dm.ws)
+    torch.cuda.synchronize()
+    ctx.poll()
+    ref_w, ref_v = [], []
+    reg0 = reg1 = 0.0
+    for li, l in enumerate(net.layers):
+        reg_in = net.space_stage[l.in_space] != 0
+        w1, v1, s_out, s_in, reg = oracle.lasso_sgd(model.w[li].numpy(), model.g[li].numpy(), model.v[li].numpy(), lam, lr, mu, wd,
+                                                     reg_in=reg_in, reg_out=True)
+        reg0 += reg
+        Hh.check_update(dm.w[li], w1, f"{l.name} w step 1")
+        Hh.check_update(dm.v[li], v1, f"{l.name} v step 1")
+        # sums of squares of the NEW weights, as the carried form leaves them
+        w1f = w1.astype(np.float32).astype(np.float64)
+        np.testing.assert_allclose(dm.sq_out[li].cpu().numpy(), (w1f ** 2).sum(axis=(1, 2, 3)), rtol=3e-5, atol=1e-30)
+        np.testing.assert_allclose(dm.sq_in[li].cpu().numpy(), (w1f ** 2).sum(axis=(0, 1, 2)), rtol=3e-5, atol=1e-30)
+        w2, v2, _, _, r1 = oracle.lasso_sgd(w1.astype(np.float32), model.g[li].numpy(), v1.astype(np.float32), lam, lr, mu, wd,
+                                            reg_in=reg_in, reg_out=True)
+        reg1 += r1
+        ref_w.append(w2)
+        ref_v.append(v2)
+    assert abs(dm.reg.item() - reg0) <= 1e-5 * reg0
+    assert abs(reg_next.item() - reg1) <= 2e-5 * reg1          # Eq. 2's sum of the new weights
+    B.pt_group_lasso_sgd_step_carried(ctx, dm.arr, lam, lr, mu, wd, reg_next, dm.ws, with_maxima=True)
+    torch.cuda.synchronize()
+    ctx.poll()
+    for li, l in enumerate(net.layers):
+        # the second step starts from the first step's fp32 results, which differ from the oracle's fp64 ones by rounding
+        g = dm.w[li].cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(g - ref_w[li]) <= 2e-5 * np.linalg.norm(ref_w[li]), l.name
+        assert torch.equal(dm.wb[li][..., :l.C], dm.w[li].to(torch.bfloat16)), l.name
+        # zero groups stay exactly zero
+        zo = (model.w[li].abs().amax(dim=(1, 2, 3)) == 0) & (model.g[li].abs().amax(dim=(1, 2, 3)) == 0) & \
+             (model.v[li].abs().amax(dim=(1, 2, 3)) == 0)
+        if zo.any():
+            assert torch.all(dm.w[li][zo.cuda()] == 0)
+    # detection from the maxima the step left behind
+    B.pt_find_zero_groups_carried(ctx, dm.arr, 1e-4, False, dm.ws)
+    torch.cuda.synchronize()
+    carried = [(dm.z_out[li].clone(), dm.z_in[li].clone()) for li in range(len(net.layers))]
+    n_zero = 0
+    for li, l in enumerate(net.layers):
+        zo, zi = oracle.find_zero_groups(dm.w[li].cpu().numpy(), 1e-4)
+        assert carried[li][0].cpu().numpy().tolist() == zo.tolist(), l.name
+        assert carried[li][1].cpu().numpy().tolist() == zi.tolist(), l.name
+        n_zero += int(zo.sum()) + int(zi.sum())
+    assert n_zero > 0
+    B.pt_find_zero_groups(ctx, dm.arr, 1e-4, False, dm.ws)
+    torch.cuda.synchronize()
+    ctx.poll()
+    for li in range(len(net.layers)):
+        assert torch.equal(dm.z_out[li], carried[li][0]) and torch.equal(dm.z_in[li], carried[li][1])
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (64, 7, 3), (7, 3, 300), (33, 1, 143), (300, 1, 2500)])
+def test_carried_step_odd_shapes(shape):
+    K, R, C = shape
+    ctx = Hh.ctx()
+    net = W.single_layer(C, K, R, 8)
+    model = W.gen_model(net, W.BASE_SEED + 80 + K)
+    dm = DevModel(model)
+    B.pt_group_lasso_norms(ctx, dm.arr, dm.reg, dm.ws)
+    B.pt_group_lasso_sgd_step_carried(ctx, dm.arr, 3e-3, 0.05, 0.9, 1e-4, None, dm.ws, with_maxima=True)
+    torch.cuda.synchronize()
+    ctx.poll()
+    reg_in = net.space_stage[net.layers[0].in_space] != 0
+    w1, v1, *_ = oracle.lasso_sgd(model.w[0].numpy(), model.g[0].numpy(), model.v[0].numpy(), 3e-3, 0.05, 0.9, 1e-4, reg_in=reg_in, reg_out=True)
+    Hh.check_update(dm.w[0], w1, "w")
+    Hh.check_update(dm.v[0], v1, "v")
+    wf = dm.w[0].cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(dm.sq_out[0].cpu().numpy(), (wf ** 2).sum(axis=(1, 2, 3)), rtol=3e-5, atol=1e-30)
+    np.testing.assert_allclose(dm.sq_in[0].cpu().numpy(), (wf ** 2).sum(axis=(0, 1, 2)), rtol=3e-5, atol=1e-30)
+    B.pt_find_zero_groups_carried(ctx, dm.arr, 1e-4, False, dm.ws)
+    torch.cuda.synchronize()
+    zo, zi = oracle.find_zero_groups(dm.w[0].cpu().numpy(), 1e-4)
+    assert dm.z_out[0].cpu().numpy().tolist() == zo.tolist() and dm.z_in[0].cpu().numpy().tolist() == zi.tolist()

@@ -62,3 +62,33 @@ def test_single_rank_is_the_identity():
     import bench
     assert bench.max_over_ranks(7.5, 1, device="cpu") == 7.5
     assert abs(bench.whole_job_value(1e12, 1, 10.0, 10) - 1.0e12 / 1e-3 / 1e12) < 1e-9
+
+
+def _spawned_rank(path):
+    """What a rank started by bench.spawn_ranks sees: the launcher's environment, and a working rendezvous."""
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    assert os.environ["MASTER_ADDR"] == "127.0.0.1" and int(os.environ["LOCAL_RANK"]) == rank
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    t = torch.tensor([float(rank + 1)])
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    with open(f"{path}.{rank}", "w") as f:
+        f.write(f"{world} {t.item()}")
+    dist.destroy_process_group()
+
+
+def test_bench_spawns_the_ranks_itself_when_no_launcher_did(tmp_path):
+    """`bench.py --gpus N` without torchrun starts N ranks (one per GPU) instead of silently running one."""
+    sys.path.insert(0, ROOT)
+    import bench
+    path = str(tmp_path / "rank")
+    bench.spawn_ranks(2, _spawned_rank, (path,))
+    for rank in range(2):
+        world, total = open(f"{path}.{rank}").read().split()
+        assert int(world) == 2 and float(total) == 3.0
+
+
+def test_bench_refuses_a_world_size_that_contradicts_gpus():
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"], env=env, capture_output=True, text=True)
+    assert r.returncode != 0 and "--gpus 2" in (r.stderr + r.stdout)
