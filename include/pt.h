@@ -337,7 +337,11 @@ pt_status pt_reconfigure_plan(pt_ctx *ctx, const pt_graph *g, int32_t *new2old, 
  * new_g must have the same topology, and each space size equal to the count pt_reconfigure_plan returned.
  * Layers whose new K or C is 0 are skipped. A new space larger than its planned count makes the gather meet the -1 padding of
  * the map: such entries are skipped (the destination elements stay as they were) and pt_poll_device_status reports
- * PT_ERR_INVALID_ARG. */
+ * PT_ERR_INVALID_ARG.
+ * The graphs may hold a subset of a model's layers (the spaces stay whole), so a model can be gathered in parts, e.g. the first
+ * layers ahead of the forward pass and the rest beside it. The library keeps the device tables of the last four distinct
+ * argument sets; a CUDA graph captured around this call embeds its table's address, which stays valid until four other
+ * argument sets have been used with the context. */
 pt_status pt_reconfigure(pt_ctx *ctx, const pt_graph *old_g, const int32_t *new2old, const pt_graph *new_g, void *stream);
 
 /* ------------------------------------------------------------------------------------------

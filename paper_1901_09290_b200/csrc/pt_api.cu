@@ -1,8 +1,8 @@
 // Context management, status handling, table upload and the conv entry points' dispatch.
 #include "pt_internal.h"
 
-static const size_t kArenaBytes = 4u << 20;     // 4 MiB of tables
-static const size_t kSlotBytes = 512u << 10;    // eight slots of 512 KiB
+static const size_t kArenaBytes = 5u << 20;     // 5 MiB of tables: ten slots of 512 KiB
+static const size_t kSlotBytes = 512u << 10;
 static const size_t kSyncWords = 16384;         // arrival counters of the split weight gradients
 
 extern "C" const char *pt_status_string(pt_status s)
@@ -47,7 +47,7 @@ extern "C" pt_status pt_create(pt_ctx **out, int device)
     for (int i = 0; i < 3; ++i) { c->lasso_tab[i].off = off; c->lasso_tab[i].cap = kSlotBytes; off += kSlotBytes; }
     for (int i = 0; i < 2; ++i) { c->detect_tab[i].off = off; c->detect_tab[i].cap = kSlotBytes; off += kSlotBytes; }
     c->graph_tab.off = off;  c->graph_tab.cap = kSlotBytes; off += kSlotBytes;
-    c->gather_tab.off = off; c->gather_tab.cap = 2 * kSlotBytes;
+    for (int i = 0; i < 4; ++i) { c->gather_slot[i].reg.off = off; c->gather_slot[i].reg.cap = kSlotBytes; off += kSlotBytes; }
     // Driver entry points for tensor-map encoding, looked up at run time so the library loads without libcuda.
     cudaDriverEntryPointQueryResult qr;
     void *fn = nullptr;

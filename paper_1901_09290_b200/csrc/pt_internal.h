@@ -37,13 +37,18 @@ struct pt_ctx {
     bool upload_pending = false;
     // Cached device tables. A captured CUDA graph embeds the device address of the table its kernels read, so tables of
     // different callers must not evict each other: the lasso step and the detection have their own slot sets.
-    pt_region lasso_tab[3], detect_tab[2], graph_tab, gather_tab;
+    pt_region lasso_tab[3], detect_tab[2], graph_tab;
     int lasso_next = 0, detect_next = 0;
-    // pt_reconfigure: the argument bytes the gather table in `gather_tab` was built from, and its launch shape. A call with
-    // the same arguments (every reconfiguration of a fixed pair of models) launches straight from the cached table.
-    std::vector<char> gather_args;
-    unsigned gather_chunks = 0;
-    size_t gather_jobs_bytes = 0;
+    // pt_reconfigure: four cached gather tables, each with the argument bytes it was built from and its launch shape. A call
+    // with the same arguments (every reconfiguration of a fixed pair of models, or of a fixed part of them) launches straight
+    // from its table; a caller that gathers a model in two parts keeps both tables alive.
+    struct GatherSlot {
+        pt_region reg;
+        std::vector<char> args;
+        unsigned chunks = 0;
+        size_t jobs_bytes = 0;
+    } gather_slot[4];
+    int gather_next = 0;
     int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan: [0] = flag the kernel raises, [16..] = counts
     unsigned int plan_seq = 0;          // sequence number the next plan's flag carries
     unsigned int *d_sync = nullptr;     // zero-initialised, self-resetting arrival counters of the split weight gradient

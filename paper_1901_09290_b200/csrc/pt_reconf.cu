@@ -300,11 +300,13 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         memcpy(a, og->links, nk); a += nk; memcpy(a, ng->links, nk); a += nk;
         memcpy(a, &new2old, sizeof(new2old));
     }
-    if (c->gather_tab.valid && c->gather_chunks && args == c->gather_args) {
-        const char *dev = c->d_arena + c->gather_tab.off;
-        const unsigned grid = c->gather_chunks < (unsigned)(4 * c->sm_count) ? c->gather_chunks : (unsigned)(4 * c->sm_count);
-        gather_kernel<<<grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + c->gather_jobs_bytes),
-                                                  (int)c->gather_chunks, c->d_status);
+    for (int i = 0; i < 4; ++i) {
+        pt_ctx::GatherSlot &gs = c->gather_slot[i];
+        if (!(gs.reg.valid && gs.chunks && args == gs.args)) continue;
+        const char *dev = c->d_arena + gs.reg.off;
+        const unsigned grid = gs.chunks < (unsigned)(4 * c->sm_count) ? gs.chunks : (unsigned)(4 * c->sm_count);
+        gather_kernel<<<grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + gs.jobs_bytes), (int)gs.chunks,
+                                                  c->d_status);
         c->launches += 1;
         PT_CUDA_OK(cudaGetLastError());
         return PT_OK;
@@ -364,8 +366,10 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
     memcpy(buf.data(), jobs.data(), jobs.size() * sizeof(GatherJob));
     memcpy(buf.data() + jb, chunks.data(), cb);
     char *dev = nullptr;
-    c->gather_chunks = 0;
-    s = pt_upload_table(c, &c->gather_tab, buf.data(), buf.size(), st, &dev);
+    pt_ctx::GatherSlot &gs = c->gather_slot[c->gather_next];
+    c->gather_next = (c->gather_next + 1) & 3;
+    gs.chunks = 0;
+    s = pt_upload_table(c, &gs.reg, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
     {
         const unsigned nchk = (unsigned)chunks.size();
@@ -374,8 +378,8 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
     }
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
-    c->gather_args.swap(args);
-    c->gather_chunks = (unsigned)chunks.size();
-    c->gather_jobs_bytes = jb;
+    gs.args.swap(args);
+    gs.chunks = (unsigned)chunks.size();
+    gs.jobs_bytes = jb;
     return PT_OK;
 }

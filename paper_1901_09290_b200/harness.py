@@ -51,6 +51,7 @@ class DeviceModel:
         self.ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
         self.reg = torch.zeros(1, dtype=torch.float64, device="cuda")
         self._graph = None
+        self._subgraphs = {}
 
     def reg_in(self, li: int) -> bool:
         return bool(self.layers[li].reg_in)
@@ -60,6 +61,16 @@ class DeviceModel:
             links = [(l.in_space, l.out_space) for l in self.net.layers]
             self._graph = B.GraphHandle(self.net.space_sizes, self.net.space_fixed, self.layers, links, self.bn)
         return self._graph
+
+    def subgraph(self, first: int, count: int) -> B.GraphHandle:
+        """The same channel spaces with layers [first, first + count) only (for a compaction done in parts)."""
+        key = (first, count)
+        if key not in self._subgraphs:
+            ls = self.net.layers[first:first + count]
+            links = [(l.in_space, l.out_space) for l in ls]
+            self._subgraphs[key] = B.GraphHandle(self.net.space_sizes, self.net.space_fixed, self.layers[first:first + count], links,
+                                                 self.bn[first:first + count])
+        return self._subgraphs[key]
 
     def n_params(self) -> int:
         return sum(l.K * l.C * l.R * l.R for l in self.net.layers)
@@ -112,6 +123,7 @@ class TrainStep:
         # that can be in flight then fits on the device together, whatever order the hardware picks its CTAs in.
         # `wgrad_ctas` is the nominal share; _wgrad_limits() refines it per launch under the same constraint.
         self.wgrad_ctas, self.wgrad_streams = wgrad_ctas, max(1, wgrad_streams)
+        self.gather_split = 4       # layers whose weights are gathered before the forward pass starts (the rest beside it)
         ctx.set_wgrad_cta_limit(wgrad_ctas)
         self.dense_net = dense_net
         self.net = W.with_sizes(dense_net, counts)
@@ -268,13 +280,26 @@ class TrainStep:
         return 4 * self.md.n_params() + 18 * self.mp.n_params()
 
     # ---- the path
-    def reconfigure(self, stream=None):
+    def reconfigure_plan(self, stream=None):
+        """Detection and keep-set scan: everything up to (and including) the host synchronisation that returns the new sizes."""
         c = self.ctx
         B.pt_find_zero_groups(c, self.md.arr, 1e-4, False, self.md.ws, stream)
         sizes = B.pt_reconfigure_plan(c, self.md.graph(), self.new2old, stream)
         if sizes != self.counts:
             raise RuntimeError(f"reconfiguration plan returned {sizes}, expected {self.counts}")
-        B.pt_reconfigure(c, self.md.graph(), self.new2old, self.mp.graph(), stream)
+
+    def gather(self, first: int = 0, count: Optional[int] = None, stream=None):
+        """The compaction gather of layers [first, first + count) into the pruned model."""
+        n = len(self.net.layers)
+        count = n - first if count is None else count
+        if first == 0 and count == n:
+            B.pt_reconfigure(self.ctx, self.md.graph(), self.new2old, self.mp.graph(), stream)
+        else:
+            B.pt_reconfigure(self.ctx, self.md.subgraph(first, count), self.new2old, self.mp.subgraph(first, count), stream)
+
+    def reconfigure(self, stream=None):
+        self.reconfigure_plan(stream)
+        self.gather(stream=stream)
 
     def conv_fwd(self, li, stream=None):
         B.pt_conv_fwd(self.ctx, self.desc[li], self.x[li], self.mp.wb[li], self.y[li], self.ws, stream)
@@ -327,7 +352,7 @@ class TrainStep:
                 out.append((first, d))
         return out
 
-    def train_two_streams(self, fwd: bool = True, dgrad: bool = True, wgrad: bool = True, lasso: bool = True):
+    def train_two_streams(self, fwd: bool = True, dgrad: bool = True, wgrad: bool = True, lasso: bool = True, gather: bool = False):
         """The same launches on several streams, following the network's own data dependencies: the weight gradient of a
         layer needs only x_l and dy_l, so it starts when dy_l exists and runs beside the data gradients below it (round-robin
         over the weight-gradient streams, each with its own workspace); a block's projection shortcut is independent of
@@ -339,13 +364,31 @@ class TrainStep:
         fork_at = {f: d for f, d in br}          # before layer f: start shortcut d on the aux stream
         ds_set = {d for _, d in br}
         forked = set()                           # streams that joined this launch sequence and must be joined back
+        gather_join = None
+        if gather:
+            # The gather needs no host: the first layers' weights are gathered on the main stream, the rest on a side stream
+            # beside the first forward layers (large maps, latency bound, SMs to spare), joined back before their first use.
+            k = min(self.gather_split, n)
+            self.gather(0, k, main)
+            if k < n:
+                gstream = ws[0]
+                gstream.wait_stream(main)
+                forked.add(gstream)
+                self.gather(k, n - k, gstream)
+                gather_join = (k, gstream)
         if lasso and fwd:
             # the group norms need the weights only (GroupLassoReg(W_i) of Algorithm 1): they run beside the forward pass
             nstream = ws[-1]
             nstream.wait_stream(main)
+            if gather_join is not None:
+                nstream.wait_stream(gather_join[1])      # the norms read every layer's gathered weights
             forked.add(nstream)
             self.lasso_norms(nstream)
         for li in range(n if fwd else 0):
+            if gather_join is not None and li == gather_join[0]:
+                main.wait_stream(gather_join[1])
+                aux.wait_stream(gather_join[1])
+                gather_join = None
             if li in fork_at:
                 aux.wait_stream(main)
                 forked.add(aux)
@@ -381,6 +424,8 @@ class TrainStep:
             if join_after == li:
                 main.wait_stream(aux)            # the gradient of the block's input sums both branches
                 join_after = None
+        if gather_join is not None:
+            main.wait_stream(gather_join[1])
         for w in forked:
             main.wait_stream(w)
         if lasso:
@@ -396,7 +441,7 @@ class TrainStep:
             self.train_two_streams(fwd=kind == "fwd", dgrad=kind == "dgrad", wgrad=kind == "wgrad", lasso=False)
         return g
 
-    def build_graph(self, two_streams: bool = True):
+    def build_graph(self, two_streams: bool = True, gather_in_graph: bool = True):
         """Captures the training part of the step (every launch after the reconfiguration's host sync) into a CUDA graph.
         Call after at least one eager step, so that every table and kernel attribute is already set up."""
         self._side = torch.cuda.Stream()
@@ -406,19 +451,32 @@ class TrainStep:
         l0 = self.ctx.launch_count()
         self.graph = torch.cuda.CUDAGraph()
         self._graph_has_update = self.world <= 1
+        self._graph_has_gather = bool(two_streams and gather_in_graph)
+        if self._graph_has_gather:
+            # the part gathers once eagerly: their device tables are then cached and the capture records kernels only
+            n = len(self.net.layers)
+            k = min(self.gather_split, n)
+            self.gather(0, k)
+            if k < n:
+                self.gather(k, n - k)
+            torch.cuda.synchronize()
+            l0 = self.ctx.launch_count()
         with torch.cuda.graph(self.graph):
             if self.world > 1:
                 # data parallel: the graph ends with the weight gradients; the collective and the update follow it eagerly
-                self.train_two_streams(lasso=False)
+                self.train_two_streams(lasso=False, gather=self._graph_has_gather)
             elif two_streams:
-                self.train_two_streams()
+                self.train_two_streams(gather=self._graph_has_gather)
             else:
                 self.train()
         self.graph_launches = self.ctx.launch_count() - l0
         return self.graph
 
     def step(self, stream=None, before_train=None):
-        self.reconfigure(stream)
+        if getattr(self, "graph", None) is not None and getattr(self, "_graph_has_gather", False):
+            self.reconfigure_plan(stream)                 # the gather is part of the graph (in two parts, beside the first layers)
+        else:
+            self.reconfigure(stream)
         if before_train is not None:
             torch.cuda.current_stream().wait_event(before_train)     # e.g. the image batch has reached the stem's input
         if getattr(self, "graph", None) is not None:
@@ -454,7 +512,7 @@ class TrainStep:
         self.x[0] = self._xbuf[cur]
         if getattr(self, "graph", None) is not None:
             if self._xgraph[cur] is None:
-                self.build_graph(self._graph_two)        # the launches that read this buffer
+                self.build_graph(self._graph_two, self._graph_has_gather)        # the launches that read this buffer
                 self._xgraph[cur] = self.graph
             self.graph = self._xgraph[cur]
         cs.wait_stream(main)                             # the previous step, the last reader of the other buffer, is done
