@@ -121,6 +121,17 @@ int32_t pt_conv_wgrad_ctas(const pt_ctx *ctx, const pt_conv_desc *d, int32_t *wa
 pt_status pt_conv_fwd(pt_ctx *ctx, const pt_conv_desc *d, const void *x, const void *w, void *y,
                       void *ws, size_t ws_bytes, void *stream);
 
+/* The same forward convolution (bf16 output, tcgen05 kernels only: PT_ERR_UNSUPPORTED otherwise) that also takes the
+ * statistics the batch normalisation after it needs (Sec. 2.1: the normalisation layers are bound by memory bandwidth because
+ * they read their input several times): every epilogue warp adds, per output channel, the sum and the sum of squares of the bf16
+ * values it stores -- from the tile that is still in shared memory -- into a row of its own. stats receives *n_parts (host, out)
+ * rows of [2][ldy] floats (row r: sums, then sums of squares; columns >= K are zero); pt_bn_relu_fwd_stats combines them in a
+ * fixed order. stats must hold pt_conv_fwd_stats_bytes(ctx, d) bytes (an upper bound that does not depend on which kernel
+ * serves the layer); PT_ERR_WORKSPACE if it is smaller than this launch needs. Run-to-run identical. */
+size_t pt_conv_fwd_stats_bytes(const pt_ctx *ctx, const pt_conv_desc *d);
+pt_status pt_conv_fwd_stats(pt_ctx *ctx, const pt_conv_desc *d, const void *x, const void *w, void *y, float *stats,
+                            size_t stats_bytes, int32_t *n_parts /*host*/, void *ws, size_t ws_bytes, void *stream);
+
 /* dx[n,h,w,c] = sum over (k,r,s,p,q) with p*stride-pad+r = h and q*stride-pad+s = w of dy[n,p,q,k] * w[k,r,s,c].
  * Back-propagation through the layer (Sec. 2.1). Pixels no tap reaches are written as 0.
  * dy: bf16 [N][P][Q][ldy]; dx: [N][H][W][ldx] bf16 or fp32. */
@@ -198,6 +209,13 @@ size_t pt_bn_workspace_bytes(const pt_ctx *ctx, const pt_bn_desc *d);
 pt_status pt_bn_relu_fwd(pt_ctx *ctx, const pt_bn_desc *d, const void *x, const void *residual, const float *gamma,
                          const float *beta, float *running_mean, float *running_var, float *save_mean, float *save_invstd,
                          void *y, void *ws, size_t ws_bytes, void *stream);
+
+/* The same forward pass without its reduction over x: the batch statistics come from the rows of partial sums the producing
+ * convolution left (pt_conv_fwd_stats: stats, n_parts; the sums are those of the stored bf16 values, exactly what the
+ * reduction pass of pt_bn_relu_fwd would read). Two launches instead of three, one pass over x instead of two; no workspace. */
+pt_status pt_bn_relu_fwd_stats(pt_ctx *ctx, const pt_bn_desc *d, const void *x, const void *residual, const float *gamma,
+                               const float *beta, float *running_mean, float *running_var, float *save_mean, float *save_invstd,
+                               void *y, const float *stats, int32_t n_parts, void *stream);
 
 /* Gradients of the call above. y is the forward output (only its sign is used, and only with relu = 1; may be NULL
  * otherwise); dresidual may be NULL when the block has no residual input. */

@@ -78,6 +78,11 @@ EXPORTS = {
     "pt_conv_wgrad_ctas": (c_int32, [c_void_p, POINTER(pt_conv_desc), POINTER(c_int32)]),
     "pt_conv_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_conv_desc), c_int32]),
     "pt_conv_fwd": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "pt_conv_fwd_stats_bytes": (c_size_t, [c_void_p, POINTER(pt_conv_desc)]),
+    "pt_conv_fwd_stats": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, POINTER(c_int32),
+                                    c_void_p, c_size_t, c_void_p]),
+    "pt_bn_relu_fwd_stats": (c_int32, [c_void_p, POINTER(pt_bn_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                       c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "pt_conv_dgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_conv_wgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_group_lasso_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_layer), c_int32]),
@@ -205,6 +210,26 @@ def _ws(ws):
 def pt_conv_fwd(ctx, d, x, w, y, ws=None, stream=None):
     p, n = _ws(ws)
     _check(lib().pt_conv_fwd(ctx.handle, byref(d), _ptr(x), _ptr(w), _ptr(y), p, n, _stream(stream)), "pt_conv_fwd")
+
+
+def pt_conv_fwd_stats_bytes(ctx, d) -> int:
+    return int(lib().pt_conv_fwd_stats_bytes(ctx.handle, byref(d)))
+
+
+def pt_conv_fwd_stats(ctx, d, x, w, y, stats, ws=None, stream=None) -> int:
+    """Returns the number of rows of partial sums the launch left in `stats`."""
+    p, n = _ws(ws)
+    parts = c_int32(0)
+    _check(lib().pt_conv_fwd_stats(ctx.handle, byref(d), _ptr(x), _ptr(w), _ptr(y), _ptr(stats), stats.numel() * stats.element_size(),
+                                   byref(parts), p, n, _stream(stream)), "pt_conv_fwd_stats")
+    return int(parts.value)
+
+
+def pt_bn_relu_fwd_stats(ctx, d, x, residual, gamma, beta, running_mean, running_var, save_mean, save_invstd, y, stats, n_parts,
+                         stream=None):
+    _check(lib().pt_bn_relu_fwd_stats(ctx.handle, byref(d), _ptr(x), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(running_mean),
+                                      _ptr(running_var), _ptr(save_mean), _ptr(save_invstd), _ptr(y), _ptr(stats), n_parts,
+                                      _stream(stream)), "pt_bn_relu_fwd_stats")
 
 
 def pt_conv_dgrad(ctx, d, dy, w, dx, ws=None, stream=None):

@@ -223,6 +223,27 @@ extern "C" pt_status pt_conv_fwd(pt_ctx *c, const pt_conv_desc *d, const void *x
     return conv_dispatch(c, d, PT_CONV_FWD, x, w, y, ws, ws_bytes, stream);
 }
 
+extern "C" size_t pt_conv_fwd_stats_bytes(const pt_ctx *c, const pt_conv_desc *d)
+{
+    int P, Q;
+    if (pt_conv_validate(c, d, &P, &Q) != PT_OK) return 0;
+    return (size_t)c->sm_count * 12 * 2 * (size_t)d->ldy * sizeof(float);      // at most twelve epilogue warps per SM
+}
+
+extern "C" pt_status pt_conv_fwd_stats(pt_ctx *c, const pt_conv_desc *d, const void *x, const void *w, void *y, float *stats,
+                                       size_t stats_bytes, int32_t *n_parts, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!c || !d || !stats || !n_parts) return PT_ERR_INVALID_ARG;
+    if (d->out_f32 || d->algo == 1) return PT_ERR_UNSUPPORTED;
+    pt_conv_desc dd = *d;
+    dd.algo = 2;                                    // the statistics come out of the tcgen05 kernels' epilogues only
+    c->stats_mode = 2; c->stats_out = stats; c->stats_cap = stats_bytes; c->stats_parts = 0;
+    const pt_status r = conv_dispatch(c, &dd, PT_CONV_FWD, x, w, y, ws, ws_bytes, stream);
+    c->stats_mode = 0; c->stats_out = nullptr; c->stats_cap = 0;
+    *n_parts = r == PT_OK ? c->stats_parts : 0;
+    return r;
+}
+
 extern "C" pt_status pt_conv_dgrad(pt_ctx *c, const pt_conv_desc *d, const void *dy, const void *w, void *dx,
                                    void *ws, size_t ws_bytes, void *stream)
 {

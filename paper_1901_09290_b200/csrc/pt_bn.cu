@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(1024) bn_fwd_finish_kernel(const BnP p, const 
     const double d = s0 / M;
     double var = s1 / M - d * d;
     if (var < 0.0) var = 0.0;
-    const double mean = (double)__bfloat162float(x[c]) + d;
+    const double mean = (x ? (double)__bfloat162float(x[c]) : 0.0) + d;     // sums about a pivot (the channel's first value) or about 0
     save_mean[c] = (float)mean;
     save_invstd[c] = (float)(1.0 / sqrt(var + (double)p.eps));
     if (running_mean && running_var) {
@@ -341,6 +341,30 @@ extern "C" pt_status pt_bn_relu_bwd(pt_ctx *c, const pt_bn_desc *d, const void *
     bn_apply_kernel<1><<<p.blocks, kBnThreads, 0, st>>>(p, (const uint4 *)x, yv, (const uint4 *)dy, gamma, nullptr, save_mean, save_invstd,
                                                         dgamma, dbeta, (uint4 *)dx, (uint4 *)dresidual);
     c->launches += 3;
+    PT_CUDA_OK(cudaGetLastError());
+    return PT_OK;
+}
+
+// The forward pass when the convolution that produced x already took the channel sums (pt_conv_fwd_stats): no reduction pass
+// over x, only the short finish over the convolution's rows of partial sums and the apply pass.
+extern "C" pt_status pt_bn_relu_fwd_stats(pt_ctx *c, const pt_bn_desc *d, const void *x, const void *residual, const float *gamma,
+                                          const float *beta, float *running_mean, float *running_var, float *save_mean,
+                                          float *save_invstd, void *y, const float *stats, int32_t n_parts, void *stream)
+{
+    BnP p;
+    pt_status r = bn_params(c, d, &p);
+    if (r != PT_OK) return r;
+    if (!x || !gamma || !beta || !save_mean || !save_invstd || !y || !stats || n_parts < 1 ||
+        (running_mean == nullptr) != (running_var == nullptr))
+        return PT_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y) || (residual && !aligned16(residual))) return PT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    BnP pf = p;
+    pf.blocks = n_parts;                            // rows of [2][ld] partial sums, taken about 0
+    bn_fwd_finish_kernel<<<pt_ceil_div(p.C, 32), 1024, 0, st>>>(pf, nullptr, stats, save_mean, save_invstd, running_mean, running_var);
+    bn_apply_kernel<0><<<p.blocks, kBnThreads, 0, st>>>(p, (const uint4 *)x, nullptr, (const uint4 *)residual, gamma, beta, save_mean,
+                                                        save_invstd, nullptr, nullptr, (uint4 *)y, nullptr);
+    c->launches += 2;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
 }

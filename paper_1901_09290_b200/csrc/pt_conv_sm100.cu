@@ -75,6 +75,8 @@ struct GemmP {
     int acc_per;        // two issuers: accumulator buffers per issuer (1 or 2)
     int alias_staging;  // 1: the CTA has a single tile; the epilogue's staging slabs lie in the (then idle) ring
     int test_skip;      // test hook (pt_test_skip_next_arrive): the A producer leaves out the first stage of its first tile
+    float *stats;       // optional: per (pixel tile, warp quarter) and output channel, sum and sum of squares of the bf16 values
+                        // stored, as [part][2][ld_out] floats (the batch-normalisation statistics of the layer that follows)
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // im2col offsets of each visited tap
@@ -101,6 +103,31 @@ struct __align__(8) PCtl {
 };
 
 constexpr uint32_t kSlabs = 2;                          // staging slabs per epilogue warp (TMA stores in flight)
+
+// Batch-normalisation statistics of a staged output chunk: `rows` is a bit mask of the warp's 32 staged rows (128 bytes each,
+// 128-byte swizzle, first row `row0` of the slab) that are real output pixels. Lane l owns channels 2l and 2l + 1 of the
+// 64-channel chunk and adds the bf16 values exactly as they were stored, rows in ascending order: sum and sum of squares, added
+// to dst[0][c] and dst[1][c] (dst rows ld apart) for the channels that exist. Feature normalisation (Sec. 2.1) reads its input
+// twice; taking the sums here, from the tile that is still in shared memory, removes the first of the two passes.
+__device__ __forceinline__ void chunk_stats(uint32_t slab, int row0, uint32_t rows, int lane, float *dst, int ld, int c0, int n_cols)
+{
+    float s0a = 0.f, s1a = 0.f, s0b = 0.f, s1b = 0.f;
+    const uint32_t jj = (uint32_t)lane >> 2, wi = ((uint32_t)lane & 3u) << 2;
+    while (rows) {
+        const int r = __ffs(rows) - 1;
+        rows &= rows - 1u;
+        const uint32_t m = (uint32_t)(row0 + r);
+        uint32_t word;
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(word) : "r"(slab + m * 128u + ((jj ^ (m & 7u)) << 4) + wi) : "memory");
+        const float a = __uint_as_float(word << 16), b = __uint_as_float(word & 0xffff0000u);
+        s0a += a; s1a = fmaf(a, a, s1a);
+        s0b += b; s1b = fmaf(b, b, s1b);
+    }
+    // the warp's own row of partial sums (zeroed by the warp at kernel start; a column is always this lane's): read, add, write
+    const int c = c0 + 2 * lane;
+    if (c < n_cols) { dst[c] += s0a; dst[ld + c] += s1a; }
+    if (c + 1 < n_cols) { dst[c + 1] += s0b; dst[ld + c + 1] += s1b; }
+}
 
 // Device-side timeline of CTA 0 (a build with -DPT_DEVICE_TRACE; read back with pt_debug_gemm_trace): per pipeline stage in
 // issue order, when the A producer found it free / issued it, when the MMA issuer found it full / committed it; per tile, when
@@ -304,6 +331,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         // i.e. the tiles tc = g, g + G, g + 2G, ... of this CTA
         const int quarter = warp & 3, group = (warp - 2) >> 2, G = p.epi_groups;
         const uint32_t slab0 = (p.alias_staging ? data_base : staging_base) + (uint32_t)(warp - 2) * (kSlabs * 4096u);
+        // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
+        float *my_stats = p.stats ? p.stats + ((size_t)blockIdx.x * (4 * G) + (warp - 2)) * 2 * p.ld_out : nullptr;
+        if (my_stats) {
+            for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
+            __syncwarp();
+        }
         int tc = group, sl = 0;
         bool ok = true;
         for (int tile = blockIdx.x + group * gridDim.x; tile < total_tiles && ok; tile += G * gridDim.x, tc += G) {
@@ -401,6 +434,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         if (m0 + quarter * 32 < p.M_total) tma_store_2d(&tmC, slab, n0 + ch * 64, m0 + quarter * 32);
                         tma_store_commit();
                     }
+                    if (p.stats) {
+                        const int left = p.M_total - (m0 + quarter * 32);
+                        const uint32_t rows = left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
+                        chunk_stats(slab, 0, rows, lane, my_stats, p.ld_out, n0 + ch * 64, p.n_cols);
+                    }
                 }
                 if (quarter == 0) GTRACE(7, tc);
                 continue;
@@ -482,6 +520,7 @@ struct HaloP {
     int b_slot, b_rows, staging;         // bytes reserved per weight tile, rows a K-major weight box brings, bytes of an epilogue group's staging slab
     int tmem_cols, tma_store, out_f32, ld_out;
     int oH, oW, o_step, o_h0, o_w0;      // direct stores: raster (n, i, j) -> out[((n*oH + i*o_step + o_h0)*oW + j*o_step + o_w0)*ld_out]
+    float *stats;                        // optional: per (tile, warp quarter) and channel, sum and sum of squares of the stored bf16
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];
@@ -768,6 +807,12 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         const int quarter = warp & 3, group = (warp - 2) >> 2;
         const int gtid = (warp - 2 - group * 4) * 32 + lane;         // 0..127 within the group
         const uint32_t slab = staging_base + (uint32_t)group * (uint32_t)p.staging;
+        // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
+        float *my_stats = p.stats ? p.stats + ((size_t)blockIdx.x * 8 + (warp - 2)) * 2 * p.ld_out : nullptr;
+        if (my_stats) {
+            for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
+            __syncwarp();
+        }
         bool ok = true;
         const int ni_shift = NI == 4 ? 2 : NI == 2 ? 1 : 0;   // NI is 1, 2 or 4
         TileWalk tw;
@@ -829,6 +874,12 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         tma_store_4d(&tmC, slab, n0 + ch * 64, 0, p0, img);
                         tma_store_commit();
                         HTRACE(7, tc);
+                    }
+                    if (p.stats) {
+                        // this thread's raster position is a real output pixel iff it lies inside the row and the image
+                        const int ri = m / p.Wp, rj = m - ri * p.Wp;
+                        const uint32_t rows = __ballot_sync(0xffffffffu, m < p.nr * p.Wp && rj < p.Q && p0 + ri < p.P);
+                        chunk_stats(slab, quarter * 32, rows, lane, my_stats, p.ld_out, n0 + ch * 64, p.n_cols);
                     }
                 }
                 continue;
@@ -1740,6 +1791,12 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
         attr_set[B_MN ? 1 : 0] = true;
     }
     const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
+    if (c->stats_mode) {
+        if (!p.tma_store) return PT_ERR_UNSUPPORTED;
+        c->stats_parts = grid * 4 * p.epi_groups;
+        if ((size_t)c->stats_parts * 2 * p.ld_out * sizeof(float) > c->stats_cap) return PT_ERR_WORKSPACE;
+        p.stats = c->stats_out;
+    }
     if (c->test_skip == 2) { p.test_skip = 1; c->test_skip = 0; }
     PT_CUDA_OK(launch_pdl(conv_gemm_kernel<B_MN>, dim3((unsigned)grid), dim3(kGemmThreads), smem, st, tmA, tmB, tmC, p));
     c->launches += 1;
@@ -1906,6 +1963,12 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     const int total_tiles = p.N * p.row_tiles * p.n_tiles;
     int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
     if (h.max_ctas > 0 && grid > h.max_ctas) grid = h.max_ctas;
+    if (c->stats_mode) {
+        if (!p.tma_store || B_MN) return PT_ERR_UNSUPPORTED;
+        c->stats_parts = grid * 8;
+        if ((size_t)c->stats_parts * 2 * p.ld_out * sizeof(float) > c->stats_cap) return PT_ERR_WORKSPACE;
+        p.stats = c->stats_out;
+    }
     PT_CUDA_OK(launch_pdl(conv_halo_kernel<B_MN>, dim3((unsigned)grid), dim3(kHaloThreads), smem, st, tmA, tmB, tmC, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());

@@ -55,6 +55,12 @@ struct pt_ctx {
     unsigned int sync_next = 0;         // ring position in d_sync
     uint64_t launches = 0;
     int wgrad_ctas = 0;                 // CTA limit of a weight-gradient launch (0 = all SMs)
+    // pt_conv_fwd_stats: non-zero while that call runs: the forward kernels also leave per-warp channel sums in stats_out
+    // (stats_cap bytes) and the launcher records how many rows of partial sums there are
+    int stats_mode = 0;
+    int stats_parts = 0;
+    float *stats_out = nullptr;
+    size_t stats_cap = 0;
     int test_skip = 0;                  // pt_test_skip_next_arrive: 1 = next split weight gradient, 2 = next fwd/dgrad GEMM-form launch
     // Helper streams for independent launches inside one call (the parity classes of a stride-2 data gradient): the caller's
     // stream forks to them and joins them back through events, which a stream capture records as graph edges.
