@@ -353,6 +353,46 @@ def bn_relu_bwd(x, y, dy, gamma, mean, invstd, relu: bool = True):
     return dx, dz, dgamma, dbeta
 
 
+# --------------------------------------------------------------------------- pooling (Sec. 2.1)
+def maxpool_fwd(x, R: int = 3, stride: int = 2, pad: int = 1):
+    """Max pooling of x [N][H][W][C] (Sec. 2.1 lists pooling among the layers of a CNN; ResNet pools once, after its first
+    convolution). y[n,p,q,c] = the maximum over the R x R window at (p*stride - pad, q*stride - pad); positions outside
+    the image are never selected; of equal maxima the first in scan order (window rows, then columns) is the selected one.
+    Returns y (fp64) and sel, the selected position h*W + w of every output element."""
+    x = np.asarray(x, np.float64)
+    N, H, W, C = x.shape
+    P, Q = out_dim(H, R, stride, pad), out_dim(W, R, stride, pad)
+    y = np.full((N, P, Q, C), -np.inf)
+    sel = np.full((N, P, Q, C), -1, np.int64)
+    for p in range(P):
+        for q in range(Q):
+            for r in range(R):
+                h = p * stride - pad + r
+                if h < 0 or h >= H:
+                    continue
+                for s in range(R):
+                    w = q * stride - pad + s
+                    if w < 0 or w >= W:
+                        continue
+                    v = x[:, h, w, :]
+                    better = (v > y[:, p, q, :]) | (sel[:, p, q, :] < 0)      # strictly greater: the first maximum stays
+                    y[:, p, q, :] = np.where(better, v, y[:, p, q, :])
+                    sel[:, p, q, :] = np.where(better, h * W + w, sel[:, p, q, :])
+    return y, sel
+
+
+def maxpool_bwd(dy, sel, H: int, W: int) -> np.ndarray:
+    """Back-propagation through the pooling: every output position hands its gradient to the input position it selected,
+    dx[n,h,w,c] = sum of dy[n,p,q,c] over the (p,q) with sel[n,p,q,c] == h*W + w."""
+    dy = np.asarray(dy, np.float64)
+    N, P, Q, C = dy.shape
+    dx = np.zeros((N, H * W, C))
+    for n in range(N):
+        for c in range(C):
+            np.add.at(dx[n, :, c], sel[n, :, :, c].ravel(), dy[n, :, :, c].ravel())
+    return dx.reshape(N, H, W, C)
+
+
 # --------------------------------------------------------------------------- channel gating (Sec. 4.2)
 def dense_channel_list(zero_flags) -> np.ndarray:
     """Ascending positions of the groups that are NOT sparsified: the "dense channel indices" a gating layer gathers

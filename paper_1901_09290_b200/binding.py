@@ -49,6 +49,10 @@ class pt_bn_desc(Structure):
                 ("eps", c_float), ("momentum", c_float), ("relu", c_int32)]
 
 
+class pt_pool_desc(Structure):
+    _fields_ = [(n, c_int32) for n in ("N", "H", "W", "C", "ld", "R", "stride", "pad")]
+
+
 class pt_layer_shape(Structure):
     _fields_ = [(n, c_int32) for n in ("H", "W", "C", "K", "R", "S", "stride", "pad")]
 
@@ -83,6 +87,8 @@ EXPORTS = {
                                     c_void_p, c_size_t, c_void_p]),
     "pt_bn_relu_fwd_stats": (c_int32, [c_void_p, POINTER(pt_bn_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
+    "pt_maxpool_fwd": (c_int32, [c_void_p, POINTER(pt_pool_desc), c_void_p, c_void_p, c_void_p]),
+    "pt_maxpool_bwd": (c_int32, [c_void_p, POINTER(pt_pool_desc), c_void_p, c_void_p, c_void_p, c_void_p]),
     "pt_conv_dgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_conv_wgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_group_lasso_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_layer), c_int32]),
@@ -334,6 +340,18 @@ def pt_bn_relu_bwd(ctx, d, x, y, dy, gamma, save_mean, save_invstd, dx, dresidua
     p, n = _ws(ws)
     _check(lib().pt_bn_relu_bwd(ctx.handle, byref(d), _ptr(x), _ptr(y), _ptr(dy), _ptr(gamma), _ptr(save_mean), _ptr(save_invstd),
                                 _ptr(dx), _ptr(dresidual), _ptr(dgamma), _ptr(dbeta), p, n, _stream(stream)), "pt_bn_relu_bwd")
+
+
+def make_pool_desc(N, H, W, C, ld=None, R=3, stride=2, pad=1) -> pt_pool_desc:
+    return pt_pool_desc(N, H, W, C, ld or (C + 7) // 8 * 8, R, stride, pad)
+
+
+def pt_maxpool_fwd(ctx, d, x, y, stream=None):
+    _check(lib().pt_maxpool_fwd(ctx.handle, byref(d), _ptr(x), _ptr(y), _stream(stream)), "pt_maxpool_fwd")
+
+
+def pt_maxpool_bwd(ctx, d, x, dy, dx, stream=None):
+    _check(lib().pt_maxpool_bwd(ctx.handle, byref(d), _ptr(x), _ptr(dy), _ptr(dx), _stream(stream)), "pt_maxpool_bwd")
 
 
 def shape_array(shapes) -> "ctypes.Array":

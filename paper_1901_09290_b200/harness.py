@@ -525,3 +525,196 @@ class TrainStep:
 
     def e2e_bytes(self):
         return self.h_image.numel() * self.h_image.element_size(), 8 + 4 * len(self.counts)
+
+
+class ChainedStep:
+    """A ResNet conv stack chained from the image to the last feature map through the C ABI: every convolution is followed
+    by batch normalisation (training statistics) and ReLU, blocks end with the residual add, the stem is followed by the
+    3x3 / stride-2 max pooling where the shape table halves there, and the backward pass runs the whole chain in reverse
+    down to every weight gradient; the group-lasso SGD step closes the iteration. With `fused_stats` the convolutions take
+    the normalisation statistics in their epilogues (pt_conv_fwd_stats + pt_bn_relu_fwd_stats: one pass over each
+    convolution output instead of two). The classifier is not part of the library: the gradient with respect to the last
+    feature map is a seeded input. Marshalling only: every tensor operation is an ABI call.
+
+    Block structure is read from the layer names: "stem", then "<block>.c1", "<block>.c2", ... and an optional "<block>.ds"
+    (projection shortcut) per block, in order."""
+
+    def __init__(self, ctx: B.Context, net: W.Net, N: int, seed: int, fused_stats: bool = True, algo: int = 0,
+                 max_blocks: Optional[int] = None, model: Optional[W.Model] = None, x0: Optional[torch.Tensor] = None,
+                 g_last: Optional[torch.Tensor] = None):
+        self.ctx, self.net, self.N, self.fused = ctx, net, N, fused_stats
+        names = [l.name for l in net.layers]
+        self.blocks = []                                   # (main conv indices, shortcut index or None)
+        for i, nm in enumerate(names):
+            if nm == "stem" or nm.endswith(".ds"):
+                continue
+            pre = nm.rsplit(".", 1)[0]
+            if not self.blocks or self.blocks[-1][2] != pre:
+                ds = names.index(pre + ".ds") if pre + ".ds" in names else None
+                self.blocks.append(([], ds, pre))
+            self.blocks[-1][0].append(i)
+        if max_blocks is not None:
+            self.blocks = self.blocks[:max_blocks]
+        self.used = [0] + [i for b in self.blocks for i in b[0]] + [b[1] for b in self.blocks if b[1] is not None]
+        self.model = model if model is not None else W.gen_model(net, seed)
+        self.dm = DeviceModel(ctx, self.model)
+        L = net.layers
+        self.ld = {i: W.pad16(L[i].K) for i in self.used}          # pitch of a layer's outputs
+        l0 = L[0]
+        self.ld_img = 8 if l0.C <= 4 else W.pad16(l0.C)
+        dev = "cuda"
+        bf = lambda n, h, ld: torch.zeros((n, h, h, ld), dtype=torch.bfloat16, device=dev)
+        if x0 is None:
+            x0 = W.gen_image(N, l0.H, l0.H, l0.C, seed + 11)
+        self.x0 = torch.zeros((N, l0.H, l0.H, self.ld_img), dtype=torch.bfloat16, device=dev)
+        self.x0[..., :l0.C] = x0.to(torch.bfloat16).cuda()
+        first_h = L[self.blocks[0][0][0]].H if self.blocks else l0.P
+        self.pool = l0.P != first_h
+        if self.pool:
+            self.pool_desc = B.make_pool_desc(N, l0.P, l0.P, l0.K, self.ld[0], 3, 2, 1)
+            assert (l0.P + 2 - 3) // 2 + 1 == first_h
+        self.desc, self.bn_desc, self.y, self.a, self.dy, self.gamma, self.beta, self.sm, self.si, self.dg, self.db = ({} for _ in range(11))
+        ws_conv, ws_bn, st_bytes = 16, 16, 16
+        gen = torch.Generator().manual_seed(seed + 12)
+        for i in self.used:
+            l = L[i]
+            ldx = self.ld_img if i == 0 else W.pad16(l.C)
+            self.desc[i] = B.make_conv_desc(N, l.H, l.H, l.C, l.K, l.R, l.R, l.stride, l.pad, ldx, self.ld[i], W.pad8(l.C), 0, algo)
+            self.bn_desc[i] = None
+            self.y[i] = bf(N, l.P, self.ld[i])             # convolution output
+            self.a[i] = bf(N, l.P, self.ld[i])             # after normalisation (+ residual) (+ ReLU)
+            self.dy[i] = bf(N, l.P, self.ld[i])            # gradient with respect to the convolution output
+            self.gamma[i] = (torch.rand(l.K, generator=gen) + 0.5).cuda()
+            self.beta[i] = (torch.rand(l.K, generator=gen) - 0.5).cuda()
+            self.sm[i], self.si[i] = torch.empty(l.K, device=dev), torch.empty(l.K, device=dev)
+            self.dg[i], self.db[i] = torch.empty(l.K, device=dev), torch.empty(l.K, device=dev)
+            for which in range(3):
+                ws_conv = max(ws_conv, B.pt_conv_workspace_bytes(ctx, self.desc[i], which))
+            st_bytes = max(st_bytes, B.pt_conv_fwd_stats_bytes(ctx, self.desc[i]))
+        ds_set = {b[1] for b in self.blocks if b[1] is not None}
+        last_of = {b[0][-1] for b in self.blocks}
+        for i in self.used:
+            l = L[i]
+            relu = i not in ds_set                         # the projection shortcut is normalised but not rectified
+            self.bn_desc[i] = B.make_bn_desc(N, l.P, l.P, l.K, self.ld[i], 1e-5, 0.1, relu)
+            ws_bn = max(ws_bn, B.pt_bn_workspace_bytes(ctx, self.bn_desc[i]))
+        self.last_of = last_of
+        self.ws = torch.empty(ws_conv, dtype=torch.uint8, device=dev)
+        self.ws_bn = torch.empty(ws_bn, dtype=torch.uint8, device=dev)
+        self.stats = torch.empty(st_bytes // 4, dtype=torch.float32, device=dev)
+        if self.pool:
+            self.pooled = bf(N, first_h, self.ld[0])
+            self.d_pooled = bf(N, first_h, self.ld[0])
+        # gradients with respect to activations: one buffer per distinct activation a convolution reads
+        # gradient with respect to a convolution's INPUT (its data gradient), and with respect to the stem's activation
+        self.da = {i: bf(N, L[i].H, W.pad16(L[i].C)) for i in self.used if i != 0}
+        self.d_a0 = bf(N, l0.P, self.ld[0])
+        self.da_tmp = {}
+        self.dres = {}
+        for main, ds, _ in self.blocks:
+            lo = L[main[-1]]
+            self.dres[main[-1]] = bf(N, lo.P, self.ld[main[-1]])             # gradient handed to the residual branch
+        out_i = self.blocks[-1][0][-1] if self.blocks else 0
+        lo = L[out_i]
+        if g_last is None:
+            g_last = W.gen_dy(N, lo.P, lo.P, lo.K, seed + 13) * 64.0
+        self.g_last = torch.zeros((N, lo.P, lo.P, self.ld[out_i]), dtype=torch.bfloat16, device=dev)
+        self.g_last[..., :lo.K] = g_last.to(torch.bfloat16).cuda()
+        self.out_index = out_i
+        self._idx = {}
+
+    # ---- helpers
+    def _arange(self, n):
+        if n not in self._idx:
+            self._idx[n] = torch.arange(n, dtype=torch.int32, device="cuda")
+        return self._idx[n]
+
+    def _add(self, a, b, out, C, ld, npix, stream=None):
+        """out = a + b (bf16, one rounding) through the scatter-add with the identity selection."""
+        B.pt_channel_scatter_add(self.ctx, b, ld, self._arange(C), C, a, out, ld, C, npix, False, stream)
+
+    def _conv_bn(self, i, x, residual=None, stream=None):
+        c = self.ctx
+        if self.fused:
+            n_parts = B.pt_conv_fwd_stats(c, self.desc[i], x, self.dm.wb[i], self.y[i], self.stats, self.ws, stream)
+            B.pt_bn_relu_fwd_stats(c, self.bn_desc[i], self.y[i], residual, self.gamma[i], self.beta[i], None, None, self.sm[i], self.si[i],
+                                   self.a[i], self.stats, n_parts, stream)
+        else:
+            B.pt_conv_fwd(c, self.desc[i], x, self.dm.wb[i], self.y[i], self.ws, stream)
+            B.pt_bn_relu_fwd(c, self.bn_desc[i], self.y[i], residual, self.gamma[i], self.beta[i], None, None, self.sm[i], self.si[i],
+                             self.a[i], self.ws_bn, stream)
+        return self.a[i]
+
+    # ---- the chain
+    def forward(self, stream=None):
+        cur = self._conv_bn(0, self.x0, None, stream)
+        if self.pool:
+            B.pt_maxpool_fwd(self.ctx, self.pool_desc, cur, self.pooled, stream)
+            cur = self.pooled
+        self.block_in = []
+        for main, ds, _ in self.blocks:
+            self.block_in.append(cur)
+            res = self._conv_bn(ds, cur, None, stream) if ds is not None else cur
+            t = cur
+            for i in main[:-1]:
+                t = self._conv_bn(i, t, None, stream)
+            cur = self._conv_bn(main[-1], t, res, stream)
+        return cur
+
+    def _bn_bwd(self, i, d_out, dres, stream=None):
+        B.pt_bn_relu_bwd(self.ctx, self.bn_desc[i], self.y[i], self.a[i], d_out, self.gamma[i], self.sm[i], self.si[i], self.dy[i], dres,
+                         self.dg[i], self.db[i], self.ws_bn, stream)
+
+    def backward(self, stream=None):
+        c, L = self.ctx, self.net.layers
+        d_cur = self.g_last                                   # gradient w.r.t. the current block's output
+        for bi in range(len(self.blocks) - 1, -1, -1):
+            main, ds, _ = self.blocks[bi]
+            x_in = self.block_in[bi]
+            last = main[-1]
+            self._bn_bwd(last, d_cur, self.dres[last], stream)
+            d_t = None
+            for k in range(len(main) - 1, -1, -1):
+                i = main[k]
+                x_i = x_in if k == 0 else self.a[main[k - 1]]
+                if k < len(main) - 1:
+                    self._bn_bwd(i, d_t, None, stream)
+                B.pt_conv_wgrad(c, self.desc[i], x_i, self.dy[i], self.dm.g[i], self.ws, stream)
+                d_t = self.da[i]
+                B.pt_conv_dgrad(c, self.desc[i], self.dy[i], self.dm.wb[i], d_t, self.ws, stream)
+            # d_t: gradient w.r.t. the block input through the main branch; the shortcut adds its own
+            li = L[main[0]]
+            npix, Cin, ld_in = self.N * li.H * li.H, li.C, W.pad16(li.C)
+            if ds is not None:
+                self._bn_bwd(ds, self.dres[last], None, stream)
+                B.pt_conv_wgrad(c, self.desc[ds], x_in, self.dy[ds], self.dm.g[ds], self.ws, stream)
+                B.pt_conv_dgrad(c, self.desc[ds], self.dy[ds], self.dm.wb[ds], self.da[ds], self.ws, stream)
+                sc = self.da[ds]
+            else:
+                sc = self.dres[last]
+            key = ("sum", bi)
+            if key not in self.da_tmp:
+                self.da_tmp[key] = torch.zeros_like(d_t)
+            self._add(d_t, sc, self.da_tmp[key], Cin, ld_in, npix, stream)
+            d_cur = self.da_tmp[key]
+        if self.pool:
+            B.pt_maxpool_bwd(c, self.pool_desc, self.a[0], d_cur, self.d_a0, stream)
+            d_cur = self.d_a0
+        self._bn_bwd(0, d_cur, None, stream)
+        B.pt_conv_wgrad(c, self.desc[0], self.x0, self.dy[0], self.dm.g[0], self.ws, stream)
+
+    def update(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
+        B.pt_group_lasso_sgd_step(self.ctx, self.dm.arr, lam, lr, mu, 0.0, self.dm.reg, self.dm.ws, stream)
+
+    def step(self, stream=None):
+        self.forward(stream)
+        self.backward(stream)
+        self.update(stream)
+
+    def conv_flops(self) -> int:
+        f = 0
+        for i in self.used:
+            l = self.net.layers[i]
+            fl = 2 * self.N * l.P * l.P * l.K * l.C * l.R * l.R
+            f += (2 if i == 0 else 3) * fl
+        return f

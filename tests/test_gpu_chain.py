@@ -147,3 +147,128 @@ def test_chained_bottleneck_block_forward_and_backward():
     for bn, dg, db, nm in ((b3, dg3, db3, "bn3"), (bs, dgs, dbs, "bn_ds"), (b2, dg2, db2, "bn2"), (b1, dg1, db1, "bn1")):
         assert _rel(bn.dg.cpu().numpy().astype(np.float64), dg) < 2e-2, nm
         assert _rel(bn.db.cpu().numpy().astype(np.float64), db) < 2e-2, nm
+
+
+# ------------------------------------------------------------------------------------------ a whole chained stage
+def _oracle_chain(cs, model, x0, g_last):
+    """The composition ChainedStep runs, written with the oracle's functions; bf16 storage rounding where the CUDA path
+    stores bf16 (convolution outputs, activations, activation gradients). Returns the block output and the gradients.
+
+    The forward pass is the oracle's own chain from the image (compared at the stage's output). The backward pass is then
+    evaluated on the forward state the CUDA path stored (its convolution outputs, activations, batch statistics and pooled
+    map, copied back): a ReLU or pooling decision is a comparison of stored values, and two forward chains that differ by
+    rounding take it differently at a few near-zero elements, each of which changes the gradient by a whole term. Fed the
+    same stored bits, both sides take every decision alike and what remains is the arithmetic of the backward chain."""
+    L = cs.net.layers
+    gam = {i: cs.gamma[i].cpu().numpy().astype(np.float64) for i in cs.used}
+    bet = {i: cs.beta[i].cpu().numpy().astype(np.float64) for i in cs.used}
+    w = {i: W.bf16_round(model.w[i]).numpy() for i in cs.used}
+    ds_set = {b[1] for b in cs.blocks if b[1] is not None}
+    y, a, st = {}, {}, {}
+
+    def conv_bn(i, x, res=None):
+        l = L[i]
+        y[i] = _r(oracle.conv_fwd(x.astype(np.float32), w[i], l.stride, l.pad))
+        out, mean, invstd, _ = oracle.bn_relu_fwd(y[i], gam[i], bet[i], 1e-5, res, i not in ds_set)
+        a[i] = _r(out)
+        st[i] = (mean.astype(np.float32).astype(np.float64), invstd.astype(np.float32).astype(np.float64))
+        return a[i]
+
+    cur = conv_bn(0, x0)
+    sel = None
+    if cs.pool:
+        pooled, sel = oracle.maxpool_fwd(cur, 3, 2, 1)
+        cur = _r(pooled)
+    block_in = []
+    for main, ds, _ in cs.blocks:
+        block_in.append(cur)
+        res = conv_bn(ds, cur) if ds is not None else cur
+        t = cur
+        for i in main[:-1]:
+            t = conv_bn(i, t)
+        cur = conv_bn(main[-1], t, res)
+    out = cur
+    dw, dgm, dbt = {}, {}, {}
+    # the stored forward state of the CUDA path
+    g64 = lambda t, C: t.float().cpu().numpy()[..., :C].astype(np.float64)
+    for i in cs.used:
+        y[i], a[i] = g64(cs.y[i], L[i].K), g64(cs.a[i], L[i].K)
+        st[i] = (cs.sm[i].cpu().numpy().astype(np.float64), cs.si[i].cpu().numpy().astype(np.float64))
+    if cs.pool:
+        _, sel = oracle.maxpool_fwd(a[0], 3, 2, 1)
+    block_in = [g64(t, L[b[0][0]].C) for t, b in zip(cs.block_in, cs.blocks)]
+
+    def bn_bwd(i, d_out):
+        dx, dres, dg, db = oracle.bn_relu_bwd(y[i], a[i], d_out, gam[i], st[i][0], st[i][1], i not in ds_set)
+        dgm[i], dbt[i] = dg, db
+        return _r(dx), _r(dres)
+
+    d_cur = g_last
+    for bi in range(len(cs.blocks) - 1, -1, -1):
+        main, ds, _ = cs.blocks[bi]
+        x_in = block_in[bi]
+        dyl, dres = bn_bwd(main[-1], d_cur)
+        d_t = None
+        for k in range(len(main) - 1, -1, -1):
+            i, l = main[k], L[main[k]]
+            x_i = x_in if k == 0 else a[main[k - 1]]
+            if k < len(main) - 1:
+                dyl, _ = bn_bwd(i, d_t)
+            dw[i] = oracle.conv_wgrad(x_i.astype(np.float32), dyl.astype(np.float32), l.R, l.R, l.stride, l.pad)
+            d_t = _r(oracle.conv_dgrad(dyl.astype(np.float32), w[i], l.H, l.H, l.stride, l.pad))
+        if ds is not None:
+            l = L[ds]
+            dys, _ = bn_bwd(ds, dres)
+            dw[ds] = oracle.conv_wgrad(x_in.astype(np.float32), dys.astype(np.float32), l.R, l.R, l.stride, l.pad)
+            sc = _r(oracle.conv_dgrad(dys.astype(np.float32), w[ds], l.H, l.H, l.stride, l.pad))
+        else:
+            sc = dres
+        d_cur = _r(d_t + sc)
+    if cs.pool:
+        d_cur = _r(oracle.maxpool_bwd(d_cur, sel, L[0].P, L[0].P))
+    dy0, _ = bn_bwd(0, d_cur)
+    l0 = L[0]
+    dw[0] = oracle.conv_wgrad(x0.astype(np.float32), dy0.astype(np.float32), l0.R, l0.R, l0.stride, l0.pad)
+    return out, dw, dgm, dbt
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_chained_stage_stem_pool_and_three_blocks(fused):
+    """Stem, max pooling and the whole first stage of a pruned ResNet-50 (a projection-shortcut block and two identity blocks),
+    forward and backward, through the chained step -- with the normalisation statistics taken in the convolution epilogues
+    and with the stand-alone normalisation -- against the oracle's composition."""
+    from paper_1901_09290_b200 import harness
+    c = Hh.ctx()
+    N = 4
+    dense = W.resnet50(64)                                   # 64x64 images: stem 32x32, pooled 16x16
+    seed = W.BASE_SEED + 4200
+    net = W.with_sizes(dense, W.random_keep(dense, seed, 0.3, 0.6))
+    model = W.gen_model(net, seed)
+    l0 = net.layers[0]
+    x0 = _r(W.gen_image(N, l0.H, l0.H, l0.C, seed + 1).numpy())
+    cs = harness.ChainedStep(c, net, N, seed, fused_stats=fused, algo=2, max_blocks=3, model=model,
+                             x0=torch.from_numpy(x0.astype(np.float32)))
+    lo = net.layers[cs.out_index]
+    g_last = _r(W.gen_dy(N, lo.P, lo.P, lo.K, seed + 2).numpy() * 64)
+    cs.g_last.zero_()
+    cs.g_last[..., :lo.K] = torch.from_numpy(g_last.astype(np.float32)).to(torch.bfloat16).cuda()
+    out_d = cs.forward()
+    cs.backward()
+    torch.cuda.synchronize()
+    c.poll()
+    out, dw, dgm, dbt = _oracle_chain(cs, model, x0, g_last)
+    f = lambda t, C: t.float().cpu().numpy()[..., :C].astype(np.float64)
+    assert _rel(f(out_d, lo.K), out) < 1e-2
+    # the backward chain on identical forward state: rounding of the stored gradients compounds along the eleven layers
+    order = [i for b in reversed(cs.blocks) for i in ([b[1]] if b[1] is not None else []) + list(reversed(b[0]))] + [0]
+    for rank, i in enumerate(order):
+        tol = 5e-3 + 1e-3 * rank
+        nm = net.layers[i].name
+        assert _rel(cs.dm.g[i].cpu().numpy().astype(np.float64), dw[i]) < tol, (nm, _rel(cs.dm.g[i].cpu().numpy().astype(np.float64), dw[i]))
+        assert _rel(cs.dg[i].cpu().numpy().astype(np.float64), dgm[i]) < tol, nm
+        # the stem's dbeta sums 4096 signed terms that nearly cancel: its error is measured against a small number
+        assert _rel(cs.db[i].cpu().numpy().astype(np.float64), dbt[i]) < (tol if i else 8e-2), nm
+    # the lasso step still closes the iteration
+    cs.update()
+    torch.cuda.synchronize()
+    c.poll()
