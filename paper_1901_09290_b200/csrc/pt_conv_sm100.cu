@@ -75,6 +75,7 @@ struct GemmP {
     int acc_per;        // two issuers: accumulator buffers per issuer (1 or 2)
     int alias_staging;  // 1: the CTA has a single tile; the epilogue's staging slabs lie in the (then idle) ring
     int test_skip;      // test hook (pt_test_skip_next_arrive): the A producer leaves out the first stage of its first tile
+    int stats_off;      // byte offset in shared memory of the epilogue warps' statistics accumulators (stats != nullptr)
     float *stats;       // optional: per (pixel tile, warp quarter) and output channel, sum and sum of squares of the bf16 values
                         // stored, as [part][2][ld_out] floats (the batch-normalisation statistics of the layer that follows)
     void *out;
@@ -106,27 +107,78 @@ constexpr uint32_t kSlabs = 2;                          // staging slabs per epi
 
 // Batch-normalisation statistics of a staged output chunk: `rows` is a bit mask of the warp's 32 staged rows (128 bytes each,
 // 128-byte swizzle, first row `row0` of the slab) that are real output pixels. Lane l owns channels 2l and 2l + 1 of the
-// 64-channel chunk and adds the bf16 values exactly as they were stored, rows in ascending order: sum and sum of squares, added
-// to dst[0][c] and dst[1][c] (dst rows ld apart) for the channels that exist. Feature normalisation (Sec. 2.1) reads its input
-// twice; taking the sums here, from the tile that is still in shared memory, removes the first of the two passes.
-__device__ __forceinline__ void chunk_stats(uint32_t slab, int row0, uint32_t rows, int lane, float *dst, int ld, int c0, int n_cols)
+// 64-channel chunk and adds the bf16 values exactly as they were stored, rows in ascending order: sum and sum of squares,
+// accumulated in the warp's own shared-memory slots (acc: 128 floats per chunk of the tile, four per lane) and written to the
+// warp's row of partial sums by stats_flush. Feature normalisation (Sec. 2.1) reads its input twice; taking the sums here,
+// from the tile that is still in shared memory, removes the first of the two passes.
+constexpr uint32_t kStatsWarpBytes = 4u * 128u * 4u;          // four chunks x 32 lanes x (sum, sum of squares) x two channels
+
+__device__ __forceinline__ void chunk_stats(uint32_t slab, int row0, uint32_t rows, int lane, uint32_t acc)
 {
     float s0a = 0.f, s1a = 0.f, s0b = 0.f, s1b = 0.f;
     const uint32_t jj = (uint32_t)lane >> 2, wi = ((uint32_t)lane & 3u) << 2;
-    while (rows) {
-        const int r = __ffs(rows) - 1;
-        rows &= rows - 1u;
-        const uint32_t m = (uint32_t)(row0 + r);
-        uint32_t word;
-        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(word) : "r"(slab + m * 128u + ((jj ^ (m & 7u)) << 4) + wi) : "memory");
-        const float a = __uint_as_float(word << 16), b = __uint_as_float(word & 0xffff0000u);
-        s0a += a; s1a = fmaf(a, a, s1a);
-        s0b += b; s1b = fmaf(b, b, s1b);
+    if (rows == 0xffffffffu) {
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+            const uint32_t m = (uint32_t)(row0 + r);
+            uint32_t word;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(word) : "r"(slab + m * 128u + ((jj ^ (m & 7u)) << 4) + wi) : "memory");
+            const float a = __uint_as_float(word << 16), b = __uint_as_float(word & 0xffff0000u);
+            s0a += a; s1a = fmaf(a, a, s1a);
+            s0b += b; s1b = fmaf(b, b, s1b);
+        }
+    } else {
+        while (rows) {
+            const int r = __ffs(rows) - 1;
+            rows &= rows - 1u;
+            const uint32_t m = (uint32_t)(row0 + r);
+            uint32_t word;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(word) : "r"(slab + m * 128u + ((jj ^ (m & 7u)) << 4) + wi) : "memory");
+            const float a = __uint_as_float(word << 16), b = __uint_as_float(word & 0xffff0000u);
+            s0a += a; s1a = fmaf(a, a, s1a);
+            s0b += b; s1b = fmaf(b, b, s1b);
+        }
     }
-    // the warp's own row of partial sums (zeroed by the warp at kernel start; a column is always this lane's): read, add, write
-    const int c = c0 + 2 * lane;
-    if (c < n_cols) { dst[c] += s0a; dst[ld + c] += s1a; }
-    if (c + 1 < n_cols) { dst[c + 1] += s0b; dst[ld + c + 1] += s1b; }
+    float4 t;
+    const uint32_t slot = acc + (uint32_t)lane * 16u;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "r"(slot) : "memory");
+    t.x += s0a; t.y += s1a; t.z += s0b; t.w += s1b;
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(slot), "f"(t.x), "f"(t.y), "f"(t.z), "f"(t.w) : "memory");
+}
+
+__device__ __forceinline__ void stats_clear(uint32_t acc0, int lane)
+{
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch)
+        asm volatile("st.shared.v4.f32 [%0], {%1, %1, %1, %1};" ::"r"(acc0 + (uint32_t)ch * 512u + (uint32_t)lane * 16u), "f"(0.f) : "memory");
+}
+
+// Adds the warp's shared-memory sums of the channels n0 .. n0 + 64 * n_chunks into its row of partial sums (zeroed by the warp
+// at kernel start; a column is always this lane's: read, add, write) and clears them.
+__device__ __forceinline__ void stats_flush(uint32_t acc0, int lane, float *dst, int ld, int n0, int n_chunks, int n_cols, bool add)
+{
+    float4 t[4];
+    float o[4][4];
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
+        if (ch >= n_chunks) break;
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t[ch].x), "=f"(t[ch].y), "=f"(t[ch].z), "=f"(t[ch].w)
+                     : "r"(acc0 + (uint32_t)ch * 512u + (uint32_t)lane * 16u) : "memory");
+        const int c = n0 + ch * 64 + 2 * lane;
+        // (a warp that visits its columns once, at the very end, has nothing to add to: the row still holds its zeros)
+        o[ch][0] = (add && c < n_cols) ? dst[c] : 0.f;
+        o[ch][1] = (add && c < n_cols) ? dst[ld + c] : 0.f;
+        o[ch][2] = (add && c + 1 < n_cols) ? dst[c + 1] : 0.f;
+        o[ch][3] = (add && c + 1 < n_cols) ? dst[ld + c + 1] : 0.f;
+    }
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
+        if (ch >= n_chunks) break;
+        const int c = n0 + ch * 64 + 2 * lane;
+        if (c < n_cols) { dst[c] = o[ch][0] + t[ch].x; dst[ld + c] = o[ch][1] + t[ch].y; }
+        if (c + 1 < n_cols) { dst[c + 1] = o[ch][2] + t[ch].z; dst[ld + c + 1] = o[ch][3] + t[ch].w; }
+    }
+    stats_clear(acc0, lane);
 }
 
 // Device-side timeline of CTA 0 (a build with -DPT_DEVICE_TRACE; read back with pt_debug_gemm_trace): per pipeline stage in
@@ -333,8 +385,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         const uint32_t slab0 = (p.alias_staging ? data_base : staging_base) + (uint32_t)(warp - 2) * (kSlabs * 4096u);
         // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
         float *my_stats = p.stats ? p.stats + ((size_t)blockIdx.x * (4 * G) + (warp - 2)) * 2 * p.ld_out : nullptr;
+        const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * kStatsWarpBytes;
         if (my_stats) {
             for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
+            stats_clear(st_acc, lane);
             __syncwarp();
         }
         int tc = group, sl = 0;
@@ -437,9 +491,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     if (p.stats) {
                         const int left = p.M_total - (m0 + quarter * 32);
                         const uint32_t rows = left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
-                        chunk_stats(slab, 0, rows, lane, my_stats, p.ld_out, n0 + ch * 64, p.n_cols);
+                        chunk_stats(slab, 0, rows, lane, st_acc + (uint32_t)ch * 512u);
                     }
                 }
+                // several channel tiles: the sums of this tile's columns leave shared memory now; one tile: after the last tile
+                if (my_stats && p.n_tiles > 1) stats_flush(st_acc, lane, my_stats, p.ld_out, n0, n_chunks, p.n_cols, true);
                 if (quarter == 0) GTRACE(7, tc);
                 continue;
             }
@@ -488,6 +544,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                 }
             }
         }
+        if (my_stats && p.n_tiles == 1) stats_flush(st_acc, lane, my_stats, p.ld_out, 0, (p.BN + 63) / 64, p.n_cols, false);
         if (p.tma_store && lane == 0) tma_store_wait_read();     // the staging slabs must outlive the stores' reads
         tc_fence_before();
     }
@@ -520,7 +577,8 @@ struct HaloP {
     int b_slot, b_rows, staging;         // bytes reserved per weight tile, rows a K-major weight box brings, bytes of an epilogue group's staging slab
     int tmem_cols, tma_store, out_f32, ld_out;
     int oH, oW, o_step, o_h0, o_w0;      // direct stores: raster (n, i, j) -> out[((n*oH + i*o_step + o_h0)*oW + j*o_step + o_w0)*ld_out]
-    float *stats;                        // optional: per (tile, warp quarter) and channel, sum and sum of squares of the stored bf16
+    int stats_off;                       // byte offset in shared memory of the epilogue warps' statistics accumulators
+    float *stats;                        // optional: per epilogue warp and channel, sum and sum of squares of the stored bf16
     void *out;
     unsigned int *status;
     unsigned char tap_oh[kMaxTaps], tap_ow[kMaxTaps];
@@ -809,8 +867,10 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         const uint32_t slab = staging_base + (uint32_t)group * (uint32_t)p.staging;
         // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
         float *my_stats = p.stats ? p.stats + ((size_t)blockIdx.x * 8 + (warp - 2)) * 2 * p.ld_out : nullptr;
+        const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * kStatsWarpBytes;
         if (my_stats) {
             for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
+            stats_clear(st_acc, lane);
             __syncwarp();
         }
         bool ok = true;
@@ -879,9 +939,10 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         // this thread's raster position is a real output pixel iff it lies inside the row and the image
                         const int ri = m / p.Wp, rj = m - ri * p.Wp;
                         const uint32_t rows = __ballot_sync(0xffffffffu, m < p.nr * p.Wp && rj < p.Q && p0 + ri < p.P);
-                        chunk_stats(slab, quarter * 32, rows, lane, my_stats, p.ld_out, n0 + ch * 64, p.n_cols);
+                        chunk_stats(slab, quarter * 32, rows, lane, st_acc + (uint32_t)ch * 512u);
                     }
                 }
+                if (my_stats && p.n_tiles > 1) stats_flush(st_acc, lane, my_stats, p.ld_out, n0, n_chunks, p.n_cols, true);
                 continue;
             }
             // ---- direct stores (fp32 outputs)
@@ -909,6 +970,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                 }
             }
         }
+        if (my_stats && p.n_tiles == 1) stats_flush(st_acc, lane, my_stats, p.ld_out, 0, (p.BN + 63) / 64, p.n_cols, false);
         if (p.tma_store && gtid == 0) tma_store_wait_read();
         tc_fence_before();
     }
@@ -1769,17 +1831,20 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     // one tile per CTA and streamed weights: the output is staged in the ring (all of its stages have been consumed when the
     // accumulator is complete), which leaves room for one more stage
     p.alias_staging = (per_cta == 1 && !p.resident) ? 1 : 0;
+    // statistics mode: the epilogue warps' accumulators sit at the end of the shared memory (taken from the ring's room)
+    const size_t st_smem = c->stats_mode ? (size_t)12 * kStatsWarpBytes : 0;
     size_t staging2 = p.alias_staging ? 0 : (size_t)p.epi_groups * 4 * kSlabs * 4096;
-    if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all, &smem);
+    if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all + st_smem, &smem);
     else {
-        p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2, &smem);
+        p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2 + st_smem, &smem);
         if (p.stages < 4 && p.epi_groups == 3 && p.taps * p.k_chunks * per_cta >= 4) {
             // a third epilogue group costs 32 KB of staging: with wide weight tiles that is the fourth pipeline stage
             p.epi_groups = 2;
             staging2 = (size_t)p.epi_groups * 4 * kSlabs * 4096;
-            p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2, &smem);
+            p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2 + st_smem, &smem);
         }
     }
+    p.stats_off = (int)(smem - st_smem);
     if (p.n_issuers == 2) {
         p.stages = p.stages / 2 * 2;
         if (p.stages < 2) { p.n_issuers = 1; p.acc_per = 1; p.stages = 2; }
@@ -1873,7 +1938,8 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     p.b_slot = (int)b_bytes;
     // epilogue staging: one slab of the tile's raster rows x 128 bytes per group (direct-store launches use none)
     p.staging = d->out_f32 ? 0 : (int)pt_align_up((size_t)(p.nr * Wp < 128 ? p.nr * Wp : 128) * 128, 1024);
-    const size_t budget = 227 * 1024 - 2048 - 2 * (size_t)p.staging - a_tail;
+    const size_t st_smem = c->stats_mode ? (size_t)8 * kStatsWarpBytes : 0;     // statistics accumulators of the eight epilogue warps
+    const size_t budget = 227 * 1024 - 2048 - 2 * (size_t)p.staging - a_tail - st_smem;
     const size_t w_all = (size_t)h.n_taps * p.k_chunks * b_bytes;
     p.resident = (p.n_tiles == 1 && w_all + 2 * (size_t)p.a_alloc <= budget) ? 1 : 0;
     size_t left = budget - (p.resident ? w_all : 0);
@@ -1954,7 +2020,9 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
                                                       CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
     }
-    const size_t smem = 2048 + 2 * (size_t)p.staging + (p.resident ? w_all : (size_t)p.stages_b * b_bytes) + (size_t)p.stages_a * p.a_alloc + a_tail;
+    const size_t smem = 2048 + 2 * (size_t)p.staging + (p.resident ? w_all : (size_t)p.stages_b * b_bytes) + (size_t)p.stages_a * p.a_alloc + a_tail +
+                        st_smem;
+    p.stats_off = (int)(smem - st_smem);
     static bool attr_set[2] = {false, false};
     if (!attr_set[B_MN ? 1 : 0]) {
         PT_CUDA_OK(cudaFuncSetAttribute(conv_halo_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));

@@ -543,6 +543,7 @@ class ChainedStep:
                  max_blocks: Optional[int] = None, model: Optional[W.Model] = None, x0: Optional[torch.Tensor] = None,
                  g_last: Optional[torch.Tensor] = None):
         self.ctx, self.net, self.N, self.fused = ctx, net, N, fused_stats
+        ctx.set_wgrad_cta_limit(0)                      # one stream: every weight gradient may take all SMs (sizes the workspaces)
         names = [l.name for l in net.layers]
         self.blocks = []                                   # (main conv indices, shortcut index or None)
         for i, nm in enumerate(names):
@@ -707,6 +708,7 @@ class ChainedStep:
         B.pt_group_lasso_sgd_step(self.ctx, self.dm.arr, lam, lr, mu, 0.0, self.dm.reg, self.dm.ws, stream)
 
     def step(self, stream=None):
+        self.ctx.set_wgrad_cta_limit(0)               # one stream: every weight gradient may take all SMs
         self.forward(stream)
         self.backward(stream)
         self.update(stream)
