@@ -57,6 +57,9 @@ typedef struct pt_ctx pt_ctx;  /* opaque: device id, SM count, status word, tabl
 pt_status pt_create(pt_ctx **ctx, int device);
 pt_status pt_destroy(pt_ctx *ctx);
 const char *pt_status_string(pt_status s);
+/* After a call returned PT_ERR_CUDA: the CUDA error's name and the runtime call that returned it, as text, for the calling
+ * thread (an empty string if none failed yet). The pointer stays valid; the text changes with the thread's next failure. */
+const char *pt_last_cuda_error(void);
 /* Synchronises `stream`, reads and clears the device status word. PT_OK if no kernel recorded an error; PT_ERR_TIMEOUT for
  * an expired device-side wait; PT_ERR_INVALID_ARG for a channel index outside its tensor (pt_channel_gather,
  * pt_channel_scatter_add and pt_reconfigure skip such an entry). */

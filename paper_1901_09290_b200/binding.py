@@ -25,7 +25,10 @@ class PtError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
         name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
-        super().__init__(f"{what} failed: {name}")
+        detail = ""
+        if name == "PT_ERR_CUDA":
+            detail = ": " + (lib().pt_last_cuda_error() or b"").decode()
+        super().__init__(f"{what} failed: {name}{detail}")
 
 
 class pt_conv_desc(Structure):
@@ -74,6 +77,7 @@ EXPORTS = {
     "pt_create": (c_int32, [POINTER(c_void_p), c_int32]),
     "pt_destroy": (c_int32, [c_void_p]),
     "pt_status_string": (c_char_p, [c_int32]),
+    "pt_last_cuda_error": (c_char_p, []),
     "pt_poll_device_status": (c_int32, [c_void_p, c_void_p]),
     "pt_launch_count": (c_uint64, [c_void_p]),
     "pt_test_set_wait_limit": (c_int32, [c_void_p, ctypes.c_uint32]),

@@ -1,9 +1,21 @@
 // Context management, status handling, table upload and the conv entry points' dispatch.
 #include "pt_internal.h"
+#include <stdio.h>
 
 static const size_t kArenaBytes = 5u << 20;     // 5 MiB of tables: ten slots of 512 KiB
 static const size_t kSlotBytes = 512u << 10;
 static const size_t kSyncWords = 16384;         // arrival counters of the split weight gradients
+
+static thread_local char g_last_cuda[384] = "";
+
+void pt_note_cuda_error(cudaError_t e, const char *call, const char *file, int line)
+{
+    const char *base = strrchr(file, '/');
+    snprintf(g_last_cuda, sizeof(g_last_cuda), "%s (%d) from %.200s at %s:%d", cudaGetErrorName(e), (int)e, call,
+             base ? base + 1 : file, line);
+}
+
+extern "C" const char *pt_last_cuda_error(void) { return g_last_cuda; }
 
 extern "C" const char *pt_status_string(pt_status s)
 {

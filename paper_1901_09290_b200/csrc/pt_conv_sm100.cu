@@ -41,6 +41,13 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// A tensor-map encode that the driver refused is kept, with its line, for pt_last_cuda_error.
+bool map_ok(CUresult r, int line)
+{
+    if (r != CUDA_SUCCESS) pt_note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncode* (refused by the driver)", __FILE__, line);
+    return r == CUDA_SUCCESS;
+}
+
 
 constexpr int kBM = 128;            // output pixels per CTA tile
 constexpr int kKC = 64;             // reduction channels per stage (one 128-byte swizzle row)
@@ -1699,7 +1706,7 @@ bool make_im2col_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, 
                                                     up, (cuuint32_t)kKC, (cuuint32_t)pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return map_ok(r, __LINE__);
 }
 
 // bf16 activations as a plain 2-D tensor (channels, pixels) with row pitch ld: box 64 channels x `pixels`.
@@ -1714,7 +1721,7 @@ bool make_act2d_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, l
                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill))c->encode_tiled)(
         tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return map_ok(r, __LINE__);
 }
 
 // bf16 weight shadow as (C, R*S, K) with row pitch ldw: box (64, 1, box_k).
@@ -1728,7 +1735,7 @@ bool make_weight_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C, 
     CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box,
                                                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return map_ok(r, __LINE__);
 }
 
 // Tile width along the output channels. One tile: the ragged count rounded up to 16. Several tiles: a multiple of
@@ -1797,7 +1804,7 @@ bool make_out_map(const pt_ctx *c, CUtensorMap *tm, void *base, int cols, int ro
     CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
                                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return map_ok(r, __LINE__);
 }
 
 template <bool B_MN>
@@ -1883,7 +1890,7 @@ bool make_halo_in_map(const pt_ctx *c, CUtensorMap *tm, const void *base, int C,
     CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box,
                                                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, lanes == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return map_ok(r, __LINE__);
 }
 
 // One launch of the halo kernel: a stride-1 correlation of `src` with a list of taps, written to a (possibly strided)
@@ -2002,7 +2009,7 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
         CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w), dims, strides, box,
                                                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
                                                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+        if (!map_ok(r, __LINE__)) return PT_ERR_CUDA;
     } else {
         if (!make_halo_in_map(c, &tmA, h.src, h.Cs, h.Ws, h.Hs, d->N, h.lds, Wp, box_h)) return PT_ERR_CUDA;
         if (!make_weight_map(c, &tmB, w, d->C, d->R * d->S, d->K, d->ldw, B_MN ? kKC : p.b_rows)) return PT_ERR_CUDA;
@@ -2018,7 +2025,7 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
         CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmC, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
                                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                       CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+        if (!map_ok(r, __LINE__)) return PT_ERR_CUDA;
     }
     const size_t smem = 2048 + 2 * (size_t)p.staging + (p.resident ? w_all : (size_t)p.stages_b * b_bytes) + (size_t)p.stages_a * p.a_alloc + a_tail +
                         st_smem;
@@ -2195,7 +2202,7 @@ bool make_partial_map(const pt_ctx *c, CUtensorMap *tm, void *ws, int bn, size_t
     CUresult r = ((EncodeTiledFn)c->encode_tiled)(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ws, dims, strides, box, estr,
                                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return map_ok(r, __LINE__);
 }
 
 // Launches the weight-gradient kernel for a problem whose x operand is described by `tmX` (64 pixels x 64 channels boxes).
@@ -2243,7 +2250,7 @@ pt_status run_wgrad(pt_ctx *c, const pt_conv_desc *d, int P, int Q, int stride, 
         CUresult r = ((EncodeTiledFn)c->encode_tiled)(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(dy), dims, strides, box,
                                                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return PT_ERR_CUDA;
+        if (!map_ok(r, __LINE__)) return PT_ERR_CUDA;
     }
     size_t smem = 0;
     const size_t stage = 2 * 8192 + (size_t)p.tpc * pt_ceil_div(p.BN, 64) * 8192;

@@ -8,10 +8,17 @@
 
 #include "../../include/pt.h"
 
+// The CUDA call that last failed on this thread: kept for pt_last_cuda_error.
+void pt_note_cuda_error(cudaError_t e, const char *call, const char *file, int line);
+
 #define PT_CUDA_OK(call)                                   \
     do {                                                   \
         cudaError_t e__ = (call);                          \
-        if (e__ != cudaSuccess) { (void)cudaGetLastError(); return PT_ERR_CUDA; } \
+        if (e__ != cudaSuccess) {                          \
+            pt_note_cuda_error(e__, #call, __FILE__, __LINE__); \
+            (void)cudaGetLastError();                      \
+            return PT_ERR_CUDA;                            \
+        }                                                  \
     } while (0)
 
 // Device status word layout: [0] = first error code recorded (0 = none), [1] = detail (where), [2] = ticket of the

@@ -38,7 +38,8 @@ def test_binding_covers_every_declared_symbol(built):
     assert sorted(binding.EXPORTS) == _declared()
     binding.lib()
     for n in _declared():
-        if n in ("pt_create", "pt_destroy", "pt_status_string", "pt_launch_count", "pt_poll_device_status"):
+        if n in ("pt_create", "pt_destroy", "pt_status_string", "pt_last_cuda_error", "pt_launch_count",
+                 "pt_poll_device_status"):
             continue
         assert hasattr(binding, n), n
 
@@ -47,6 +48,7 @@ def test_status_strings(built):
     from paper_1901_09290_b200 import binding
     L = binding.lib()
     assert L.pt_status_string(0) == b"PT_OK" and L.pt_status_string(5) == b"PT_ERR_TIMEOUT"
+    assert L.pt_last_cuda_error() == b""            # nothing failed on this thread yet
 
 
 def test_create_without_gpu_fails_loudly(built):
