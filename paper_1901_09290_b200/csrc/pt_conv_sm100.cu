@@ -108,6 +108,9 @@ struct __align__(8) PCtl {
     uint64_t w_full;            // resident weights have landed
     uint32_t tmem_base;
     int abort_flag;
+#ifdef PT_DEVICE_TRACE
+    unsigned int chain_seq;
+#endif
 };
 
 constexpr uint32_t kSlabs = 2;                          // staging slabs per epilogue warp (TMA stores in flight)
@@ -194,8 +197,15 @@ __device__ __forceinline__ void stats_flush(uint32_t acc0, int lane, float *dst,
 #ifdef PT_DEVICE_TRACE
 __device__ unsigned long long g_gemm_trace[8][64];
 #define GTRACE(role, idx) do { if (blockIdx.x == 0 && (idx) < 64 && (threadIdx.x & 31) == 0) g_gemm_trace[role][idx] = globaltimer_ns(); } while (0)
+// Timeline of a chain of launches: launch number seq (a device counter, taken by CTA 0 at entry) stamps its entry, the end of
+// its prologue, the return of its dependency wait, its first activation load, its first full stage, its last commit, the end
+// of its last epilogue and its exit.
+__device__ unsigned long long g_chain_trace[256][12];
+__device__ unsigned int g_chain_seq;
+#define CTRACE(ev) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && ctl->chain_seq < 256) g_chain_trace[ctl->chain_seq][ev] = globaltimer_ns(); } while (0)
 #else
 #define GTRACE(role, idx) do { } while (0)
+#define CTRACE(ev) do { } while (0)
 #endif
 
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... The TMA ring runs continuously across
@@ -228,6 +238,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     const int nb_b = (p.BN + 63) / 64;
     const bool two_b = B_MN && !p.resident && nb_b > 1;
 
+#ifdef PT_DEVICE_TRACE
+    if (threadIdx.x == 0) {
+        ctl->chain_seq = blockIdx.x == 0 ? atomicAdd(&g_chain_seq, 1u) : 0xffffffffu;
+        CTRACE(0);
+    }
+#endif
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), p.resident ? 1 : (two_b ? 3 : 2));   // the A producer and, with streamed weights, the B producer(s)
@@ -255,7 +271,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
     // The weights are not written by the kernels that precede a convolution in a stream (those that trigger their dependents
     // early are convolutions themselves), so the weight producers start loading at once; everybody else waits for the
     // previous kernel's results here.
-    if (!(warp == 14 || (warp == 15 && two_b))) grid_dependency_wait();
+    // The activation producer (warp 0) waits just before its first load instead: its set-up (tile coordinates, tap tables: a
+    // few hundred cycles of divisions and first-touch parameter reads) then runs while the previous kernel drains.
+    if (!(warp == 0 || warp == 14 || (warp == 15 && two_b))) grid_dependency_wait();
     grid_launch_dependents();
 
     if (warp == 0 || warp == 14 || (warp == 15 && two_b)) {
@@ -263,10 +281,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             // ---------------- TMA producers: warp 0 brings the A tile of every stage, warp 14 the B tile (issuing a TMA
             // instruction costs its thread about 200 cycles, so the two operands are issued side by side)
             const bool is_a = warp == 0;
+            if (is_a) CTRACE(8);
             const int bsel = warp == 15 ? 1 : 0, nbp = two_b ? 2 : 1;         // this B producer's boxes: bsel, bsel + nbp, ...
             const uint32_t my_bytes = is_a ? a_bytes : (two_b ? (uint32_t)((nb_b + 1 - bsel) / 2) * 8192u : b_bytes);
             int s = 0, ph = 0, issued = 0;   // stage-ring position, continuous across tiles
             int s1 = 0, ph1 = 0;             // position in the second issuer's ring
+            bool dep_waited = false;         // the activation producer has waited for the previous kernel's results
             const int SR = p.stages / p.n_issuers;
             if (!is_a && p.resident) {
                 // n_tiles == 1 here: every weight tile of the launch, once
@@ -298,8 +318,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     const int wtap = p.tap_wt[tap];
                     const uint16_t ow = (uint16_t)p.tap_ow[tap], oh = (uint16_t)p.tap_oh[tap];
                     for (int kc = 0; kc < p.k_chunks; ++kc) {
+                        if (is_a && issued == 0) CTRACE(9);
                         ok = mbar_wait(smem_u32(&ctl->empty[sbase + s]), ph ^ 1, abort_flag, p.status, 1);
                         if (!ok) break;
+                        if (is_a && issued == 0) CTRACE(10);
                         if (is_a) GTRACE(0, issued); else if (warp == 14) GTRACE(2, issued);
                         const uint32_t bar = smem_u32(&ctl->full[sbase + s]);
                         const uint32_t a_dst = data_base + (uint32_t)(sbase + s) * stage_bytes, b_dst = a_dst + a_bytes;
@@ -309,6 +331,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                             continue;
                         }
                         mbar_arrive_expect_tx(bar, my_bytes);
+                        if (is_a && !dep_waited) { CTRACE(1); grid_dependency_wait(); CTRACE(2); dep_waited = true; }
                         if (is_a) {
                             if (p.a_tiled) tma_load_2d(a_dst, &tmA, bar, kc * kKC, m0);
                             else tma_load_im2col_4d(a_dst, &tmA, bar, kc * kKC, w0, h0, n, ow, oh);
@@ -319,6 +342,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                                 tma_load_3d(b_dst + (uint32_t)nb * 8192u, &tmB, bar, n0 + nb * 64, wtap, kc * kKC);
                         }
                         if (is_a) GTRACE(1, issued); else if (warp == 14) GTRACE(3, issued);
+                        if (is_a && issued == 0) CTRACE(3);
                         ++issued;
                         if (++s == SR) { s = 0; ph ^= 1; }
                     }
@@ -361,6 +385,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                     ok = mbar_wait(smem_u32(&ctl->full[sbase + s]), ph, abort_flag, p.status, 2);
                     if (!ok) break;
                     if (warp == 1) GTRACE(4, consumed);
+                    if (warp == 1 && consumed == 0) CTRACE(4);
                     tc_fence_after();
                     const uint32_t a_src = data_base + (uint32_t)(sbase + s) * stage_bytes;
                     const uint32_t b_src = p.resident ? w_base + (uint32_t)(tap * p.k_chunks + kc) * b_slot : a_src + a_bytes;
@@ -384,6 +409,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
             }
             if (ok) umma_commit_lead(smem_u32(&ctl->acc_full[b]), leader);   // this tile's accumulator is complete
             if (NI == 1 && ++b == p.epi_groups) { b = 0; aph ^= 1; }
+            if (warp == 1) CTRACE(5);
         }
     } else if (warp - 2 < 4 * p.epi_groups) {
         // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; group g drains accumulator buffer g,
@@ -553,9 +579,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         }
         if (my_stats && p.n_tiles == 1) stats_flush(st_acc, lane, my_stats, p.ld_out, 0, (p.BN + 63) / 64, p.n_cols, false);
         if (p.tma_store && lane == 0) tma_store_wait_read();     // the staging slabs must outlive the stores' reads
+        if (warp == 2) CTRACE(6);
         tc_fence_before();
     }
     __syncthreads();
+    if (warp == 0) CTRACE(7);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
@@ -691,7 +719,8 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
     const int issuer = warp == 1 ? 0 : warp - 9;             // warps 10, 11, 12 -> issuers 1, 2, 3
     // the weight producers do not read the previous kernel's output: resident weights are issued first and the wait follows
     // them (below); the producers of streamed weights never need it
-    if (!(warp == 0 || (warp == 13 && !p.resident))) grid_dependency_wait();
+    // Warps that load activations wait just before their first activation load, after their set-up (tile walk, ring positions).
+    if (!(warp == 0 || ((warp == 13 || warp == 14 || warp == 15) && !p.resident))) grid_dependency_wait();
     grid_launch_dependents();
 
     // Streamed weights with two issuers: two complete pipelines (producer warp, A ring, B ring, issuer warp, accumulators),
@@ -720,8 +749,8 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         if (!B_MN) tma_load_3d(dst, &tmB, bar, kc * kKC, wtap, 0);
                         else for (int nb = 0; nb < (p.BN + 63) / 64; ++nb) tma_load_3d(dst + (uint32_t)nb * 8192u, &tmB, bar, nb * 64, wtap, kc * kKC);
                     }
-                grid_dependency_wait();          // the activations are the previous kernel's output
             }
+            bool dep_waited = false;             // the activations are the previous kernel's output
             int tc = pid;
             TileWalk tw;
             tw.init((int)blockIdx.x + pid * (int)gridDim.x, n_prod * (int)gridDim.x, p.n_tiles, p.row_tiles);
@@ -744,6 +773,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         const uint32_t bar = smem_u32(&ctl->full_a[sa]);
                         HTRACE(0, tc);
                         mbar_arrive_expect_tx(bar, (uint32_t)p.a_box_bytes);
+                        if (!dep_waited) { grid_dependency_wait(); dep_waited = true; }
                         tma_load_4d(a_base + (uint32_t)sa * (uint32_t)p.a_alloc, &tmA, bar, kc * kKC, p.lo_w, p0 + p.lo_h, img);
                     }
                     if (!b_role) continue;
@@ -1317,7 +1347,9 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int issuer = warp == 1 ? 0 : warp - 5;                      // warps 6, 7, 8 -> issuers 1, 2, 3
-    grid_dependency_wait();              // nothing above touches global memory
+    // Nothing above touches global memory. The producer threads wait for the previous kernel after their set-up (pixel
+    // coordinates of the first stage: several divisions) instead of before it.
+    if (!((warp == 0 || (warp >= 2 && warp < 2 + NXP)) && lane == 0)) grid_dependency_wait();
     grid_launch_dependents();
     if (threadIdx.x == 0) WTRACE(0);
 
@@ -1346,6 +1378,7 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_kernel(const __grid_const
                     box_sh[n_mine] = (uint16_t)r; box_sw[n_mine] = (uint16_t)((tap0 + tt) - r * p.S);
                 }
             int s = 0, ph = 0, issued = 0;
+            grid_dependency_wait();
             for (int it = 0; it < iters; ++it) {
                 if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 4)) break;
                 const uint32_t bar = smem_u32(&ctl->full[s]);
@@ -1487,7 +1520,8 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_rows_kernel(const __grid_
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int issuer = warp == 1 ? 0 : warp - 5;                      // warps 6, 7, 8 -> issuers 1, 2, 3
-    grid_dependency_wait();              // nothing above touches global memory
+    // nothing above touches global memory; the producer threads wait after their set-up
+    if (!((warp == 0 || warp == 2) && lane == 0)) grid_dependency_wait();
     grid_launch_dependents();
     if (threadIdx.x == 0) WTRACE(0);
 
@@ -1500,6 +1534,7 @@ __global__ void __launch_bounds__(kThreads) conv_wgrad_rows_kernel(const __grid_
                                             : nb_b * (uint32_t)((p.nr + p.lo_span) * p.Wp) * 128u;
             int n = u_beg / p.RB, rb = u_beg - n * p.RB;
             int s = 0, ph = 0, issued = 0;
+            grid_dependency_wait();
             for (int it = 0; it < iters; ++it) {
                 if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag, p.status, 4)) break;
                 const uint32_t bar = smem_u32(&ctl->full[s]);
@@ -2705,6 +2740,17 @@ pt_status pt_sm100_set_wait_limit_ns(unsigned long long ns, cudaStream_t st)
 extern "C" int pt_debug_wgrad_trace(unsigned long long *host_out)
 {
     return (int)cudaMemcpyFromSymbol(host_out, g_wg_trace, sizeof(unsigned long long) * 8 * 64);
+}
+extern "C" int pt_debug_chain_trace(unsigned long long *host_out, int reset)
+{
+    cudaError_t e = cudaMemcpyFromSymbol(host_out, g_chain_trace, sizeof(unsigned long long) * 256 * 12);
+    if (reset) {
+        static const unsigned long long zeros[256 * 12] = {0};
+        const unsigned int z = 0;
+        (void)cudaMemcpyToSymbol(g_chain_trace, zeros, sizeof(zeros));
+        (void)cudaMemcpyToSymbol(g_chain_seq, &z, sizeof(z));
+    }
+    return (int)e;
 }
 extern "C" int pt_debug_gemm_trace(unsigned long long *host_out)
 {
