@@ -3,6 +3,7 @@
     python -m paper_1901_09290_b200.layerbench --layer s1b1.c3 --passes fwd,dgrad,wgrad --iters 20
     python -m paper_1901_09290_b200.layerbench --shape 64,56,36,143,1,1 --passes fwd      # N,H,C,K,R,stride
     python -m paper_1901_09290_b200.layerbench --bn 64,56,143                              # batch norm + ReLU + residual: N,H,C
+    python -m paper_1901_09290_b200.layerbench --model --iters 5      # lasso step, detection, compaction of the whole model alone
 
 It is also the small case ncu captures are taken on.
 """
@@ -15,6 +16,37 @@ import torch
 
 from . import binding as B
 from . import workloads as W
+
+
+def model_main(args):
+    """The HBM-bound model passes alone, in the order a step runs them, each timed with CUDA events after an L2 flush."""
+    from .harness import TrainStep
+    net = W.resnet50()
+    seed = W.BASE_SEED + 4
+    counts = W.staged_keep_to_flops(net, seed, 0.60)
+    ctx = B.Context(0)
+    ts = TrainStep(ctx, net, counts, W.choose_kept(net, counts, seed), 1, seed)
+    md = ts.md
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    ops = [("detect", lambda: B.pt_find_zero_groups(ctx, md.arr, 1e-4, False, md.ws)),
+           ("plan_incl_host_sync", lambda: B.pt_reconfigure_plan(ctx, md.graph(), ts.new2old)),
+           ("gather", lambda: ts.gather()),
+           ("lasso", lambda: ts.lasso()),
+           ("lasso_norms", lambda: ts.lasso_norms()),
+           ("lasso_carried", lambda: ts.lasso_carried())]
+    tot = {k: 0.0 for k, _ in ops}
+    for it in range(args.iters + 1):                    # the first round is the warm-up
+        for k, fn in ops:
+            flush.fill_(it)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            if it:
+                tot[k] += a.elapsed_time(b) * 1e3 / args.iters
+    ctx.poll()
+    print(json.dumps({"model": "resnet50 keep drawn to 0.60", "dense_params": md.n_params(), "kept_params": ts.mp.n_params(),
+                      "us": {k: round(v, 1) for k, v in tot.items()},
+                      "note": "eager launches with events around each call (host launch cost included)"}))
 
 
 def main():
@@ -30,7 +62,12 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager launches (includes host launch cost)")
     ap.add_argument("--bn", default=None, help="N,H,C: time pt_bn_relu_fwd / pt_bn_relu_bwd instead of a convolution")
     ap.add_argument("--gate", default=None, help="N,H,C,S: time pt_channel_gather / pt_channel_scatter_add of S of a node's C channels")
+    ap.add_argument("--model", action="store_true",
+                    help="time detection, plan, gather, the lasso step and its carried form over the bench's ResNet-50 model "
+                         "alone (batch 1 activations: ~0.7 GB on the device, the model itself larger than L2)")
     args = ap.parse_args()
+    if args.model:
+        return model_main(args)
     if args.gate:
         return gate_main(args)
     if args.bn:
