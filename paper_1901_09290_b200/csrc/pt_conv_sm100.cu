@@ -211,7 +211,8 @@ __device__ unsigned int g_chain_seq;
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... The TMA ring runs continuously across
 // tiles. The accumulator has G = 2 or 3 buffers in TMEM and buffer b has its own group of four epilogue warps, so the
 // loads and MMAs of the next tiles overlap the epilogues of the previous ones.
-template <bool B_MN>
+// STATS: the epilogue also takes the batch-normalisation statistics (a variant of its own: the plain kernels keep their registers).
+template <bool B_MN, bool STATS>
 __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                  const __grid_constant__ CUtensorMap tmB,
                                                                  const __grid_constant__ CUtensorMap tmC, const GemmP p)
@@ -417,7 +418,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         const int quarter = warp & 3, group = (warp - 2) >> 2, G = p.epi_groups;
         const uint32_t slab0 = (p.alias_staging ? data_base : staging_base) + (uint32_t)(warp - 2) * (kSlabs * 4096u);
         // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
-        float *my_stats = p.stats ? p.stats + ((size_t)blockIdx.x * (4 * G) + (warp - 2)) * 2 * p.ld_out : nullptr;
+        float *my_stats = (STATS && p.stats) ? p.stats + ((size_t)blockIdx.x * (4 * G) + (warp - 2)) * 2 * p.ld_out : nullptr;
         const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * kStatsWarpBytes;
         if (my_stats) {
             for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
@@ -521,7 +522,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
                         if (m0 + quarter * 32 < p.M_total) tma_store_2d(&tmC, slab, n0 + ch * 64, m0 + quarter * 32);
                         tma_store_commit();
                     }
-                    if (p.stats) {
+                    if (STATS && p.stats) {
                         const int left = p.M_total - (m0 + quarter * 32);
                         const uint32_t rows = left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
                         chunk_stats(slab, 0, rows, lane, st_acc + (uint32_t)ch * 512u);
@@ -674,7 +675,7 @@ constexpr int kHaloThreads = 512;
 // kernel therefore runs up to four issuer warps, each on its own scheduler: issuer i owns accumulator buffer i and
 // an A ring of its own (a waiter may lag an mbarrier by at most one phase, so issuers cannot share a ring), and takes
 // the tiles i, i + I, i + 2I, ... of the CTA. Weights that stream through a ring keep a single issuer.
-template <bool B_MN>
+template <bool B_MN, bool STATS>
 __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                      const __grid_constant__ CUtensorMap tmB,
                                                                      const __grid_constant__ CUtensorMap tmC, const HaloP p)
@@ -903,7 +904,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         const int gtid = (warp - 2 - group * 4) * 32 + lane;         // 0..127 within the group
         const uint32_t slab = staging_base + (uint32_t)group * (uint32_t)p.staging;
         // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
-        float *my_stats = p.stats ? p.stats + ((size_t)blockIdx.x * 8 + (warp - 2)) * 2 * p.ld_out : nullptr;
+        float *my_stats = (STATS && p.stats) ? p.stats + ((size_t)blockIdx.x * 8 + (warp - 2)) * 2 * p.ld_out : nullptr;
         const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * kStatsWarpBytes;
         if (my_stats) {
             for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
@@ -972,7 +973,7 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
                         tma_store_commit();
                         HTRACE(7, tc);
                     }
-                    if (p.stats) {
+                    if (STATS && p.stats) {
                         // this thread's raster position is a real output pixel iff it lies inside the row and the image
                         const int ri = m / p.Wp, rj = m - ri * p.Wp;
                         const uint32_t rows = __ballot_sync(0xffffffffu, m < p.nr * p.Wp && rj < p.Q && p0 + ri < p.P);
@@ -1892,10 +1893,14 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
         if (p.stages < 2) { p.n_issuers = 1; p.acc_per = 1; p.stages = 2; }
     }
     p.tmem_cols = pow2_cols((p.n_issuers == 2 ? 2 * p.acc_per : p.epi_groups) * p.BN);
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[B_MN ? 1 : 0]) {
-        PT_CUDA_OK(cudaFuncSetAttribute(conv_gemm_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set[B_MN ? 1 : 0] = true;
+    // the statistics variant exists for the forward kernel only
+    void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, GemmP) =
+        (!B_MN && c->stats_mode) ? conv_gemm_kernel<false, true> : conv_gemm_kernel<B_MN, false>;
+    const int kid = (!B_MN && c->stats_mode) ? 2 : (B_MN ? 1 : 0);
+    static bool attr_set[3] = {false, false, false};
+    if (!attr_set[kid]) {
+        PT_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set[kid] = true;
     }
     const int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
     if (c->stats_mode) {
@@ -1905,7 +1910,7 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
         p.stats = c->stats_out;
     }
     if (c->test_skip == 2) { p.test_skip = 1; c->test_skip = 0; }
-    PT_CUDA_OK(launch_pdl(conv_gemm_kernel<B_MN>, dim3((unsigned)grid), dim3(kGemmThreads), smem, st, tmA, tmB, tmC, p));
+    PT_CUDA_OK(launch_pdl(kernel, dim3((unsigned)grid), dim3(kGemmThreads), smem, st, tmA, tmB, tmC, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
@@ -2065,10 +2070,13 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     const size_t smem = 2048 + 2 * (size_t)p.staging + (p.resident ? w_all : (size_t)p.stages_b * b_bytes) + (size_t)p.stages_a * p.a_alloc + a_tail +
                         st_smem;
     p.stats_off = (int)(smem - st_smem);
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[B_MN ? 1 : 0]) {
-        PT_CUDA_OK(cudaFuncSetAttribute(conv_halo_kernel<B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set[B_MN ? 1 : 0] = true;
+    void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, HaloP) =
+        (!B_MN && c->stats_mode) ? conv_halo_kernel<false, true> : conv_halo_kernel<B_MN, false>;
+    const int kid = (!B_MN && c->stats_mode) ? 2 : (B_MN ? 1 : 0);
+    static bool attr_set[3] = {false, false, false};
+    if (!attr_set[kid]) {
+        PT_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set[kid] = true;
     }
     const int total_tiles = p.N * p.row_tiles * p.n_tiles;
     int grid = total_tiles < c->sm_count ? total_tiles : c->sm_count;
@@ -2079,7 +2087,7 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
         if ((size_t)c->stats_parts * 2 * p.ld_out * sizeof(float) > c->stats_cap) return PT_ERR_WORKSPACE;
         p.stats = c->stats_out;
     }
-    PT_CUDA_OK(launch_pdl(conv_halo_kernel<B_MN>, dim3((unsigned)grid), dim3(kHaloThreads), smem, st, tmA, tmB, tmC, p));
+    PT_CUDA_OK(launch_pdl(kernel, dim3((unsigned)grid), dim3(kHaloThreads), smem, st, tmA, tmB, tmC, p));
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     return PT_OK;
