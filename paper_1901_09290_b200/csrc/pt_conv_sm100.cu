@@ -1812,9 +1812,11 @@ int pow2_cols(int bn)
 }
 
 // Pipeline depth for a kernel that owns the SM: as many stages as fit beside `reserved` bytes, at most kMaxStages.
-int pick_stages(size_t stage_bytes, int iters, size_t reserved, size_t *smem)
+// The GEMM-form kernel may take all but 1 KB of the 227 KB a CTA can have (one more stage for the wide 1x1 layers).
+constexpr size_t kGemmSmemCap = (size_t)226 * 1024;
+int pick_stages(size_t stage_bytes, int iters, size_t reserved, size_t *smem, size_t cap = (size_t)220 * 1024)
 {
-    int st = (int)((220 * 1024 - 2048 - reserved) / stage_bytes);
+    int st = (int)((cap - 2048 - reserved) / stage_bytes);
     if (st > kMaxStages) st = kMaxStages;
     if (st > iters && iters >= 2) st = iters;
     if (st < 2) st = 2;
@@ -1877,14 +1879,14 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     // statistics mode: the epilogue warps' accumulators sit at the end of the shared memory (taken from the ring's room)
     const size_t st_smem = c->stats_mode ? (size_t)12 * kStatsWarpBytes : 0;
     size_t staging2 = p.alias_staging ? 0 : (size_t)p.epi_groups * 4 * kSlabs * 4096;
-    if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all + st_smem, &smem);
+    if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all + st_smem, &smem, kGemmSmemCap);
     else {
-        p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2 + st_smem, &smem);
+        p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2 + st_smem, &smem, kGemmSmemCap);
         if (p.stages < 4 && p.epi_groups == 3 && p.taps * p.k_chunks * per_cta >= 4) {
             // a third epilogue group costs 32 KB of staging: with wide weight tiles that is the fourth pipeline stage
             p.epi_groups = 2;
             staging2 = (size_t)p.epi_groups * 4 * kSlabs * 4096;
-            p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2 + st_smem, &smem);
+            p.stages = pick_stages(a_bytes + b_bytes, p.taps * p.k_chunks * per_cta, staging2 + st_smem, &smem, kGemmSmemCap);
         }
     }
     p.stats_off = (int)(smem - st_smem);
