@@ -117,8 +117,11 @@ int32_t pt_conv_wgrad_ctas(const pt_ctx *ctx, const pt_conv_desc *d, int32_t *wa
 
 /* Stream order: the three calls below are ordinary stream work. Their kernels are launched with programmatic stream
  * serialization and read the WEIGHTS before waiting for the preceding kernel of the stream; that is invisible to callers
- * because only kernels that release their dependents early can be overtaken, and the only such kernels are this library's
- * convolutions, which never write weights. */
+ * because only kernels that release their dependents early (griddepcontrol.launch_dependents before their last store) can be
+ * overtaken: of this library's kernels the convolutions and the read-only sweeps of the lasso step do that, and none of them
+ * writes weights (the update of pt_group_lasso_sgd_step and the gather of pt_reconfigure complete before their successors
+ * start). A caller's own kernel that writes w and releases its dependents early must be followed by an event or another
+ * kernel before a convolution reads w. */
 /* y[n,p,q,k] = sum_{r,s,c} x[n, p*stride-pad+r, q*stride-pad+s, c] * w[k,r,s,c], zero outside the image.
  * x: bf16 [N][H][W][ldx]; w: bf16 shadow [K][R][S][ldw]; y: [N][P][Q][ldy] bf16 or fp32. fp32 accumulation. */
 pt_status pt_conv_fwd(pt_ctx *ctx, const pt_conv_desc *d, const void *x, const void *w, void *y,

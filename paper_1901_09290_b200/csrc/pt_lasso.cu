@@ -108,7 +108,10 @@ __global__ void __launch_bounds__(kThreads) sweep_kernel(const LayerDev *__restr
     const int c = ch.col0 + tx;
     const bool cv = c < L.C;
     pdl_wait();
-    pdl_trigger();
+    // A sweep that writes the weights lets its dependents start only when it has completed: the convolution kernels' weight
+    // producers do not wait for their predecessor (weights are never written by a kernel that releases its dependents early),
+    // and a convolution may well be the next launch of the stream.
+    if (!UPD) pdl_trigger();
     if (RED && blockIdx.x == 0 && threadIdx.x == 0) *ticket = 0u;          // for the finish kernel that follows
     float ci = 0.f;
     if (UPD && cv) ci = inv_in[L.c_off + c];

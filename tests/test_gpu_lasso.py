@@ -303,3 +303,29 @@ def test_carried_step_odd_shapes(shape):
     torch.cuda.synchronize()
     zo, zi = oracle.find_zero_groups(dm.w[0].cpu().numpy(), 1e-4)
     assert dm.z_out[0].cpu().numpy().tolist() == zo.tolist() and dm.z_in[0].cpu().numpy().tolist() == zi.tolist()
+
+
+def test_conv_right_behind_the_update_reads_the_new_weights():
+    """Stream order: the update writes the bf16 shadow, and a convolution launched right behind it on the same stream must
+    read the new values, although its weight producers do not wait for the kernel before them (the update therefore does
+    not release its dependents early). The last layer of the table is updated by the last blocks of the sweep."""
+    net = W.resnet50(image=32)
+    counts = W.uniform_keep(net, 0.3)
+    model = W.gen_model(W.with_sizes(net, counts), W.BASE_SEED + 77)
+    dm = DevModel(model)
+    li = len(model.net.layers) - 1
+    l = model.net.layers[li]
+    N, H = 2, 7
+    d = B.make_conv_desc(N, H, H, l.C, l.K, l.R, l.R, 1, l.pad, W.pad16(l.C), W.pad16(l.K), W.pad8(l.C), 0, 2)
+    x = W.gen_act(N, H, H, l.C, W.BASE_SEED + 78)
+    xd = Hh.to_dev_padded(x, d.ldx)
+    ws = Hh.conv_ws(d, 0)
+    for it in range(6):
+        y = Hh.out_buffer((N, H, H), l.K, d.ldy, False)
+        B.pt_group_lasso_sgd_step(Hh.ctx(), dm.arr, 1e-4, 0.5, 0.9, 0.0, dm.reg, dm.ws)     # lr 0.5: every step moves the weights visibly
+        B.pt_conv_fwd(Hh.ctx(), d, xd, dm.wb[li], y, ws)
+        torch.cuda.synchronize()
+        Hh.ctx().poll()
+        w_now = dm.wb[li][..., :l.C].float().cpu().numpy()
+        ref = oracle.conv_fwd(x.numpy(), w_now, 1, l.pad)
+        Hh.check_conv(y, l.K, ref, what=f"iteration {it}")
