@@ -52,8 +52,8 @@ struct pt_ctx {
     struct GatherSlot {
         pt_region reg;
         std::vector<char> args;
-        unsigned chunks = 0;
-        size_t jobs_bytes = 0;
+        unsigned chunks = 0, grid = 0;
+        size_t jobs_bytes = 0, first_off = 0;
     } gather_slot[4];
     int gather_next = 0;
     int32_t *h_counts = nullptr;        // pinned, for pt_reconfigure_plan: [0] = flag the kernel raises, [16..] = counts

@@ -108,12 +108,12 @@ __device__ __forceinline__ void bad_map_entry(unsigned int *status, unsigned int
 }
 
 __global__ void __launch_bounds__(kGThreads, 4) gather_kernel(const GatherJob *__restrict__ jobs, const GatherChunk *__restrict__ chunks,
-                                                            int n_chunks, unsigned int *status)
+                                                            const int *__restrict__ block_first, unsigned int *status)
 {
     __shared__ int s_oline[kGMaxLines];          // old line of each new line of the chunk (-1: skipped)
     __shared__ int s_co[kGMaxC];                 // old column of each new column (-1: skipped)
-    const int c_beg = (int)((long long)blockIdx.x * n_chunks / gridDim.x);
-    const int c_end = (int)((long long)(blockIdx.x + 1) * n_chunks / gridDim.x);
+    // block b takes chunks [block_first[b], block_first[b + 1]): consecutive chunks with about the same number of elements
+    const int c_beg = block_first[blockIdx.x], c_end = block_first[blockIdx.x + 1];
     int cur_job = -1;
     for (int ci = c_beg; ci < c_end; ++ci) {
         const GatherChunk ch = chunks[ci];
@@ -304,9 +304,8 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         pt_ctx::GatherSlot &gs = c->gather_slot[i];
         if (!(gs.reg.valid && gs.chunks && args == gs.args)) continue;
         const char *dev = c->d_arena + gs.reg.off;
-        const unsigned grid = gs.chunks < (unsigned)(4 * c->sm_count) ? gs.chunks : (unsigned)(4 * c->sm_count);
-        gather_kernel<<<grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + gs.jobs_bytes), (int)gs.chunks,
-                                                  c->d_status);
+        gather_kernel<<<gs.grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + gs.jobs_bytes),
+                                                     (const int *)(dev + gs.first_off), c->d_status);
         c->launches += 1;
         PT_CUDA_OK(cudaGetLastError());
         return PT_OK;
@@ -345,7 +344,7 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         const int job = (int)jobs.size();
         jobs.push_back(J);
         {
-            int per = 16384 / n.C;                       // whole lines, about 16K elements per chunk
+            int per = 8192 / n.C;                        // whole lines, about 8K elements per chunk
             if (per < 1) per = 1;
             if (per > kGMaxLines) per = kGMaxLines;
             for (int l0 = 0; l0 < J.lines; l0 += per) chunks.push_back(GatherChunk{job, l0, J.lines - l0 < per ? J.lines - l0 : per, 0});
@@ -361,25 +360,50 @@ extern "C" pt_status pt_reconfigure(pt_ctx *c, const pt_graph *og, const int32_t
         }
     }
     if (chunks.empty()) return PT_OK;
-    size_t jb = pt_align_up(jobs.size() * sizeof(GatherJob), 256), cb = chunks.size() * sizeof(GatherChunk);
-    std::vector<char> buf(jb + cb, 0);
+    // Blocks are persistent (at most four per SM) and take consecutive chunks; the list is cut where the running element
+    // count passes the next multiple of total / grid, so that every block moves about the same number of elements (a
+    // per-channel vector counts as one block-wide step).
+    const unsigned nchk = (unsigned)chunks.size();
+    const unsigned grid = nchk < (unsigned)(4 * c->sm_count) ? nchk : (unsigned)(4 * c->sm_count);
+    std::vector<int> first(grid + 1, 0);
+    {
+        std::vector<long long> cost(nchk);
+        long long total = 0;
+        for (unsigned i = 0; i < nchk; ++i) {
+            const GatherJob &J = jobs[chunks[i].job];
+            cost[i] = J.kind == 1 ? kGThreads : (long long)chunks[i].n_lines * J.Cn;
+            total += cost[i];
+        }
+        long long run = 0;
+        unsigned b = 1;
+        for (unsigned i = 0; i < nchk && b < grid; ++i) {
+            run += cost[i];
+            // chunk i ends block b - 1 once the running count reaches that block's share (and enough chunks remain for the rest)
+            while (b < grid && (run * grid >= total * b || nchk - (i + 1) <= grid - b)) first[b++] = (int)(i + 1);
+        }
+        while (b <= grid) first[b++] = (int)nchk;
+        first[grid] = (int)nchk;
+    }
+    size_t jb = pt_align_up(jobs.size() * sizeof(GatherJob), 256), cb = pt_align_up(chunks.size() * sizeof(GatherChunk), 256);
+    const size_t fb = first.size() * sizeof(int);
+    std::vector<char> buf(jb + cb + fb, 0);
     memcpy(buf.data(), jobs.data(), jobs.size() * sizeof(GatherJob));
-    memcpy(buf.data() + jb, chunks.data(), cb);
+    memcpy(buf.data() + jb, chunks.data(), chunks.size() * sizeof(GatherChunk));
+    memcpy(buf.data() + jb + cb, first.data(), fb);
     char *dev = nullptr;
     pt_ctx::GatherSlot &gs = c->gather_slot[c->gather_next];
     c->gather_next = (c->gather_next + 1) & 3;
     gs.chunks = 0;
     s = pt_upload_table(c, &gs.reg, buf.data(), buf.size(), st, &dev);
     if (s != PT_OK) return s;
-    {
-        const unsigned nchk = (unsigned)chunks.size();
-        const unsigned grid = nchk < (unsigned)(4 * c->sm_count) ? nchk : (unsigned)(4 * c->sm_count);
-        gather_kernel<<<grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + jb), (int)nchk, c->d_status);
-    }
+    gather_kernel<<<grid, kGThreads, 0, st>>>((const GatherJob *)dev, (const GatherChunk *)(dev + jb), (const int *)(dev + jb + cb),
+                                              c->d_status);
     c->launches += 1;
     PT_CUDA_OK(cudaGetLastError());
     gs.args.swap(args);
-    gs.chunks = (unsigned)chunks.size();
+    gs.chunks = nchk;
     gs.jobs_bytes = jb;
+    gs.first_off = jb + cb;
+    gs.grid = grid;
     return PT_OK;
 }
