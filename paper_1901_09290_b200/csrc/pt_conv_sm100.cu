@@ -83,6 +83,7 @@ struct GemmP {
     int alias_staging;  // 1: the CTA has a single tile; the epilogue's staging slabs lie in the (then idle) ring
     int test_skip;      // test hook (pt_test_skip_next_arrive): the A producer leaves out the first stage of its first tile
     int stats_off;      // byte offset in shared memory of the epilogue warps' statistics accumulators (stats != nullptr)
+    int stats_warp;     // bytes of one warp's accumulators: 512 per 64-channel chunk of the tile
     float *stats;       // optional: per (pixel tile, warp quarter) and output channel, sum and sum of squares of the bf16 values
                         // stored, as [part][2][ld_out] floats (the batch-normalisation statistics of the layer that follows)
     void *out;
@@ -121,30 +122,27 @@ constexpr uint32_t kSlabs = 2;                          // staging slabs per epi
 // accumulated in the warp's own shared-memory slots (acc: 128 floats per chunk of the tile, four per lane) and written to the
 // warp's row of partial sums by stats_flush. Feature normalisation (Sec. 2.1) reads its input twice; taking the sums here,
 // from the tile that is still in shared memory, removes the first of the two passes.
-constexpr uint32_t kStatsWarpBytes = 4u * 128u * 4u;          // four chunks x 32 lanes x (sum, sum of squares) x two channels
+constexpr uint32_t kStatsChunkBytes = 128u * 4u;              // per 64-channel chunk: 32 lanes x (sum, sum of squares) x two channels
 
 __device__ __forceinline__ void chunk_stats(uint32_t slab, int row0, uint32_t rows, int lane, uint32_t acc)
 {
     float s0a = 0.f, s1a = 0.f, s0b = 0.f, s1b = 0.f;
     const uint32_t jj = (uint32_t)lane >> 2, wi = ((uint32_t)lane & 3u) << 2;
-    if (rows == 0xffffffffu) {
+    // Eight loads are issued before the first is used (one at a time, each waits out the shared-memory latency: 1500 cycles
+    // per chunk in the first version, more than the rest of the epilogue). Rows that are not output pixels (the halo tiles'
+    // raster has some) are loaded too and count as zeros.
 #pragma unroll
-        for (int r = 0; r < 32; ++r) {
-            const uint32_t m = (uint32_t)(row0 + r);
-            uint32_t word;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(word) : "r"(slab + m * 128u + ((jj ^ (m & 7u)) << 4) + wi) : "memory");
-            const float a = __uint_as_float(word << 16), b = __uint_as_float(word & 0xffff0000u);
-            s0a += a; s1a = fmaf(a, a, s1a);
-            s0b += b; s1b = fmaf(b, b, s1b);
+    for (int r0 = 0; r0 < 32; r0 += 8) {
+        uint32_t word[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t m = (uint32_t)(row0 + r0 + j);
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(word[j]) : "r"(slab + m * 128u + ((jj ^ (m & 7u)) << 4) + wi));
         }
-    } else {
-        while (rows) {
-            const int r = __ffs(rows) - 1;
-            rows &= rows - 1u;
-            const uint32_t m = (uint32_t)(row0 + r);
-            uint32_t word;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(word) : "r"(slab + m * 128u + ((jj ^ (m & 7u)) << 4) + wi) : "memory");
-            const float a = __uint_as_float(word << 16), b = __uint_as_float(word & 0xffff0000u);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const bool on = (rows >> (r0 + j)) & 1u;
+            const float a = on ? __uint_as_float(word[j] << 16) : 0.f, b = on ? __uint_as_float(word[j] & 0xffff0000u) : 0.f;
             s0a += a; s1a = fmaf(a, a, s1a);
             s0b += b; s1b = fmaf(b, b, s1b);
         }
@@ -156,11 +154,12 @@ __device__ __forceinline__ void chunk_stats(uint32_t slab, int row0, uint32_t ro
     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(slot), "f"(t.x), "f"(t.y), "f"(t.z), "f"(t.w) : "memory");
 }
 
-__device__ __forceinline__ void stats_clear(uint32_t acc0, int lane)
+__device__ __forceinline__ void stats_clear(uint32_t acc0, int lane, int n_chunks)
 {
 #pragma unroll
     for (int ch = 0; ch < 4; ++ch)
-        asm volatile("st.shared.v4.f32 [%0], {%1, %1, %1, %1};" ::"r"(acc0 + (uint32_t)ch * 512u + (uint32_t)lane * 16u), "f"(0.f) : "memory");
+        if (ch < n_chunks)
+            asm volatile("st.shared.v4.f32 [%0], {%1, %1, %1, %1};" ::"r"(acc0 + (uint32_t)ch * 512u + (uint32_t)lane * 16u), "f"(0.f) : "memory");
 }
 
 // Adds the warp's shared-memory sums of the channels n0 .. n0 + 64 * n_chunks into its row of partial sums (zeroed by the warp
@@ -188,7 +187,7 @@ __device__ __forceinline__ void stats_flush(uint32_t acc0, int lane, float *dst,
         if (c < n_cols) { dst[c] = o[ch][0] + t[ch].x; dst[ld + c] = o[ch][1] + t[ch].y; }
         if (c + 1 < n_cols) { dst[c + 1] = o[ch][2] + t[ch].z; dst[ld + c + 1] = o[ch][3] + t[ch].w; }
     }
-    stats_clear(acc0, lane);
+    stats_clear(acc0, lane, n_chunks);
 }
 
 // Device-side timeline of CTA 0 (a build with -DPT_DEVICE_TRACE; read back with pt_debug_gemm_trace): per pipeline stage in
@@ -419,10 +418,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) conv_gemm_kernel(const __grid
         const uint32_t slab0 = (p.alias_staging ? data_base : staging_base) + (uint32_t)(warp - 2) * (kSlabs * 4096u);
         // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
         float *my_stats = (STATS && p.stats) ? p.stats + ((size_t)blockIdx.x * (4 * G) + (warp - 2)) * 2 * p.ld_out : nullptr;
-        const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * kStatsWarpBytes;
+        const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * (uint32_t)p.stats_warp;
         if (my_stats) {
             for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
-            stats_clear(st_acc, lane);
+            stats_clear(st_acc, lane, (p.BN + 63) / 64);
             __syncwarp();
         }
         int tc = group, sl = 0;
@@ -614,6 +613,7 @@ struct HaloP {
     int tmem_cols, tma_store, out_f32, ld_out;
     int oH, oW, o_step, o_h0, o_w0;      // direct stores: raster (n, i, j) -> out[((n*oH + i*o_step + o_h0)*oW + j*o_step + o_w0)*ld_out]
     int stats_off;                       // byte offset in shared memory of the epilogue warps' statistics accumulators
+    int stats_warp;                      // bytes of one warp's accumulators: 512 per 64-channel chunk of the tile
     float *stats;                        // optional: per epilogue warp and channel, sum and sum of squares of the stored bf16
     void *out;
     unsigned int *status;
@@ -905,10 +905,10 @@ __global__ void __launch_bounds__(kHaloThreads, 1) conv_halo_kernel(const __grid
         const uint32_t slab = staging_base + (uint32_t)group * (uint32_t)p.staging;
         // statistics: one row of partial sums per epilogue warp of the grid, [2][ld_out] floats, accumulated over the warp's tiles
         float *my_stats = (STATS && p.stats) ? p.stats + ((size_t)blockIdx.x * 8 + (warp - 2)) * 2 * p.ld_out : nullptr;
-        const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * kStatsWarpBytes;
+        const uint32_t st_acc = smem_base + (uint32_t)p.stats_off + (uint32_t)(warp - 2) * (uint32_t)p.stats_warp;
         if (my_stats) {
             for (int e = lane; e < 2 * p.ld_out; e += 32) my_stats[e] = 0.f;
-            stats_clear(st_acc, lane);
+            stats_clear(st_acc, lane, (p.BN + 63) / 64);
             __syncwarp();
         }
         bool ok = true;
@@ -1877,7 +1877,8 @@ pt_status launch_gemm(pt_ctx *c, const CUtensorMap &tmA, const CUtensorMap &tmB,
     // accumulator is complete), which leaves room for one more stage
     p.alias_staging = (per_cta == 1 && !p.resident) ? 1 : 0;
     // statistics mode: the epilogue warps' accumulators sit at the end of the shared memory (taken from the ring's room)
-    const size_t st_smem = c->stats_mode ? (size_t)12 * kStatsWarpBytes : 0;
+    p.stats_warp = pt_ceil_div(p.BN, 64) * (int)kStatsChunkBytes;
+    const size_t st_smem = c->stats_mode ? (size_t)4 * p.epi_groups * p.stats_warp : 0;     // (the group count can only shrink below)
     size_t staging2 = p.alias_staging ? 0 : (size_t)p.epi_groups * 4 * kSlabs * 4096;
     if (p.resident) p.stages = pick_stages(a_bytes, p.taps * p.k_chunks * per_cta, staging2 + w_all + st_smem, &smem, kGemmSmemCap);
     else {
@@ -1987,7 +1988,8 @@ pt_status launch_halo(pt_ctx *c, const pt_conv_desc *d, const HaloSpec &h, const
     p.b_slot = (int)b_bytes;
     // epilogue staging: one slab of the tile's raster rows x 128 bytes per group (direct-store launches use none)
     p.staging = d->out_f32 ? 0 : (int)pt_align_up((size_t)(p.nr * Wp < 128 ? p.nr * Wp : 128) * 128, 1024);
-    const size_t st_smem = c->stats_mode ? (size_t)8 * kStatsWarpBytes : 0;     // statistics accumulators of the eight epilogue warps
+    p.stats_warp = pt_ceil_div(p.BN, 64) * (int)kStatsChunkBytes;
+    const size_t st_smem = c->stats_mode ? (size_t)8 * p.stats_warp : 0;        // statistics accumulators of the eight epilogue warps
     const size_t budget = 227 * 1024 - 2048 - 2 * (size_t)p.staging - a_tail - st_smem;
     const size_t w_all = (size_t)h.n_taps * p.k_chunks * b_bytes;
     p.resident = (p.n_tiles == 1 && w_all + 2 * (size_t)p.a_alloc <= budget) ? 1 : 0;

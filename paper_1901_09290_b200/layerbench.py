@@ -62,6 +62,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager launches (includes host launch cost)")
     ap.add_argument("--bn", default=None, help="N,H,C: time pt_bn_relu_fwd / pt_bn_relu_bwd instead of a convolution")
     ap.add_argument("--gate", default=None, help="N,H,C,S: time pt_channel_gather / pt_channel_scatter_add of S of a node's C channels")
+    ap.add_argument("--stats", action="store_true",
+                    help="the forward pass through pt_conv_fwd_stats (batch-norm statistics taken in the epilogue)")
     ap.add_argument("--model", action="store_true",
                     help="time detection, plan, gather, the lasso step and its carried form over the bench's ResNet-50 model "
                          "alone (batch 1 activations: ~0.7 GB on the device, the model itself larger than L2)")
@@ -95,13 +97,19 @@ def main():
         w = (torch.randn((K, R, R, d.ldw), generator=g, device="cuda") * (2.0 / (C * R * R)) ** 0.5).to(torch.bfloat16)
         sets.append((x, dy, w, torch.empty_like(dy), torch.empty_like(x), torch.empty((K, R, R, C), device="cuda")))
     ws = torch.empty(max(16, max(B.pt_conv_workspace_bytes(ctx, d, i) for i in range(3))), dtype=torch.uint8, device="cuda")
+    stats = None
+    if args.stats:
+        d.algo = 2                               # the statistics epilogue exists in the tcgen05 kernels only
+        stats = torch.empty(B.pt_conv_fwd_stats_bytes(ctx, d) // 4, dtype=torch.float32, device="cuda")
     flops = 2 * N * P * P * K * C * R * R
     act = N * H * H * C * 2 + N * P * P * K * 2
     out = {"layer": name, "N": N, "H": H, "C": C, "K": K, "R": R, "stride": stride}
     for ps in args.passes.split(","):
         def run(i):
             x, dy, w, y, dx, dw = sets[i % len(sets)]
-            if ps == "fwd":
+            if ps == "fwd" and stats is not None:
+                B.pt_conv_fwd_stats(ctx, d, x, w, y, stats, ws)
+            elif ps == "fwd":
                 B.pt_conv_fwd(ctx, d, x, w, y, ws)
             elif ps == "dgrad":
                 B.pt_conv_dgrad(ctx, d, dy, w, dx, ws)
