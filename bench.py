@@ -307,6 +307,17 @@ def run_ours(args):
             return first, 1
         return run(steps * r) / r, r
 
+    if args.profile_steps and args.profile_chained:
+        # the same for the chained step (convolutions + batch norm + pooling + residual adds, forward and backward)
+        from paper_1901_09290_b200 import harness
+        cs = harness.ChainedStep(ctx, ts.net, args.batch, seed + 5, fused_stats=True, algo=args.algo)
+        for _ in range(1 + args.profile_steps):
+            cs.step()
+            torch.cuda.synchronize()
+        ctx.poll()
+        if rank == 0:
+            print(json.dumps({"profile_steps": args.profile_steps, "step": "chained", "workload": name}))
+        return
     if args.profile_steps:
         # a short run for profilers: one warm-up step, then the requested steps, nothing else
         ts.step()
@@ -586,6 +597,7 @@ def main():
     ap.add_argument("--no-chained", action="store_true", help="skip the chained-step timing (conv + batch norm + pooling + residuals)")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel eagerly instead of replaying a CUDA graph")
     ap.add_argument("--one-stream", action="store_true", help="capture the step on one stream (no dgrad/wgrad overlap)")
+    ap.add_argument("--profile-chained", action="store_true", help="with --profile-steps: run the chained step instead")
     ap.add_argument("--profile-steps", type=int, default=0,
                     help="run only this many steps after one warm-up and print no timing: for a launch list (the one-pass "
                          "gpu__time_duration capture); captures with more metrics belong on a small case (layerbench, --net resnet32)")

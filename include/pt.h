@@ -235,13 +235,17 @@ pt_status pt_bn_relu_bwd(pt_ctx *ctx, const pt_bn_desc *d, const void *x, const 
  * [N][H][W][ld] bf16, 16-byte aligned, ld a multiple of 8; square window R, stride, padding pad < R; output
  * [N][P][Q][ld] with P = floor((H + 2*pad - R)/stride) + 1. Positions outside the image are never selected; of equal maxima the
  * first in scan order (rows, then columns of the window) is the selected one and receives the gradient. Pad lanes of the
- * outputs are written as zeros. The backward pass recomputes the selections from x (no index tensor) and adds nothing
- * atomically. PT_ERR_INVALID_ARG for bad sizes, pitches, alignment or null pointers.
+ * outputs are written as zeros. Nothing is added atomically. `index` (device, optional, 8-byte aligned, uint8
+ * [N][P][Q][ld], R*R <= 255): the forward pass leaves the selected position r*R + s of every window there (255: none, and in
+ * the pad lanes) and the backward pass reads it; with index = NULL the backward pass recomputes the selections from x (R*R
+ * loads per window instead of one). PT_ERR_INVALID_ARG for bad sizes, pitches, alignment or null pointers.
  * ------------------------------------------------------------------------------------------ */
 typedef struct { int32_t N, H, W, C, ld, R, stride, pad; } pt_pool_desc;
-pt_status pt_maxpool_fwd(pt_ctx *ctx, const pt_pool_desc *d, const void *x, void *y, void *stream);
-/* dx[n,h,w,c] = sum of dy[n,p,q,c] over the windows (p,q) whose selected position is (h,w); x is the forward input. */
-pt_status pt_maxpool_bwd(pt_ctx *ctx, const pt_pool_desc *d, const void *x, const void *dy, void *dx, void *stream);
+pt_status pt_maxpool_fwd(pt_ctx *ctx, const pt_pool_desc *d, const void *x, void *y, void *index, void *stream);
+/* dx[n,h,w,c] = sum of dy[n,p,q,c] over the windows (p,q) whose selected position is (h,w); x is the forward input (may be
+ * NULL when index is given). */
+pt_status pt_maxpool_bwd(pt_ctx *ctx, const pt_pool_desc *d, const void *x, const void *dy, const void *index, void *dx,
+                         void *stream);
 
 /* ------------------------------------------------------------------------------------------
  * Dynamic mini-batch adjustment (Sec. 4.3; Algorithm 1, "UpdateMiniBatch(system_memory, Net)"): after every reconfiguration

@@ -91,8 +91,8 @@ EXPORTS = {
                                     c_void_p, c_size_t, c_void_p]),
     "pt_bn_relu_fwd_stats": (c_int32, [c_void_p, POINTER(pt_bn_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
-    "pt_maxpool_fwd": (c_int32, [c_void_p, POINTER(pt_pool_desc), c_void_p, c_void_p, c_void_p]),
-    "pt_maxpool_bwd": (c_int32, [c_void_p, POINTER(pt_pool_desc), c_void_p, c_void_p, c_void_p, c_void_p]),
+    "pt_maxpool_fwd": (c_int32, [c_void_p, POINTER(pt_pool_desc), c_void_p, c_void_p, c_void_p, c_void_p]),
+    "pt_maxpool_bwd": (c_int32, [c_void_p, POINTER(pt_pool_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "pt_conv_dgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_conv_wgrad": (c_int32, [c_void_p, POINTER(pt_conv_desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "pt_group_lasso_workspace_bytes": (c_size_t, [c_void_p, POINTER(pt_layer), c_int32]),
@@ -350,12 +350,12 @@ def make_pool_desc(N, H, W, C, ld=None, R=3, stride=2, pad=1) -> pt_pool_desc:
     return pt_pool_desc(N, H, W, C, ld or (C + 7) // 8 * 8, R, stride, pad)
 
 
-def pt_maxpool_fwd(ctx, d, x, y, stream=None):
-    _check(lib().pt_maxpool_fwd(ctx.handle, byref(d), _ptr(x), _ptr(y), _stream(stream)), "pt_maxpool_fwd")
+def pt_maxpool_fwd(ctx, d, x, y, stream=None, index=None):
+    _check(lib().pt_maxpool_fwd(ctx.handle, byref(d), _ptr(x), _ptr(y), _ptr(index), _stream(stream)), "pt_maxpool_fwd")
 
 
-def pt_maxpool_bwd(ctx, d, x, dy, dx, stream=None):
-    _check(lib().pt_maxpool_bwd(ctx.handle, byref(d), _ptr(x), _ptr(dy), _ptr(dx), _stream(stream)), "pt_maxpool_bwd")
+def pt_maxpool_bwd(ctx, d, x, dy, dx, stream=None, index=None):
+    _check(lib().pt_maxpool_bwd(ctx.handle, byref(d), _ptr(x), _ptr(dy), _ptr(index), _ptr(dx), _stream(stream)), "pt_maxpool_bwd")
 
 
 def shape_array(shapes) -> "ctypes.Array":

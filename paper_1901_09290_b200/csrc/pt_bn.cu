@@ -133,6 +133,16 @@ __device__ __forceinline__ bool bn_sum_partials(const BnP &p, const float *__res
     double a0 = 0.0, a1 = 0.0;
     if (c < p.C) {
         int b = ty;
+        for (; b + 224 < p.blocks; b += 256) {           // sixteen loads in flight (the rows of a convolution's epilogue warps: up to 1776)
+            float v0[8], v1[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                v0[u] = partial[(size_t)(b + 32 * u) * 2 * p.ld + c];
+                v1[u] = partial[(size_t)(b + 32 * u) * 2 * p.ld + p.ld + c];
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { a0 += (double)v0[u]; a1 += (double)v1[u]; }
+        }
         for (; b + 96 < p.blocks; b += 128) {
             float v0[4], v1[4];
 #pragma unroll

@@ -605,6 +605,7 @@ class ChainedStep:
         self.stats = torch.empty(st_bytes // 4, dtype=torch.float32, device=dev)
         if self.pool:
             self.pooled = bf(N, first_h, self.ld[0])
+            self.pool_index = torch.empty((N, first_h, first_h, self.ld[0]), dtype=torch.uint8, device="cuda")   # selections of the forward pass
             self.d_pooled = bf(N, first_h, self.ld[0])
         # gradients with respect to activations: one buffer per distinct activation a convolution reads
         # gradient with respect to a convolution's INPUT (its data gradient), and with respect to the stem's activation
@@ -650,7 +651,7 @@ class ChainedStep:
     def forward(self, stream=None):
         cur = self._conv_bn(0, self.x0, None, stream)
         if self.pool:
-            B.pt_maxpool_fwd(self.ctx, self.pool_desc, cur, self.pooled, stream)
+            B.pt_maxpool_fwd(self.ctx, self.pool_desc, cur, self.pooled, stream, index=self.pool_index)
             cur = self.pooled
         self.block_in = []
         for main, ds, _ in self.blocks:
@@ -699,7 +700,7 @@ class ChainedStep:
             self._add(d_t, sc, self.da_tmp[key], Cin, ld_in, npix, stream)
             d_cur = self.da_tmp[key]
         if self.pool:
-            B.pt_maxpool_bwd(c, self.pool_desc, self.a[0], d_cur, self.d_a0, stream)
+            B.pt_maxpool_bwd(c, self.pool_desc, self.a[0], d_cur, self.d_a0, stream, index=self.pool_index)
             d_cur = self.d_a0
         self._bn_bwd(0, d_cur, None, stream)
         B.pt_conv_wgrad(c, self.desc[0], self.x0, self.dy[0], self.dm.g[0], self.ws, stream)
