@@ -124,47 +124,58 @@ __global__ void __launch_bounds__(kBnThreads) bn_reduce_kernel(const BnP p, cons
     }
 }
 
-// Sums the block partials of 32 channels per CTA: thread (tx, ty) adds the blocks ty, ty + 32, ... of channel tx in ascending
-// order in fp64, then the 32 slices are added in order (a chain of dependent L2 loads is what costs time here). Returns the two sums to the threads with ty == 0.
+// Sums the block partials of kFinC channels per CTA: thread (tx, ty) adds the rows ty, ty + kFinS, ... of channel tx in ascending
+// order in fp64 (eight loads in flight: a chain of dependent L2 loads is what costs time here), then the kFinS slices are added
+// in a fixed order in two steps. 8 channels x 128 slices: a convolution's epilogue warps leave up to 1776 rows, 14 per slice
+// (32 channels x 32 slices took 9 us per call, 55 rows per slice). Returns the two sums to the threads with ty == 0.
+constexpr int kFinC = 8, kFinS = 128;
 __device__ __forceinline__ bool bn_sum_partials(const BnP &p, const float *__restrict__ partial, int c, double &s0, double &s1)
 {
-    __shared__ double sh[2][32][32];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    __shared__ double sh[2][kFinS][kFinC];
+    __shared__ double sh2[2][16][kFinC];
+    const int tx = threadIdx.x & (kFinC - 1), ty = threadIdx.x / kFinC;
     double a0 = 0.0, a1 = 0.0;
     if (c < p.C) {
         int b = ty;
-        for (; b + 224 < p.blocks; b += 256) {           // sixteen loads in flight (the rows of a convolution's epilogue warps: up to 1776)
+        for (; b + 7 * kFinS < p.blocks; b += 8 * kFinS) {
             float v0[8], v1[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                v0[u] = partial[(size_t)(b + 32 * u) * 2 * p.ld + c];
-                v1[u] = partial[(size_t)(b + 32 * u) * 2 * p.ld + p.ld + c];
+                v0[u] = partial[(size_t)(b + kFinS * u) * 2 * p.ld + c];
+                v1[u] = partial[(size_t)(b + kFinS * u) * 2 * p.ld + p.ld + c];
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) { a0 += (double)v0[u]; a1 += (double)v1[u]; }
         }
-        for (; b + 96 < p.blocks; b += 128) {
-            float v0[4], v1[4];
+        {
+            // the remaining rows (fewer than eight): loaded together, added in the same ascending order
+            float v0[8], v1[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                v0[u] = partial[(size_t)(b + 32 * u) * 2 * p.ld + c];
-                v1[u] = partial[(size_t)(b + 32 * u) * 2 * p.ld + p.ld + c];
+            for (int u = 0; u < 8; ++u) {
+                const int bb = b + kFinS * u;
+                v0[u] = bb < p.blocks ? partial[(size_t)bb * 2 * p.ld + c] : 0.f;
+                v1[u] = bb < p.blocks ? partial[(size_t)bb * 2 * p.ld + p.ld + c] : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { a0 += (double)v0[u]; a1 += (double)v1[u]; }
-        }
-        for (; b < p.blocks; b += 32) {
-            a0 += (double)partial[(size_t)b * 2 * p.ld + c];
-            a1 += (double)partial[(size_t)b * 2 * p.ld + p.ld + c];
+            for (int u = 0; u < 8; ++u)
+                if (b + kFinS * u < p.blocks) { a0 += (double)v0[u]; a1 += (double)v1[u]; }
         }
     }
     sh[0][ty][tx] = a0;
     sh[1][ty][tx] = a1;
     __syncthreads();
+    if (ty < 16) {
+        double t0 = 0.0, t1 = 0.0;
+#pragma unroll
+        for (int r = 0; r < kFinS / 16; ++r) { t0 += sh[0][ty * (kFinS / 16) + r][tx]; t1 += sh[1][ty * (kFinS / 16) + r][tx]; }
+        sh2[0][ty][tx] = t0;
+        sh2[1][ty][tx] = t1;
+    }
+    __syncthreads();
     if (ty != 0 || c >= p.C) return false;
     s0 = 0.0; s1 = 0.0;
 #pragma unroll
-    for (int r = 0; r < 32; ++r) { s0 += sh[0][r][tx]; s1 += sh[1][r][tx]; }
+    for (int r = 0; r < 16; ++r) { s0 += sh2[0][r][tx]; s1 += sh2[1][r][tx]; }
     return true;
 }
 
@@ -172,7 +183,7 @@ __global__ void __launch_bounds__(1024) bn_fwd_finish_kernel(const BnP p, const 
                                                             float *__restrict__ save_mean, float *__restrict__ save_invstd,
                                                             float *__restrict__ running_mean, float *__restrict__ running_var)
 {
-    const int c = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int c = blockIdx.x * kFinC + (threadIdx.x & (kFinC - 1));
     double s0, s1;
     if (!bn_sum_partials(p, partial, c, s0, s1)) return;
     const double M = (double)p.M;
@@ -192,7 +203,7 @@ __global__ void __launch_bounds__(1024) bn_fwd_finish_kernel(const BnP p, const 
 __global__ void __launch_bounds__(1024) bn_bwd_finish_kernel(const BnP p, const float *__restrict__ partial, float *__restrict__ dgamma,
                                                             float *__restrict__ dbeta)
 {
-    const int c = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int c = blockIdx.x * kFinC + (threadIdx.x & (kFinC - 1));
     double s0, s1;
     if (!bn_sum_partials(p, partial, c, s0, s1)) return;
     dbeta[c] = (float)s0;
@@ -323,7 +334,7 @@ extern "C" pt_status pt_bn_relu_fwd(pt_ctx *c, const pt_bn_desc *d, const void *
     cudaStream_t st = (cudaStream_t)stream;
     float *partial = (float *)ws;
     bn_reduce_kernel<0><<<p.blocks, kBnThreads, 0, st>>>(p, (const uint4 *)x, nullptr, nullptr, nullptr, nullptr, partial);
-    bn_fwd_finish_kernel<<<pt_ceil_div(p.C, 32), 1024, 0, st>>>(p, (const __nv_bfloat16 *)x, partial, save_mean, save_invstd, running_mean,
+    bn_fwd_finish_kernel<<<pt_ceil_div(p.C, kFinC), kFinC * kFinS, 0, st>>>(p, (const __nv_bfloat16 *)x, partial, save_mean, save_invstd, running_mean,
                                                                running_var);
     bn_apply_kernel<0><<<p.blocks, kBnThreads, 0, st>>>(p, (const uint4 *)x, nullptr, (const uint4 *)residual, gamma, beta, save_mean,
                                                         save_invstd, nullptr, nullptr, (uint4 *)y, nullptr);
@@ -347,7 +358,7 @@ extern "C" pt_status pt_bn_relu_bwd(pt_ctx *c, const pt_bn_desc *d, const void *
     float *partial = (float *)ws;
     const uint4 *yv = (const uint4 *)(y ? y : dy);          // without ReLU the mask input is never looked at
     bn_reduce_kernel<1><<<p.blocks, kBnThreads, 0, st>>>(p, (const uint4 *)x, yv, (const uint4 *)dy, save_mean, save_invstd, partial);
-    bn_bwd_finish_kernel<<<pt_ceil_div(p.C, 32), 1024, 0, st>>>(p, partial, dgamma, dbeta);
+    bn_bwd_finish_kernel<<<pt_ceil_div(p.C, kFinC), kFinC * kFinS, 0, st>>>(p, partial, dgamma, dbeta);
     bn_apply_kernel<1><<<p.blocks, kBnThreads, 0, st>>>(p, (const uint4 *)x, yv, (const uint4 *)dy, gamma, nullptr, save_mean, save_invstd,
                                                         dgamma, dbeta, (uint4 *)dx, (uint4 *)dresidual);
     c->launches += 3;
@@ -371,7 +382,7 @@ extern "C" pt_status pt_bn_relu_fwd_stats(pt_ctx *c, const pt_bn_desc *d, const 
     cudaStream_t st = (cudaStream_t)stream;
     BnP pf = p;
     pf.blocks = n_parts;                            // rows of [2][ld] partial sums, taken about 0
-    bn_fwd_finish_kernel<<<pt_ceil_div(p.C, 32), 1024, 0, st>>>(pf, nullptr, stats, save_mean, save_invstd, running_mean, running_var);
+    bn_fwd_finish_kernel<<<pt_ceil_div(p.C, kFinC), kFinC * kFinS, 0, st>>>(pf, nullptr, stats, save_mean, save_invstd, running_mean, running_var);
     bn_apply_kernel<0><<<p.blocks, kBnThreads, 0, st>>>(p, (const uint4 *)x, nullptr, (const uint4 *)residual, gamma, beta, save_mean,
                                                         save_invstd, nullptr, nullptr, (uint4 *)y, nullptr);
     c->launches += 2;
