@@ -218,8 +218,8 @@ def chained_step_times(ctx, ts, args, seed):
     import torch
     from paper_1901_09290_b200 import harness
     res = {}
-    for fused in (True, False):
-        cs = harness.ChainedStep(ctx, ts.net, args.batch, seed + 5, fused_stats=fused, algo=args.algo)
+    for fused, ws_n, key in ((True, 2, "fused_statistics"), (False, 2, "stand_alone_normalisation"), (True, 0, "fused_statistics_one_stream")):
+        cs = harness.ChainedStep(ctx, ts.net, args.batch, seed + 5, fused_stats=fused, algo=args.algo, wgrad_streams=ws_n)
         cs.step()
         torch.cuda.synchronize()
         l0 = ctx.launch_count()
@@ -239,13 +239,13 @@ def chained_step_times(ctx, ts, args, seed):
         torch.cuda.synchronize()
         ctx.poll()
         ms = a.elapsed_time(b) / n
-        res["fused_statistics" if fused else "stand_alone_normalisation"] = {
+        res[key] = {
             "ms_per_step": ms, "launches": launches, "conv_tflops_over_step": cs.conv_flops() / (ms * 1e-3) / 1e12}
         del cs, g
         torch.cuda.empty_cache()
     ctx.set_wgrad_cta_limit(ts.wgrad_ctas)
     res["note"] = ("53 convolutions each followed by batch norm (training statistics) + ReLU, 3x3/2 max pooling after the stem, 16 "
-                   "residual adds, backward to every weight / gamma / beta gradient, lasso step; one stream, CUDA graph replay")
+                   "residual adds, backward to every weight / gamma / beta gradient, lasso step; CUDA graph replay; the weight gradients on two side streams beside the backward chain (one stream in the third entry)")
     return res
 
 

@@ -541,9 +541,14 @@ class ChainedStep:
 
     def __init__(self, ctx: B.Context, net: W.Net, N: int, seed: int, fused_stats: bool = True, algo: int = 0,
                  max_blocks: Optional[int] = None, model: Optional[W.Model] = None, x0: Optional[torch.Tensor] = None,
-                 g_last: Optional[torch.Tensor] = None):
+                 g_last: Optional[torch.Tensor] = None, wgrad_streams: int = 0):
         self.ctx, self.net, self.N, self.fused = ctx, net, N, fused_stats
-        ctx.set_wgrad_cta_limit(0)                      # one stream: every weight gradient may take all SMs (sizes the workspaces)
+        # wgrad_streams > 0: a layer's weight gradient needs only its input and dy, so it goes to a side stream (round robin,
+        # a workspace each) and runs beside the rest of the backward chain; the launches are held to SMs / streams CTAs so
+        # that the split ones, whose CTAs wait for one another, always fit on the device together
+        self.wgrad_streams = wgrad_streams
+        self.wgrad_limit = 0 if wgrad_streams <= 0 else max(1, 148 // wgrad_streams)
+        ctx.set_wgrad_cta_limit(self.wgrad_limit)       # sizes the workspaces (0: one stream, every weight gradient may take all SMs)
         names = [l.name for l in net.layers]
         self.blocks = []                                   # (main conv indices, shortcut index or None)
         for i, nm in enumerate(names):
@@ -601,6 +606,9 @@ class ChainedStep:
             ws_bn = max(ws_bn, B.pt_bn_workspace_bytes(ctx, self.bn_desc[i]))
         self.last_of = last_of
         self.ws = torch.empty(ws_conv, dtype=torch.uint8, device=dev)
+        self.ws_side = [torch.empty(ws_conv, dtype=torch.uint8, device=dev) for _ in range(max(0, wgrad_streams))]
+        self._side = [torch.cuda.Stream() for _ in range(max(0, wgrad_streams))]
+        self._wi = 0
         self.ws_bn = torch.empty(ws_bn, dtype=torch.uint8, device=dev)
         self.stats = torch.empty(st_bytes // 4, dtype=torch.float32, device=dev)
         if self.pool:
@@ -667,8 +675,21 @@ class ChainedStep:
         B.pt_bn_relu_bwd(self.ctx, self.bn_desc[i], self.y[i], self.a[i], d_out, self.gamma[i], self.sm[i], self.si[i], self.dy[i], dres,
                          self.dg[i], self.db[i], self.ws_bn, stream)
 
+    def _wgrad(self, i, x_i, stream):
+        """The weight gradient of layer i: on the caller's stream, or on the next side stream once that stream has dy_i."""
+        if not self._side:
+            B.pt_conv_wgrad(self.ctx, self.desc[i], x_i, self.dy[i], self.dm.g[i], self.ws, stream)
+            return
+        main = stream if stream is not None else torch.cuda.current_stream()
+        k = self._wi % len(self._side)
+        self._wi += 1
+        side = self._side[k]
+        side.wait_stream(main)
+        B.pt_conv_wgrad(self.ctx, self.desc[i], x_i, self.dy[i], self.dm.g[i], self.ws_side[k], side)
+
     def backward(self, stream=None):
         c, L = self.ctx, self.net.layers
+        self._wi = 0
         d_cur = self.g_last                                   # gradient w.r.t. the current block's output
         for bi in range(len(self.blocks) - 1, -1, -1):
             main, ds, _ = self.blocks[bi]
@@ -681,7 +702,7 @@ class ChainedStep:
                 x_i = x_in if k == 0 else self.a[main[k - 1]]
                 if k < len(main) - 1:
                     self._bn_bwd(i, d_t, None, stream)
-                B.pt_conv_wgrad(c, self.desc[i], x_i, self.dy[i], self.dm.g[i], self.ws, stream)
+                self._wgrad(i, x_i, stream)
                 d_t = self.da[i]
                 B.pt_conv_dgrad(c, self.desc[i], self.dy[i], self.dm.wb[i], d_t, self.ws, stream)
             # d_t: gradient w.r.t. the block input through the main branch; the shortcut adds its own
@@ -689,7 +710,7 @@ class ChainedStep:
             npix, Cin, ld_in = self.N * li.H * li.H, li.C, W.pad16(li.C)
             if ds is not None:
                 self._bn_bwd(ds, self.dres[last], None, stream)
-                B.pt_conv_wgrad(c, self.desc[ds], x_in, self.dy[ds], self.dm.g[ds], self.ws, stream)
+                self._wgrad(ds, x_in, stream)
                 B.pt_conv_dgrad(c, self.desc[ds], self.dy[ds], self.dm.wb[ds], self.da[ds], self.ws, stream)
                 sc = self.da[ds]
             else:
@@ -703,13 +724,16 @@ class ChainedStep:
             B.pt_maxpool_bwd(c, self.pool_desc, self.a[0], d_cur, self.d_a0, stream, index=self.pool_index)
             d_cur = self.d_a0
         self._bn_bwd(0, d_cur, None, stream)
-        B.pt_conv_wgrad(c, self.desc[0], self.x0, self.dy[0], self.dm.g[0], self.ws, stream)
+        self._wgrad(0, self.x0, stream)
+        main = stream if stream is not None else torch.cuda.current_stream()
+        for side in self._side:
+            main.wait_stream(side)                        # the update needs every weight gradient
 
     def update(self, stream=None, lam=1e-4, lr=0.1, mu=0.9):
         B.pt_group_lasso_sgd_step(self.ctx, self.dm.arr, lam, lr, mu, 0.0, self.dm.reg, self.dm.ws, stream)
 
     def step(self, stream=None):
-        self.ctx.set_wgrad_cta_limit(0)               # one stream: every weight gradient may take all SMs
+        self.ctx.set_wgrad_cta_limit(self.wgrad_limit)
         self.forward(stream)
         self.backward(stream)
         self.update(stream)
