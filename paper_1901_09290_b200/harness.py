@@ -609,6 +609,12 @@ class ChainedStep:
         self.ws_side = [torch.empty(ws_conv, dtype=torch.uint8, device=dev) for _ in range(max(0, wgrad_streams))]
         self._side = [torch.cuda.Stream() for _ in range(max(0, wgrad_streams))]
         self._wi = 0
+        # in the same mode a block's projection shortcut (convolution + batch norm) runs on a stream of its own beside the block's
+        # main branch, in both directions, with workspaces of its own
+        self._aux = torch.cuda.Stream() if wgrad_streams > 0 else None
+        self.ws_aux = torch.empty(ws_conv, dtype=torch.uint8, device=dev) if self._aux else None
+        self.ws_bn_aux = torch.empty(ws_bn, dtype=torch.uint8, device=dev) if self._aux else None
+        self.stats_aux = torch.empty(st_bytes // 4, dtype=torch.float32, device=dev) if self._aux else None
         self.ws_bn = torch.empty(ws_bn, dtype=torch.uint8, device=dev)
         self.stats = torch.empty(st_bytes // 4, dtype=torch.float32, device=dev)
         if self.pool:
@@ -643,16 +649,17 @@ class ChainedStep:
         """out = a + b (bf16, one rounding) through the scatter-add with the identity selection."""
         B.pt_channel_scatter_add(self.ctx, b, ld, self._arange(C), C, a, out, ld, C, npix, False, stream)
 
-    def _conv_bn(self, i, x, residual=None, stream=None):
+    def _conv_bn(self, i, x, residual=None, stream=None, aux=False):
         c = self.ctx
+        ws, ws_bn, stats = (self.ws_aux, self.ws_bn_aux, self.stats_aux) if aux else (self.ws, self.ws_bn, self.stats)
         if self.fused:
-            n_parts = B.pt_conv_fwd_stats(c, self.desc[i], x, self.dm.wb[i], self.y[i], self.stats, self.ws, stream)
+            n_parts = B.pt_conv_fwd_stats(c, self.desc[i], x, self.dm.wb[i], self.y[i], stats, ws, stream)
             B.pt_bn_relu_fwd_stats(c, self.bn_desc[i], self.y[i], residual, self.gamma[i], self.beta[i], None, None, self.sm[i], self.si[i],
-                                   self.a[i], self.stats, n_parts, stream)
+                                   self.a[i], stats, n_parts, stream)
         else:
-            B.pt_conv_fwd(c, self.desc[i], x, self.dm.wb[i], self.y[i], self.ws, stream)
+            B.pt_conv_fwd(c, self.desc[i], x, self.dm.wb[i], self.y[i], ws, stream)
             B.pt_bn_relu_fwd(c, self.bn_desc[i], self.y[i], residual, self.gamma[i], self.beta[i], None, None, self.sm[i], self.si[i],
-                             self.a[i], self.ws_bn, stream)
+                             self.a[i], ws_bn, stream)
         return self.a[i]
 
     # ---- the chain
@@ -664,16 +671,24 @@ class ChainedStep:
         self.block_in = []
         for main, ds, _ in self.blocks:
             self.block_in.append(cur)
-            res = self._conv_bn(ds, cur, None, stream) if ds is not None else cur
+            side = self._aux if ds is not None else None
+            ms = stream if stream is not None else torch.cuda.current_stream()
+            if side is not None:
+                side.wait_stream(ms)
+                res = self._conv_bn(ds, cur, None, side, aux=True)
+            else:
+                res = self._conv_bn(ds, cur, None, stream) if ds is not None else cur
             t = cur
             for i in main[:-1]:
                 t = self._conv_bn(i, t, None, stream)
+            if side is not None:
+                ms.wait_stream(side)                      # the block's last batch norm adds the shortcut
             cur = self._conv_bn(main[-1], t, res, stream)
         return cur
 
-    def _bn_bwd(self, i, d_out, dres, stream=None):
+    def _bn_bwd(self, i, d_out, dres, stream=None, aux=False):
         B.pt_bn_relu_bwd(self.ctx, self.bn_desc[i], self.y[i], self.a[i], d_out, self.gamma[i], self.sm[i], self.si[i], self.dy[i], dres,
-                         self.dg[i], self.db[i], self.ws_bn, stream)
+                         self.dg[i], self.db[i], self.ws_bn_aux if aux else self.ws_bn, stream)
 
     def _wgrad(self, i, x_i, stream):
         """The weight gradient of layer i: on the caller's stream, or on the next side stream once that stream has dy_i."""
@@ -696,6 +711,14 @@ class ChainedStep:
             x_in = self.block_in[bi]
             last = main[-1]
             self._bn_bwd(last, d_cur, self.dres[last], stream)
+            ms = stream if stream is not None else torch.cuda.current_stream()
+            side = self._aux if ds is not None else None
+            if side is not None:
+                # the shortcut's backward (batch norm, weight and data gradient) beside the main branch's
+                side.wait_stream(ms)
+                self._bn_bwd(ds, self.dres[last], None, side, aux=True)
+                self._wgrad(ds, x_in, side)
+                B.pt_conv_dgrad(c, self.desc[ds], self.dy[ds], self.dm.wb[ds], self.da[ds], self.ws_aux, side)
             d_t = None
             for k in range(len(main) - 1, -1, -1):
                 i = main[k]
@@ -708,7 +731,10 @@ class ChainedStep:
             # d_t: gradient w.r.t. the block input through the main branch; the shortcut adds its own
             li = L[main[0]]
             npix, Cin, ld_in = self.N * li.H * li.H, li.C, W.pad16(li.C)
-            if ds is not None:
+            if side is not None:
+                ms.wait_stream(side)
+                sc = self.da[ds]
+            elif ds is not None:
                 self._bn_bwd(ds, self.dres[last], None, stream)
                 self._wgrad(ds, x_in, stream)
                 B.pt_conv_dgrad(c, self.desc[ds], self.dy[ds], self.dm.wb[ds], self.da[ds], self.ws, stream)

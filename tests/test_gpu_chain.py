@@ -232,11 +232,12 @@ def _oracle_chain(cs, model, x0, g_last):
     return out, dw, dgm, dbt
 
 
-@pytest.mark.parametrize("fused", [True, False])
-def test_chained_stage_stem_pool_and_three_blocks(fused):
+@pytest.mark.parametrize("fused,streams", [(True, 0), (False, 0), (True, 2)], ids=["fused", "stand-alone", "fused-side-streams"])
+def test_chained_stage_stem_pool_and_three_blocks(fused, streams):
     """Stem, max pooling and the whole first stage of a pruned ResNet-50 (a projection-shortcut block and two identity blocks),
     forward and backward, through the chained step -- with the normalisation statistics taken in the convolution epilogues
-    and with the stand-alone normalisation -- against the oracle's composition."""
+    and with the stand-alone normalisation, on one stream and with the weight gradients and the projection shortcut on side
+    streams -- against the oracle's composition."""
     from paper_1901_09290_b200 import harness
     c = Hh.ctx()
     N = 4
@@ -247,7 +248,7 @@ def test_chained_stage_stem_pool_and_three_blocks(fused):
     l0 = net.layers[0]
     x0 = _r(W.gen_image(N, l0.H, l0.H, l0.C, seed + 1).numpy())
     cs = harness.ChainedStep(c, net, N, seed, fused_stats=fused, algo=2, max_blocks=3, model=model,
-                             x0=torch.from_numpy(x0.astype(np.float32)))
+                             x0=torch.from_numpy(x0.astype(np.float32)), wgrad_streams=streams)
     lo = net.layers[cs.out_index]
     g_last = _r(W.gen_dy(N, lo.P, lo.P, lo.K, seed + 2).numpy() * 64)
     cs.g_last.zero_()
@@ -256,6 +257,7 @@ def test_chained_stage_stem_pool_and_three_blocks(fused):
     cs.backward()
     torch.cuda.synchronize()
     c.poll()
+    c.set_wgrad_cta_limit(0)                                 # the context is shared with the other tests
     out, dw, dgm, dbt = _oracle_chain(cs, model, x0, g_last)
     f = lambda t, C: t.float().cpu().numpy()[..., :C].astype(np.float64)
     assert _rel(f(out_d, lo.K), out) < 1e-2
