@@ -226,7 +226,9 @@ __global__ void __launch_bounds__(kThreads) finish_kernel(const LayerDev *__rest
                 const int np = L.RS * L.n_cb;                             // one partial per (line, column block)
                 const float *p = linesum + L.line_off + (long long)i * np;
                 float s = 0.f;
-#pragma unroll 4
+                // (a thread's partials are consecutive, the lanes' are np apart: every load is a round trip to L2, so many are
+                // kept in flight; a 3x3 layer has 9 to 72 of them, the 7x7 stem 49)
+#pragma unroll 16
                 for (int e = 0; e < np; ++e) s += p[e];                   // fixed order
                 L.sumsq_out[i] = s;
                 inv_out[L.k_off + i] = (L.reg_out && s > 1e-24f) ? rsqrtf(s) : 0.f;
@@ -236,7 +238,7 @@ __global__ void __launch_bounds__(kThreads) finish_kernel(const LayerDev *__rest
                 const int np = L.RS * L.n_cb;
                 const unsigned *p = linemax + L.line_off + (long long)i * np;
                 unsigned m = 0u;
-#pragma unroll 4
+#pragma unroll 16
                 for (int e = 0; e < np; ++e) m = max(m, p[e]);
                 if (flags & 2) gmax_out[L.k_off + i] = m;
                 if (flags & 4) L.zero_out[i] = (__uint_as_float(m) < thr) ? 1 : 0;
