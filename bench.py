@@ -591,7 +591,8 @@ def main():
     ap.add_argument("--wgrad-ctas", type=int, default=49, help="CTA limit of a weight-gradient launch")
     ap.add_argument("--wgrad-streams", type=int, default=3,
                     help="streams the weight gradients go round-robin on; streams x CTA limit must not exceed the SM count")
-    ap.add_argument("--algo", type=int, default=0)
+    ap.add_argument("--algo", type=int, default=2,
+                    help="2 (default): the tcgen05 kernels only, a shape they decline is an error; 0: fall back to the CUDA-core kernels; 1: CUDA-core kernels")
     ap.add_argument("--per-layer", default=None, help="write the per-layer table (JSON) here")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chained", action="store_true", help="skip the chained-step timing (conv + batch norm + pooling + residuals)")
