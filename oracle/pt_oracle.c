@@ -21,7 +21,7 @@
  *   group-lasso regulariser          Eq. 1, Eq. 2
  *   optimiser                        Algorithm 1 (Optimizer step), momentum SGD
  *   threshold zeroing                Sec. 4.1 ("threshold of 1e-4"), Sec. 4.2 / Fig. 4 (max-abs per channel)
- *   gather of surviving channels     Sec. 4.2 ("training variables of the remaining channels are kept as is")
+ *   gather of surviving channels     Sec. 4.2 (the surviving channels keep their weights and momentum unchanged)
  *
  * Parity pins: every function below is pinned by tests/test_oracle_*.py
  * (closed forms, adjoint identities, finite differences, hand examples,
