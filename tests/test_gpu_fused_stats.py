@@ -116,3 +116,40 @@ def test_statistics_are_run_to_run_identical_and_refuse_what_they_cannot_serve()
     assert e.value.status == 2                                   # fp32 outputs: PT_ERR_UNSUPPORTED
     torch.cuda.synchronize()
     c.poll()
+
+
+def test_every_layer_of_the_bench_workload_at_full_size():
+    """All 53 layers of the pruned ResNet-50 at batch 64 (the launch shapes of the chained bench step): the forward with the
+    statistics epilogue stores bit for bit what the plain forward stores (which the network tests hold against the oracle at
+    this size), and its rows of partial sums add up to the sums of those stored values."""
+    c = Hh.ctx()
+    net = W.resnet50()
+    seed = W.BASE_SEED + 4
+    counts = W.staged_keep_to_flops(net, seed, 0.60)
+    netp = W.with_sizes(net, counts)
+    N = 64
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    for li, l in enumerate(netp.layers):
+        ldx, ldy = (8 if l.C <= 4 else W.pad16(l.C)), W.pad16(l.K)
+        d = B.make_conv_desc(N, l.H, l.H, l.C, l.K, l.R, l.R, l.stride, l.pad, ldx, ldy, W.pad8(l.C), 0, 2)
+        x = torch.randn((N, l.H, l.H, ldx), generator=g, device="cuda")
+        if li:
+            x.clamp_(min=0)
+        x = x.to(torch.bfloat16)
+        w = (torch.randn((l.K, l.R, l.R, W.pad8(l.C)), generator=g, device="cuda") * (2.0 / (l.C * l.R * l.R)) ** 0.5).to(torch.bfloat16)
+        y = torch.full((N, l.P, l.P, ldy), 7680.0, dtype=torch.bfloat16, device="cuda")
+        y2 = torch.full_like(y, 7680.0)
+        stats = torch.full((B.pt_conv_fwd_stats_bytes(c, d) // 4,), float("nan"), dtype=torch.float32, device="cuda")
+        ws = Hh.conv_ws(d, B.PT_CONV_FWD)
+        n_parts = B.pt_conv_fwd_stats(c, d, x, w, y, stats, ws)
+        B.pt_conv_fwd(c, d, x, w, y2, ws)
+        torch.cuda.synchronize()
+        c.poll()
+        assert torch.equal(y[..., :l.K], y2[..., :l.K]), l.name
+        st = stats[: n_parts * 2 * ldy].view(n_parts, 2, ldy).double().sum(dim=0).cpu().numpy()
+        ys = y[..., :l.K].reshape(-1, l.K).float().cpu().numpy().astype(np.float64)
+        s0, s1 = ys.sum(axis=0), (ys ** 2).sum(axis=0)
+        assert np.allclose(st[0, :l.K], s0, rtol=2e-5, atol=2e-5 * np.abs(ys).sum(axis=0).max()), l.name
+        assert np.allclose(st[1, :l.K], s1, rtol=2e-5), l.name
+        assert np.all(st[:, l.K:] == 0), l.name
+        del x, w, y, y2, stats
