@@ -274,3 +274,39 @@ def test_chained_stage_stem_pool_and_three_blocks(fused, streams):
     cs.update()
     torch.cuda.synchronize()
     c.poll()
+
+
+def test_chained_step_at_bench_size_is_the_same_on_side_streams():
+    """The whole pruned ResNet-50 at batch 64 as the bench chains it: with the weight gradients and the projection shortcuts on
+    side streams every result must be what it is on one stream (a missing dependency between the streams would show as a
+    difference): activations, data gradients, gamma/beta gradients bit for bit (the same launches); weight gradients to
+    rounding (their CTA limit, hence the split of their sums, differs between the two modes) and bit for bit between two runs
+    of the same mode."""
+    from paper_1901_09290_b200 import harness
+    c = Hh.ctx()
+    net = W.resnet50()
+    seed = W.BASE_SEED + 4
+    netp = W.with_sizes(net, W.staged_keep_to_flops(net, seed, 0.60))
+    model = W.gen_model(netp, seed + 5)
+    runs = []
+    for streams in (0, 2, 2):
+        cs = harness.ChainedStep(c, netp, 64, seed + 5, fused_stats=True, algo=2, model=model, wgrad_streams=streams)
+        out = cs.forward()
+        cs.backward()
+        torch.cuda.synchronize()
+        c.poll()
+        runs.append(dict(out=out.clone(), dw=[cs.dm.g[i].clone() for i in cs.used], dg=[cs.dg[i].clone() for i in cs.used],
+                         db=[cs.db[i].clone() for i in cs.used], dy0=cs.dy[0].clone()))
+        del cs
+        torch.cuda.empty_cache()
+    c.set_wgrad_cta_limit(0)
+    one, a, b = runs
+    for r in (a, b):
+        assert torch.equal(r["out"], one["out"]) and torch.equal(r["dy0"], one["dy0"])
+        for x, y in zip(r["dg"] + r["db"], one["dg"] + one["db"]):
+            assert torch.equal(x, y)
+        for x, y in zip(r["dw"], one["dw"]):
+            scale = float(y.abs().max()) + 1e-30
+            assert float((x - y).abs().max()) <= 2e-4 * scale           # fp32 sums over up to 800 K pixels, split differently
+    for x, y in zip(a["dw"], b["dw"]):
+        assert torch.equal(x, y)
