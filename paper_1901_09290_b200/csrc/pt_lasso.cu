@@ -47,8 +47,10 @@ struct WsLayout { size_t linesum, colpart, linemax, colmax, inv_out, inv_in, gma
 
 constexpr int kThreads = 256;
 constexpr int kUnroll = 8;                // lines in flight per thread
-constexpr int kSweeps = 8;                // unrolled sweeps per chunk (16384 thread slots; 4 measured 4 % slower, 16 and more slower again)
-constexpr int kUpdateSplit = 4;           // blocks per chunk in the plain update
+constexpr int kSweeps = 8;                // unrolled sweeps per chunk of a large model (16384 thread slots; 4 measured 4 % slower, 16 slower again)
+constexpr int kSweepsSmall = 4;           // ... of a model with fewer than kSmallModel parameters (more, smaller blocks: 8 measured 7-10 % slower there)
+constexpr long long kSmallModel = 12ll << 20;
+// The plain update has no per-chunk results to combine: sweeps / 2 blocks share a chunk (two sweeps each).
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -90,10 +92,10 @@ __global__ void __launch_bounds__(kThreads) sweep_kernel(const LayerDev *__restr
                                                          const float *__restrict__ inv_out, const float *__restrict__ inv_in,
                                                          pt_sgd_hparams hp, float *__restrict__ linesum, float *__restrict__ colpart,
                                                          unsigned *__restrict__ linemax, unsigned *__restrict__ colmax,
-                                                         unsigned *__restrict__ ticket)
+                                                         unsigned *__restrict__ ticket, int split)
 {
     constexpr bool RED = SUM || MAX;
-    constexpr int SPLIT = RED ? 1 : kUpdateSplit;      // the plain update has no per-chunk results: kUpdateSplit blocks share a chunk
+    const int SPLIT = RED ? 1 : split;                 // the plain update has no per-chunk results: `split` blocks share a chunk
     __shared__ float s_col[RED ? kThreads : 1];
     __shared__ unsigned s_colm[MAX ? kThreads : 1];
     __shared__ float s_line[SUM ? 2 * kThreads : 1];       // [line in chunk][warp along the line]: at most 64 lines per TY x 8 warps
@@ -354,6 +356,7 @@ struct Tables {
     std::vector<int> first_chunk;          // per layer
     std::vector<FinishJob> jobs;
     WsLayout ws;
+    int sweeps = kSweeps;                  // base sweeps per chunk of this model; the plain update runs sweeps / 2 blocks per chunk
 };
 
 pt_status build_tables(const pt_layer *layers, int n, Tables *t)
@@ -364,6 +367,9 @@ pt_status build_tables(const pt_layer *layers, int n, Tables *t)
     t->chunks.clear();
     t->jobs.clear();
     long long line_off = 0, col_off = 0, k_off = 0, c_off = 0;
+    long long params = 0;
+    for (int i = 0; i < n; ++i) params += (long long)layers[i].K * layers[i].RS * layers[i].C;
+    t->sweeps = params >= kSmallModel ? kSweeps : kSweepsSmall;
     for (int i = 0; i < n; ++i) {
         const pt_layer &s = layers[i];
         if (!s.w || !s.v || s.K <= 0 || s.C <= 0 || s.RS <= 0) return PT_ERR_INVALID_ARG;
@@ -386,9 +392,9 @@ pt_status build_tables(const pt_layer *layers, int n, Tables *t)
         d.tx_log2 = lg;
         const int TX = 1 << lg, TY = kThreads / TX;
         const int lines = s.K * s.RS;
-        // a chunk is TY*kUnroll*sweeps lines x TX columns; sweeps = 8 (16384 thread slots: the most the line staging holds), so that no
-        // column has more than ~32 chunk partials to add up in the finish (the line staging holds at most 512 entries)
-        int sweeps = kSweeps;
+        // a chunk is TY*kUnroll*sweeps lines x TX columns; sweeps = 8 or 4 by the model's size (at most 8: the line staging
+        // holds 512 entries), more than the base for tall tensors so that no column has more than ~32 chunk partials to add up
+        int sweeps = t->sweeps;
         while (sweeps < 8 && lines > 32 * TY * kUnroll * sweeps) sweeps *= 2;
         const int lines_per_chunk = TY * kUnroll * sweeps;
         d.n_cb = pt_ceil_div(s.C, TX);
@@ -524,7 +530,7 @@ static pt_status lasso_phases(pt_ctx *c, const pt_layer *layers, int32_t n, cons
     memset(&none, 0, sizeof(none));
     if (phases & 1) {
         PT_CUDA_OK(launch_pdl(sweep_kernel<false, true, false>, nch, kThreads, st, b.dl, b.dc, (const float *)b.inv_out,
-                              (const float *)b.inv_in, none, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket));
+                              (const float *)b.inv_in, none, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket, 1));
         c->launches += 1;
         s = launch_finish(c, b, nj, reg_sum_out, 1, 0.f, st);
         if (s != PT_OK) return s;
@@ -538,14 +544,14 @@ static pt_status lasso_phases(pt_ctx *c, const pt_layer *layers, int32_t n, cons
         if (c1 > c0) {
             if ((phases & 4) && (phases & 8))
                 PT_CUDA_OK(launch_pdl(sweep_kernel<true, true, true>, c1 - c0, kThreads, st, b.dl, b.dc + c0, (const float *)b.inv_out,
-                                      (const float *)b.inv_in, *hp, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket));
+                                      (const float *)b.inv_in, *hp, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket, 1));
             else if (phases & 4)
                 PT_CUDA_OK(launch_pdl(sweep_kernel<true, true, false>, c1 - c0, kThreads, st, b.dl, b.dc + c0, (const float *)b.inv_out,
-                                      (const float *)b.inv_in, *hp, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket));
+                                      (const float *)b.inv_in, *hp, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket, 1));
             else
-                PT_CUDA_OK(launch_pdl(sweep_kernel<true, false, false>, (c1 - c0) * kUpdateSplit, kThreads, st, b.dl, b.dc + c0,
+                PT_CUDA_OK(launch_pdl(sweep_kernel<true, false, false>, (c1 - c0) * (unsigned)(t.sweeps / 2), kThreads, st, b.dl, b.dc + c0,
                                       (const float *)b.inv_out, (const float *)b.inv_in, *hp, b.linesum, b.colpart, b.linemax, b.colmax,
-                                      b.ticket));
+                                      b.ticket, t.sweeps / 2));
             c->launches += 1;
         }
         if (phases & 4) {
@@ -607,7 +613,7 @@ extern "C" pt_status pt_find_zero_groups(pt_ctx *c, const pt_layer *layers, int3
     pt_sgd_hparams none;
     memset(&none, 0, sizeof(none));
     PT_CUDA_OK(launch_pdl(sweep_kernel<false, false, true>, nch, kThreads, st, b.dl, b.dc, (const float *)b.inv_out,
-                          (const float *)b.inv_in, none, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket));
+                          (const float *)b.inv_in, none, b.linesum, b.colpart, b.linemax, b.colmax, b.ticket, 1));
     c->launches += 1;
     s = launch_finish(c, b, nj, nullptr, 4, threshold, st);
     if (s != PT_OK) return s;
