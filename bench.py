@@ -548,7 +548,7 @@ def run_ours(args):
                      "frac_all_passes": sum(floor_ms.values()) / conv_total_ms,
                      "tensor_only": {"achieved_tflops": dom_flops / dom_t / 1e12, "frac_of_sustained_bf16": dom_flops / dom_t / tc_peak},
                      "hbm_only": {"achieved_gbs": dom_bytes / dom_t / 1e9, "frac_of_copy_rate": dom_bytes / dom_t / bw_peak},
-                     "traffic": ncu_pass_traffic(dom) if (args.net == "resnet50" and args.keep is None and args.batch == 64 and args.algo == 0) else None,
+                     "traffic": ncu_pass_traffic(dom) if (args.net == "resnet50" and args.keep is None and args.batch == 64 and args.algo in (0, 2)) else None,
                      "traffic_note": "dram bytes of the pass's launches in the tracked ncu summary (profiles/); mostly reads: a launch's "
                                      "writes retire from L2 after it has ended",
                      "algorithmic_bytes": dom_bytes,
