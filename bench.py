@@ -212,9 +212,10 @@ def whole_job_value(flops_per_rank: float, world: int, ms_total: float, steps: i
 
 def chained_step_times(ctx, ts, args, seed):
     """The same pruned network as ONE chained training step (convolution -> batch norm -> ReLU, max pooling after the stem,
-    residual adds, the whole backward pass, the lasso step), replayed from a CUDA graph on one stream: with the normalisation
-    statistics taken in the convolution epilogues and with the stand-alone normalisation. Not the headline metric (which, as
-    the benchmark spec defines it, has no normalisation layers in it); reported beside it."""
+    residual adds, the whole backward pass, the lasso step), replayed from a CUDA graph: with the normalisation statistics
+    taken in the convolution epilogues and with the stand-alone normalisation (weight gradients and projection shortcuts on
+    side streams), and once more with everything on one stream. Not the headline metric (whose workload has no
+    normalisation layers in it); reported beside it."""
     import torch
     from paper_1901_09290_b200 import harness
     res = {}
